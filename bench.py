@@ -1,0 +1,387 @@
+"""Throughput of the G-CADA step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config cfg3] [--impl ours|reference]
+
+A step is one full G-CADA iteration (minibatch draw, dual-point gradients of
+all groups, innovation test, lazy aggregation, AMSGrad update, straggler
+clock) on the named synthetic workload.  One JSON line is printed by rank 0.
+
+--impl reference times the fp64 CPU oracle on the host cores instead (a
+deliberately plain program: its ratio to the CUDA path says nothing about
+kernel quality; the roofline fraction does).
+"""
+import argparse
+import hashlib
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+sys.path.insert(0, os.path.join(ROOT, "tests"))
+
+METRIC = "G-CADA iterations/sec (all groups)"
+UNIT = "it/s"
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant
+# kernel, from the ncu capture summarised under profiles/; valid only for the
+# kernel source whose digest is recorded with it.
+NCU_TRAFFIC = {
+    # config: (kernel source file, sha256 of that file at capture time, bytes per launch)
+}
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm=float(p["hbm_gbs"]), bf16=float(p["bf16_tflops"]),
+                    bf16_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    return dict(hbm=FALLBACK_HBM_GBS, bf16=FALLBACK_BF16_TFLOPS, bf16_sustained=1400.0, source="fallback")
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while running."""
+
+    def __init__(self, index):
+        super().__init__(daemon=True)
+        self.index, self.samples, self.reasons, self.stop_flag, self.max_mhz = index, [], set(), False, None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.handle = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def run(self):
+        if self.nv is None:
+            return
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+            "hw_power_brake_slowdown": getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80),
+        }
+        while not self.stop_flag:
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.handle, nv.NVML_CLOCK_SM))
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.handle)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle)
+                for n, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(n)
+            except Exception:
+                pass
+            time.sleep(0.02)
+
+    def result(self):
+        s = sorted(self.samples)
+        return {"sm_mhz": (s[len(s) // 2] if s else None), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(s)}
+
+
+def _dist_setup(n_gpus):
+    import torch
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    return rank, local, world
+
+
+def _barrier_max(world, value_ms, device):
+    import torch
+    if world == 1:
+        return value_ms
+    import torch.distributed as dist
+    t = torch.tensor([value_ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def _barrier(world):
+    import torch
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    torch.cuda.synchronize()
+
+
+def algorithmic_bytes_per_launch(w):
+    """Bytes the dominant (gradient) kernel must move per launch: every sampled
+    row once (it serves both points) plus its label."""
+    rows = (w["M"] // w["M_G"]) * w["batch"]
+    esz = 2 if w["compute"] == "bf16" else 4
+    return rows * (w["dims"][0] * esz + 4)
+
+
+def mlp_flops_per_iteration(w):
+    """Dense flops of the dual-point forward/backward as specified: per row and
+    point 2*n_in*n_out forward, the same for dW, and for dA except at layer 1."""
+    dims = w["dims"]
+    rows = (w["M"] // w["M_G"]) * w["batch"] * 2
+    f = 0
+    for l in range(1, len(dims)):
+        f += 2 * dims[l - 1] * dims[l] * (3 if l > 1 else 2)
+    return rows * f
+
+
+def run_ours(args):
+    import torch
+    from paper_2201_04301_b200 import binding
+    from paper_2201_04301_b200 import build as _build
+    from paper_2201_04301_b200.workloads import make_workload
+
+    rank, local, world = _dist_setup(args.gpus)
+    dev = torch.device("cuda", local)
+    if rank == 0:
+        _build.build()
+    _barrier(world)
+    binding.load()
+    t0 = time.time()
+    w = make_workload(args.config, device=dev, data_seed=rank, rows=args.rows)
+    stream = torch.cuda.Stream(device=dev)
+    torch.cuda.synchronize()
+    g = binding.from_workload(w, stream=stream)
+    gen_s = time.time() - t0
+    G = g.G
+
+    # --- device-resident timing ------------------------------------------------
+    g.step(args.warmup)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    l0 = g.get_launch_count()
+    _barrier(world)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    g.step(args.steps)
+    e1.record(stream)
+    e1.synchronize()
+    _barrier(world)
+    sampler.stop_flag = True
+    sampler.join()
+    ms = _barrier_max(world, e0.elapsed_time(e1), dev)
+    launches = g.get_launch_count() - l0
+    value = world * args.steps / (ms * 1e-3)
+
+    # --- per-kernel times (plain launches bracketed by events) -------------------
+    g.set_option(binding.OPT_TIMING, 1)
+    g.step(min(args.steps, 256))
+    (ms_grad, ms_sel, ms_upd), n_timed = g.get_kernel_times()
+    g.set_option(binding.OPT_TIMING, 0)
+
+    # --- end to end: minibatches fed from pinned host memory, theta read back ----
+    e2e = None
+    if not args.no_e2e:
+        rows = G * w["batch"]
+        d = w["dims"][0]
+        n_g = w["X"].shape[0] // G
+        idx = torch.cat([torch.randint(0, n_g, (w["batch"],), device=dev) + gi * n_g for gi in range(G)])
+        Xb = w["X"].index_select(0, idx)[:, :d].contiguous().cpu().pin_memory()
+        yb = w["y"].index_select(0, idx).contiguous().cpu().pin_memory()
+        h = binding.GCada(w["kind"], w["dims"], w["M"], w["M_G"], w["D"], w["c"], w["alpha"], w["beta1"],
+                          w["beta2"], w["eps"], compute=w["compute"], stream=stream)
+        h.set_batch(w["batch"])
+        h.set_theta(w["theta0"])
+        n_e2e = max(3, min(args.steps, args.e2e_steps))
+        for _ in range(3):
+            h.step_host_batch(Xb, yb)
+            h.get_theta()
+        _barrier(world)
+        t_a = time.perf_counter()
+        for _ in range(n_e2e):
+            h.step_host_batch(Xb, yb)
+            h.get_theta()
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t_a
+        _barrier(world)
+        dt = _barrier_max(world, dt * 1e3, dev) * 1e-3
+        e2e = {"value": world * n_e2e / dt, "unit": UNIT, "steps": n_e2e,
+               "h2d_bytes_per_step": int(Xb.numel() * Xb.element_size() + yb.numel() * yb.element_size()),
+               "d2h_bytes_per_step": int(g.p * 4 + 64)}
+        h.close()
+
+    if rank != 0:
+        return
+    peaks = _peaks()
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16" if w["compute"] == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": "%s: %s dims=%s N=%d M=%d M_G=%d batch=%d D=%d c=%g" % (
+            args.config, w["kind"], list(w["dims"]), w["X"].shape[0], w["M"], w["M_G"], w["batch"], w["D"], w["c"]),
+            "parallelism": "replicas only (%d)" % world,
+            "l2": "inputs larger than L2: each step gathers its rows from the resident training set"
+                  if w["X"].numel() * w["X"].element_size() > 126e6 else "training set smaller than L2 (latency-bound workload)",
+            "setup_s": round(gen_s, 1)},
+        "clocks": sampler.result(),
+        "gpu_launches": int(launches),
+        "kernel_ms": {"gradient": ms_grad, "select": ms_sel, "update": ms_upd, "timed_iterations": n_timed},
+    }
+    if e2e:
+        out["e2e"] = e2e
+    if w["kind"] != "mlp" or w["compute"] == "fp32":
+        bytes_launch = algorithmic_bytes_per_launch(w)
+        achieved = bytes_launch / (ms_grad * 1e-3) / 1e9 if ms_grad > 0 else None
+        traffic = None
+        rec = NCU_TRAFFIC.get(args.config)
+        if rec:
+            src = os.path.join(ROOT, "paper_2201_04301_b200", "csrc", rec[0])
+            if hashlib.sha256(open(src, "rb").read()).hexdigest() == rec[1]:
+                traffic = rec[2]
+        out["roofline"] = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm"], "unit": "GB/s",
+                           "frac": achieved / peaks["hbm"] if achieved else None, "traffic": traffic,
+                           "kernel": "gradient", "peak_source": peaks["source"],
+                           "algorithmic_bytes_per_launch": bytes_launch,
+                           "frac_of_nominal_8TBs": achieved / 8000.0 if achieved else None}
+    else:
+        flops = mlp_flops_per_iteration(w)
+        achieved = flops / (ms_grad * 1e-3) / 1e12 if ms_grad > 0 else None
+        out["roofline"] = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_sustained"],
+                           "unit": "TFLOP/s", "frac": achieved / peaks["bf16_sustained"] if achieved else None,
+                           "traffic": None, "kernel": "gradient (all GEMM launches of one iteration)",
+                           "peak_source": peaks["source"] + " (sustained)", "flops_per_iteration": flops}
+    if world == 1 and not args.no_cpu:
+        out["cpu_baseline"] = cpu_baseline(args.config, budget_s=args.cpu_budget)
+    print(json.dumps(out), flush=True)
+
+
+# ------------------------------------------------------------------------------
+# CPU oracle timing
+# ------------------------------------------------------------------------------
+def _oracle_workload(config, shard_rows):
+    """The named workload with every shard cut to `shard_rows` rows (same model,
+    groups, batch): what one oracle iteration costs does not depend on the shard size."""
+    from paper_2201_04301_b200.workloads import CONFIGS, make_workload
+    from parity import make_oracle
+    G = CONFIGS[config]["M"] // CONFIGS[config]["M_G"]
+    n_full = CONFIGS[config]["N"]
+    rows = min(n_full, G * shard_rows)
+    w = make_workload(config, device="cpu", rows=rows)
+    return w, make_oracle(w), G
+
+
+def _cores_used():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def _time_groups(o, n_groups):
+    """Time the dual-point gradients of `n_groups` groups plus the server update:
+    n_groups / G of one oracle iteration."""
+    import numpy as np
+    t0 = time.perf_counter()
+    theta_k = o.thetas[o.k]
+    for g in range(n_groups):
+        _, Xb, yb = o.minibatch(g)
+        old = o.theta_at(o.k - int(o.tau[g]))
+        a = o.model.grad(theta_k, Xb, yb, o.reduction)
+        b = o.model.grad(old, Xb, yb, o.reduction)
+        d = a - b
+        float(d @ d)
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(config, budget_s=15.0):
+    from paper_2201_04301_b200.workloads import CONFIGS
+    c = CONFIGS[config]
+    G = c["M"] // c["M_G"]
+    heavy = c["kind"] == "mlp" and c["compute"] == "bf16"
+    w, o, G = _oracle_workload(config, shard_rows=max(c["batch"], 256) if heavy else max(c["batch"] * 2, 1024))
+    t_one = _time_groups(o, 1)                       # calibration
+    if t_one * G <= budget_s / 3:
+        n = max(1, int(budget_s / (t_one * G)))
+        n = min(n, 200)
+        t0 = time.perf_counter()
+        for _ in range(n):
+            o.step()
+        dt = time.perf_counter() - t0
+        value, sample = n / dt, "%d full oracle iterations, shards cut to %d rows" % (n, w["X"].shape[0] // G)
+    else:
+        ng = max(1, min(G, int(budget_s / t_one)))
+        dt = _time_groups(o, ng)
+        value = 1.0 / (dt * G / ng)
+        sample = "dual-point gradients of %d of %d groups, extrapolated to a full iteration" % (ng, G)
+    return {"value": value, "unit": UNIT, "cores": _cores_used(), "kind": "oracle", "sample": sample}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2201_04301_b200.workloads import CONFIGS
+    c = CONFIGS[args.config]
+    G = c["M"] // c["M_G"]
+    w, o, G = _oracle_workload(args.config, shard_rows=max(c["batch"], 256))
+    total_budget = 150.0
+    per_step = total_budget / (args.steps + args.warmup)
+    t_one = _time_groups(o, 1)
+    ng = max(1, min(G, int(per_step / t_one)))
+    full = ng == G
+    for _ in range(args.warmup):
+        o.step() if full else _time_groups(o, ng)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        o.step() if full else _time_groups(o, ng)
+    dt = time.perf_counter() - t0
+    step_s = dt / args.steps
+    value = 1.0 / (step_s * G / ng)
+    sample = ("full oracle iterations" if full else
+              "each step = dual-point gradients of %d of %d groups, scaled to a full iteration" % (ng, G))
+    sample += ", shards cut to %d rows" % (w["X"].shape[0] // G)
+    out = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_s * 1e3 * G / ng,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "%s (CPU oracle, fp64 numpy)" % args.config},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": _cores_used(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(out), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--config", default="cfg3")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--rows", type=int, default=None, help="cut the training set to this many rows")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=60)
+    ap.add_argument("--cpu-budget", type=float, default=15.0)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        args.steps = args.steps if args.steps is not None else 20
+        args.warmup = args.warmup if args.warmup is not None else 3
+        run_reference(args)
+    else:
+        args.steps = args.steps if args.steps is not None else 10000
+        args.warmup = max(3, args.warmup if args.warmup is not None else 50)
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

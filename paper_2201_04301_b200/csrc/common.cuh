@@ -1,0 +1,151 @@
+// Shared device-side declarations of the G-CADA step library: the state that
+// lives in device memory, the parameter block handed to every kernel, the
+// counter-based generator and a few reduction helpers.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace gcada {
+
+// Device error words (DevState::err).
+enum { DEV_OK = 0, DEV_ERR_COPY_TIMEOUT = 1, DEV_ERR_BOUNDS = 2 };
+
+// Mutable run state kept in device memory so that a captured graph can be
+// replayed without changing kernel arguments.
+struct DevState {
+  long long k;                    // iteration about to run
+  unsigned long long uploads;     // sum of selection masks
+  unsigned long long comm;        // (M_G + 1) * uploads, Eq. (5)/(19)
+  unsigned long long comp;        // M_G * uploads, Eq. (6)/(22)
+  double wall;                    // simulated wall-clock, Eq. (4) summed
+  double last_dt;                 // its last increment
+  double rhs;                     // right side of Eq. (9), last iteration
+  int err;                        // DEV_*
+  int err_info;
+  unsigned int ticket_select;     // "last block done" counters
+  unsigned int ticket_update;
+  unsigned int ticket_aux;
+  unsigned int pad_;
+};
+
+// How a per-group gradient is spread over partial-sum slots by the linear
+// (logistic / quadratic) gradient kernels: CTA c owns the rows
+// [c*R/n, (c+1)*R/n) of the G*B minibatch rows and writes one slot per group
+// it touches, slot = c*maxseg + (g - first group of c).
+struct PartialMap {
+  int n_cta;      // 0 = gradients are already whole (one "slot" per group)
+  int maxseg;
+  int rows_per_group;  // B
+};
+
+struct Params {
+  DevState* st;
+  // problem
+  int G, M, M_G, D, B;
+  long long n_g;        // shard rows per group
+  long long p, p_pad;   // parameters; padded row stride of every p-vector (multiple of 4)
+  int d;                // features (linear models)
+  long long ld;         // row stride of X in elements
+  const void* X;
+  const void* y;
+  int identity_batch;   // 1: minibatch of group g = rows g*B .. of X (host-fed step)
+  // constants
+  double c;
+  float alpha, beta1, beta2, omb1, omb2, eps;
+  float scale;          // 1/B (mean) or 1 (sum)
+  uint32_t seed_lo, seed_hi;
+  double shift, inv_rate;
+  // state vectors (stride p_pad)
+  float* theta_ring;    // (D+1) iterates; slot j mod (D+1) holds theta^j
+  float* h;
+  float* vhat;
+  float* agg_hi;        // lazily aggregated gradient, Eq. (3), as an unevaluated sum hi + lo
+  float* agg_lo;
+  float* g_last;        // [G] last uploaded gradient
+  float* fresh;         // [G] gradient at theta^k
+  float* stale;         // [G] gradient at the stale iterate (optional, may be null)
+  float* partial;       // [slots][2] partial sums of (fresh, stale)
+  PartialMap pm;
+  // scheduler
+  int* tau;             // [G] age of information
+  double* lhs;          // [G]
+  double* t_g;          // [G]
+  double* s_ring;       // [D] squared step norms, slot j mod D holds ||theta^{j+1}-theta^j||^2
+  double* lhs_part;     // [G][nblk_select]
+  double* upd_part;     // [nblk_update]
+  unsigned char* mask_cur;  // [G]
+  unsigned char* hist;      // [hist_cap][G]
+  long long hist_cap;
+  const unsigned char* forced;  // [n][G] or null
+  long long forced_base;        // iteration of forced row 0
+};
+
+// ---------------------------------------------------------------------------
+// Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11).
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ uint4 philox4x32_10(uint4 ctr, uint32_t k0, uint32_t k1) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, ctr.x), lo0 = 0xD2511F53u * ctr.x;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, ctr.z), lo1 = 0xCD9E8D57u * ctr.z;
+    ctr = make_uint4(hi1 ^ ctr.y ^ k0, lo1, hi0 ^ ctr.w ^ k1, lo0);
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  return ctr;
+}
+
+__device__ __forceinline__ uint32_t philox_word(uint32_t a, uint32_t b, uint32_t k, uint32_t stream,
+                                                uint32_t k0, uint32_t k1) {
+  const uint4 o = philox4x32_10(make_uint4(a >> 2, b, k, stream), k0, k1);
+  const uint32_t s = a & 3u;
+  return s == 0 ? o.x : (s == 1 ? o.y : (s == 2 ? o.z : o.w));
+}
+
+// Global row of draw j of group g at iteration k (Section II-A: a minibatch
+// drawn at random from the group's shard; uniform with replacement).
+__device__ __forceinline__ long long batch_row(const Params& P, uint32_t k, int g, int j) {
+  if (P.identity_batch) return (long long)g * P.B + j;
+  const uint32_t w = philox_word((uint32_t)j, (uint32_t)g, k, 0u, P.seed_lo, P.seed_hi);
+  return (long long)g * P.n_g + (long long)(((unsigned long long)w * (unsigned long long)P.n_g) >> 32);
+}
+
+// Computing time of worker m at iteration k (Section II-B).
+__device__ __forceinline__ double worker_time(const Params& P, uint32_t k, int m) {
+  const uint32_t w = philox_word((uint32_t)m, 0u, k, 1u, P.seed_lo, P.seed_hi);
+  const double u = ((double)w + 0.5) * 2.3283064365386963e-10;  // 2^-32
+  return P.shift - log1p(-u) * P.inv_rate;
+}
+
+// ---------------------------------------------------------------------------
+// Reductions with a fixed order (bitwise reproducible).
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Sum over a block of up to 1024 threads; result valid in every thread.
+// `scratch` holds at least 33 doubles of shared memory.
+__device__ __forceinline__ double block_sum(double v, double* scratch) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+  v = warp_sum(v);
+  __syncthreads();
+  if (lane == 0) scratch[w] = v;
+  __syncthreads();
+  if (w == 0) {
+    double t = lane < nw ? scratch[lane] : 0.0;
+    t = warp_sum(t);
+    if (lane == 0) scratch[32] = t;
+  }
+  __syncthreads();
+  return scratch[32];
+}
+
+}  // namespace gcada

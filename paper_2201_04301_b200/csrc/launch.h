@@ -1,0 +1,36 @@
+// Host-side launch plans and launcher declarations shared by the translation
+// units of the library.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+
+#include "common.cuh"
+
+namespace gcada {
+
+struct LinearPlan {
+  bool small;       // d <= 256: warp-per-row kernel, else the row-ring kernel
+  int cpl;          // small: columns per lane
+  int cpt, threads, R, nslot;  // large: 16-byte chunks per thread, CTA size, rows per batch, ring slots
+  size_t smem_bytes;
+  int n_cta;
+  int maxseg;       // partial slots per CTA
+};
+
+// Chooses the kernel and its shape; false (with *why) if the shape is not supported.
+bool plan_linear(int d, long long ld, const void* X, int G, int B, int sm_count, size_t smem_optin,
+                 LinearPlan* plan, const char** why);
+// One-time function attributes (dynamic shared memory size); call before the first launch.
+cudaError_t prepare_grad_linear(const LinearPlan& plan, bool quad);
+cudaError_t launch_grad_linear(const Params& P, const LinearPlan& plan, bool quad, cudaStream_t st);
+
+struct TailPlan {
+  int select_cols4_per_block;  // float4 columns per block of the selection kernel
+  int select_blocks_x;         // blocks per group
+  int update_blocks;
+};
+void plan_tail(long long p_pad, int G, int sm_count, TailPlan* plan);
+cudaError_t launch_select(const Params& P, const TailPlan& plan, cudaStream_t st);
+cudaError_t launch_update(const Params& P, const TailPlan& plan, cudaStream_t st);
+
+}  // namespace gcada

@@ -1,0 +1,272 @@
+// Server-side kernels of one G-CADA iteration.
+//
+// select_kernel: adds the gradient partial sums of every group in a fixed
+//   order, forms LHS_g = ||fresh_g - stale_g||^2 (the gradient innovation the
+//   left side of Eq. (9) estimates; the linear-model kernels hand over the
+//   innovation itself, the MLP kernels both gradients), and its last block
+//   evaluates the right side c * sum_d ||theta^{k+1-d} - theta^{k-d}||^2, the age rule tau_g >= D
+//   (Section IV), the selection mask, the ages for the next iteration
+//   (Algorithm 1, last step), the workers' computing times with the
+//   fastest-in-group / slowest-selected-group wall-clock (Section II-B,
+//   Section V-A) and the load counters (Eqs. 5, 6, 19, 22).
+// update_kernel: swaps the selected groups' fresh gradients into the lazily
+//   aggregated gradient (Eq. 3), applies Eq. (8a)-(8c), stores theta^{k+1} in
+//   the iterate ring and ||theta^{k+1} - theta^k||^2 in the ring of squared
+//   step norms that feeds the next D right sides.
+#include "common.cuh"
+#include "launch.h"
+
+namespace gcada {
+
+__device__ __forceinline__ float4 ld4(const float* p) { return *reinterpret_cast<const float4*>(p); }
+__device__ __forceinline__ void st4(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
+
+template <int U>
+__global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_x) {
+  __shared__ double scratch[40];
+  __shared__ int sh_nsel[8];
+  __shared__ double sh_tmax[8];
+  __shared__ bool is_last;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int g = blockIdx.y;
+  const long long cols4 = P.p_pad >> 2;
+  const long long k = P.st->k;
+
+  // ---- phase 1: partial sums -> fresh_g (and stale_g), innovation norm
+  int c_lo = 0, c_hi = -1;
+  const long long Rtot = (long long)P.G * P.pm.rows_per_group;
+  const int n = P.pm.n_cta;
+  if (n > 0) {
+    const long long x0 = (long long)g * P.pm.rows_per_group;
+    const long long x1 = x0 + P.pm.rows_per_group - 1;
+    c_lo = (int)(((x0 + 1) * n - 1) / Rtot);
+    c_hi = (int)(((x1 + 1) * n - 1) / Rtot);
+  }
+  double local = 0.0;
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+    const long long i4 = ((long long)blockIdx.x * U + u) * 256 + tid;
+    if (i4 >= cols4) continue;
+    float4 f, s;
+    if (n > 0) {
+      f = make_float4(0.f, 0.f, 0.f, 0.f);
+      s = f;
+      for (int c = c_lo; c <= c_hi; ++c) {
+        const int gf = (int)(((long long)c * Rtot / n) / P.pm.rows_per_group);
+        const float* src = P.partial + ((long long)(c * P.pm.maxseg + (g - gf)) * 2) * P.p_pad + i4 * 4;
+        const float4 a = ld4(src), b = ld4(src + P.p_pad);
+        f.x += a.x; f.y += a.y; f.z += a.z; f.w += a.w;
+        s.x += b.x; s.y += b.y; s.z += b.z; s.w += b.w;
+      }
+      // second slot half = innovation; the stale-point gradient is fresh - innovation
+      st4(P.fresh + (long long)g * P.p_pad + i4 * 4, f);
+      if (P.stale)
+        st4(P.stale + (long long)g * P.p_pad + i4 * 4, make_float4(f.x - s.x, f.y - s.y, f.z - s.z, f.w - s.w));
+    } else {
+      f = ld4(P.fresh + (long long)g * P.p_pad + i4 * 4);
+      s = ld4(P.stale + (long long)g * P.p_pad + i4 * 4);
+      s = make_float4(f.x - s.x, f.y - s.y, f.z - s.z, f.w - s.w);
+    }
+    const float dx = s.x, dy = s.y, dz = s.z, dw = s.w;  // the innovation
+    local += (double)dx * dx + (double)dy * dy + (double)dz * dz + (double)dw * dw;
+  }
+  const double tot = block_sum(local, scratch);
+  if (tid == 0) {
+    P.lhs_part[(long long)g * blocks_x + blockIdx.x] = tot;
+    __threadfence();
+    const unsigned int total = (unsigned int)blocks_x * (unsigned int)P.G;
+    is_last = atomicAdd(&P.st->ticket_select, 1u) == total - 1u;
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+
+  // ---- phase 2 (last block only): the server's scheduling decision
+  double rhs = 0.0;
+  for (int i = 0; i < P.D; ++i) rhs += P.s_ring[i];
+  rhs *= P.c;
+  const volatile double* parts = P.lhs_part;
+  int nsel = 0;
+  double tmax = 0.0;
+  const uint32_t k32 = (uint32_t)k;
+  for (int gg = warp; gg < P.G; gg += 8) {
+    double s = 0.0;
+    for (int b = lane; b < blocks_x; b += 32) s += parts[(long long)gg * blocks_x + b];
+    s = warp_sum(s);
+    double t = 1.0e300;
+    for (int j = lane; j < P.M_G; j += 32) t = fmin(t, worker_time(P, k32, gg * P.M_G + j));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) t = fmin(t, __shfl_xor_sync(0xffffffffu, t, o));
+    if (lane == 0) {
+      const int tau = P.tau[gg];
+      bool sel;
+      if (P.forced)
+        sel = P.forced[(k - P.forced_base) * P.G + gg] != 0;
+      else
+        sel = (tau >= P.D) || (s > rhs);
+      P.lhs[gg] = s;
+      P.t_g[gg] = t;
+      P.mask_cur[gg] = sel ? 1 : 0;
+      P.hist[(k % P.hist_cap) * P.G + gg] = sel ? 1 : 0;
+      P.tau[gg] = sel ? 1 : tau + 1;
+      if (sel) {
+        ++nsel;
+        tmax = fmax(tmax, t);
+      }
+    }
+  }
+  if (lane == 0) {
+    sh_nsel[warp] = nsel;
+    sh_tmax[warp] = tmax;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int ns = 0;
+    double tm = 0.0;
+    for (int w = 0; w < 8; ++w) {
+      ns += sh_nsel[w];
+      tm = fmax(tm, sh_tmax[w]);
+    }
+    DevState* st = P.st;
+    st->uploads += (unsigned long long)ns;
+    st->comm += (unsigned long long)ns * (unsigned long long)(P.M_G + 1);
+    st->comp += (unsigned long long)ns * (unsigned long long)P.M_G;
+    st->wall += tm;
+    st->last_dt = tm;
+    st->rhs = rhs;
+    st->ticket_select = 0u;
+  }
+}
+
+// Error-free difference and compensated accumulation: (hi, lo) += f - l with
+// the rounding errors of both operations kept in lo (Knuth's TwoSum), so that
+// the aggregate stays equal to the sum of the last uploaded gradients however
+// many swaps have been folded in.
+__device__ __forceinline__ void fold(float& hi, float& lo, float f, float l) {
+  const float dff = f - l;
+  const float bb = dff - f;
+  const float e1 = (f - (dff - bb)) + (-l - bb);
+  const float s = hi + dff;
+  const float b2 = s - hi;
+  const float e2 = (hi - (s - b2)) + (dff - b2);
+  hi = s;
+  lo += e1 + e2;
+}
+__device__ __forceinline__ void renorm(float& hi, float& lo) {
+  const float t = hi + lo;
+  lo = lo - (t - hi);
+  hi = t;
+}
+
+__global__ void __launch_bounds__(256) update_kernel(const Params P) {
+  extern __shared__ int sel_list[];  // selected groups, ascending
+  __shared__ int n_sel_sh;
+  __shared__ double scratch[40];
+  __shared__ bool is_last;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const long long cols4 = P.p_pad >> 2;
+  const long long k = P.st->k;
+  const int ring = P.D + 1;
+
+  if (warp == 0) {
+    int cnt = 0;
+    for (int g0 = 0; g0 < P.G; g0 += 32) {
+      const int gg = g0 + lane;
+      const bool s = gg < P.G && P.mask_cur[gg] != 0;
+      const unsigned int b = __ballot_sync(0xffffffffu, s);
+      if (s) sel_list[cnt + __popc(b & ((1u << lane) - 1u))] = gg;
+      cnt += __popc(b);
+    }
+    if (lane == 0) n_sel_sh = cnt;
+  }
+  __syncthreads();
+  const int n_sel = n_sel_sh;
+
+  const long long i4 = (long long)blockIdx.x * 256 + tid;
+  double local = 0.0;
+  if (i4 < cols4) {
+    const long long o = i4 * 4;
+    float4 hi = ld4(P.agg_hi + o), lo = ld4(P.agg_lo + o);
+    for (int j = 0; j < n_sel; ++j) {
+      const long long go = (long long)sel_list[j] * P.p_pad + o;
+      const float4 f = ld4(P.fresh + go), l = ld4(P.g_last + go);
+      st4(P.g_last + go, f);
+      fold(hi.x, lo.x, f.x, l.x);
+      fold(hi.y, lo.y, f.y, l.y);
+      fold(hi.z, lo.z, f.z, l.z);
+      fold(hi.w, lo.w, f.w, l.w);
+    }
+    renorm(hi.x, lo.x);
+    renorm(hi.y, lo.y);
+    renorm(hi.z, lo.z);
+    renorm(hi.w, lo.w);
+    st4(P.agg_hi + o, hi);
+    st4(P.agg_lo + o, lo);
+    // Eq. (8a)-(8c)
+    float4 h = ld4(P.h + o), vh = ld4(P.vhat + o);
+    const float4 th = ld4(P.theta_ring + (k % ring) * P.p_pad + o);
+    float4 tn;
+#define GCADA_AMSGRAD(c)                                   \
+  {                                                        \
+    const float gr = hi.c;                                 \
+    h.c = P.beta1 * h.c + P.omb1 * gr;                     \
+    const float v = P.beta2 * vh.c + P.omb2 * (gr * gr);   \
+    vh.c = fmaxf(vh.c, v);                                 \
+    const float up = P.alpha * h.c / sqrtf(P.eps + vh.c);  \
+    tn.c = th.c - up;                                      \
+    local += (double)up * (double)up;                      \
+  }
+    GCADA_AMSGRAD(x)
+    GCADA_AMSGRAD(y)
+    GCADA_AMSGRAD(z)
+    GCADA_AMSGRAD(w)
+#undef GCADA_AMSGRAD
+    st4(P.h + o, h);
+    st4(P.vhat + o, vh);
+    st4(P.theta_ring + ((k + 1) % ring) * P.p_pad + o, tn);
+  }
+  const double tot = block_sum(local, scratch);
+  if (tid == 0) {
+    P.upd_part[blockIdx.x] = tot;
+    __threadfence();
+    is_last = atomicAdd(&P.st->ticket_update, 1u) == gridDim.x - 1u;
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  const volatile double* parts = P.upd_part;
+  double s = 0.0;
+  for (unsigned int b = tid; b < gridDim.x; b += 256) s += parts[b];
+  s = block_sum(s, scratch);
+  if (tid == 0) {
+    P.s_ring[k % P.D] = s;
+    P.st->k = k + 1;
+    P.st->ticket_update = 0u;
+  }
+}
+
+void plan_tail(long long p_pad, int G, int sm_count, TailPlan* plan) {
+  (void)G;
+  (void)sm_count;
+  const long long cols4 = p_pad / 4;
+  const int U = cols4 > 256 * 1024 ? 4 : 1;
+  plan->select_cols4_per_block = 256 * U;
+  plan->select_blocks_x = (int)((cols4 + 256 * U - 1) / (256 * U));
+  plan->update_blocks = (int)((cols4 + 255) / 256);
+}
+
+cudaError_t launch_select(const Params& P, const TailPlan& plan, cudaStream_t st) {
+  dim3 grid(plan.select_blocks_x, P.G);
+  if (plan.select_cols4_per_block == 256)
+    select_kernel<1><<<grid, 256, 0, st>>>(P, plan.select_blocks_x);
+  else
+    select_kernel<4><<<grid, 256, 0, st>>>(P, plan.select_blocks_x);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_update(const Params& P, const TailPlan& plan, cudaStream_t st) {
+  update_kernel<<<plan.update_blocks, 256, (size_t)P.G * sizeof(int), st>>>(P);
+  return cudaGetLastError();
+}
+
+}  // namespace gcada

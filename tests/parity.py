@@ -1,0 +1,114 @@
+"""Helpers shared by the GPU parity tests: build the CPU oracle and the CUDA
+context from the same seeded workload and compare them step by step."""
+import numpy as np
+import torch
+
+from oracle.gcada import GCadaOracle
+from oracle.models import make_model
+from paper_2201_04301_b200 import binding
+
+TOL_FP32 = 1e-5      # relative L2, gradients and parameters, fp32 paths
+TOL_BF16 = 2e-2      # relative L2 with bf16 operands
+MARGIN = 1e-4        # selection test: relative margin below which a flip is allowed
+
+
+def rel_l2(a, b):
+    a = np.asarray(a, dtype=np.float64).ravel()
+    b = np.asarray(b, dtype=np.float64).ravel()
+    den = np.linalg.norm(b)
+    return float(np.linalg.norm(a - b) / den) if den > 0 else float(np.linalg.norm(a))
+
+
+class DeviceRows:
+    """Rows of a CUDA matrix fetched on demand (for data sets too large to copy)."""
+
+    def __init__(self, X, d):
+        self.X, self.d = X, d
+
+    def __getitem__(self, idx):
+        t = torch.as_tensor(np.asarray(idx), device=self.X.device)
+        return self.X.index_select(0, t)[:, :self.d].float().cpu().numpy()
+
+
+def make_oracle(w, lazy=False, **kw):
+    d = w["dims"][0]
+    model = make_model(w["kind"], w["dims"], bf16=(w["compute"] == "bf16"))
+    if lazy:
+        X, y = DeviceRows(w["X"], d), DeviceRows(w["y"].reshape(-1, 1), 1)
+
+        class _Y:
+            def __init__(self, t):
+                self.t = t
+
+            def __len__(self):
+                return self.t.shape[0]
+
+            def __getitem__(self, idx):
+                i = torch.as_tensor(np.asarray(idx), device=self.t.device)
+                return self.t.index_select(0, i).cpu().numpy()
+        y = _Y(w["y"])
+    else:
+        X = w["X"][:, :d].float().cpu().numpy().astype(np.float64)
+        y = w["y"].cpu().numpy()
+    args = dict(X=X, y=y, batch=w["batch"], theta0=w["theta0"].cpu().numpy().astype(np.float64),
+                seed=w["seed"], shift=w["shift"], rate=w["rate"])
+    args.update(kw)
+    return GCadaOracle(model, w["M"], w["M_G"], w["D"], w["c"], w["alpha"], w["beta1"], w["beta2"], w["eps"],
+                       **args)
+
+
+def to_cuda(w):
+    w = dict(w)
+    for key in ("X", "y", "theta0"):
+        w[key] = w[key].cuda()
+    return w
+
+
+def forced_parity(w, K, tol=TOL_FP32, stream=None, reduction="mean", check_stale=True):
+    """Run the oracle free for K steps and the CUDA path teacher-forced with the
+    oracle's masks; compare every step.  Returns the number of steps at which
+    the CUDA path's own test outcome differed from the oracle's (only allowed
+    within MARGIN)."""
+    o = make_oracle(w, reduction=reduction)
+    wc = to_cuda(w)
+    opts = {binding.OPT_KEEP_STALE: 1.0, binding.OPT_REDUCTION: 0.0 if reduction == "mean" else 1.0}
+    g = binding.from_workload(wc, stream=stream, options=opts)
+    flips = 0
+    worst = dict(fresh=0.0, stale=0.0, theta=0.0, lhs=0.0)
+    for k in range(K):
+        tau_before = g.get_debug(binding.DBG_TAU)
+        rec = o.step()
+        g.step_forced(rec["mask"][None, :])
+        fresh, stale = g.get_debug(binding.DBG_FRESH), g.get_debug(binding.DBG_STALE)
+        for gi in range(o.G):
+            e = rel_l2(fresh[gi], rec["fresh"][gi])
+            worst["fresh"] = max(worst["fresh"], e)
+            assert e <= tol, ("fresh", k, gi, e)
+            if check_stale:
+                e = rel_l2(stale[gi], rec["stale"][gi])
+                worst["stale"] = max(worst["stale"], e)
+                assert e <= tol, ("stale", k, gi, e)
+        lhs, rhs = g.get_debug(binding.DBG_LHS), g.get_debug(binding.DBG_RHS)[0]
+        assert np.array_equal(tau_before, rec["tau"]), (k, tau_before, rec["tau"])
+        assert rhs == np.float64(rhs) and abs(rhs - rec["rhs"]) <= 1e-4 * max(rec["rhs"], 1e-300), (k, rhs, rec["rhs"])
+        # the CUDA path's own decision, from its own numbers
+        own = (tau_before >= o.D) | (lhs > rhs)
+        for gi in range(o.G):
+            if bool(own[gi]) != bool(rec["mask"][gi]):
+                margin = abs(rec["lhs"][gi] - rec["rhs"]) / max(rec["lhs"][gi], rec["rhs"], 1e-300)
+                assert margin < MARGIN, ("mask", k, gi, lhs[gi], rhs, rec["lhs"][gi], rec["rhs"])
+                flips += 1
+            if rec["lhs"][gi] > 0:
+                worst["lhs"] = max(worst["lhs"], abs(lhs[gi] - rec["lhs"][gi]) / rec["lhs"][gi])
+        e = rel_l2(g.get_theta(), rec["theta"])
+        worst["theta"] = max(worst["theta"], e)
+        assert e <= tol, ("theta", k, e)
+        assert np.allclose(g.get_debug(binding.DBG_TGROUP), rec["t_g"], rtol=1e-12, atol=0)
+    assert np.array_equal(g.get_selection_mask(0, K), np.stack(o.masks))
+    assert g.get_comm_count() == (o.uploads, o.comm, o.comp)
+    wall, last = g.get_wallclock()
+    assert abs(wall - o.wall) <= 1e-12 * max(o.wall, 1.0) and abs(last - rec["dt"]) <= 1e-12 * max(rec["dt"], 1.0)
+    assert g.get_iteration() == K
+    assert rel_l2(g.get_debug(binding.DBG_AGG), rec["agg"]) <= tol
+    g.close()
+    return flips, worst

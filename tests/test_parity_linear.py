@@ -1,0 +1,153 @@
+"""CUDA path vs CPU oracle, logistic and quadratic models, element by element
+on the same seeded inputs (through the C ABI)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2201_04301_b200 import binding
+from paper_2201_04301_b200.workloads import make_workload
+
+from parity import MARGIN, TOL_FP32, forced_parity, make_oracle, rel_l2, to_cuda
+
+pytestmark = pytest.mark.gpu
+
+
+def _stream():
+    return torch.cuda.Stream()
+
+
+def test_cfg1_teacher_forced_full_run():
+    w = make_workload("cfg1")
+    flips, worst = forced_parity(w, w["K"], stream=_stream())
+    print("cfg1 worst", worst, "flips", flips)
+    assert flips <= 2
+
+
+def test_cfg2_teacher_forced():
+    """d = 54 in rows padded to 56 floats, batch 1024: several CTAs per group."""
+    w = make_workload("cfg2", rows=100000)
+    flips, worst = forced_parity(w, 60, stream=_stream())
+    print("cfg2 worst", worst, "flips", flips)
+
+
+def test_cfg3_shape_small_shards():
+    """d = 4096, 64 groups of 512 rows per batch as in the large workload, but
+    shards of 600 rows so that the oracle can hold the data."""
+    w = make_workload("cfg3", rows=64 * 600)
+    flips, worst = forced_parity(w, 12, stream=_stream())
+    print("cfg3-small worst", worst, "flips", flips)
+
+
+@pytest.mark.parametrize("d,ld,batch,M,M_G,D", [
+    (1, 1, 5, 2, 1, 1),         # scalar model, one worker per group, D = 1
+    (7, 9, 33, 3, 3, 2),        # G = 1, odd sizes, stride > d
+    (33, 40, 100, 8, 2, 3),     # two columns per lane with a ragged tail
+    (200, 200, 17, 6, 2, 4),    # widest warp-per-row shape
+    (257, 260, 37, 4, 2, 3),    # smallest row-ring shape, ragged 16-byte chunk
+    (1000, 1000, 70, 10, 2, 5),
+    (3001, 3004, 19, 6, 3, 2),  # ragged tail, four chunks per thread
+])
+def test_odd_shapes(d, ld, batch, M, M_G, D):
+    G = M // M_G
+    w = make_workload("cfg1", rows=G * 50, dims=(d,), M=M, M_G=M_G, D=D, batch=batch, c=0.5)
+    if ld != d:
+        Xp = torch.full((w["X"].shape[0], ld), float("nan"))
+        Xp[:, :d] = w["X"]
+        w["X"], w["ld"] = Xp, ld
+        w["X"][:, d:] = 7.0      # padding must never be read into a result
+    forced_parity(w, 3 * D + 2, stream=_stream())
+
+
+@pytest.mark.parametrize("reduction", ["mean", "sum"])
+def test_quadratic_model(reduction):
+    w = make_workload("cfg1", rows=3000, kind="quadratic", alpha=0.002)
+    forced_parity(w, 25, stream=_stream(), reduction=reduction)
+
+
+def test_free_running_masks_match_until_a_near_tie():
+    w = make_workload("cfg1")
+    o = make_oracle(w)
+    g = binding.from_workload(to_cuda(w), stream=_stream())
+    K = w["K"]
+    g.step(K)
+    got = g.get_selection_mask(0, K)
+    for k in range(K):
+        rec = o.step()
+        if not np.array_equal(got[k], rec["mask"]):
+            bad = np.nonzero(got[k] != rec["mask"])[0]
+            for gi in bad:
+                margin = abs(rec["lhs"][gi] - rec["rhs"]) / max(rec["lhs"][gi], rec["rhs"])
+                assert margin < MARGIN, (k, gi, margin)
+            break
+    else:
+        assert rel_l2(g.get_theta(), o.theta) <= TOL_FP32
+        assert g.get_comm_count() == (o.uploads, o.comm, o.comp)
+    assert got.sum() < K * o.G          # the rule skipped uploads
+    assert got[0].all()                 # first iteration selects every group
+
+
+def test_graph_replay_equals_plain_launches_bitwise():
+    w = to_cuda(make_workload("cfg2", rows=50000))
+    runs = []
+    for graph, chunks in ((1.0, [37]), (0.0, [37]), (1.0, [16, 5, 16])):
+        g = binding.from_workload(w, stream=_stream(), options={binding.OPT_GRAPH: graph})
+        for n in chunks:
+            g.step(n)
+        runs.append((g.get_theta(), g.get_selection_mask(0, 37), g.get_wallclock(), g.get_comm_count()))
+        g.close()
+    for r in runs[1:]:
+        assert np.array_equal(r[0], runs[0][0]) and np.array_equal(r[1], runs[0][1])
+        assert r[2] == runs[0][2] and r[3] == runs[0][3]
+
+
+def test_host_fed_step_equals_resident_step():
+    from oracle import philox
+    w = make_workload("cfg1", rows=3000)
+    wc = to_cuda(w)
+    a = binding.from_workload(wc, stream=_stream())
+    b = binding.GCada(w["kind"], w["dims"], w["M"], w["M_G"], w["D"], w["c"], w["alpha"], w["beta1"],
+                      w["beta2"], w["eps"], stream=_stream())
+    b.set_batch(w["batch"])
+    b.set_theta(w["theta0"])
+    G, n_g = a.G, w["X"].shape[0] // a.G
+    for k in range(15):
+        idx = np.concatenate([philox.batch_indices(w["seed"], k, g, w["batch"], n_g) for g in range(G)])
+        Xb = w["X"][idx].contiguous().pin_memory()
+        yb = w["y"][idx].contiguous().pin_memory()
+        a.step(1)
+        b.step_host_batch(Xb, yb)
+        assert np.array_equal(a.get_theta(), b.get_theta())
+        assert np.array_equal(a.get_selection_mask(k, 1), b.get_selection_mask(k, 1))
+    assert a.get_wallclock() == b.get_wallclock()
+
+
+def test_state_errors_and_history_window():
+    w = to_cuda(make_workload("cfg1", rows=600))
+    g = binding.GCada(w["kind"], w["dims"], w["M"], w["M_G"], w["D"], w["c"], w["alpha"], w["beta1"],
+                      w["beta2"], w["eps"])
+    with pytest.raises(binding.GCadaError) as e:
+        g.step(1)
+    assert e.value.status == binding.ESTATE
+    g.set_option(binding.OPT_HISTORY, 8)
+    g.set_theta(w["theta0"])
+    with pytest.raises(binding.GCadaError) as e:
+        g.step(1)
+    assert e.value.status == binding.ESTATE        # no data yet
+    with pytest.raises(binding.GCadaError) as e:
+        g.set_data(w["X"], w["y"], 0)
+    assert e.value.status == binding.EINVAL
+    g.set_data(w["X"], w["y"], w["batch"])
+    g.step(20)                                     # legacy default stream, plain launches
+    assert g.get_iteration() == 20
+    assert g.get_selection_mask(12, 8).shape == (8, g.G)
+    for first, n in ((11, 8), (15, 6), (-1, 1)):
+        with pytest.raises(binding.GCadaError) as e:
+            g.get_selection_mask(first, n)
+        assert e.value.status == binding.EINVAL
+    with pytest.raises(binding.GCadaError):
+        g.set_option(binding.OPT_REDUCTION, 1)     # fixed once stepping has begun
+    up, comm, comp = g.get_comm_count()
+    assert comm == (g.M_G + 1) * up and comp == g.M_G * up
+    assert g.get_launch_count() == 60
+    g.set_theta(w["theta0"])                       # restart
+    assert g.get_iteration() == 0 and g.get_comm_count() == (0, 0, 0)
