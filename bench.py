@@ -156,7 +156,7 @@ def run_ours(args):
     w = make_workload(args.config, device=dev, data_seed=rank, rows=args.rows)
     stream = torch.cuda.Stream(device=dev)
     torch.cuda.synchronize()
-    g = binding.from_workload(w, stream=stream)
+    g = binding.from_workload(w, stream=stream, options={binding.OPT_GRAPH: 0.0 if args.no_graph else 1.0})
     gen_s = time.time() - t0
     G = g.G
 
@@ -370,6 +370,7 @@ def main():
     ap.add_argument("--rows", type=int, default=None, help="cut the training set to this many rows")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="plain launches instead of graph replay")
     ap.add_argument("--e2e-steps", type=int, default=60)
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     args = ap.parse_args()

@@ -147,7 +147,8 @@ __global__ void __launch_bounds__(THREADS, 1) grad_linear_large_kernel(const Par
 
   const int g_first = (int)(r0 / P.B);
   int cur_g = -1;
-  long long rowctr = 0;  // rows consumed by this CTA so far (slot / parity bookkeeping)
+  int cslot = 0;          // ring slot of the next row to consume
+  uint32_t cphase = 0;    // barrier parity of that slot's current fill
   int failed = 0;
 
   auto flush = [&](int g) {
@@ -185,7 +186,8 @@ __global__ void __launch_bounds__(THREADS, 1) grad_linear_large_kernel(const Par
     if (tid == 0) {
       const int n0 = nrows < nslot ? nrows : nslot;
       for (; issued < n0; ++issued) {
-        const int s = (int)((rowctr + issued) % nslot);
+        int s = cslot + issued;
+        if (s >= nslot) s -= nslot;
         mbar_expect_tx(&bars[s], rowbytes);
         bulk_load(slots + (size_t)s * rowbytes, Xf + row_sm[issued] * P.ld, rowbytes, &bars[s]);
       }
@@ -224,9 +226,13 @@ __global__ void __launch_bounds__(THREADS, 1) grad_linear_large_kernel(const Par
         pz[r] = 0.f;
         pz[R + r] = 0.f;
         if (r < nb) {
-          const long long rc = rowctr + r;
-          const int s = (int)(rc % nslot);
-          if (!mbar_wait_bounded(&bars[s], (uint32_t)((rc / nslot) & 1))) failed = 1;
+          int s = cslot + r;
+          uint32_t ph = cphase;
+          if (s >= nslot) {
+            s -= nslot;
+            ph ^= 1u;
+          }
+          if (!mbar_wait_bounded(&bars[s], ph)) failed = 1;
           const float4* src = reinterpret_cast<const float4*>(slots + (size_t)s * rowbytes);
 #pragma unroll
           for (int i = 0; i < CPT; ++i) {
@@ -251,7 +257,8 @@ __global__ void __launch_bounds__(THREADS, 1) grad_linear_large_kernel(const Par
       if (failed) break;
       if (tid == 0) {
         for (int r = 0; r < nb && issued < nrows; ++r, ++issued) {
-          const int s = (int)((rowctr + r) % nslot);  // slot of a row consumed just now
+          int s = cslot + r;  // slot of a row consumed just now
+          if (s >= nslot) s -= nslot;
           mbar_expect_tx(&bars[s], rowbytes);
           bulk_load(slots + (size_t)s * rowbytes, Xf + row_sm[issued] * P.ld, rowbytes, &bars[s]);
         }
@@ -292,15 +299,24 @@ __global__ void __launch_bounds__(THREADS, 1) grad_linear_large_kernel(const Par
         }
       }
       consumed += nb;
-      rowctr += nb;
+      cslot += nb;
+      if (cslot >= nslot) {
+        cslot -= nslot;
+        cphase ^= 1u;
+      }
     }
     if (failed) {
       // give copies already in flight a bounded chance to land before leaving
       if (tid == 0) {
         atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
         for (int j = consumed; j < issued; ++j) {
-          const long long rc = rowctr + (j - consumed);
-          mbar_wait_bounded(&bars[rc % nslot], (uint32_t)((rc / nslot) & 1));
+          int s = cslot + (j - consumed);
+          uint32_t ph = cphase;
+          if (s >= nslot) {
+            s -= nslot;
+            ph ^= 1u;
+          }
+          mbar_wait_bounded(&bars[s], ph);
         }
       }
       return;
