@@ -37,6 +37,8 @@
 #ifndef GCADA_H
 #define GCADA_H
 
+#include <stddef.h>
+
 #ifdef __cplusplus
 extern "C" {
 #endif
@@ -193,6 +195,42 @@ gcada_status gcada_get_launch_count(gcada_ctx *ctx, unsigned long long *launches
  * ms[2] update kernel, over the (at most 512) most recent timed iterations,
  * whose number goes to *n_timed.  Synchronises the stream. */
 gcada_status gcada_get_kernel_times(gcada_ctx *ctx, double ms[3], int *n_timed);
+
+/*
+ * Innovation norms without any allocation.  (The paper has no counterpart of
+ * this call; it exists for the sake of callers, not of the method.)
+ *
+ * Some users of this library run where device memory may not be allocated:
+ * inside a region whose memory plan is frozen (a serving process that
+ * pre-allocated its pool, a real-time loop, code running between the capture
+ * and replay of someone else's graph) or under an allocator they do not
+ * control.  gcada_create and gcada_set_theta allocate, so such callers cannot
+ * use a context.  This call gives them the test quantity of the selection
+ * rule on gradients they already hold:
+ *     lhs_dev[g] = || fresh_dev[g*ld .. g*ld+p) - stale_dev[g*ld .. g*ld+p) ||^2
+ * for g < G, the same arithmetic as the selection kernel (float difference,
+ * double accumulation, fixed summation order).  All three pointers are device
+ * memory of the CURRENT device, owned by the caller; lhs_dev receives G
+ * doubles.  The work is enqueued on cuda_stream (cudaStream_t as void*, NULL =
+ * legacy default stream) and is asynchronous.
+ *
+ * Scratch space is a fixed 512 KiB array inside the library image: every GPU
+ * that loads the library carries it until the process exits.  Limit:
+ * G <= GCADA_NOALLOC_MAX_GROUPS, otherwise GCADA_EINVAL and nothing runs (p
+ * is not limited).  All calls on one device share that array, so two calls
+ * whose kernels may overlap on the GPU (different streams without ordering
+ * between them) race and give wrong sums; order them.  The array keeps the
+ * previous call's contents; the one word that must start at zero is cleared
+ * on the stream by every call.  The first call on each device looks up the
+ * array's device address (cudaGetSymbolAddress, with that device current):
+ * make that first call outside any stream capture.  No call here uses
+ * cudaMalloc, cudaFree or any other allocating routine.
+ * On failure a message is written to errbuf (if non-NULL, errbuf_len bytes).
+ */
+#define GCADA_NOALLOC_MAX_GROUPS 1024
+gcada_status gcada_innovation_norms_noalloc(const float *fresh_dev, const float *stale_dev, int G,
+                                            long long p, long long ld, double *lhs_dev,
+                                            void *cuda_stream, char *errbuf, size_t errbuf_len);
 
 /* Text of the last error of this context ("" if none); valid until the next
  * call on the context.  ctx == NULL returns the text of the last failed

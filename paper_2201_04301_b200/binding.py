@@ -56,6 +56,7 @@ SIGNATURES = {
     "gcada_get_debug": (C.c_int, [_VP, C.c_int, _VP, _LL]),
     "gcada_get_launch_count": (C.c_int, [_VP, _ULLP]),
     "gcada_get_kernel_times": (C.c_int, [_VP, C.POINTER(C.c_double), C.POINTER(C.c_int)]),
+    "gcada_innovation_norms_noalloc": (C.c_int, [_VP, _VP, C.c_int, _LL, _LL, _VP, _VP, C.c_char_p, C.c_size_t]),
     "gcada_last_error": (C.c_char_p, [_VP]),
     "gcada_destroy": (None, [_VP]),
 }
@@ -216,6 +217,27 @@ class GCada:
         out = np.empty(shape, dtype=dt)
         self._ck(self.lib.gcada_get_debug(self.h, int(what), _VP(out.ctypes.data), out.nbytes))
         return out
+
+
+NOALLOC_MAX_GROUPS = 1024
+
+
+def innovation_norms_noalloc(fresh, stale, lhs_out, stream=None):
+    """lhs_out[g] = ||fresh[g] - stale[g]||^2 through gcada_innovation_norms_noalloc.
+
+    fresh, stale: CUDA float32 tensors [G, p] with the same row stride; lhs_out:
+    CUDA float64 tensor [G].  All of them are the caller's; the call itself
+    allocates nothing on the device (its scratch is a fixed array inside the
+    library, shared by every call: do not overlap calls on one GPU)."""
+    lib = load()
+    G, p = fresh.shape
+    assert stale.shape == fresh.shape and fresh.stride(0) == stale.stride(0) and fresh.stride(1) == 1
+    buf = C.create_string_buffer(256)
+    raw = getattr(stream, "cuda_stream", stream)
+    st = lib.gcada_innovation_norms_noalloc(_VP(fresh.data_ptr()), _VP(stale.data_ptr()), int(G), int(p),
+                                            int(fresh.stride(0)), _VP(lhs_out.data_ptr()), _VP(raw or 0), buf, 256)
+    if st != OK:
+        raise GCadaError(st, buf.value.decode())
 
 
 def from_workload(w, stream=None, options=None):
