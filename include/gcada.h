@@ -79,6 +79,10 @@ typedef struct {
 #define GCADA_OPT_TIMING 5     /* 1 = bracket each kernel phase with CUDA events (plain launches; see
                                   gcada_get_kernel_times); may be switched at any time (default 0) */
 
+#define GCADA_OPT_LINEAR_VARIANT 6 /* tuning knob of the d > 256 gradient kernel: 0 = default, 1 = one CTA per
+                                      SM with 4-row batches, 2 = two CTAs per SM with 2-row batches; results
+                                      differ only in summation order */
+
 /* Items for gcada_get_debug.  Sizes are in elements of the stated type. */
 #define GCADA_DBG_FRESH 0   /* float [G][p]: gradient of each group at theta^k, last iteration run */
 #define GCADA_DBG_STALE 1   /* float [G][p]: gradient at the stale iterate (needs GCADA_OPT_KEEP_STALE) */

@@ -36,7 +36,7 @@ struct gcada_ctx {
   double c = 0, alpha = 0, beta1 = 0, beta2 = 0, eps = 0;
   unsigned long long seed = 0;
   double shift = 1.0, rate = 1.0;
-  int rule = 0, reduction = 0, keep_stale = 0, use_graph = 1;
+  int rule = 0, reduction = 0, keep_stale = 0, use_graph = 1, linear_variant = 0;
   long long hist_cap = 65536;
   // data
   const void* X = nullptr;
@@ -219,7 +219,8 @@ gcada_status make_plans(gcada_ctx* ctx) {
     // the plan must also hold for the staging buffer of host-fed steps
     const void* xa = ctx->have_data ? ctx->X : nullptr;
     const long long ld = ctx->have_data ? ctx->ld : ((ctx->dims[0] + 3) / 4) * 4;
-    if (!plan_linear(ctx->dims[0], ld, xa, ctx->G, ctx->B, ctx->sm_count, ctx->smem_optin, &ctx->lin, &why))
+    if (!plan_linear(ctx->dims[0], ld, xa, ctx->G, ctx->B, ctx->sm_count, ctx->smem_optin, ctx->linear_variant,
+                     &ctx->lin, &why))
       return fail(ctx, GCADA_EINVAL, "%s", why);
     CK(prepare_grad_linear(ctx->lin, ctx->kind == GCADA_MODEL_QUADRATIC));
     P.pm.n_cta = ctx->lin.n_cta;
@@ -476,6 +477,10 @@ gcada_status gcada_set_option(gcada_ctx* ctx, int key, double value) {
     case GCADA_OPT_HISTORY:
       if (!(value >= 1) || value > 1e9) return fail(ctx, GCADA_EINVAL, "history must be in [1, 1e9]");
       ctx->hist_cap = (long long)value;
+      break;
+    case GCADA_OPT_LINEAR_VARIANT:
+      if (value != 0 && value != 1 && value != 2) return fail(ctx, GCADA_EINVAL, "variant must be 0, 1 or 2");
+      ctx->linear_variant = (int)value;
       break;
     case GCADA_OPT_KEEP_STALE:
       ctx->keep_stale = value != 0;

@@ -81,24 +81,25 @@ __device__ __forceinline__ void coefficients(float z, float dz, float y, float& 
 // ---------------------------------------------------------------------------
 // Large-d kernel (256 < d <= THREADS*CPT*4).  Thread t owns the 16-byte
 // column chunks t + THREADS*i, i < CPT, of every row: theta, the stale iterate
-// (as theta^k minus it) and both accumulators stay in registers; rows arrive in a shared-memory
-// ring through bulk asynchronous copies (one per 4*d-byte row) issued ahead
-// by thread 0, so each row crosses HBM -> SM exactly once.
+// (as theta^k minus it) and both accumulators stay in registers; rows arrive
+// in a shared-memory ring through bulk asynchronous copies (one per 4*d-byte
+// row) issued ahead by thread 0, so each row crosses HBM -> SM exactly once.
+// FULL = the row is exactly THREADS*CPT chunks (no column predicates).
 // ---------------------------------------------------------------------------
 constexpr int LG_CHUNK_ROWS = 256;  // rows whose indices / labels are staged at once
 
-template <int THREADS, int CPT, int R, bool QUAD>
-__global__ void __launch_bounds__(THREADS, 1) grad_linear_large_kernel(const Params P, int nslot) {
+template <int THREADS, int CPT, int R, int MINB, bool QUAD, bool FULL>
+__global__ void __launch_bounds__(THREADS, MINB) grad_linear_large_kernel(const Params P, int nslot) {
   constexpr int V = 2 * R;
   constexpr int NW = THREADS / 32;
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int d = P.d;
-  const int nchunks = (d + 3) >> 2;
+  const int nchunks = FULL ? THREADS * CPT : (d + 3) >> 2;
   const uint32_t rowbytes = (uint32_t)nchunks * 16u;
 
   // shared memory carve-up
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_raw);                       // nslot
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_raw);                       // nslot (<= 32)
   long long* row_sm = reinterpret_cast<long long*>(smem_raw + 8 * 32);          // LG_CHUNK_ROWS
   float* y_sm = reinterpret_cast<float*>(row_sm + LG_CHUNK_ROWS);               // LG_CHUNK_ROWS
   float* part = y_sm + LG_CHUNK_ROWS;                                           // V * THREADS
@@ -112,11 +113,15 @@ __global__ void __launch_bounds__(THREADS, 1) grad_linear_large_kernel(const Par
   const float* theta_k = P.theta_ring + (k % ring) * P.p_pad;
   const float* Xf = reinterpret_cast<const float*>(P.X);
   const float* yf = reinterpret_cast<const float*>(P.y);
+  const int B = P.B;
 
-  const long long Rtot = (long long)P.G * P.B;
+  const long long Rtot = (long long)P.G * B;
   const long long r0 = (long long)blockIdx.x * Rtot / gridDim.x;
   const long long r1 = (long long)(blockIdx.x + 1) * Rtot / gridDim.x;
   if (r0 >= r1) return;
+  const int rows_cta = (int)(r1 - r0);
+  const int g_first = (int)(r0 / B);
+  const int in_g0 = (int)(r0 - (long long)g_first * B);  // position of the CTA's first row in its group
 
   if (tid == 0) {
     for (int s = 0; s < nslot; ++s) mbar_init(&bars[s], 1);
@@ -127,26 +132,30 @@ __global__ void __launch_bounds__(THREADS, 1) grad_linear_large_kernel(const Par
   bool own[CPT];
   float4 th[CPT], ths[CPT], acc0[CPT], acc1[CPT];
   const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+  const bool ragged = !FULL && (d & 3) != 0;
 #pragma unroll
   for (int i = 0; i < CPT; ++i) {
     const int q = tid + THREADS * i;
-    own[i] = q < nchunks;
+    own[i] = FULL || q < nchunks;
     th[i] = zero4;
     if (own[i]) {
       const int c0 = q * 4;
-      th[i].x = theta_k[c0];
-      th[i].y = c0 + 1 < d ? theta_k[c0 + 1] : 0.f;
-      th[i].z = c0 + 2 < d ? theta_k[c0 + 2] : 0.f;
-      th[i].w = c0 + 3 < d ? theta_k[c0 + 3] : 0.f;
+      if (FULL) {
+        th[i] = *reinterpret_cast<const float4*>(theta_k + c0);
+      } else {
+        th[i].x = theta_k[c0];
+        th[i].y = c0 + 1 < d ? theta_k[c0 + 1] : 0.f;
+        th[i].z = c0 + 2 < d ? theta_k[c0 + 2] : 0.f;
+        th[i].w = c0 + 3 < d ? theta_k[c0 + 3] : 0.f;
+      }
     }
     ths[i] = zero4;
     acc0[i] = zero4;
     acc1[i] = zero4;
   }
-  const bool ragged = (d & 3) != 0;
 
-  const int g_first = (int)(r0 / P.B);
   int cur_g = -1;
+  int g_end = 0;          // CTA-local row at which the current group ends
   int cslot = 0;          // ring slot of the next row to consume
   uint32_t cphase = 0;    // barrier parity of that slot's current fill
   int failed = 0;
@@ -171,14 +180,14 @@ __global__ void __launch_bounds__(THREADS, 1) grad_linear_large_kernel(const Par
     }
   };
 
-  for (long long cs = r0; cs < r1 && !failed; cs += LG_CHUNK_ROWS) {
-    const int nrows = (int)((r1 - cs) < LG_CHUNK_ROWS ? (r1 - cs) : LG_CHUNK_ROWS);
+  for (int cs = 0; cs < rows_cta && !failed; cs += LG_CHUNK_ROWS) {
+    const int nrows = rows_cta - cs < LG_CHUNK_ROWS ? rows_cta - cs : LG_CHUNK_ROWS;
     __syncthreads();  // previous chunk fully consumed; barriers initialised (first pass)
     for (int i = tid; i < nrows; i += THREADS) {
-      const long long gr = cs + i;
-      const int g = (int)(gr / P.B);
-      const long long row = batch_row(P, k32, g, (int)(gr - (long long)g * P.B));
-      row_sm[i] = row;
+      const int pos = in_g0 + cs + i;
+      const int gi = pos / B;
+      const long long row = batch_row(P, k32, g_first + gi, pos - gi * B);
+      row_sm[i] = row * P.ld;
       y_sm[i] = yf[row];
     }
     __syncthreads();
@@ -189,17 +198,17 @@ __global__ void __launch_bounds__(THREADS, 1) grad_linear_large_kernel(const Par
         int s = cslot + issued;
         if (s >= nslot) s -= nslot;
         mbar_expect_tx(&bars[s], rowbytes);
-        bulk_load(slots + (size_t)s * rowbytes, Xf + row_sm[issued] * P.ld, rowbytes, &bars[s]);
+        bulk_load(slots + (size_t)s * rowbytes, Xf + row_sm[issued], rowbytes, &bars[s]);
       }
     }
     int consumed = 0;
     while (consumed < nrows) {
-      const long long gr = cs + consumed;
-      const int g = (int)(gr / P.B);
-      if (g != cur_g) {
+      const int lr = cs + consumed;
+      if (lr == g_end) {  // first row of a group (g_end starts at 0)
         if (cur_g >= 0) flush(cur_g);
-        cur_g = g;
-        long long js = k - P.tau[g];
+        cur_g = cur_g < 0 ? g_first : cur_g + 1;
+        g_end = (cur_g + 1 - g_first) * B - in_g0;
+        long long js = k - P.tau[cur_g];
         if (js < 0) js = 0;
         const float* theta_s = P.theta_ring + (js % ring) * P.p_pad;
 #pragma unroll
@@ -208,17 +217,22 @@ __global__ void __launch_bounds__(THREADS, 1) grad_linear_large_kernel(const Par
           acc1[i] = zero4;
           if (own[i]) {
             const int c0 = (tid + THREADS * i) * 4;
-            ths[i].x = th[i].x - theta_s[c0];
-            ths[i].y = c0 + 1 < d ? th[i].y - theta_s[c0 + 1] : 0.f;
-            ths[i].z = c0 + 2 < d ? th[i].z - theta_s[c0 + 2] : 0.f;
-            ths[i].w = c0 + 3 < d ? th[i].w - theta_s[c0 + 3] : 0.f;
+            if (FULL) {
+              const float4 t = *reinterpret_cast<const float4*>(theta_s + c0);
+              ths[i] = make_float4(th[i].x - t.x, th[i].y - t.y, th[i].z - t.z, th[i].w - t.w);
+            } else {
+              ths[i].x = th[i].x - theta_s[c0];
+              ths[i].y = c0 + 1 < d ? th[i].y - theta_s[c0 + 1] : 0.f;
+              ths[i].z = c0 + 2 < d ? th[i].z - theta_s[c0 + 2] : 0.f;
+              ths[i].w = c0 + 3 < d ? th[i].w - theta_s[c0 + 3] : 0.f;
+            }
           }
         }
       }
-      const long long seg_end = ((long long)(g + 1) * P.B < cs + nrows ? (long long)(g + 1) * P.B : cs + nrows) - cs;
-      const int nb = (int)(seg_end - consumed) < R ? (int)(seg_end - consumed) : R;
+      int lim = (g_end < cs + nrows ? g_end : cs + nrows) - lr;
+      const int nb = lim < R ? lim : R;
 
-      // pass 1: rows -> registers, partial dot products at both points
+      // pass 1: rows -> registers, partial dot products z = x.theta and dz = x.(theta - theta_stale)
       float4 x[R][CPT];
       float pz[V];
 #pragma unroll
@@ -236,12 +250,16 @@ __global__ void __launch_bounds__(THREADS, 1) grad_linear_large_kernel(const Par
           const float4* src = reinterpret_cast<const float4*>(slots + (size_t)s * rowbytes);
 #pragma unroll
           for (int i = 0; i < CPT; ++i) {
-            x[r][i] = own[i] ? src[tid + THREADS * i] : zero4;
-            if (ragged && own[i]) {
-              const int c0 = (tid + THREADS * i) * 4;
-              if (c0 + 1 >= d) x[r][i].y = 0.f;
-              if (c0 + 2 >= d) x[r][i].z = 0.f;
-              if (c0 + 3 >= d) x[r][i].w = 0.f;
+            if (FULL) {
+              x[r][i] = src[tid + THREADS * i];
+            } else {
+              x[r][i] = own[i] ? src[tid + THREADS * i] : zero4;
+              if (ragged && own[i]) {
+                const int c0 = (tid + THREADS * i) * 4;
+                if (c0 + 1 >= d) x[r][i].y = 0.f;
+                if (c0 + 2 >= d) x[r][i].z = 0.f;
+                if (c0 + 3 >= d) x[r][i].w = 0.f;
+              }
             }
             pz[r] += x[r][i].x * th[i].x + x[r][i].y * th[i].y + x[r][i].z * th[i].z + x[r][i].w * th[i].w;
             pz[R + r] += x[r][i].x * ths[i].x + x[r][i].y * ths[i].y + x[r][i].z * ths[i].z + x[r][i].w * ths[i].w;
@@ -260,7 +278,7 @@ __global__ void __launch_bounds__(THREADS, 1) grad_linear_large_kernel(const Par
           int s = cslot + r;  // slot of a row consumed just now
           if (s >= nslot) s -= nslot;
           mbar_expect_tx(&bars[s], rowbytes);
-          bulk_load(slots + (size_t)s * rowbytes, Xf + row_sm[issued] * P.ld, rowbytes, &bars[s]);
+          bulk_load(slots + (size_t)s * rowbytes, Xf + row_sm[issued], rowbytes, &bars[s]);
         }
       }
       // stage 2: warp r finishes both dot products of row r and turns them
@@ -283,9 +301,23 @@ __global__ void __launch_bounds__(THREADS, 1) grad_linear_large_kernel(const Par
       }
       __syncthreads();  // (B)
       // pass 2: rank-one accumulation
+      float cf[V];
+      if (V % 4 == 0) {
+#pragma unroll
+        for (int v = 0; v < V; v += 4) {
+          const float4 t = *reinterpret_cast<const float4*>(res + v);
+          cf[v] = t.x;
+          cf[v + 1] = t.y;
+          cf[v + 2] = t.z;
+          cf[v + 3] = t.w;
+        }
+      } else {
+#pragma unroll
+        for (int v = 0; v < V; ++v) cf[v] = res[v];
+      }
 #pragma unroll
       for (int r = 0; r < R; ++r) {
-        const float a = res[r], b = res[R + r];
+        const float a = cf[r], b = cf[R + r];
 #pragma unroll
         for (int i = 0; i < CPT; ++i) {
           acc0[i].x += a * x[r][i].x;
@@ -440,15 +472,19 @@ static size_t large_smem_fixed(int threads, int R) {
   return 8 * 32 + LG_CHUNK_ROWS * (sizeof(long long) + sizeof(float)) + (size_t)2 * R * threads * 4 + 32 * 4 + 128;
 }
 
-template <int THREADS, int CPT, int R>
+template <int CPT, int R, int MINB>
 static cudaError_t launch_large(const Params& P, const LinearPlan& plan, bool quad, cudaStream_t st,
                                 bool attr_only) {
-  auto kq = grad_linear_large_kernel<THREADS, CPT, R, true>;
-  auto kl = grad_linear_large_kernel<THREADS, CPT, R, false>;
-  auto kern = quad ? kq : kl;
+  void (*kern)(const Params, int);
+  if (plan.full)
+    kern = quad ? grad_linear_large_kernel<256, CPT, R, MINB, true, true>
+                : grad_linear_large_kernel<256, CPT, R, MINB, false, true>;
+  else
+    kern = quad ? grad_linear_large_kernel<256, CPT, R, MINB, true, false>
+                : grad_linear_large_kernel<256, CPT, R, MINB, false, false>;
   if (attr_only)
     return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
-  kern<<<plan.n_cta, THREADS, plan.smem_bytes, st>>>(P, plan.nslot);
+  kern<<<plan.n_cta, 256, plan.smem_bytes, st>>>(P, plan.nslot);
   return cudaGetLastError();
 }
 
@@ -461,7 +497,7 @@ static cudaError_t launch_small(const Params& P, const LinearPlan& plan, bool qu
   return cudaGetLastError();
 }
 
-bool plan_linear(int d, long long ld, const void* X, int G, int B, int sm_count, size_t smem_optin,
+bool plan_linear(int d, long long ld, const void* X, int G, int B, int sm_count, size_t smem_optin, int variant,
                  LinearPlan* plan, const char** why) {
   const long long Rtot = (long long)G * B;
   plan->small = d <= 256;
@@ -484,10 +520,14 @@ bool plan_linear(int d, long long ld, const void* X, int G, int B, int sm_count,
     const int nchunks = (d + 3) / 4;
     plan->cpt = nchunks <= 256 ? 1 : (nchunks <= 512 ? 2 : 4);
     plan->threads = 256;
-    plan->R = 4;
+    plan->full = (d & 3) == 0 && nchunks == 256 * plan->cpt;
+    // variant 1: one CTA per SM, 4 rows per batch; variant 2: two CTAs per SM, 2 rows per batch
+    plan->ctas_per_sm = variant == 1 ? 1 : 2;
+    plan->R = plan->ctas_per_sm == 1 ? 4 : 2;
     const size_t rowbytes = (size_t)nchunks * 16;
     const size_t fixed = large_smem_fixed(plan->threads, plan->R);
-    long long nslot = ((long long)smem_optin - (long long)fixed) / (long long)rowbytes;
+    const long long budget = plan->ctas_per_sm == 1 ? (long long)smem_optin : ((long long)smem_optin + 1024) / 2 - 1024;
+    long long nslot = (budget - (long long)fixed) / (long long)rowbytes;
     if (nslot > 32) nslot = 32;
     if (nslot < 2 * plan->R) {
       *why = "not enough shared memory for the row ring";
@@ -495,7 +535,8 @@ bool plan_linear(int d, long long ld, const void* X, int G, int B, int sm_count,
     }
     plan->nslot = (int)nslot;
     plan->smem_bytes = fixed + (size_t)nslot * rowbytes;
-    plan->n_cta = (int)(Rtot < sm_count ? Rtot : sm_count);
+    const long long want = (long long)sm_count * plan->ctas_per_sm;
+    plan->n_cta = (int)(Rtot < want ? Rtot : want);
   }
   const long long per = (Rtot + plan->n_cta - 1) / plan->n_cta;
   plan->maxseg = (int)((per + B - 2) / B + 1);
@@ -504,10 +545,17 @@ bool plan_linear(int d, long long ld, const void* X, int G, int B, int sm_count,
 
 static cudaError_t dispatch_large(const Params& P, const LinearPlan& plan, bool quad, cudaStream_t st,
                                   bool attr_only) {
+  if (plan.ctas_per_sm == 1) {
+    switch (plan.cpt) {
+      case 1: return launch_large<1, 4, 1>(P, plan, quad, st, attr_only);
+      case 2: return launch_large<2, 4, 1>(P, plan, quad, st, attr_only);
+      default: return launch_large<4, 4, 1>(P, plan, quad, st, attr_only);
+    }
+  }
   switch (plan.cpt) {
-    case 1: return launch_large<256, 1, 4>(P, plan, quad, st, attr_only);
-    case 2: return launch_large<256, 2, 4>(P, plan, quad, st, attr_only);
-    default: return launch_large<256, 4, 4>(P, plan, quad, st, attr_only);
+    case 1: return launch_large<1, 2, 2>(P, plan, quad, st, attr_only);
+    case 2: return launch_large<2, 2, 2>(P, plan, quad, st, attr_only);
+    default: return launch_large<4, 2, 2>(P, plan, quad, st, attr_only);
   }
 }
 

@@ -12,13 +12,16 @@ struct LinearPlan {
   bool small;       // d <= 256: warp-per-row kernel, else the row-ring kernel
   int cpl;          // small: columns per lane
   int cpt, threads, R, nslot;  // large: 16-byte chunks per thread, CTA size, rows per batch, ring slots
+  int ctas_per_sm;  // large: resident CTAs per SM the shape is sized for
+  bool full;        // large: a row is exactly threads*cpt 16-byte chunks
   size_t smem_bytes;
   int n_cta;
   int maxseg;       // partial slots per CTA
 };
 
 // Chooses the kernel and its shape; false (with *why) if the shape is not supported.
-bool plan_linear(int d, long long ld, const void* X, int G, int B, int sm_count, size_t smem_optin,
+// `variant`: 0 = default shape, 1 = one CTA per SM with 4-row batches, 2 = two CTAs per SM with 2-row batches.
+bool plan_linear(int d, long long ld, const void* X, int G, int B, int sm_count, size_t smem_optin, int variant,
                  LinearPlan* plan, const char** why);
 // One-time function attributes (dynamic shared memory size); call before the first launch.
 cudaError_t prepare_grad_linear(const LinearPlan& plan, bool quad);
