@@ -26,6 +26,8 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
   __shared__ double scratch[40];
   __shared__ int sh_nsel[8];
   __shared__ double sh_tmax[8];
+  __shared__ double tw_sm[1024];
+  __shared__ double lhs_sm[256];
   __shared__ bool is_last;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = blockIdx.y;
@@ -51,12 +53,25 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
     if (n > 0) {
       f = make_float4(0.f, 0.f, 0.f, 0.f);
       s = f;
-      for (int c = c_lo; c <= c_hi; ++c) {
-        const int gf = (int)(((long long)c * Rtot / n) / P.pm.rows_per_group);
-        const float* src = P.partial + ((long long)(c * P.pm.maxseg + (g - gf)) * 2) * P.p_pad + i4 * 4;
-        const float4 a = ld4(src), b = ld4(src + P.p_pad);
-        f.x += a.x; f.y += a.y; f.z += a.z; f.w += a.w;
-        s.x += b.x; s.y += b.y; s.z += b.z; s.w += b.w;
+      for (int c0 = c_lo; c0 <= c_hi; c0 += 4) {  // four partial sums per round: loads first, adds in CTA order
+        float4 a[4], b[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int c = c0 + u;
+          if (c <= c_hi) {
+            const int gf = (int)(((long long)c * Rtot / n) / P.pm.rows_per_group);
+            const float* src = P.partial + ((long long)(c * P.pm.maxseg + (g - gf)) * 2) * P.p_pad + i4 * 4;
+            a[u] = ld4(src);
+            b[u] = ld4(src + P.p_pad);
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          if (c0 + u <= c_hi) {
+            f.x += a[u].x; f.y += a[u].y; f.z += a[u].z; f.w += a[u].w;
+            s.x += b[u].x; s.y += b[u].y; s.z += b[u].z; s.w += b[u].w;
+          }
+        }
       }
       // second slot half = innovation; the stale-point gradient is fresh - innovation
       st4(P.fresh + (long long)g * P.p_pad + i4 * 4, f);
@@ -81,30 +96,56 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
   if (!is_last) return;
   __threadfence();
 
-  // ---- phase 2 (last block only): the server's scheduling decision
+  // ---- phase 2 (last block only): the server's scheduling decision.
+  // One thread per group, 256 groups at a time; everything a group needs is
+  // fetched in one round of independent loads.
   double rhs = 0.0;
   for (int i = 0; i < P.D; ++i) rhs += P.s_ring[i];
   rhs *= P.c;
+  const uint32_t k32 = (uint32_t)k;
   const volatile double* parts = P.lhs_part;
   int nsel = 0;
   double tmax = 0.0;
-  const uint32_t k32 = (uint32_t)k;
-  for (int gg = warp; gg < P.G; gg += 8) {
-    double s = 0.0;
-    for (int b = lane; b < blocks_x; b += 32) s += parts[(long long)gg * blocks_x + b];
-    s = warp_sum(s);
+  for (int gc = 0; gc < P.G; gc += 256) {
+    const int gg = gc + tid;
+    const bool have = gg < P.G;
+    const int ng = P.G - gc < 256 ? P.G - gc : 256;
+    // loads first: age, forced bit, partial sums of the innovation norm
+    const int tau = have ? P.tau[gg] : 0;
+    bool sel_forced = false;
+    if (have && P.forced) sel_forced = P.forced[(k - P.forced_base) * P.G + gg] != 0;
+    double lhs = 0.0;
+    if (blocks_x <= 64) {
+      if (have)
+        for (int b = 0; b < blocks_x; ++b) lhs += parts[(long long)gg * blocks_x + b];
+    } else {
+      for (int lg = warp; lg < ng; lg += 8) {
+        double v = 0.0;
+        for (int b = lane; b < blocks_x; b += 32) v += parts[(long long)(gc + lg) * blocks_x + b];
+        v = warp_sum(v);
+        if (lane == 0) lhs_sm[lg] = v;
+      }
+      __syncthreads();
+      if (have) lhs = lhs_sm[tid];
+    }
+    // computing times: one thread per worker into shared memory (tiles of 1024
+    // workers), then each group's thread takes the minimum over its workers
     double t = 1.0e300;
-    for (int j = lane; j < P.M_G; j += 32) t = fmin(t, worker_time(P, k32, gg * P.M_G + j));
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) t = fmin(t, __shfl_xor_sync(0xffffffffu, t, o));
-    if (lane == 0) {
-      const int tau = P.tau[gg];
-      bool sel;
-      if (P.forced)
-        sel = P.forced[(k - P.forced_base) * P.G + gg] != 0;
-      else
-        sel = (tau >= P.D) || (s > rhs);
-      P.lhs[gg] = s;
+    const long long w_lo = (long long)gc * P.M_G, w_hi = (long long)(gc + ng) * P.M_G;
+    for (long long m0 = w_lo; m0 < w_hi; m0 += 1024) {
+      const int cnt = (int)(w_hi - m0 < 1024 ? w_hi - m0 : 1024);
+      __syncthreads();
+      for (int i = tid; i < cnt; i += 256) tw_sm[i] = worker_time(P, k32, (int)(m0 + i));
+      __syncthreads();
+      if (have) {
+        const long long lo = (long long)gg * P.M_G > m0 ? (long long)gg * P.M_G : m0;
+        const long long hi = (long long)(gg + 1) * P.M_G < m0 + cnt ? (long long)(gg + 1) * P.M_G : m0 + cnt;
+        for (long long m = lo; m < hi; ++m) t = fmin(t, tw_sm[m - m0]);
+      }
+    }
+    if (have) {
+      const bool sel = P.forced ? sel_forced : ((tau >= P.D) || (lhs > rhs));
+      P.lhs[gg] = lhs;
       P.t_g[gg] = t;
       P.mask_cur[gg] = sel ? 1 : 0;
       P.hist[(k % P.hist_cap) * P.G + gg] = sel ? 1 : 0;
@@ -114,6 +155,12 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
         tmax = fmax(tmax, t);
       }
     }
+  }
+  // block-wide count and maximum
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    nsel += __shfl_xor_sync(0xffffffffu, nsel, o);
+    tmax = fmax(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
   }
   if (lane == 0) {
     sh_nsel[warp] = nsel;
@@ -158,10 +205,14 @@ __device__ __forceinline__ void renorm(float& hi, float& lo) {
   hi = t;
 }
 
+// Block = 32 float4 columns (lanes) x 8 warps.  Warp w folds the selected
+// groups number w, w+8, ... of the (ascending) list into its own compensated
+// partial sum; the eight partial sums are then added to the aggregate in warp
+// order, so the result does not depend on timing.
 __global__ void __launch_bounds__(256) update_kernel(const Params P) {
   extern __shared__ int sel_list[];  // selected groups, ascending
   __shared__ int n_sel_sh;
-  __shared__ double scratch[40];
+  __shared__ float4 wsum_hi[8][32], wsum_lo[8][32];
   __shared__ bool is_last;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const long long cols4 = P.p_pad >> 2;
@@ -182,33 +233,67 @@ __global__ void __launch_bounds__(256) update_kernel(const Params P) {
   __syncthreads();
   const int n_sel = n_sel_sh;
 
-  const long long i4 = (long long)blockIdx.x * 256 + tid;
-  double local = 0.0;
-  if (i4 < cols4) {
-    const long long o = i4 * 4;
-    float4 hi = ld4(P.agg_hi + o), lo = ld4(P.agg_lo + o);
-    for (int j = 0; j < n_sel; ++j) {
-      const long long go = (long long)sel_list[j] * P.p_pad + o;
-      const float4 f = ld4(P.fresh + go), l = ld4(P.g_last + go);
-      st4(P.g_last + go, f);
-      fold(hi.x, lo.x, f.x, l.x);
-      fold(hi.y, lo.y, f.y, l.y);
-      fold(hi.z, lo.z, f.z, l.z);
-      fold(hi.w, lo.w, f.w, l.w);
+  const long long i4 = (long long)blockIdx.x * 32 + lane;
+  const bool active = i4 < cols4;
+  const long long o = i4 * 4;
+  float4 hi = make_float4(0.f, 0.f, 0.f, 0.f), lo = hi;
+  if (active) {
+    for (int j0 = warp; j0 < n_sel; j0 += 32) {  // four groups of this warp per round, loads first
+      float4 f[4], l[4];
+      long long go[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int j = j0 + 8 * u;
+        if (j < n_sel) {
+          go[u] = (long long)sel_list[j] * P.p_pad + o;
+          f[u] = ld4(P.fresh + go[u]);
+          l[u] = ld4(P.g_last + go[u]);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (j0 + 8 * u < n_sel) {
+          st4(P.g_last + go[u], f[u]);
+          fold(hi.x, lo.x, f[u].x, l[u].x);
+          fold(hi.y, lo.y, f[u].y, l[u].y);
+          fold(hi.z, lo.z, f[u].z, l[u].z);
+          fold(hi.w, lo.w, f[u].w, l[u].w);
+        }
+      }
     }
-    renorm(hi.x, lo.x);
-    renorm(hi.y, lo.y);
-    renorm(hi.z, lo.z);
-    renorm(hi.w, lo.w);
-    st4(P.agg_hi + o, hi);
-    st4(P.agg_lo + o, lo);
-    // Eq. (8a)-(8c)
-    float4 h = ld4(P.h + o), vh = ld4(P.vhat + o);
-    const float4 th = ld4(P.theta_ring + (k % ring) * P.p_pad + o);
-    float4 tn;
+  }
+  wsum_hi[warp][lane] = hi;
+  wsum_lo[warp][lane] = lo;
+  __syncthreads();
+  if (warp == 0) {
+    double local = 0.0;
+    if (active) {
+      float4 ahi = ld4(P.agg_hi + o), alo = ld4(P.agg_lo + o);
+#pragma unroll
+      for (int w = 0; w < 8; ++w) {
+        const float4 h2 = wsum_hi[w][lane], l2 = wsum_lo[w][lane];
+        fold(ahi.x, alo.x, h2.x, 0.f);
+        fold(ahi.y, alo.y, h2.y, 0.f);
+        fold(ahi.z, alo.z, h2.z, 0.f);
+        fold(ahi.w, alo.w, h2.w, 0.f);
+        alo.x += l2.x;
+        alo.y += l2.y;
+        alo.z += l2.z;
+        alo.w += l2.w;
+      }
+      renorm(ahi.x, alo.x);
+      renorm(ahi.y, alo.y);
+      renorm(ahi.z, alo.z);
+      renorm(ahi.w, alo.w);
+      st4(P.agg_hi + o, ahi);
+      st4(P.agg_lo + o, alo);
+      // Eq. (8a)-(8c)
+      float4 h = ld4(P.h + o), vh = ld4(P.vhat + o);
+      const float4 th = ld4(P.theta_ring + (k % ring) * P.p_pad + o);
+      float4 tn;
 #define GCADA_AMSGRAD(c)                                   \
   {                                                        \
-    const float gr = hi.c;                                 \
+    const float gr = ahi.c;                                \
     h.c = P.beta1 * h.c + P.omb1 * gr;                     \
     const float v = P.beta2 * vh.c + P.omb2 * (gr * gr);   \
     vh.c = fmaxf(vh.c, v);                                 \
@@ -216,20 +301,21 @@ __global__ void __launch_bounds__(256) update_kernel(const Params P) {
     tn.c = th.c - up;                                      \
     local += (double)up * (double)up;                      \
   }
-    GCADA_AMSGRAD(x)
-    GCADA_AMSGRAD(y)
-    GCADA_AMSGRAD(z)
-    GCADA_AMSGRAD(w)
+      GCADA_AMSGRAD(x)
+      GCADA_AMSGRAD(y)
+      GCADA_AMSGRAD(z)
+      GCADA_AMSGRAD(w)
 #undef GCADA_AMSGRAD
-    st4(P.h + o, h);
-    st4(P.vhat + o, vh);
-    st4(P.theta_ring + ((k + 1) % ring) * P.p_pad + o, tn);
-  }
-  const double tot = block_sum(local, scratch);
-  if (tid == 0) {
-    P.upd_part[blockIdx.x] = tot;
-    __threadfence();
-    is_last = atomicAdd(&P.st->ticket_update, 1u) == gridDim.x - 1u;
+      st4(P.h + o, h);
+      st4(P.vhat + o, vh);
+      st4(P.theta_ring + ((k + 1) % ring) * P.p_pad + o, tn);
+    }
+    local = warp_sum(local);
+    if (lane == 0) {
+      P.upd_part[blockIdx.x] = local;
+      __threadfence();
+      is_last = atomicAdd(&P.st->ticket_update, 1u) == gridDim.x - 1u;
+    }
   }
   __syncthreads();
   if (!is_last) return;
@@ -237,7 +323,7 @@ __global__ void __launch_bounds__(256) update_kernel(const Params P) {
   const volatile double* parts = P.upd_part;
   double s = 0.0;
   for (unsigned int b = tid; b < gridDim.x; b += 256) s += parts[b];
-  s = block_sum(s, scratch);
+  s = block_sum(s, reinterpret_cast<double*>(&wsum_hi[0][0]));
   if (tid == 0) {
     P.s_ring[k % P.D] = s;
     P.st->k = k + 1;
@@ -252,7 +338,7 @@ void plan_tail(long long p_pad, int G, int sm_count, TailPlan* plan) {
   const int U = cols4 > 256 * 1024 ? 4 : 1;
   plan->select_cols4_per_block = 256 * U;
   plan->select_blocks_x = (int)((cols4 + 256 * U - 1) / (256 * U));
-  plan->update_blocks = (int)((cols4 + 255) / 256);
+  plan->update_blocks = (int)((cols4 + 31) / 32);
 }
 
 cudaError_t launch_select(const Params& P, const TailPlan& plan, cudaStream_t st) {
