@@ -237,7 +237,19 @@ def run_ours(args):
     }
     if e2e:
         out["e2e"] = e2e
-    if w["kind"] != "mlp" or w["compute"] == "fp32":
+    if w["kind"] == "mlp" and w["compute"] == "fp32":
+        # plain fp32 FFMA tiles (a 1e-5 tolerance rules out single-pass tensor-core arithmetic):
+        # peak = SMs x 128 FMA lanes x 2 flop x max SM clock
+        flops = mlp_flops_per_iteration(w)
+        import torch
+        sms = torch.cuda.get_device_properties(0).multi_processor_count
+        peak = sms * 128 * 2 * (sampler.max_mhz or 1965) * 1e6 / 1e12
+        achieved = flops / (ms_grad * 1e-3) / 1e12 if ms_grad > 0 else None
+        out["roofline"] = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                           "frac": achieved / peak if achieved else None, "traffic": None,
+                           "kernel": "gradient (all launches of one iteration; latency-bound at this size)",
+                           "peak_source": "derived: SMs x 128 lanes x 2 x max SM clock", "flops_per_iteration": flops}
+    elif w["kind"] != "mlp":
         bytes_launch = algorithmic_bytes_per_launch(w)
         achieved = bytes_launch / (ms_grad * 1e-3) / 1e9 if ms_grad > 0 else None
         traffic = None

@@ -125,7 +125,21 @@ class MLP:
         per = -logp[np.arange(len(yb)), np.asarray(yb, dtype=np.int64)]
         return _scale(reduction, len(yb)) * per.sum()
 
-    def grad(self, theta, Xb, yb, reduction="mean"):
+    def near_kinks(self, theta, Xb, tol):
+        """Hidden units (layer index, row, unit) whose pre-activation is within
+        `tol` of zero: there the ReLU derivative is a matter of rounding, and
+        either choice (0 or 1) is a valid subgradient."""
+        _, _, zs = self._forward(theta, Xb)
+        out = []
+        for l, z in enumerate(zs[:-1]):
+            r, u = np.nonzero(np.abs(z) <= tol)
+            out += [(l, int(a), int(b)) for a, b in zip(r, u)]
+        return out
+
+    def grad(self, theta, Xb, yb, reduction="mean", flip=()):
+        """Gradient of the minibatch loss.  `flip` lists hidden units
+        (layer index, row, unit) whose ReLU derivative is taken as the other
+        admissible value (see near_kinks); the forward pass is unaffected."""
         layers, acts, zs = self._forward(theta, Xb)
         s = zs[-1]
         s = s - s.max(axis=1, keepdims=True)
@@ -142,7 +156,11 @@ class MLP:
             pieces[l] = (dW, db)
             if l > 0:
                 da = dz @ W
-                dz = da * (zs[l - 1] > 0.0)
+                on = zs[l - 1] > 0.0
+                for (fl, fr, fu) in flip:
+                    if fl == l - 1:
+                        on[fr, fu] = ~on[fr, fu]
+                dz = da * on
         return np.concatenate([np.concatenate([dW.ravel(), db]) for dW, db in pieces])
 
 

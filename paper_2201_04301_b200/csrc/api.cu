@@ -328,6 +328,7 @@ gcada_status gcada_create(const gcada_model* model, int M, int M_G, int D, doubl
   if (!(c >= 0) || !(alpha > 0) || !(beta1 > 0 && beta1 < 1) || !(beta2 > 0 && beta2 < 1) || !(eps > 0))
     return fail(ctx, GCADA_EINVAL, "need c >= 0, alpha > 0, 0 < beta1, beta2 < 1, eps > 0");
   if (M / M_G > 65535) return fail(ctx, GCADA_EINVAL, "at most 65535 groups");
+  if (model->kind == GCADA_MODEL_MLP && M / M_G > 32767) return fail(ctx, GCADA_EINVAL, "at most 32767 groups for an MLP");
   long long p = 0;
   if (model->kind == GCADA_MODEL_LOGISTIC || model->kind == GCADA_MODEL_QUADRATIC) {
     if (model->n_dims != 1 || model->dims[0] < 1 || model->dims[0] > 4096)

@@ -1,8 +1,329 @@
-// placeholder
+// Dual-point minibatch gradients of the multilayer perceptron (ReLU hidden
+// layers, softmax cross-entropy) for all groups: the gradient step of
+// Algorithm 1 evaluated at theta^k (point 0) and at each group's stale
+// iterate theta^{k - tau_g} (point 1) on the same gathered samples.
+//
+// fp32 path (this file): plain FFMA tiles, because single-pass tensor-core
+// arithmetic (tf32 / bf16 operands) cannot hold a 1e-5 relative tolerance.
+// The bf16 path lives in mlp_bf16.cu.
+//
+// theta layout: for l = 1..L, W_l (n_l rows of n_{l-1}) then b_l (n_l).
+// Batch index z = q * G + g (q = point, g = group).
 #include "mlp.h"
+
+#include "mlp_bf16.h"
+
 namespace gcada {
-const char* mlp_supported(const std::vector<int>&, int) { return "the MLP path is not built yet"; }
-cudaError_t mlp_plan_create(const std::vector<int>&, int, int, int, int, long long, int, cudaStream_t, MlpPlan*,
-                            std::vector<void*>*, const char** why) { *why = "the MLP path is not built yet"; return cudaSuccess; }
-cudaError_t launch_grad_mlp(const Params&, const MlpPlan&, cudaStream_t, int* n) { *n = 0; return cudaErrorNotSupported; }
+
+namespace {
+
+__device__ __forceinline__ const float* ring_ptr(const Params& P, int g, int q, long long k) {
+  long long j = q == 0 ? k : k - P.tau[g];
+  if (j < 0) j = 0;
+  return P.theta_ring + (j % (P.D + 1)) * P.p_pad;
 }
+
+// ------------------------------------------------------------------ gather
+// Warp per sampled row: xb[r] = X[row(r)], yb[r] = y[row(r)].
+__global__ void __launch_bounds__(256) mlp_gather_kernel(const Params P, float* xb, int* yb, int d) {
+  const int warp = (int)((blockIdx.x * 256 + threadIdx.x) >> 5), lane = threadIdx.x & 31;
+  const long long rows = (long long)P.G * P.B;
+  if (warp >= rows) return;
+  const int g = warp / P.B, j = warp - g * P.B;
+  const long long row = batch_row(P, (uint32_t)P.st->k, g, j);
+  const float* src = reinterpret_cast<const float*>(P.X) + row * P.ld;
+  float* dst = xb + (long long)warp * d;
+  for (int c = lane; c < d; c += 32) dst[c] = src[c];
+  if (lane == 0) yb[warp] = reinterpret_cast<const int*>(P.y)[row];
+}
+
+// ------------------------------------------------------------------ GEMM
+struct Operand {
+  const float* base;  // plain buffer, or unused when ring != 0
+  long long off;      // ring != 0: offset inside theta
+  long long zg, zq;   // batch strides (group, point)
+  long long rs, cs;   // strides of the first / second matrix index
+  int ring;           // 1: the operand lives in the iterate ring (theta^k for q = 0, theta^{k-tau_g} for q = 1)
+};
+
+struct GemmArgs {
+  int M, N, K;
+  Operand A;   // A(m, k)
+  Operand Bm;  // B(k, n)
+  float* C;    // plain output (c_grad == 0): C + g*c_zg + q*c_zq + m*c_rs + n
+  long long c_zg, c_zq, c_rs;
+  int c_grad;  // 1: output goes to the gradient vectors, (q == 0 ? fresh : stale) + g*p_pad + c_off
+  long long c_off;
+  int bias;    // add b[n] from the iterate ring at bias_off
+  long long bias_off;
+  int relu;
+  const float* mask;  // multiply by (mask(m, n) > 0); same indexing as C
+};
+
+constexpr int TM = 64, TN = 64, TK = 16;
+
+__global__ void __launch_bounds__(256) mlp_sgemm_kernel(const Params P, const GemmArgs a) {
+  __shared__ float As[TK][TM + 4];
+  __shared__ float Bs[TK][TN + 4];
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const int z = blockIdx.z, q = z / P.G, g = z - q * P.G;
+  const int m0 = blockIdx.y * TM, n0 = blockIdx.x * TN;
+  const long long k_it = P.st->k;
+  const float* Ab = a.A.ring ? ring_ptr(P, g, q, k_it) + a.A.off : a.A.base + g * a.A.zg + q * a.A.zq;
+  const float* Bb = a.Bm.ring ? ring_ptr(P, g, q, k_it) + a.Bm.off : a.Bm.base + g * a.Bm.zg + q * a.Bm.zq;
+  float acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+  for (int k0 = 0; k0 < a.K; k0 += TK) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int e = tid + 256 * i;
+      int mm, kk;
+      if (a.A.cs == 1) {
+        kk = e & (TK - 1);
+        mm = e >> 4;
+      } else {
+        mm = e & (TM - 1);
+        kk = e >> 6;
+      }
+      const int m = m0 + mm, kx = k0 + kk;
+      As[kk][mm] = (m < a.M && kx < a.K) ? Ab[m * a.A.rs + kx * a.A.cs] : 0.f;
+      int nn, kb;
+      if (a.Bm.cs == 1) {
+        nn = e & (TN - 1);
+        kb = e >> 6;
+      } else {
+        kb = e & (TK - 1);
+        nn = e >> 4;
+      }
+      const int n = n0 + nn, ky = k0 + kb;
+      Bs[kb][nn] = (n < a.N && ky < a.K) ? Bb[ky * a.Bm.rs + n * a.Bm.cs] : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < TK; ++kk) {
+      float av[4], bv[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) av[i] = As[kk][ty * 4 + i];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) bv[j] = Bs[kk][tx * 4 + j];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] += av[i] * bv[j];
+    }
+    __syncthreads();
+  }
+
+  float* Cb;
+  if (a.c_grad)
+    Cb = (q == 0 ? P.fresh : P.stale) + (long long)g * P.p_pad + a.c_off;
+  else
+    Cb = a.C + g * a.c_zg + q * a.c_zq;
+  const float* Mb = a.mask ? a.mask + g * a.c_zg + q * a.c_zq : nullptr;
+  const float* bias = a.bias ? ring_ptr(P, g, q, k_it) + a.bias_off : nullptr;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int m = m0 + ty * 4 + i;
+    if (m >= a.M) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int n = n0 + tx * 4 + j;
+      if (n >= a.N) continue;
+      float v = acc[i][j];
+      if (bias) v += bias[n];
+      if (a.relu) v = fmaxf(v, 0.f);
+      if (Mb) v = Mb[m * a.c_rs + n] > 0.f ? v : 0.f;
+      Cb[m * a.c_rs + n] = v;
+    }
+  }
+}
+
+// ------------------------------------------------------------------ loss
+// Warp per (point, row): dz = (softmax(scores) - onehot(y)) * scale.  Class ids outside [0, n_cls) are
+// the caller's error (undefined result).
+__global__ void __launch_bounds__(256) mlp_softmax_grad_kernel(const Params P, const float* scores, const int* yb,
+                                                               float* dz, int n_cls) {
+  const long long rows = (long long)P.G * P.B;
+  const long long w = ((long long)blockIdx.x * 256 + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (w >= 2 * rows) return;
+  const long long r = w % rows;
+  const float* s = scores + w * n_cls;
+  float* o = dz + w * n_cls;
+  float mx = -3.0e38f;
+  for (int c = lane; c < n_cls; c += 32) mx = fmaxf(mx, s[c]);
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+  // p_y - 1 = -(sum of the other classes' exponentials) / sum: formed without
+  // the cancellation that p_y - 1 suffers once a sample is classified well
+  const int y = yb[r];
+  float others = 0.f;
+  for (int c = lane; c < n_cls; c += 32)
+    if (c != y) others += expf(s[c] - mx);
+  others = warp_sum(others);
+  const float ey = expf(s[y] - mx);
+  const float inv = 1.0f / (others + ey);
+  for (int c = lane; c < n_cls; c += 32)
+    o[c] = (c == y ? -others * inv : expf(s[c] - mx) * inv) * P.scale;
+}
+
+// ------------------------------------------------------------------ bias gradients
+// db_l[n] = sum over the group's rows of dz_l[row][n]; grid (n blocks, 2G, L).
+struct BiasArgs {
+  const float* dz[MLP_MAX_LAYERS + 1];
+  int n[MLP_MAX_LAYERS + 1];
+  long long b_off[MLP_MAX_LAYERS + 1];
+};
+
+__global__ void __launch_bounds__(256) mlp_bias_grad_kernel(const Params P, const BiasArgs a) {
+  const int l = blockIdx.z + 1;
+  const int n = blockIdx.x * 256 + threadIdx.x;
+  if (n >= a.n[l]) return;
+  const int z = blockIdx.y, q = z / P.G, g = z - q * P.G;
+  const float* src = a.dz[l] + ((long long)z * P.B) * a.n[l] + n;
+  float s = 0.f;
+  for (int r = 0; r < P.B; ++r) s += src[(long long)r * a.n[l]];
+  ((q == 0 ? P.fresh : P.stale) + (long long)g * P.p_pad + a.b_off[l])[n] = s;
+}
+
+cudaError_t launch_gemm(const Params& P, const GemmArgs& a, cudaStream_t st) {
+  dim3 grid((a.N + TN - 1) / TN, (a.M + TM - 1) / TM, 2 * P.G);
+  mlp_sgemm_kernel<<<grid, 256, 0, st>>>(P, a);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+const char* mlp_supported(const std::vector<int>& dims, int compute) {
+  if ((int)dims.size() - 1 > MLP_MAX_LAYERS) return "too many layers (at most 15)";
+  if (compute == 1) return mlp_bf16_supported(dims);
+  return nullptr;
+}
+
+cudaError_t mlp_plan_create(const std::vector<int>& dims, int compute, int G, int B, int D, long long p_pad,
+                            int sm_count, cudaStream_t st, MlpPlan* plan, std::vector<void*>* owned,
+                            const char** why) {
+  *why = "";
+  const int L = (int)dims.size() - 1;
+  plan->n_layers = L;
+  plan->compute = compute;
+  plan->G = G;
+  plan->B = B;
+  plan->D = D;
+  plan->p_pad = p_pad;
+  plan->sm_count = sm_count;
+  long long off = 0;
+  for (int l = 0; l <= L; ++l) plan->dims[l] = dims[l];
+  for (int l = 1; l <= L; ++l) {
+    plan->w_off[l] = off;
+    off += (long long)dims[l] * dims[l - 1];
+    plan->b_off[l] = off;
+    off += dims[l];
+  }
+  if (compute == 1) return mlp_bf16_plan_create(plan, st, owned, why);
+  const long long rows = (long long)G * B;
+  auto alloc = [&](void** q, size_t bytes) -> cudaError_t {
+    cudaError_t e = cudaMalloc(q, bytes);
+    if (e != cudaSuccess) return e;
+    owned->push_back(*q);
+    return cudaMemsetAsync(*q, 0, bytes, st);
+  };
+  cudaError_t e;
+  if ((e = alloc(reinterpret_cast<void**>(&plan->xb), sizeof(float) * rows * dims[0])) != cudaSuccess) return e;
+  if ((e = alloc(reinterpret_cast<void**>(&plan->yb), sizeof(int) * rows)) != cudaSuccess) return e;
+  for (int l = 1; l <= L; ++l) {
+    if ((e = alloc(reinterpret_cast<void**>(&plan->act[l]), sizeof(float) * 2 * rows * dims[l])) != cudaSuccess) return e;
+    if ((e = alloc(reinterpret_cast<void**>(&plan->dz[l]), sizeof(float) * 2 * rows * dims[l])) != cudaSuccess) return e;
+  }
+  plan->launches_per_iter = 3 * L + 2;
+  return cudaSuccess;
+}
+
+cudaError_t launch_grad_mlp(const Params& P, const MlpPlan& pl, cudaStream_t st, int* n_launches) {
+  if (pl.compute == 1) return mlp_bf16_launch(P, pl, st, n_launches);
+  const int L = pl.n_layers, G = P.G, B = P.B;
+  const long long rows = (long long)G * B;
+  int n = 0;
+  cudaError_t e;
+  mlp_gather_kernel<<<(unsigned)((rows * 32 + 255) / 256), 256, 0, st>>>(P, pl.xb, pl.yb, pl.dims[0]);
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  ++n;
+  // forward
+  for (int l = 1; l <= L; ++l) {
+    const int ni = pl.dims[l - 1], no = pl.dims[l];
+    GemmArgs a{};
+    a.M = B;
+    a.N = no;
+    a.K = ni;
+    if (l == 1)
+      a.A = Operand{pl.xb, 0, (long long)B * ni, 0, ni, 1, 0};
+    else
+      a.A = Operand{pl.act[l - 1], 0, (long long)B * ni, rows * ni, ni, 1, 0};
+    a.Bm = Operand{nullptr, pl.w_off[l], 0, 0, 1, ni, 1};  // B(k, n) = W_l[n][k]
+    a.C = pl.act[l];
+    a.c_zg = (long long)B * no;
+    a.c_zq = rows * no;
+    a.c_rs = no;
+    a.bias = 1;
+    a.bias_off = pl.b_off[l];
+    a.relu = l < L;
+    if ((e = launch_gemm(P, a, st)) != cudaSuccess) return e;
+    ++n;
+  }
+  mlp_softmax_grad_kernel<<<(unsigned)((2 * rows * 32 + 255) / 256), 256, 0, st>>>(P, pl.act[L], pl.yb, pl.dz[L],
+                                                                                  pl.dims[L]);
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  ++n;
+  // backward
+  for (int l = L; l >= 1; --l) {
+    const int ni = pl.dims[l - 1], no = pl.dims[l];
+    GemmArgs w{};  // dW_l = dz_l^T a_{l-1}
+    w.M = no;
+    w.N = ni;
+    w.K = B;
+    w.A = Operand{pl.dz[l], 0, (long long)B * no, rows * no, 1, no, 0};  // A(m, k) = dz_l[k][m]
+    if (l == 1)
+      w.Bm = Operand{pl.xb, 0, (long long)B * ni, 0, ni, 1, 0};
+    else
+      w.Bm = Operand{pl.act[l - 1], 0, (long long)B * ni, rows * ni, ni, 1, 0};
+    w.c_grad = 1;
+    w.c_off = pl.w_off[l];
+    w.c_rs = ni;
+    if ((e = launch_gemm(P, w, st)) != cudaSuccess) return e;
+    ++n;
+    if (l > 1) {
+      GemmArgs d{};  // dz_{l-1} = (dz_l W_l) masked by a_{l-1} > 0
+      d.M = B;
+      d.N = ni;
+      d.K = no;
+      d.A = Operand{pl.dz[l], 0, (long long)B * no, rows * no, no, 1, 0};
+      d.Bm = Operand{nullptr, pl.w_off[l], 0, 0, ni, 1, 1};  // B(k, n) = W_l[k][n]
+      d.C = pl.dz[l - 1];
+      d.c_zg = (long long)B * ni;
+      d.c_zq = rows * ni;
+      d.c_rs = ni;
+      d.mask = pl.act[l - 1];
+      if ((e = launch_gemm(P, d, st)) != cudaSuccess) return e;
+      ++n;
+    }
+  }
+  BiasArgs ba{};
+  int maxn = 0;
+  for (int l = 1; l <= L; ++l) {
+    ba.dz[l] = pl.dz[l];
+    ba.n[l] = pl.dims[l];
+    ba.b_off[l] = pl.b_off[l];
+    if (pl.dims[l] > maxn) maxn = pl.dims[l];
+  }
+  mlp_bias_grad_kernel<<<dim3((maxn + 255) / 256, 2 * G, L), 256, 0, st>>>(P, ba);
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  ++n;
+  *n_launches = n;
+  return cudaSuccess;
+}
+
+}  // namespace gcada

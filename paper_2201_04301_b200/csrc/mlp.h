@@ -8,19 +8,24 @@
 
 namespace gcada {
 
+constexpr int MLP_MAX_LAYERS = 15;
+
 struct MlpPlan {
-  int n_layers = 0;
+  int n_layers = 0;           // L
   int launches_per_iter = 0;
-  int compute = 0;
-  int dims[16] = {0};
-  long long w_off[16] = {0};  // offset of W_l inside theta
-  long long b_off[16] = {0};  // offset of b_l inside theta
-  // workspaces (device)
-  void* xb = nullptr;         // gathered minibatch rows
-  int* yb = nullptr;          // gathered labels
-  float* act[16] = {nullptr}; // act[l]: [2][G*B][dims[l]] post-activation of layer l (l >= 1)
-  float* dz[16] = {nullptr};  // dz[l]: [2][G*B][dims[l]] gradient w.r.t. pre-activation of layer l
+  int compute = 0;            // 0 fp32, 1 bf16 operands
+  int G = 0, B = 0, D = 0;
+  long long p_pad = 0;
+  int dims[MLP_MAX_LAYERS + 1] = {0};
+  long long w_off[MLP_MAX_LAYERS + 1] = {0};  // offset of W_l inside theta (l = 1..L)
+  long long b_off[MLP_MAX_LAYERS + 1] = {0};  // offset of b_l inside theta
   int sm_count = 0;
+  // fp32 workspaces (device)
+  float* xb = nullptr;                        // [G*B][dims[0]] gathered minibatch rows
+  int* yb = nullptr;                          // [G*B] gathered class ids
+  float* act[MLP_MAX_LAYERS + 1] = {nullptr}; // act[l], 1 <= l < L: [2][G*B][dims[l]] after ReLU; act[L]: class scores
+  float* dz[MLP_MAX_LAYERS + 1] = {nullptr};  // dz[l], 1 <= l <= L: [2][G*B][dims[l]] gradient w.r.t. z_l
+  void* bf16_impl = nullptr;                  // opaque state of the bf16 tensor-core path
 };
 
 // nullptr if the architecture is supported, else the reason.

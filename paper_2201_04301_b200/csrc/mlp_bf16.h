@@ -1,0 +1,9 @@
+// bf16 tensor-core path of the MLP gradients (tcgen05 + TMA); see mlp_bf16.cu.
+#pragma once
+#include "mlp.h"
+
+namespace gcada {
+const char* mlp_bf16_supported(const std::vector<int>& dims);
+cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<void*>* owned, const char** why);
+cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& plan, cudaStream_t st, int* n_launches);
+}  // namespace gcada

