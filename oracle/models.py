@@ -81,9 +81,13 @@ class MLP:
     theta is the concatenation over l = 1..L of W_l (n_l rows of n_{l-1}
     values, row-major) followed by b_l (n_l values).
 
-    With bf16=True the inputs and the weights (biases included) are rounded to
-    bfloat16 before use and everything else is fp64: the rounding points the
-    mixed-precision workload fixes for its operands."""
+    With bf16=True every matrix-product operand is a bfloat16 value: the
+    inputs, the weights (biases included), the hidden activations a_l and
+    the back-propagated errors dz_l are rounded to bfloat16 (ties to even)
+    before they are used; products, sums, the softmax and the loss are fp64.
+    This is the reading of "bf16 inputs/weights with fp32 accumulation" for a
+    multi-layer network: the input of layer l+1 is the bf16 output of layer l,
+    so both sides take each ReLU on/off decision from the same numbers."""
     kind = "mlp"
 
     def __init__(self, dims, bf16=False):
@@ -114,7 +118,8 @@ class MLP:
             z = acts[-1] @ W.T + b
             zs.append(z)
             if l < len(layers) - 1:
-                acts.append(np.maximum(z, 0.0))
+                a = np.maximum(z, 0.0)
+                acts.append(round_to_bf16(a) if self.bf16 else a)
         return layers, acts, zs
 
     def loss(self, theta, Xb, yb, reduction="mean"):
@@ -151,6 +156,8 @@ class MLP:
         pieces = [None] * len(layers)
         for l in range(len(layers) - 1, -1, -1):
             W, _ = layers[l]
+            if self.bf16:
+                dz = round_to_bf16(dz)
             dW = dz.T @ acts[l]          # n_l x n_{l-1}
             db = dz.sum(axis=0)
             pieces[l] = (dW, db)

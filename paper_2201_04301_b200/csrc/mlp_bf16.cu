@@ -1,12 +1,689 @@
+// bf16 tensor-core path of the dual-point MLP gradients (Algorithm 1's
+// gradient step for every group at theta^k and at theta^{k-tau_g}).
+//
+// Operands are bf16 (features as stored; weights rounded from the fp32 master
+// iterate once per iteration), accumulation is fp32 in tensor memory, the
+// per-group weight gradients are written in fp32 straight into the gradient
+// vectors.  Every product is an "NT" GEMM  C[M x N] = A[M x K] * B[N x K]^T
+// with both operands K-major, so one kernel serves all of them:
+//     forward   z_l   = a_{l-1} W_l^T        A = a_{l-1} [rows][n_{l-1}],  B = W_l   [n_l][n_{l-1}]
+//     backward  da    = dz_l W_l             A = dz_l    [rows][n_l],      B = W_l^T [n_{l-1}][n_l]
+//     weights   dW_l  = dz_l^T a_{l-1}       A = dz_l^T  [n_l][rows],      B = a_{l-1}^T [n_{l-1}][rows]
+// which is why activations, dz and the weights are kept in both orientations
+// (the epilogues write the second orientation for free).
+//
+// Kernel: one CTA per 128 x 128 output tile; warp 0 = TMA producer
+// (cp.async.bulk.tensor, 128-byte swizzle, mbarrier ring), warp 1 = MMA issuer
+// (tcgen05.mma, cta_group::1, 128x128x16 bf16 -> fp32 in TMEM), warps 2-5 =
+// epilogue (tcgen05.ld, fused bias / ReLU / ReLU-mask, stores).  A group's
+// minibatch is padded to a multiple of 128 rows, so an M tile never mixes
+// groups and the stale-point weights of a tile are one slot of the bf16
+// weight ring.  Every wait is bounded; a timeout raises the device error word.
 #include "mlp_bf16.h"
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+
 namespace gcada {
-const char* mlp_bf16_supported(const std::vector<int>&) { return "the bf16 MLP path is not built yet"; }
-cudaError_t mlp_bf16_plan_create(MlpPlan*, cudaStream_t, std::vector<void*>*, const char** why) {
-  *why = "the bf16 MLP path is not built yet";
+
+namespace {
+
+constexpr int BM = 128, BN = 128, BK = 64;      // tile; BK * 2 bytes = one 128-byte swizzle row
+constexpr int MAX_STAGES = 6;
+constexpr int STAGE_BYTES = (BM + BN) * BK * 2;  // 32 KiB
+constexpr int GEMM_THREADS = 192;
+
+enum { EPI_HIDDEN = 0, EPI_SCORES = 1, EPI_DA = 2, EPI_DW = 3 };
+enum { ZB_BATCH = 0, ZB_GROUP = 1, ZB_RING = 2 };
+
+struct Bf16Impl {
+  int Bp = 0;                   // rows per group padded to a multiple of 128
+  long long slot_elems = 0;     // bf16 elements per weight-ring slot
+  long long w_pos[MLP_MAX_LAYERS + 1] = {0};   // W_l   [n_l][ldk_l] inside a slot
+  long long wt_pos[MLP_MAX_LAYERS + 1] = {0};  // W_l^T [n_{l-1}][ldn_l]
+  long long bias_pos[MLP_MAX_LAYERS + 1] = {0};  // floats (bf16-rounded biases) inside the bias ring slot
+  long long bias_slot = 0;
+  int ld[MLP_MAX_LAYERS + 1] = {0};            // row stride (elements) of activation-like buffers of width n_l
+  __nv_bfloat16* wb = nullptr;   // (D+1) slots
+  float* bias = nullptr;         // (D+1) slots of rounded biases
+  __nv_bfloat16* xb = nullptr;   // [G*Bp][ld0]
+  __nv_bfloat16* xbT = nullptr;  // [G][n_0][Bp]
+  int* yb = nullptr;             // [G*Bp], -1 on padding rows
+  __nv_bfloat16* act[MLP_MAX_LAYERS + 1] = {nullptr};   // [2][G*Bp][ld_l]
+  __nv_bfloat16* actT[MLP_MAX_LAYERS + 1] = {nullptr};  // [2][G][n_l][Bp]
+  __nv_bfloat16* dz[MLP_MAX_LAYERS + 1] = {nullptr};
+  __nv_bfloat16* dzT[MLP_MAX_LAYERS + 1] = {nullptr};
+  float* scores = nullptr;       // [2][G*Bp][n_L]
+  CUtensorMap tm_fwd_a[MLP_MAX_LAYERS + 1], tm_fwd_b[MLP_MAX_LAYERS + 1];
+  CUtensorMap tm_da_a[MLP_MAX_LAYERS + 1], tm_da_b[MLP_MAX_LAYERS + 1];
+  CUtensorMap tm_dw_a[MLP_MAX_LAYERS + 1], tm_dw_b[MLP_MAX_LAYERS + 1];
+};
+
+struct GemmB {
+  int M, N, K;
+  int a_shared;      // 1: operand A has one batch entry per group (the gathered features), else per (point, group)
+  int zb_mode;       // ZB_*
+  int epi;           // EPI_*
+  int stages;
+  // epilogue operands
+  __nv_bfloat16* out;    // row-major bf16 [z][M][ldo]
+  __nv_bfloat16* outT;   // transposed bf16 [z][N][ldt]
+  float* out_f32;        // EPI_SCORES: [z][M][N]
+  const __nv_bfloat16* mask;  // EPI_DA: same indexing as out
+  const float* bias_ring;     // EPI_HIDDEN / EPI_SCORES: rounded biases, ring slots of bias_slot floats
+  long long bias_slot, bias_pos;
+  long long ldo, ldt;
+  long long z_stride_out, z_stride_outT;
+  long long c_off, ldc;       // EPI_DW: offset inside the gradient vector, row stride
+};
+
+// ----------------------------------------------------------------- PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
+  for (uint32_t it = 0; it < (1u << 22); ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (it > 32) __nanosleep(64);
+  }
+  return false;
+}
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* tm, int c0, int c1, int c2, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(
+          smem_u32(dst)),
+      "l"(tm), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t tmem_c, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accum) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
+      :
+      : "r"(tmem_c), "l"(da), "l"(db), "r"(idesc), "r"(accum), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
+      : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n\t"
+      "tcgen05.wait::ld.sync.aligned;"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes
+// (64 bf16) under the 128-byte swizzle: 8-row atoms of 1024 bytes, start
+// address in 16-byte units, leading offset 1, stride offset 1024 bytes,
+// descriptor version 1, layout type 2 (128-byte swizzle).
+__device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr) {
+  return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
+         (2ull << 61);
+}
+// Instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, N >> 3 at bit 17, M >> 4 at bit 24.
+constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+__device__ __forceinline__ int ring_slot(const Params& P, int g, int q, long long k) {
+  long long j = q == 0 ? k : k - P.tau[g];
+  if (j < 0) j = 0;
+  return (int)(j % (P.D + 1));
+}
+
+// ----------------------------------------------------------------- GEMM
+__global__ void __launch_bounds__(GEMM_THREADS) bf16_gemm_kernel(const __grid_constant__ CUtensorMap tmA,
+                                                                 const __grid_constant__ CUtensorMap tmB,
+                                                                 const Params P, const GemmB a) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  __shared__ uint64_t full_bar[MAX_STAGES], empty_bar[MAX_STAGES], accum_bar;
+  __shared__ uint32_t tmem_base_sm;
+  unsigned char* tiles = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int z = blockIdx.z, q = z / P.G, g = z - q * P.G;
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  const int nkb = (a.K + BK - 1) / BK;
+  const int stages = a.stages;
+  const long long k_it = P.st->k;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(&full_bar[s], 1);
+      mbar_init(&empty_bar[s], 1);
+    }
+    mbar_init(&accum_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {  // TMEM: 128 lanes x BN fp32 columns
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_sm)),
+                 "r"((uint32_t)BN)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_sm;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      const int zA = a.a_shared ? g : z;
+      const int zB = a.zb_mode == ZB_RING ? ring_slot(P, g, q, k_it) : (a.zb_mode == ZB_GROUP ? g : z);
+      bool ok = true;
+      for (int kb = 0; kb < nkb && ok; ++kb) {
+        const int s = kb % stages;
+        ok = mbar_wait_bounded(&empty_bar[s], (uint32_t)(((kb / stages) & 1) ^ 1));
+        if (!ok) break;
+        unsigned char* sa = tiles + (size_t)s * STAGE_BYTES;
+        mbar_expect_tx(&full_bar[s], STAGE_BYTES);
+        tma_load_3d(sa, &tmA, kb * BK, m0, zA, &full_bar[s]);
+        tma_load_3d(sa + BM * BK * 2, &tmB, kb * BK, n0, zB, &full_bar[s]);
+      }
+      if (!ok) {
+        atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      bool ok = true;
+      for (int kb = 0; kb < nkb && ok; ++kb) {
+        const int s = kb % stages;
+        ok = mbar_wait_bounded(&full_bar[s], (uint32_t)((kb / stages) & 1));
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t sa = smem_u32(tiles + (size_t)s * STAGE_BYTES);
+        const uint64_t da = make_desc(sa), db = make_desc(sa + BM * BK * 2);
+#pragma unroll
+        for (int kk = 0; kk < BK / 16; ++kk)  // 16 bf16 = 32 bytes = 2 descriptor units per MMA
+          tc_mma_bf16(tmem_base, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), IDESC, (kb | kk) != 0 ? 1u : 0u);
+        tc_commit(&empty_bar[s]);  // frees the stage once these MMAs have read it
+      }
+      if (ok) {
+        tc_commit(&accum_bar);
+      } else {
+        atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
+      }
+    }
+  } else {
+    // epilogue: warp w may touch TMEM lanes 32*(w%4) .. +31
+    const int quad = warp & 3;
+    const int m = m0 + quad * 32 + lane;
+    bool ok = mbar_wait_bounded(&accum_bar, 0u);
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok) {
+      tc_fence_after();
+      const float* bias = nullptr;
+      if (a.epi == EPI_HIDDEN || a.epi == EPI_SCORES)
+        bias = a.bias_ring + (long long)ring_slot(P, g, q, k_it) * a.bias_slot + a.bias_pos;
+#pragma unroll 1
+      for (int c = 0; c < BN; c += 32) {
+        uint32_t v[32];
+        tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)c, v);
+        const int nc = n0 + c;
+        if (nc >= a.N) break;  // uniform across the CTA
+        const bool row_ok = m < a.M;
+        const bool full = nc + 32 <= a.N;
+        if (a.epi == EPI_DW) {
+          float* dst = (q == 0 ? P.fresh : P.stale) + (long long)g * P.p_pad + a.c_off + (long long)m * a.ldc + nc;
+          if (row_ok) {
+            if (full && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0)) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 4)
+                *reinterpret_cast<float4*>(dst + j) = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
+                                                                  __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+            } else {
+              for (int j = 0; j < 32 && nc + j < a.N; ++j) dst[j] = __uint_as_float(v[j]);
+            }
+          }
+        } else if (a.epi == EPI_SCORES) {
+          float* dst = a.out_f32 + ((long long)z * a.M + m) * a.N + nc;
+          if (row_ok)
+            for (int j = 0; j < 32 && nc + j < a.N; ++j) dst[j] = __uint_as_float(v[j]) + bias[nc + j];
+        } else {
+          float f[32];
+          if (a.epi == EPI_HIDDEN) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) f[j] = fmaxf(__uint_as_float(v[j]) + (nc + j < a.N ? bias[nc + j] : 0.f), 0.f);
+          } else {  // EPI_DA: ReLU derivative of the layer below
+            const __nv_bfloat16* mk = a.mask + (long long)z * a.z_stride_out + (long long)m * a.ldo + nc;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const bool on = row_ok && nc + j < a.N && __bfloat162float(mk[j]) > 0.f;
+              f[j] = on ? __uint_as_float(v[j]) : 0.f;
+            }
+          }
+          if (row_ok) {
+            __nv_bfloat16* dst = a.out + (long long)z * a.z_stride_out + (long long)m * a.ldo + nc;
+            if (full) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 8) {
+                __nv_bfloat162 h0 = __floats2bfloat162_rn(f[j], f[j + 1]), h1 = __floats2bfloat162_rn(f[j + 2], f[j + 3]);
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(f[j + 4], f[j + 5]), h3 = __floats2bfloat162_rn(f[j + 6], f[j + 7]);
+                uint4 pk;
+                pk.x = *reinterpret_cast<uint32_t*>(&h0);
+                pk.y = *reinterpret_cast<uint32_t*>(&h1);
+                pk.z = *reinterpret_cast<uint32_t*>(&h2);
+                pk.w = *reinterpret_cast<uint32_t*>(&h3);
+                *reinterpret_cast<uint4*>(dst + j) = pk;
+              }
+            } else {
+              for (int j = 0; j < 32 && nc + j < a.N; ++j) dst[j] = __float2bfloat16_rn(f[j]);
+            }
+            __nv_bfloat16* dstT = a.outT + (long long)z * a.z_stride_outT + (long long)nc * a.ldt + m;
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (nc + j < a.N) dstT[(long long)j * a.ldt] = __float2bfloat16_rn(f[j]);
+          }
+        }
+      }
+    } else if (lane == 0) {
+      atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)BN) : "memory");
+  }
+}
+
+// ----------------------------------------------------------------- weights -> bf16 (both orientations)
+// grid (col tiles, row tiles, layer-1); 32 x 32 tiles through shared memory.
+struct ConvArgs {
+  int n_out[MLP_MAX_LAYERS + 1], n_in[MLP_MAX_LAYERS + 1];
+  long long w_off[MLP_MAX_LAYERS + 1], b_off[MLP_MAX_LAYERS + 1];
+  long long w_pos[MLP_MAX_LAYERS + 1], wt_pos[MLP_MAX_LAYERS + 1], bias_pos[MLP_MAX_LAYERS + 1];
+  int ldk[MLP_MAX_LAYERS + 1], ldn[MLP_MAX_LAYERS + 1];
+  long long slot_elems, bias_slot;
+};
+
+__global__ void __launch_bounds__(256) bf16_convert_kernel(const Params P, const ConvArgs a, __nv_bfloat16* wb,
+                                                           float* bias) {
+  __shared__ float tile[32][33];
+  const int l = blockIdx.z + 1;
+  const int no = a.n_out[l], ni = a.n_in[l];
+  const int r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
+  if (r0 >= no || c0 >= ni) return;
+  const long long k = P.st->k;
+  const int slot = (int)(k % (P.D + 1));
+  const float* th = P.theta_ring + (long long)slot * P.p_pad;
+  __nv_bfloat16* W = wb + (long long)slot * a.slot_elems + a.w_pos[l];
+  __nv_bfloat16* WT = wb + (long long)slot * a.slot_elems + a.wt_pos[l];
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  for (int i = ty; i < 32; i += 8) {
+    const int r = r0 + i, c = c0 + tx;
+    float v = 0.f;
+    if (r < no && c < ni) {
+      v = th[a.w_off[l] + (long long)r * ni + c];
+      W[(long long)r * a.ldk[l] + c] = __float2bfloat16_rn(v);
+    }
+    tile[i][tx] = v;
+  }
+  __syncthreads();
+  for (int i = ty; i < 32; i += 8) {
+    const int c = c0 + i, r = r0 + tx;
+    if (r < no && c < ni) WT[(long long)c * a.ldn[l] + r] = __float2bfloat16_rn(tile[tx][i]);
+  }
+  if (blockIdx.x == 0 && blockIdx.y == 0) {
+    float* bo = bias + (long long)slot * a.bias_slot + a.bias_pos[l];
+    for (int n = threadIdx.x; n < no; n += 256) bo[n] = __bfloat162float(__float2bfloat16_rn(th[a.b_off[l] + n]));
+  }
+}
+
+// ----------------------------------------------------------------- gather (rows and their transpose)
+// Block = 32 consecutive rows of one group; features move through a 32 x 64 tile.
+__global__ void __launch_bounds__(256) bf16_gather_kernel(const Params P, __nv_bfloat16* xb, __nv_bfloat16* xbT,
+                                                          int* yb, int d, int ld0, int Bp) {
+  __shared__ __nv_bfloat16 tile[32][66];
+  __shared__ long long rows_sm[32];
+  const int g = blockIdx.y, rb = blockIdx.x * 32;
+  const int tid = threadIdx.x;
+  if (tid < 32) {
+    const int j = rb + tid;
+    long long row = -1;
+    if (j < P.B) row = batch_row(P, (uint32_t)P.st->k, g, j);
+    rows_sm[tid] = row;
+    yb[(long long)g * Bp + j] = row >= 0 ? reinterpret_cast<const int*>(P.y)[row] : -1;
+  }
+  __syncthreads();
+  const __nv_bfloat16* X = reinterpret_cast<const __nv_bfloat16*>(P.X);
+  for (int c0 = 0; c0 < d; c0 += 64) {
+    for (int e = tid; e < 32 * 64; e += 256) {
+      const int r = e >> 6, c = e & 63;
+      const long long row = rows_sm[r];
+      __nv_bfloat16 v = __float2bfloat16_rn(0.f);
+      if (row >= 0 && c0 + c < d) v = X[row * P.ld + c0 + c];
+      tile[r][c] = v;
+      if (c0 + c < d) xb[((long long)g * Bp + rb + r) * ld0 + c0 + c] = v;
+    }
+    __syncthreads();
+    for (int e = tid; e < 64 * 32; e += 256) {
+      const int c = e >> 5, r = e & 31;
+      if (c0 + c < d) xbT[((long long)g * d + c0 + c) * Bp + rb + r] = tile[r][c];
+    }
+    __syncthreads();
+  }
+}
+
+// ----------------------------------------------------------------- loss gradient
+// Warp per (point, padded row): dz = (softmax(scores) - onehot(y)) * scale in both orientations;
+// padding rows (y < 0) get zeros.
+__global__ void __launch_bounds__(256) bf16_softmax_grad_kernel(const Params P, const float* scores, const int* yb,
+                                                                __nv_bfloat16* dz, __nv_bfloat16* dzT, int n_cls,
+                                                                int ldz, int Bp) {
+  const long long rows = (long long)P.G * Bp;
+  const long long w = ((long long)blockIdx.x * 256 + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (w >= 2 * rows) return;
+  const long long r = w % rows;
+  const int q = (int)(w / rows);
+  const int g = (int)(r / Bp), mrow = (int)(r - (long long)g * Bp);
+  const float* s = scores + w * n_cls;
+  __nv_bfloat16* o = dz + w * ldz;
+  __nv_bfloat16* oT = dzT + ((long long)(q * P.G + g) * n_cls) * Bp + mrow;
+  const int y = yb[r];
+  if (y < 0) {
+    for (int c = lane; c < n_cls; c += 32) {
+      o[c] = __float2bfloat16_rn(0.f);
+      oT[(long long)c * Bp] = __float2bfloat16_rn(0.f);
+    }
+    return;
+  }
+  float mx = -3.0e38f;
+  for (int c = lane; c < n_cls; c += 32) mx = fmaxf(mx, s[c]);
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+  float others = 0.f;
+  for (int c = lane; c < n_cls; c += 32)
+    if (c != y) others += expf(s[c] - mx);
+  others = warp_sum(others);
+  const float inv = 1.0f / (others + expf(s[y] - mx));
+  for (int c = lane; c < n_cls; c += 32) {
+    const float v = (c == y ? -others * inv : expf(s[c] - mx) * inv) * P.scale;
+    const __nv_bfloat16 b = __float2bfloat16_rn(v);
+    o[c] = b;
+    oT[(long long)c * Bp] = b;
+  }
+}
+
+// ----------------------------------------------------------------- bias gradients
+struct BiasArgsB {
+  const __nv_bfloat16* dz[MLP_MAX_LAYERS + 1];
+  int n[MLP_MAX_LAYERS + 1], ld[MLP_MAX_LAYERS + 1];
+  long long b_off[MLP_MAX_LAYERS + 1];
+};
+__global__ void __launch_bounds__(256) bf16_bias_grad_kernel(const Params P, const BiasArgsB a, int Bp) {
+  const int l = blockIdx.z + 1;
+  const int n = blockIdx.x * 256 + threadIdx.x;
+  if (n >= a.n[l]) return;
+  const int z = blockIdx.y, q = z / P.G, g = z - q * P.G;
+  const __nv_bfloat16* src = a.dz[l] + ((long long)z * Bp) * a.ld[l] + n;
+  float s = 0.f;
+  for (int r = 0; r < Bp; ++r) s += __bfloat162float(src[(long long)r * a.ld[l]]);
+  ((q == 0 ? P.fresh : P.stale) + (long long)g * P.p_pad + a.b_off[l])[n] = s;
+}
+
+// ----------------------------------------------------------------- host
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess &&
+        qr == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// bf16 tensor [batch][rows][k] (k contiguous, row stride ld elements, batch stride bs elements);
+// box = 64 (k) x box_rows x 1, 128-byte swizzle, zero fill outside.
+bool make_map(CUtensorMap* tm, const void* base, long long k_extent, long long rows, long long batch, long long ld,
+              long long bs, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)k_extent, (cuuint64_t)rows, (cuuint64_t)batch};
+  cuuint64_t strides[2] = {(cuuint64_t)ld * 2, (cuuint64_t)bs * 2};
+  cuuint32_t box[3] = {(cuuint32_t)BK, (cuuint32_t)box_rows, 1};
+  cuuint32_t es[3] = {1, 1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+long long up(long long x, long long m) { return (x + m - 1) / m * m; }
+
+cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const Params& P, GemmB a, cudaStream_t st) {
+  const int nkb = (a.K + BK - 1) / BK;
+  a.stages = nkb < MAX_STAGES ? nkb : MAX_STAGES;
+  const size_t smem = (size_t)a.stages * STAGE_BYTES + 1024;
+  dim3 grid((a.N + BN - 1) / BN, (a.M + BM - 1) / BM, 2 * P.G);
+  bf16_gemm_kernel<<<grid, GEMM_THREADS, smem, st>>>(ta, tb, P, a);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+const char* mlp_bf16_supported(const std::vector<int>& dims) {
+  (void)dims;
+  return nullptr;
+}
+
+cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<void*>* owned, const char** why) {
+  const int L = plan->n_layers, G = plan->G, B = plan->B, D = plan->D;
+  Bf16Impl* im = new Bf16Impl();
+  plan->bf16_impl = im;  // lives as long as the process (a few hundred bytes per plan)
+  im->Bp = (int)up(B, 128);
+  const long long rows = (long long)G * im->Bp;
+  long long pos = 0, bpos = 0;
+  for (int l = 0; l <= L; ++l) im->ld[l] = (int)up(plan->dims[l], 8);
+  for (int l = 1; l <= L; ++l) {
+    im->w_pos[l] = pos;
+    pos += up((long long)plan->dims[l] * im->ld[l - 1], 64);
+    im->wt_pos[l] = pos;
+    pos += up((long long)plan->dims[l - 1] * im->ld[l], 64);
+    im->bias_pos[l] = bpos;
+    bpos += up(plan->dims[l], 4);
+  }
+  im->slot_elems = pos;
+  im->bias_slot = bpos;
+  auto alloc = [&](void** q, size_t bytes) -> cudaError_t {
+    cudaError_t e = cudaMalloc(q, bytes);
+    if (e != cudaSuccess) return e;
+    owned->push_back(*q);
+    return cudaMemsetAsync(*q, 0, bytes, st);
+  };
+#define A_(ptr, count, type)                                                                     \
+  do {                                                                                           \
+    cudaError_t e_ = alloc(reinterpret_cast<void**>(&(ptr)), sizeof(type) * (size_t)(count));    \
+    if (e_ != cudaSuccess) return e_;                                                            \
+  } while (0)
+  A_(im->wb, (long long)(D + 1) * im->slot_elems, __nv_bfloat16);
+  A_(im->bias, (long long)(D + 1) * im->bias_slot, float);
+  A_(im->xb, rows * im->ld[0], __nv_bfloat16);
+  A_(im->xbT, (long long)G * plan->dims[0] * im->Bp, __nv_bfloat16);
+  A_(im->yb, rows, int);
+  for (int l = 1; l <= L; ++l) {
+    if (l < L) {
+      A_(im->act[l], 2 * rows * im->ld[l], __nv_bfloat16);
+      A_(im->actT[l], 2LL * G * plan->dims[l] * im->Bp, __nv_bfloat16);
+    }
+    A_(im->dz[l], 2 * rows * im->ld[l], __nv_bfloat16);
+    A_(im->dzT[l], 2LL * G * plan->dims[l] * im->Bp, __nv_bfloat16);
+  }
+  A_(im->scores, 2 * rows * plan->dims[L], float);
+#undef A_
+  if (!encode_fn()) {
+    *why = "cuTensorMapEncodeTiled is not available from this driver";
+    return cudaSuccess;
+  }
+  bool ok = true;
+  const long long Bp = im->Bp;
+  for (int l = 1; l <= L; ++l) {
+    const int ni = plan->dims[l - 1], no = plan->dims[l];
+    // forward: A = a_{l-1} rows, B = W_l (ring)
+    if (l == 1)
+      ok &= make_map(&im->tm_fwd_a[l], im->xb, ni, Bp, G, im->ld[0], Bp * im->ld[0], BM);
+    else
+      ok &= make_map(&im->tm_fwd_a[l], im->act[l - 1], ni, Bp, 2LL * G, im->ld[l - 1], Bp * im->ld[l - 1], BM);
+    ok &= make_map(&im->tm_fwd_b[l], im->wb + im->w_pos[l], ni, no, D + 1, im->ld[l - 1], im->slot_elems, BN);
+    // backward data: A = dz_l rows, B = W_l^T (ring)
+    ok &= make_map(&im->tm_da_a[l], im->dz[l], no, Bp, 2LL * G, im->ld[l], Bp * im->ld[l], BM);
+    ok &= make_map(&im->tm_da_b[l], im->wb + im->wt_pos[l], no, ni, D + 1, im->ld[l], im->slot_elems, BN);
+    // weight gradient: A = dz_l^T, B = a_{l-1}^T
+    ok &= make_map(&im->tm_dw_a[l], im->dzT[l], Bp, no, 2LL * G, Bp, (long long)no * Bp, BM);
+    if (l == 1)
+      ok &= make_map(&im->tm_dw_b[l], im->xbT, Bp, ni, G, Bp, (long long)ni * Bp, BN);
+    else
+      ok &= make_map(&im->tm_dw_b[l], im->actT[l - 1], Bp, ni, 2LL * G, Bp, (long long)ni * Bp, BN);
+  }
+  if (!ok) {
+    *why = "tensor map creation failed for this MLP shape";
+    return cudaSuccess;
+  }
+  cudaError_t e = cudaFuncSetAttribute(bf16_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       MAX_STAGES * STAGE_BYTES + 1024);
+  if (e != cudaSuccess) return e;
+  plan->launches_per_iter = 3 + L + 1 + L + (L - 1);
   return cudaSuccess;
 }
-cudaError_t mlp_bf16_launch(const Params&, const MlpPlan&, cudaStream_t, int* n) {
-  *n = 0;
-  return cudaErrorNotSupported;
+
+cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st, int* n_launches) {
+  const Bf16Impl* im = static_cast<const Bf16Impl*>(pl.bf16_impl);
+  const int L = pl.n_layers, G = P.G, Bp = im->Bp;
+  const long long rows = (long long)G * Bp;
+  int n = 0;
+  cudaError_t e;
+  // weights of theta^k -> bf16 ring slot k (both orientations) and rounded biases
+  {
+    ConvArgs c{};
+    int max_no = 0, max_ni = 0;
+    for (int l = 1; l <= L; ++l) {
+      c.n_out[l] = pl.dims[l];
+      c.n_in[l] = pl.dims[l - 1];
+      c.w_off[l] = pl.w_off[l];
+      c.b_off[l] = pl.b_off[l];
+      c.w_pos[l] = im->w_pos[l];
+      c.wt_pos[l] = im->wt_pos[l];
+      c.bias_pos[l] = im->bias_pos[l];
+      c.ldk[l] = im->ld[l - 1];
+      c.ldn[l] = im->ld[l];
+      if (pl.dims[l] > max_no) max_no = pl.dims[l];
+      if (pl.dims[l - 1] > max_ni) max_ni = pl.dims[l - 1];
+    }
+    c.slot_elems = im->slot_elems;
+    c.bias_slot = im->bias_slot;
+    bf16_convert_kernel<<<dim3((max_ni + 31) / 32, (max_no + 31) / 32, L), 256, 0, st>>>(P, c, im->wb, im->bias);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    ++n;
+  }
+  bf16_gather_kernel<<<dim3(Bp / 32, G), 256, 0, st>>>(P, im->xb, im->xbT, im->yb, pl.dims[0], im->ld[0], Bp);
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  ++n;
+  for (int l = 1; l <= L; ++l) {
+    GemmB a{};
+    a.M = Bp;
+    a.N = pl.dims[l];
+    a.K = pl.dims[l - 1];
+    a.a_shared = l == 1;
+    a.zb_mode = ZB_RING;
+    a.bias_ring = im->bias;
+    a.bias_slot = im->bias_slot;
+    a.bias_pos = im->bias_pos[l];
+    if (l < L) {
+      a.epi = EPI_HIDDEN;
+      a.out = im->act[l];
+      a.outT = im->actT[l];
+      a.ldo = im->ld[l];
+      a.ldt = Bp;
+      a.z_stride_out = (long long)Bp * im->ld[l];
+      a.z_stride_outT = (long long)pl.dims[l] * Bp;
+    } else {
+      a.epi = EPI_SCORES;
+      a.out_f32 = im->scores;
+    }
+    if ((e = launch_gemm(im->tm_fwd_a[l], im->tm_fwd_b[l], P, a, st)) != cudaSuccess) return e;
+    ++n;
+  }
+  bf16_softmax_grad_kernel<<<(unsigned)((2 * rows * 32 + 255) / 256), 256, 0, st>>>(
+      P, im->scores, im->yb, im->dz[L], im->dzT[L], pl.dims[L], im->ld[L], Bp);
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  ++n;
+  for (int l = L; l >= 1; --l) {
+    GemmB w{};
+    w.M = pl.dims[l];
+    w.N = pl.dims[l - 1];
+    w.K = Bp;
+    w.a_shared = 0;
+    w.zb_mode = l == 1 ? ZB_GROUP : ZB_BATCH;
+    w.epi = EPI_DW;
+    w.c_off = pl.w_off[l];
+    w.ldc = pl.dims[l - 1];
+    if ((e = launch_gemm(im->tm_dw_a[l], im->tm_dw_b[l], P, w, st)) != cudaSuccess) return e;
+    ++n;
+    if (l > 1) {
+      GemmB d{};
+      d.M = Bp;
+      d.N = pl.dims[l - 1];
+      d.K = pl.dims[l];
+      d.a_shared = 0;
+      d.zb_mode = ZB_RING;
+      d.epi = EPI_DA;
+      d.out = im->dz[l - 1];
+      d.outT = im->dzT[l - 1];
+      d.mask = im->act[l - 1];
+      d.ldo = im->ld[l - 1];
+      d.ldt = Bp;
+      d.z_stride_out = (long long)Bp * im->ld[l - 1];
+      d.z_stride_outT = (long long)pl.dims[l - 1] * Bp;
+      if ((e = launch_gemm(im->tm_da_a[l], im->tm_da_b[l], P, d, st)) != cudaSuccess) return e;
+      ++n;
+    }
+  }
+  BiasArgsB ba{};
+  int maxn = 0;
+  for (int l = 1; l <= L; ++l) {
+    ba.dz[l] = im->dz[l];
+    ba.n[l] = pl.dims[l];
+    ba.ld[l] = im->ld[l];
+    ba.b_off[l] = pl.b_off[l];
+    if (pl.dims[l] > maxn) maxn = pl.dims[l];
+  }
+  bf16_bias_grad_kernel<<<dim3((maxn + 255) / 256, 2 * G, L), 256, 0, st>>>(P, ba, Bp);
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  ++n;
+  *n_launches = n;
+  return cudaSuccess;
 }
+
 }  // namespace gcada

@@ -79,7 +79,8 @@ def _kink_match(o, got, theta, Xb, yb, reduction, tol, kink_tol):
     return False
 
 
-def forced_parity(w, K, tol=TOL_FP32, stream=None, reduction="mean", check_stale=True, kink_tol=2e-6):
+def forced_parity(w, K, tol=TOL_FP32, stream=None, reduction="mean", check_stale=True, kink_tol=2e-6,
+                  margin=MARGIN, rhs_tol=1e-4):
     """Run the oracle free for K steps and the CUDA path teacher-forced with the
     oracle's masks; compare every step.  Returns the number of steps at which
     the CUDA path's own test outcome differed from the oracle's (only allowed
@@ -112,13 +113,13 @@ def forced_parity(w, K, tol=TOL_FP32, stream=None, reduction="mean", check_stale
                 assert e <= tol, (name, k, gi, e)
         lhs, rhs = g.get_debug(binding.DBG_LHS), g.get_debug(binding.DBG_RHS)[0]
         assert np.array_equal(tau_before, rec["tau"]), (k, tau_before, rec["tau"])
-        assert rhs == np.float64(rhs) and abs(rhs - rec["rhs"]) <= 1e-4 * max(rec["rhs"], 1e-300), (k, rhs, rec["rhs"])
+        assert abs(rhs - rec["rhs"]) <= rhs_tol * max(rec["rhs"], 1e-300), (k, rhs, rec["rhs"])
         # the CUDA path's own decision, from its own numbers
         own = (tau_before >= o.D) | (lhs > rhs)
         for gi in range(o.G):
             if bool(own[gi]) != bool(rec["mask"][gi]):
-                margin = abs(rec["lhs"][gi] - rec["rhs"]) / max(rec["lhs"][gi], rec["rhs"], 1e-300)
-                assert margin < MARGIN, ("mask", k, gi, lhs[gi], rhs, rec["lhs"][gi], rec["rhs"])
+                rel = abs(rec["lhs"][gi] - rec["rhs"]) / max(rec["lhs"][gi], rec["rhs"], 1e-300)
+                assert margin is None or rel < margin, ("mask", k, gi, lhs[gi], rhs, rec["lhs"][gi], rec["rhs"])
                 flips += 1
             if rec["lhs"][gi] > 0:
                 worst["lhs"] = max(worst["lhs"], abs(lhs[gi] - rec["lhs"][gi]) / rec["lhs"][gi])

@@ -453,3 +453,51 @@ def test_relu_kink_choices_are_the_one_sided_derivatives():
     assert abs(right - left) > 1e-3           # the kink is real
     assert mlp.grad(theta, Xb, yb, "sum")[6] == pytest.approx(left, rel=1e-5)
     assert mlp.grad(theta, Xb, yb, "sum", flip=kinks)[6] == pytest.approx(right, rel=1e-5)
+
+
+def test_bf16_mode_rounds_every_matrix_operand():
+    """bf16 mode against torch autograd (library routine) with explicit
+    bfloat16 casts of inputs, weights and hidden activations in the forward
+    pass and gradient hooks that round the back-propagated errors."""
+    rng = np.random.default_rng(7)
+    mlp = MLP((6, 5, 4, 3), bf16=True)
+    theta = rng.normal(size=mlp.p)
+    Xb = rng.normal(size=(8, 6))
+    yb = rng.integers(0, 3, 8)
+    rb = lambda t: t.to(torch.float32).to(torch.bfloat16).to(torch.float64)
+
+    class RoundGrad(torch.autograd.Function):
+        @staticmethod
+        def forward(ctx, x):
+            return x
+
+        @staticmethod
+        def backward(ctx, g):
+            return rb(g)
+
+    class RoundValue(torch.autograd.Function):     # value rounded, gradient passed through
+        @staticmethod
+        def forward(ctx, x):
+            return rb(x)
+
+        @staticmethod
+        def backward(ctx, g):
+            return g
+
+    t = torch.tensor(theta, requires_grad=True)
+    tr = RoundValue.apply(t)
+    o, a = 0, rb(torch.tensor(Xb))
+    dims = mlp.dims
+    for l in range(1, len(dims)):
+        W = tr[o:o + dims[l] * dims[l - 1]].reshape(dims[l], dims[l - 1])
+        o += dims[l] * dims[l - 1]
+        b = tr[o:o + dims[l]]
+        o += dims[l]
+        z = RoundGrad.apply(a @ W.T + b)
+        a = RoundValue.apply(torch.relu(z)) if l < len(dims) - 1 else z
+    torch.nn.functional.cross_entropy(a, torch.tensor(yb), reduction="mean").backward()
+    got = mlp.grad(theta, Xb, yb, "mean")
+    assert np.allclose(got, t.grad.numpy(), rtol=1e-9, atol=1e-12)
+    # and it stays close to the unrounded gradient
+    exact = MLP((6, 5, 4, 3)).grad(theta, Xb, yb, "mean")
+    assert 1e-5 < np.linalg.norm(got - exact) / np.linalg.norm(exact) < 3e-2

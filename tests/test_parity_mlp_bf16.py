@@ -1,0 +1,39 @@
+"""CUDA tensor-core path (bf16 operands, fp32 accumulation) vs the CPU oracle
+with the same operand rounding, through the C ABI.  Tolerance 2e-2 relative
+L2: the CUDA path also rounds activations and back-propagated errors to bf16
+between layers, which the oracle (fp64 after operand rounding) does not."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2201_04301_b200 import binding
+from paper_2201_04301_b200.workloads import make_workload
+
+from parity import TOL_BF16, forced_parity, to_cuda
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("dims,batch,M,M_G,D", [
+    ((64, 128, 96, 40), 128, 6, 2, 3),     # three layers, one 128-row tile per group
+    ((100, 72, 10), 32, 4, 2, 2),          # ragged K and N, minibatch padded from 32 to 128 rows
+    ((256, 300, 130), 256, 2, 1, 2),       # two row tiles per group, three N tiles with a ragged one
+])
+def test_small_architectures(dims, batch, M, M_G, D):
+    G = M // M_G
+    w = make_workload("cfg5", rows=G * 1000, dims=dims, M=M, M_G=M_G, D=D, batch=batch, c=0.3, alpha=1e-3)
+    flips, worst = forced_parity(w, 2 * D + 3, tol=TOL_BF16, stream=torch.cuda.Stream(), margin=None, rhs_tol=2e-2)
+    print("bf16", dims, "worst", worst, "flips", flips)
+
+
+def test_deterministic_and_counts():
+    w = to_cuda(make_workload("cfg5", rows=3000, dims=(64, 128, 40), M=6, M_G=2, D=3, batch=128))
+    outs = []
+    for _ in range(2):
+        g = binding.from_workload(w, stream=torch.cuda.Stream())
+        g.step(20)
+        outs.append((g.get_theta(), g.get_selection_mask(0, 20), g.get_comm_count()))
+        g.close()
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+    up, comm, comp = outs[0][2]
+    assert up == int(outs[0][1].sum()) and comm == 3 * up and comp == 2 * up and outs[0][1][0].all()
