@@ -154,7 +154,10 @@ def run_ours(args):
     _barrier(world)
     binding.load()
     t0 = time.time()
-    w = make_workload(args.config, device=dev, data_seed=rank, rows=args.rows)
+    overrides = {}
+    if args.workers:
+        overrides["M"] = args.workers
+    w = make_workload(args.config, device=dev, data_seed=rank, rows=args.rows, **overrides)
     stream = torch.cuda.Stream(device=dev)
     torch.cuda.synchronize()
     g = binding.from_workload(w, stream=stream, options={binding.OPT_GRAPH: 0.0 if args.no_graph else 1.0,
@@ -385,6 +388,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="plain launches instead of graph replay")
+    ap.add_argument("--workers", type=int, default=None, help="override M (fewer groups, for profiling captures)")
     ap.add_argument("--variant", type=int, default=0, help="GCADA_OPT_LINEAR_VARIANT (kernel shape knob)")
     ap.add_argument("--e2e-steps", type=int, default=60)
     ap.add_argument("--cpu-budget", type=float, default=15.0)
