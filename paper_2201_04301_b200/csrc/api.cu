@@ -176,7 +176,9 @@ gcada_status make_ready(gcada_ctx* ctx, const float* theta0, int on_device) {
   TRY(dev_alloc(ctx, &P.agg_lo, (size_t)pp));
   TRY(dev_alloc(ctx, &P.g_last, (size_t)G * pp));
   TRY(dev_alloc(ctx, &P.fresh, (size_t)G * pp));
-  if (ctx->keep_stale || !is_linear(ctx)) TRY(dev_alloc(ctx, &P.stale, (size_t)G * pp));
+  // the fp32 MLP kernels hand over both gradients; the others keep the stale one only on request
+  if (ctx->keep_stale || (!is_linear(ctx) && ctx->compute == GCADA_COMPUTE_FP32))
+    TRY(dev_alloc(ctx, &P.stale, (size_t)G * pp));
   TRY(dev_alloc(ctx, &P.tau, (size_t)G));
   TRY(dev_alloc(ctx, &P.lhs, (size_t)G));
   TRY(dev_alloc(ctx, &P.t_g, (size_t)G));
@@ -238,6 +240,11 @@ gcada_status make_plans(gcada_ctx* ctx) {
     for (void* q : bufs) ctx->owned.push_back(q);
     if (e != cudaSuccess) return fail(ctx, e == cudaErrorMemoryAllocation ? GCADA_ENOMEM : GCADA_ECUDA, "MLP plan: %s (%s)", why, cudaGetErrorString(e));
     if (why[0]) return fail(ctx, GCADA_EINVAL, "%s", why);
+    if (ctx->mlp.norm_parts > 0) {  // the gradient kernels deliver the innovation-norm partial sums themselves
+      P.pm.n_cta = -1;
+      P.pm.maxseg = ctx->mlp.norm_parts;
+      TRY(dev_alloc(ctx, &P.lhs_part, (size_t)ctx->G * ctx->mlp.norm_parts));
+    }
   }
   CK(cudaStreamSynchronize(ctx->stream));
   ctx->ready = true;

@@ -33,7 +33,8 @@ struct DevState {
 // [c*R/n, (c+1)*R/n) of the G*B minibatch rows and writes one slot per group
 // it touches, slot = c*maxseg + (g - first group of c).
 struct PartialMap {
-  int n_cta;      // 0 = gradients are already whole (one "slot" per group)
+  int n_cta;      // 0 = gradients are already whole (one "slot" per group); -1 = whole, and lhs_part already
+                  // holds `maxseg` partial sums of the innovation norm per group (nothing left to reduce)
   int maxseg;
   int rows_per_group;  // B
 };

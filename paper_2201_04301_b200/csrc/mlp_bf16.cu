@@ -54,6 +54,8 @@ struct Bf16Impl {
   __nv_bfloat16* dz[MLP_MAX_LAYERS + 1] = {nullptr};
   __nv_bfloat16* dzT[MLP_MAX_LAYERS + 1] = {nullptr};
   float* scores = nullptr;       // [2][G*Bp][n_L]
+  int dw_part_base[MLP_MAX_LAYERS + 1] = {0}, bias_part_base[MLP_MAX_LAYERS + 1] = {0};
+  int n_parts = 0;               // innovation-norm partial sums per group
   CUtensorMap tm_fwd_a[MLP_MAX_LAYERS + 1], tm_fwd_b[MLP_MAX_LAYERS + 1];
   CUtensorMap tm_da_a[MLP_MAX_LAYERS + 1], tm_da_b[MLP_MAX_LAYERS + 1];
   CUtensorMap tm_dw_a[MLP_MAX_LAYERS + 1], tm_dw_b[MLP_MAX_LAYERS + 1];
@@ -313,6 +315,169 @@ __global__ void __launch_bounds__(GEMM_THREADS) bf16_gemm_kernel(const __grid_co
   }
 }
 
+// ----------------------------------------------------------------- weight gradients, both points in one CTA
+// dW_l of one group at theta^k (accumulator 0) and at the stale iterate
+// (accumulator 1) for one 128 x 128 tile.  The epilogue writes the fresh
+// gradient (and the stale one only when it is kept for inspection), forms the
+// squared norm of their difference - this tile's share of the left side of
+// Eq. (9) - and stores it in the tile's own slot of lhs_part, so the
+// per-group gradients are never re-read to build the test.  Rows reach
+// global memory as full 128-byte lines through a per-warp staging tile.
+struct DwArgs {
+  int M, N, K;            // n_l, n_{l-1}, padded rows per group
+  int b_shared;           // 1: operand B has one entry per group (the gathered features)
+  int nkb;                // K blocks per point
+  int stages;
+  long long c_off, ldc;   // position of W_l inside the gradient vector, row stride
+  int part_base, n_parts; // this layer's first slot in lhs_part and slots per group
+};
+
+constexpr int DW_PITCH = 36;  // floats per staged row (16-byte aligned, conflict-free 16-byte stores)
+
+__global__ void __launch_bounds__(GEMM_THREADS) bf16_dw_kernel(const __grid_constant__ CUtensorMap tmA,
+                                                               const __grid_constant__ CUtensorMap tmB,
+                                                               const Params P, const DwArgs a) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  __shared__ uint64_t full_bar[MAX_STAGES], empty_bar[MAX_STAGES], accum_bar;
+  __shared__ uint32_t tmem_base_sm;
+  __shared__ double norm_sm[4];
+  unsigned char* tiles = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  float* stage_all = reinterpret_cast<float*>(tiles + (size_t)a.stages * STAGE_BYTES);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = blockIdx.z;
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  const int stages = a.stages;
+  const int total_kb = 2 * a.nkb;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(&full_bar[s], 1);
+      mbar_init(&empty_bar[s], 1);
+    }
+    mbar_init(&accum_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {  // two fp32 accumulators of BN columns each
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_sm)),
+                 "r"((uint32_t)(2 * BN))
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_sm;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      bool ok = true;
+      for (int it = 0; it < total_kb && ok; ++it) {
+        const int q = it / a.nkb, kb = it - q * a.nkb;
+        const int s = it % stages;
+        ok = mbar_wait_bounded(&empty_bar[s], (uint32_t)(((it / stages) & 1) ^ 1));
+        if (!ok) break;
+        unsigned char* sa = tiles + (size_t)s * STAGE_BYTES;
+        mbar_expect_tx(&full_bar[s], STAGE_BYTES);
+        tma_load_3d(sa, &tmA, kb * BK, m0, q * P.G + g, &full_bar[s]);
+        tma_load_3d(sa + BM * BK * 2, &tmB, kb * BK, n0, a.b_shared ? g : q * P.G + g, &full_bar[s]);
+      }
+      if (!ok) atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      bool ok = true;
+      for (int it = 0; it < total_kb && ok; ++it) {
+        const int q = it / a.nkb, kb = it - q * a.nkb;
+        const int s = it % stages;
+        ok = mbar_wait_bounded(&full_bar[s], (uint32_t)((it / stages) & 1));
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t sa = smem_u32(tiles + (size_t)s * STAGE_BYTES);
+        const uint64_t da = make_desc(sa), db = make_desc(sa + BM * BK * 2);
+#pragma unroll
+        for (int kk = 0; kk < BK / 16; ++kk)
+          tc_mma_bf16(tmem_base + (uint32_t)(q * BN), da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), IDESC,
+                      (kb | kk) != 0 ? 1u : 0u);
+        tc_commit(&empty_bar[s]);
+      }
+      if (ok)
+        tc_commit(&accum_bar);
+      else
+        atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
+    }
+  } else {
+    const int quad = warp & 3;
+    float* stg = stage_all + (size_t)quad * 32 * DW_PITCH;
+    double local = 0.0;
+    bool ok = mbar_wait_bounded(&accum_bar, 0u);
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok) {
+      tc_fence_after();
+      float* fresh = P.fresh + (long long)g * P.p_pad + a.c_off;
+      float* stale = P.stale ? P.stale + (long long)g * P.p_pad + a.c_off : nullptr;
+      const int mrow = m0 + quad * 32;  // first row of this warp
+      const bool vec_ok = ((a.c_off | a.ldc) & 3) == 0 && (reinterpret_cast<uintptr_t>(P.fresh) & 15) == 0 &&
+                          (P.p_pad & 3) == 0;
+#pragma unroll 1
+      for (int c = 0; c < BN; c += 32) {
+        uint32_t v0[32], v1[32];
+        tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)c, v0);
+        tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(BN + c), v1);
+        const int nc = n0 + c;
+        if (nc >= a.N) break;
+        const bool row_ok = mrow + lane < a.M;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const float d = __uint_as_float(v0[j]) - __uint_as_float(v1[j]);
+          if (row_ok && nc + j < a.N) local += (double)d * (double)d;
+        }
+        for (int pass = 0; pass < (stale ? 2 : 1); ++pass) {
+          const uint32_t* v = pass == 0 ? v0 : v1;
+          float* out = pass == 0 ? fresh : stale;
+          __syncwarp();
+#pragma unroll
+          for (int j = 0; j < 32; j += 4)
+            *reinterpret_cast<float4*>(stg + lane * DW_PITCH + j) =
+                make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]),
+                            __uint_as_float(v[j + 3]));
+          __syncwarp();
+          // lanes 8r..8r+7 write the 128 bytes of one row
+          const int rr = lane >> 3, c4 = (lane & 7) * 4;
+#pragma unroll
+          for (int r0 = 0; r0 < 32; r0 += 4) {
+            const int r = r0 + rr;
+            const int m = mrow + r;
+            if (m >= a.M) continue;
+            const float4 t = *reinterpret_cast<const float4*>(stg + r * DW_PITCH + c4);
+            float* dst = out + (long long)m * a.ldc + nc + c4;
+            if (vec_ok && nc + c4 + 3 < a.N) {
+              *reinterpret_cast<float4*>(dst) = t;
+            } else {
+              const float tt[4] = {t.x, t.y, t.z, t.w};
+              for (int e = 0; e < 4 && nc + c4 + e < a.N; ++e) dst[e] = tt[e];
+            }
+          }
+        }
+      }
+    } else if (lane == 0) {
+      atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
+    }
+    local = warp_sum(local);
+    if (lane == 0) norm_sm[quad] = local;
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const double t = (norm_sm[0] + norm_sm[1]) + (norm_sm[2] + norm_sm[3]);
+    P.lhs_part[(long long)g * a.n_parts + a.part_base + blockIdx.y * gridDim.x + blockIdx.x] = t;
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)(2 * BN))
+                 : "memory");
+  }
+}
+
 // ----------------------------------------------------------------- weights -> bf16 (both orientations)
 // grid (col tiles, row tiles, layer-1); 32 x 32 tiles through shared memory.
 struct ConvArgs {
@@ -433,20 +598,37 @@ __global__ void __launch_bounds__(256) bf16_softmax_grad_kernel(const Params P, 
 }
 
 // ----------------------------------------------------------------- bias gradients
+// db_l at both points (column sums of dz_l over the group's rows), their
+// squared difference summed per block into the block's lhs_part slot.
 struct BiasArgsB {
   const __nv_bfloat16* dz[MLP_MAX_LAYERS + 1];
   int n[MLP_MAX_LAYERS + 1], ld[MLP_MAX_LAYERS + 1];
   long long b_off[MLP_MAX_LAYERS + 1];
+  int part_base[MLP_MAX_LAYERS + 1];
+  int n_parts;
 };
 __global__ void __launch_bounds__(256) bf16_bias_grad_kernel(const Params P, const BiasArgsB a, int Bp) {
+  __shared__ double scratch[40];
   const int l = blockIdx.z + 1;
+  if ((int)blockIdx.x * 256 >= a.n[l]) return;
   const int n = blockIdx.x * 256 + threadIdx.x;
-  if (n >= a.n[l]) return;
-  const int z = blockIdx.y, q = z / P.G, g = z - q * P.G;
-  const __nv_bfloat16* src = a.dz[l] + ((long long)z * Bp) * a.ld[l] + n;
-  float s = 0.f;
-  for (int r = 0; r < Bp; ++r) s += __bfloat162float(src[(long long)r * a.ld[l]]);
-  ((q == 0 ? P.fresh : P.stale) + (long long)g * P.p_pad + a.b_off[l])[n] = s;
+  const int g = blockIdx.y;
+  double d2 = 0.0;
+  if (n < a.n[l]) {
+    const long long rows = (long long)P.G * Bp;
+    const __nv_bfloat16* s0 = a.dz[l] + ((long long)g * Bp) * a.ld[l] + n;
+    const __nv_bfloat16* s1 = s0 + rows * a.ld[l];
+    float f = 0.f, s = 0.f;
+    for (int r = 0; r < Bp; ++r) {
+      f += __bfloat162float(s0[(long long)r * a.ld[l]]);
+      s += __bfloat162float(s1[(long long)r * a.ld[l]]);
+    }
+    (P.fresh + (long long)g * P.p_pad + a.b_off[l])[n] = f;
+    if (P.stale) (P.stale + (long long)g * P.p_pad + a.b_off[l])[n] = s;
+    d2 = (double)(f - s) * (double)(f - s);
+  }
+  d2 = block_sum(d2, scratch);
+  if (threadIdx.x == 0) P.lhs_part[(long long)g * a.n_parts + a.part_base[l] + blockIdx.x] = d2;
 }
 
 // ----------------------------------------------------------------- host
@@ -517,6 +699,17 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
   }
   im->slot_elems = pos;
   im->bias_slot = bpos;
+  int parts = 0;
+  for (int l = 1; l <= L; ++l) {
+    im->dw_part_base[l] = parts;
+    parts += ((plan->dims[l] + BM - 1) / BM) * ((plan->dims[l - 1] + BN - 1) / BN);
+  }
+  for (int l = 1; l <= L; ++l) {
+    im->bias_part_base[l] = parts;
+    parts += (plan->dims[l] + 255) / 256;
+  }
+  im->n_parts = parts;
+  plan->norm_parts = parts;
   auto alloc = [&](void** q, size_t bytes) -> cudaError_t {
     cudaError_t e = cudaMalloc(q, bytes);
     if (e != cudaSuccess) return e;
@@ -573,6 +766,9 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
   }
   cudaError_t e = cudaFuncSetAttribute(bf16_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        MAX_STAGES * STAGE_BYTES + 1024);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(bf16_dw_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           MAX_STAGES * STAGE_BYTES + 1024 + 4 * 32 * DW_PITCH * 4);
   if (e != cudaSuccess) return e;
   plan->launches_per_iter = 3 + L + 1 + L + (L - 1);
   return cudaSuccess;
@@ -640,16 +836,23 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   ++n;
   for (int l = L; l >= 1; --l) {
-    GemmB w{};
+    DwArgs w{};
     w.M = pl.dims[l];
     w.N = pl.dims[l - 1];
     w.K = Bp;
-    w.a_shared = 0;
-    w.zb_mode = l == 1 ? ZB_GROUP : ZB_BATCH;
-    w.epi = EPI_DW;
+    w.b_shared = l == 1;
+    w.nkb = Bp / BK;
+    w.stages = 2 * w.nkb < 4 ? 2 * w.nkb : 4;
     w.c_off = pl.w_off[l];
     w.ldc = pl.dims[l - 1];
-    if ((e = launch_gemm(im->tm_dw_a[l], im->tm_dw_b[l], P, w, st)) != cudaSuccess) return e;
+    w.part_base = im->dw_part_base[l];
+    w.n_parts = im->n_parts;
+    {
+      dim3 grid((w.N + BN - 1) / BN, (w.M + BM - 1) / BM, G);
+      const size_t smem = (size_t)w.stages * STAGE_BYTES + 1024 + 4 * 32 * DW_PITCH * 4;
+      bf16_dw_kernel<<<grid, GEMM_THREADS, smem, st>>>(im->tm_dw_a[l], im->tm_dw_b[l], P, w);
+      if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
     ++n;
     if (l > 1) {
       GemmB d{};
@@ -677,9 +880,11 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
     ba.n[l] = pl.dims[l];
     ba.ld[l] = im->ld[l];
     ba.b_off[l] = pl.b_off[l];
+    ba.part_base[l] = im->bias_part_base[l];
     if (pl.dims[l] > maxn) maxn = pl.dims[l];
   }
-  bf16_bias_grad_kernel<<<dim3((maxn + 255) / 256, 2 * G, L), 256, 0, st>>>(P, ba, Bp);
+  ba.n_parts = im->n_parts;
+  bf16_bias_grad_kernel<<<dim3((maxn + 255) / 256, G, L), 256, 0, st>>>(P, ba, Bp);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   ++n;
   *n_launches = n;

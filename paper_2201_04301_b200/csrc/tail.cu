@@ -35,66 +35,69 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
   const long long k = P.st->k;
 
   // ---- phase 1: partial sums -> fresh_g (and stale_g), innovation norm
-  int c_lo = 0, c_hi = -1;
-  const long long Rtot = (long long)P.G * P.pm.rows_per_group;
-  const int n = P.pm.n_cta;
-  if (n > 0) {
-    const long long x0 = (long long)g * P.pm.rows_per_group;
-    const long long x1 = x0 + P.pm.rows_per_group - 1;
-    c_lo = (int)(((x0 + 1) * n - 1) / Rtot);
-    c_hi = (int)(((x1 + 1) * n - 1) / Rtot);
-  }
-  double local = 0.0;
-#pragma unroll
-  for (int u = 0; u < U; ++u) {
-    const long long i4 = ((long long)blockIdx.x * U + u) * 256 + tid;
-    if (i4 >= cols4) continue;
-    float4 f, s;
+  // (skipped when the gradient kernels have already delivered the norm partial sums)
+  if (P.pm.n_cta >= 0) {
+    int c_lo = 0, c_hi = -1;
+    const long long Rtot = (long long)P.G * P.pm.rows_per_group;
+    const int n = P.pm.n_cta;
     if (n > 0) {
-      f = make_float4(0.f, 0.f, 0.f, 0.f);
-      s = f;
-      for (int c0 = c_lo; c0 <= c_hi; c0 += 4) {  // four partial sums per round: loads first, adds in CTA order
-        float4 a[4], b[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const int c = c0 + u;
-          if (c <= c_hi) {
-            const int gf = (int)(((long long)c * Rtot / n) / P.pm.rows_per_group);
-            const float* src = P.partial + ((long long)(c * P.pm.maxseg + (g - gf)) * 2) * P.p_pad + i4 * 4;
-            a[u] = ld4(src);
-            b[u] = ld4(src + P.p_pad);
-          }
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          if (c0 + u <= c_hi) {
-            f.x += a[u].x; f.y += a[u].y; f.z += a[u].z; f.w += a[u].w;
-            s.x += b[u].x; s.y += b[u].y; s.z += b[u].z; s.w += b[u].w;
-          }
-        }
-      }
-      // second slot half = innovation; the stale-point gradient is fresh - innovation
-      st4(P.fresh + (long long)g * P.p_pad + i4 * 4, f);
-      if (P.stale)
-        st4(P.stale + (long long)g * P.p_pad + i4 * 4, make_float4(f.x - s.x, f.y - s.y, f.z - s.z, f.w - s.w));
-    } else {
-      f = ld4(P.fresh + (long long)g * P.p_pad + i4 * 4);
-      s = ld4(P.stale + (long long)g * P.p_pad + i4 * 4);
-      s = make_float4(f.x - s.x, f.y - s.y, f.z - s.z, f.w - s.w);
+      const long long x0 = (long long)g * P.pm.rows_per_group;
+      const long long x1 = x0 + P.pm.rows_per_group - 1;
+      c_lo = (int)(((x0 + 1) * n - 1) / Rtot);
+      c_hi = (int)(((x1 + 1) * n - 1) / Rtot);
     }
-    const float dx = s.x, dy = s.y, dz = s.z, dw = s.w;  // the innovation
-    local += (double)dx * dx + (double)dy * dy + (double)dz * dz + (double)dw * dw;
-  }
-  const double tot = block_sum(local, scratch);
-  if (tid == 0) {
-    P.lhs_part[(long long)g * blocks_x + blockIdx.x] = tot;
+    double local = 0.0;
+  #pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const long long i4 = ((long long)blockIdx.x * U + u) * 256 + tid;
+      if (i4 >= cols4) continue;
+      float4 f, s;
+      if (n > 0) {
+        f = make_float4(0.f, 0.f, 0.f, 0.f);
+        s = f;
+        for (int c0 = c_lo; c0 <= c_hi; c0 += 4) {  // four partial sums per round: loads first, adds in CTA order
+          float4 a[4], b[4];
+  #pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const int c = c0 + u;
+            if (c <= c_hi) {
+              const int gf = (int)(((long long)c * Rtot / n) / P.pm.rows_per_group);
+              const float* src = P.partial + ((long long)(c * P.pm.maxseg + (g - gf)) * 2) * P.p_pad + i4 * 4;
+              a[u] = ld4(src);
+              b[u] = ld4(src + P.p_pad);
+            }
+          }
+  #pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            if (c0 + u <= c_hi) {
+              f.x += a[u].x; f.y += a[u].y; f.z += a[u].z; f.w += a[u].w;
+              s.x += b[u].x; s.y += b[u].y; s.z += b[u].z; s.w += b[u].w;
+            }
+          }
+        }
+        // second slot half = innovation; the stale-point gradient is fresh - innovation
+        st4(P.fresh + (long long)g * P.p_pad + i4 * 4, f);
+        if (P.stale)
+          st4(P.stale + (long long)g * P.p_pad + i4 * 4, make_float4(f.x - s.x, f.y - s.y, f.z - s.z, f.w - s.w));
+      } else {
+        f = ld4(P.fresh + (long long)g * P.p_pad + i4 * 4);
+        s = ld4(P.stale + (long long)g * P.p_pad + i4 * 4);
+        s = make_float4(f.x - s.x, f.y - s.y, f.z - s.z, f.w - s.w);
+      }
+      const float dx = s.x, dy = s.y, dz = s.z, dw = s.w;  // the innovation
+      local += (double)dx * dx + (double)dy * dy + (double)dz * dz + (double)dw * dw;
+    }
+    const double tot = block_sum(local, scratch);
+    if (tid == 0) {
+      P.lhs_part[(long long)g * blocks_x + blockIdx.x] = tot;
+      __threadfence();
+      const unsigned int total = (unsigned int)blocks_x * (unsigned int)P.G;
+      is_last = atomicAdd(&P.st->ticket_select, 1u) == total - 1u;
+    }
+    __syncthreads();
+    if (!is_last) return;
     __threadfence();
-    const unsigned int total = (unsigned int)blocks_x * (unsigned int)P.G;
-    is_last = atomicAdd(&P.st->ticket_select, 1u) == total - 1u;
   }
-  __syncthreads();
-  if (!is_last) return;
-  __threadfence();
 
   // ---- phase 2 (last block only): the server's scheduling decision.
   // One thread per group, 256 groups at a time; everything a group needs is
@@ -342,6 +345,10 @@ void plan_tail(long long p_pad, int G, int sm_count, TailPlan* plan) {
 }
 
 cudaError_t launch_select(const Params& P, const TailPlan& plan, cudaStream_t st) {
+  if (P.pm.n_cta < 0) {  // norm partial sums already in lhs_part: only the scheduling phase remains
+    select_kernel<1><<<dim3(1, 1), 256, 0, st>>>(P, P.pm.maxseg);
+    return cudaGetLastError();
+  }
   dim3 grid(plan.select_blocks_x, P.G);
   if (plan.select_cols4_per_block == 256)
     select_kernel<1><<<grid, 256, 0, st>>>(P, plan.select_blocks_x);
