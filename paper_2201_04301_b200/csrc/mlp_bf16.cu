@@ -317,49 +317,63 @@ __global__ void __launch_bounds__(GEMM_THREADS) bf16_gemm_kernel(const __grid_co
 
 // ----------------------------------------------------------------- weight gradients, both points in one CTA
 // dW_l of one group at theta^k (accumulator 0) and at the stale iterate
-// (accumulator 1) for one 128 x 128 tile.  The epilogue writes the fresh
-// gradient (and the stale one only when it is kept for inspection), forms the
-// squared norm of their difference - this tile's share of the left side of
-// Eq. (9) - and stores it in the tile's own slot of lhs_part, so the
-// per-group gradients are never re-read to build the test.  Rows reach
-// global memory as full 128-byte lines through a per-warp staging tile.
+// (accumulator 1), 128 x 128 tiles.  The epilogue writes the fresh gradient
+// (and the stale one only when it is kept for inspection), forms the squared
+// norm of their difference - the tile's share of the left side of Eq. (9) -
+// and stores it in the tile's own slot of lhs_part, so the per-group
+// gradients are never re-read to build the test.
+//
+// Persistent: one CTA per SM walks tiles t = blockIdx.x, + gridDim.x, ...;
+// tensor memory holds two accumulator pairs (2 x 256 columns) so that the
+// eight epilogue warps drain tile i while the producer and the MMA warp work
+// on tile i+1.  Rows reach global memory as full 128-byte lines through a
+// per-warp staging tile.
 struct DwArgs {
   int M, N, K;            // n_l, n_{l-1}, padded rows per group
   int b_shared;           // 1: operand B has one entry per group (the gathered features)
   int nkb;                // K blocks per point
   int stages;
+  int tiles_m, tiles_n, total_tiles;
   long long c_off, ldc;   // position of W_l inside the gradient vector, row stride
   int part_base, n_parts; // this layer's first slot in lhs_part and slots per group
 };
 
-constexpr int DW_PITCH = 36;  // floats per staged row (16-byte aligned, conflict-free 16-byte stores)
+constexpr int DW_PITCH = 36;   // floats per staged row (16-byte aligned, conflict-free 16-byte stores)
+constexpr int DW_EPI_WARPS = 8;
+constexpr int DW_THREADS = 64 + 32 * DW_EPI_WARPS;
+constexpr int DW_STAGE_FLOATS = DW_EPI_WARPS * 32 * DW_PITCH;
 
-__global__ void __launch_bounds__(GEMM_THREADS) bf16_dw_kernel(const __grid_constant__ CUtensorMap tmA,
-                                                               const __grid_constant__ CUtensorMap tmB,
-                                                               const Params P, const DwArgs a) {
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+__global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_constant__ CUtensorMap tmA,
+                                                                const __grid_constant__ CUtensorMap tmB,
+                                                                const Params P, const DwArgs a) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
-  __shared__ uint64_t full_bar[MAX_STAGES], empty_bar[MAX_STAGES], accum_bar;
+  __shared__ uint64_t full_bar[MAX_STAGES], empty_bar[MAX_STAGES], tfull_bar[2], tempty_bar[2];
   __shared__ uint32_t tmem_base_sm;
-  __shared__ double norm_sm[4];
+  __shared__ double norm_sm[2][DW_EPI_WARPS];
   unsigned char* tiles = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   float* stage_all = reinterpret_cast<float*>(tiles + (size_t)a.stages * STAGE_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int g = blockIdx.z;
-  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
   const int stages = a.stages;
-  const int total_kb = 2 * a.nkb;
+  const int kb_per_tile = 2 * a.nkb;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) {
       mbar_init(&full_bar[s], 1);
       mbar_init(&empty_bar[s], 1);
     }
-    mbar_init(&accum_bar, 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&tfull_bar[s], 1);
+      mbar_init(&tempty_bar[s], DW_EPI_WARPS);
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) {  // two fp32 accumulators of BN columns each
+  if (warp == 1) {  // all 512 columns: two slots of two fp32 accumulators
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_sm)),
-                 "r"((uint32_t)(2 * BN))
+                 "r"(512u)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -371,110 +385,135 @@ __global__ void __launch_bounds__(GEMM_THREADS) bf16_dw_kernel(const __grid_cons
   if (warp == 0) {
     if (lane == 0) {
       bool ok = true;
-      for (int it = 0; it < total_kb && ok; ++it) {
-        const int q = it / a.nkb, kb = it - q * a.nkb;
-        const int s = it % stages;
-        ok = mbar_wait_bounded(&empty_bar[s], (uint32_t)(((it / stages) & 1) ^ 1));
-        if (!ok) break;
-        unsigned char* sa = tiles + (size_t)s * STAGE_BYTES;
-        mbar_expect_tx(&full_bar[s], STAGE_BYTES);
-        tma_load_3d(sa, &tmA, kb * BK, m0, q * P.G + g, &full_bar[s]);
-        tma_load_3d(sa + BM * BK * 2, &tmB, kb * BK, n0, a.b_shared ? g : q * P.G + g, &full_bar[s]);
+      int it = 0;
+      for (int t = blockIdx.x; t < a.total_tiles && ok; t += gridDim.x) {
+        const int nt = t % a.tiles_n, mt = (t / a.tiles_n) % a.tiles_m, g = t / (a.tiles_n * a.tiles_m);
+        for (int j = 0; j < kb_per_tile && ok; ++j, ++it) {
+          const int q = j / a.nkb, kb = j - q * a.nkb;
+          const int s = it % stages;
+          ok = mbar_wait_bounded(&empty_bar[s], (uint32_t)(((it / stages) & 1) ^ 1));
+          if (!ok) break;
+          unsigned char* sa = tiles + (size_t)s * STAGE_BYTES;
+          mbar_expect_tx(&full_bar[s], STAGE_BYTES);
+          tma_load_3d(sa, &tmA, kb * BK, mt * BM, q * P.G + g, &full_bar[s]);
+          tma_load_3d(sa + BM * BK * 2, &tmB, kb * BK, nt * BN, a.b_shared ? g : q * P.G + g, &full_bar[s]);
+        }
       }
       if (!ok) atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
     }
   } else if (warp == 1) {
     if (lane == 0) {
       bool ok = true;
-      for (int it = 0; it < total_kb && ok; ++it) {
-        const int q = it / a.nkb, kb = it - q * a.nkb;
-        const int s = it % stages;
-        ok = mbar_wait_bounded(&full_bar[s], (uint32_t)((it / stages) & 1));
+      int it = 0, i = 0;
+      for (int t = blockIdx.x; t < a.total_tiles && ok; t += gridDim.x, ++i) {
+        const int slot = i & 1;
+        ok = mbar_wait_bounded(&tempty_bar[slot], (uint32_t)(((i >> 1) & 1) ^ 1));  // epilogue has drained the slot
         if (!ok) break;
         tc_fence_after();
-        const uint32_t sa = smem_u32(tiles + (size_t)s * STAGE_BYTES);
-        const uint64_t da = make_desc(sa), db = make_desc(sa + BM * BK * 2);
+        for (int j = 0; j < kb_per_tile && ok; ++j, ++it) {
+          const int q = j / a.nkb, kb = j - q * a.nkb;
+          const int s = it % stages;
+          ok = mbar_wait_bounded(&full_bar[s], (uint32_t)((it / stages) & 1));
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t sa = smem_u32(tiles + (size_t)s * STAGE_BYTES);
+          const uint64_t da = make_desc(sa), db = make_desc(sa + BM * BK * 2);
 #pragma unroll
-        for (int kk = 0; kk < BK / 16; ++kk)
-          tc_mma_bf16(tmem_base + (uint32_t)(q * BN), da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), IDESC,
-                      (kb | kk) != 0 ? 1u : 0u);
-        tc_commit(&empty_bar[s]);
+          for (int kk = 0; kk < BK / 16; ++kk)
+            tc_mma_bf16(tmem_base + (uint32_t)(slot * 2 * BN + q * BN), da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2),
+                        IDESC, (kb | kk) != 0 ? 1u : 0u);
+          tc_commit(&empty_bar[s]);
+        }
+        if (ok) tc_commit(&tfull_bar[slot]);
       }
-      if (ok)
-        tc_commit(&accum_bar);
-      else
-        atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
+      if (!ok) atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
     }
   } else {
-    const int quad = warp & 3;
-    float* stg = stage_all + (size_t)quad * 32 * DW_PITCH;
-    double local = 0.0;
-    bool ok = mbar_wait_bounded(&accum_bar, 0u);
-    ok = __all_sync(0xffffffffu, ok);
-    if (ok) {
-      tc_fence_after();
-      float* fresh = P.fresh + (long long)g * P.p_pad + a.c_off;
-      float* stale = P.stale ? P.stale + (long long)g * P.p_pad + a.c_off : nullptr;
-      const int mrow = m0 + quad * 32;  // first row of this warp
-      const bool vec_ok = ((a.c_off | a.ldc) & 3) == 0 && (reinterpret_cast<uintptr_t>(P.fresh) & 15) == 0 &&
-                          (P.p_pad & 3) == 0;
+    const int ew = warp - 2;           // 0..7
+    const int quad = warp & 3;         // TMEM lanes this warp may read
+    const int half = ew >> 2;          // which 64 columns of the tile
+    float* stg = stage_all + (size_t)ew * 32 * DW_PITCH;
+    const bool vec_ok = ((a.c_off | a.ldc) & 3) == 0 && (reinterpret_cast<uintptr_t>(P.fresh) & 15) == 0 &&
+                        (P.p_pad & 3) == 0;
+    bool ok = true;
+    int i = 0;
+    for (int t = blockIdx.x; t < a.total_tiles; t += gridDim.x, ++i) {
+      const int slot = i & 1;
+      const int nt = t % a.tiles_n, mt = (t / a.tiles_n) % a.tiles_m, g = t / (a.tiles_n * a.tiles_m);
+      double local = 0.0;
+      if (ok) {
+        ok = mbar_wait_bounded(&tfull_bar[slot], (uint32_t)((i >> 1) & 1));
+        ok = __all_sync(0xffffffffu, ok);
+      }
+      if (ok) {
+        tc_fence_after();
+        float* fresh = P.fresh + (long long)g * P.p_pad + a.c_off;
+        float* stale = P.stale ? P.stale + (long long)g * P.p_pad + a.c_off : nullptr;
+        const int mrow = mt * BM + quad * 32;
+        const uint32_t tbase = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(slot * 2 * BN);
 #pragma unroll 1
-      for (int c = 0; c < BN; c += 32) {
-        uint32_t v0[32], v1[32];
-        tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)c, v0);
-        tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(BN + c), v1);
-        const int nc = n0 + c;
-        if (nc >= a.N) break;
-        const bool row_ok = mrow + lane < a.M;
+        for (int c = half * 64; c < half * 64 + 64; c += 32) {
+          uint32_t v0[32], v1[32];
+          tc_ld32(tbase + (uint32_t)c, v0);
+          tc_ld32(tbase + (uint32_t)(BN + c), v1);
+          const int nc = nt * BN + c;
+          if (nc >= a.N) break;
+          const bool row_ok = mrow + lane < a.M;
+          float part = 0.f;
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const float d = __uint_as_float(v0[j]) - __uint_as_float(v1[j]);
-          if (row_ok && nc + j < a.N) local += (double)d * (double)d;
-        }
-        for (int pass = 0; pass < (stale ? 2 : 1); ++pass) {
-          const uint32_t* v = pass == 0 ? v0 : v1;
-          float* out = pass == 0 ? fresh : stale;
-          __syncwarp();
+          for (int j = 0; j < 32; ++j) {
+            const float d = __uint_as_float(v0[j]) - __uint_as_float(v1[j]);
+            if (row_ok && nc + j < a.N) part += d * d;
+          }
+          local += (double)part;
+          for (int pass = 0; pass < (stale ? 2 : 1); ++pass) {
+            const uint32_t* v = pass == 0 ? v0 : v1;
+            float* out = pass == 0 ? fresh : stale;
+            __syncwarp();
 #pragma unroll
-          for (int j = 0; j < 32; j += 4)
-            *reinterpret_cast<float4*>(stg + lane * DW_PITCH + j) =
-                make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]),
-                            __uint_as_float(v[j + 3]));
-          __syncwarp();
-          // lanes 8r..8r+7 write the 128 bytes of one row
-          const int rr = lane >> 3, c4 = (lane & 7) * 4;
+            for (int j = 0; j < 32; j += 4)
+              *reinterpret_cast<float4*>(stg + lane * DW_PITCH + j) =
+                  make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]),
+                              __uint_as_float(v[j + 3]));
+            __syncwarp();
+            const int rr = lane >> 3, c4 = (lane & 7) * 4;  // lanes 8r..8r+7 write the 128 bytes of one row
 #pragma unroll
-          for (int r0 = 0; r0 < 32; r0 += 4) {
-            const int r = r0 + rr;
-            const int m = mrow + r;
-            if (m >= a.M) continue;
-            const float4 t = *reinterpret_cast<const float4*>(stg + r * DW_PITCH + c4);
-            float* dst = out + (long long)m * a.ldc + nc + c4;
-            if (vec_ok && nc + c4 + 3 < a.N) {
-              *reinterpret_cast<float4*>(dst) = t;
-            } else {
-              const float tt[4] = {t.x, t.y, t.z, t.w};
-              for (int e = 0; e < 4 && nc + c4 + e < a.N; ++e) dst[e] = tt[e];
+            for (int r0 = 0; r0 < 32; r0 += 4) {
+              const int r = r0 + rr;
+              const int m = mrow + r;
+              if (m >= a.M) continue;
+              const float4 tv = *reinterpret_cast<const float4*>(stg + r * DW_PITCH + c4);
+              float* dst = out + (long long)m * a.ldc + nc + c4;
+              if (vec_ok && nc + c4 + 3 < a.N) {
+                *reinterpret_cast<float4*>(dst) = tv;
+              } else {
+                const float tt[4] = {tv.x, tv.y, tv.z, tv.w};
+                for (int e = 0; e < 4 && nc + c4 + e < a.N; ++e) dst[e] = tt[e];
+              }
             }
           }
         }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&tempty_bar[slot]);  // this warp is done with the slot's tensor memory
       }
-    } else if (lane == 0) {
-      atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
+      local = warp_sum(local);
+      if (lane == 0) norm_sm[slot][ew] = local;
+      asm volatile("bar.sync 1, %0;" ::"n"(32 * DW_EPI_WARPS) : "memory");
+      if (ew == 0 && lane == 0) {
+        double tsum = 0.0;
+#pragma unroll
+        for (int w = 0; w < DW_EPI_WARPS; ++w) tsum += norm_sm[slot][w];
+        P.lhs_part[(long long)g * a.n_parts + a.part_base + mt * a.tiles_n + nt] = tsum;
+      }
     }
-    local = warp_sum(local);
-    if (lane == 0) norm_sm[quad] = local;
+    if (!ok && lane == 0) atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
   }
   tc_fence_before();
   __syncthreads();
-  if (threadIdx.x == 0) {
-    const double t = (norm_sm[0] + norm_sm[1]) + (norm_sm[2] + norm_sm[3]);
-    P.lhs_part[(long long)g * a.n_parts + a.part_base + blockIdx.y * gridDim.x + blockIdx.x] = t;
-  }
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)(2 * BN))
-                 : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
   }
 }
 
@@ -768,7 +807,7 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
                                        MAX_STAGES * STAGE_BYTES + 1024);
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(bf16_dw_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           MAX_STAGES * STAGE_BYTES + 1024 + 4 * 32 * DW_PITCH * 4);
+                           4 * STAGE_BYTES + 1024 + DW_STAGE_FLOATS * 4);
   if (e != cudaSuccess) return e;
   plan->launches_per_iter = 3 + L + 1 + L + (L - 1);
   return cudaSuccess;
@@ -842,15 +881,18 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
     w.K = Bp;
     w.b_shared = l == 1;
     w.nkb = Bp / BK;
-    w.stages = 2 * w.nkb < 4 ? 2 * w.nkb : 4;
+    w.stages = 4;
+    w.tiles_m = (w.M + BM - 1) / BM;
+    w.tiles_n = (w.N + BN - 1) / BN;
+    w.total_tiles = w.tiles_m * w.tiles_n * G;
     w.c_off = pl.w_off[l];
     w.ldc = pl.dims[l - 1];
     w.part_base = im->dw_part_base[l];
     w.n_parts = im->n_parts;
     {
-      dim3 grid((w.N + BN - 1) / BN, (w.M + BM - 1) / BM, G);
-      const size_t smem = (size_t)w.stages * STAGE_BYTES + 1024 + 4 * 32 * DW_PITCH * 4;
-      bf16_dw_kernel<<<grid, GEMM_THREADS, smem, st>>>(im->tm_dw_a[l], im->tm_dw_b[l], P, w);
+      const int ctas = w.total_tiles < pl.sm_count ? w.total_tiles : pl.sm_count;
+      const size_t smem = (size_t)w.stages * STAGE_BYTES + 1024 + DW_STAGE_FLOATS * 4;
+      bf16_dw_kernel<<<ctas, DW_THREADS, smem, st>>>(im->tm_dw_a[l], im->tm_dw_b[l], P, w);
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
     ++n;
