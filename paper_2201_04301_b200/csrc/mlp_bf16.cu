@@ -12,10 +12,10 @@
 // which is why activations, dz and the weights are kept in both orientations
 // (the epilogues write the second orientation for free).
 //
-// Kernel: one CTA per 128 x 128 output tile; warp 0 = TMA producer
+// Kernels: persistent CTAs, one per SM; warp 0 = TMA producer
 // (cp.async.bulk.tensor, 128-byte swizzle, mbarrier ring), warp 1 = MMA issuer
-// (tcgen05.mma, cta_group::1, 128x128x16 bf16 -> fp32 in TMEM), warps 2-5 =
-// epilogue (tcgen05.ld, fused bias / ReLU / ReLU-mask, stores).  A group's
+// (tcgen05.mma, cta_group::1, bf16 -> fp32 in TMEM, two accumulator slots),
+// warps 2-9 = epilogue (tcgen05.ld, fused bias / ReLU / ReLU-mask, stores).  A group's
 // minibatch is padded to a multiple of 128 rows, so an M tile never mixes
 // groups and the stale-point weights of a tile are one slot of the bf16
 // weight ring.  Every wait is bounded; a timeout raises the device error word.
@@ -31,7 +31,6 @@ namespace {
 constexpr int BM = 128, BN = 128, BK = 64;      // tile; BK * 2 bytes = one 128-byte swizzle row
 constexpr int MAX_STAGES = 6;
 constexpr int STAGE_BYTES = (BM + BN) * BK * 2;  // 32 KiB
-constexpr int GEMM_THREADS = 192;
 
 enum { EPI_HIDDEN = 0, EPI_SCORES = 1, EPI_DA = 2, EPI_DW = 3 };
 enum { ZB_BATCH = 0, ZB_GROUP = 1, ZB_RING = 2 };
@@ -158,32 +157,49 @@ __device__ __forceinline__ int ring_slot(const Params& P, int g, int q, long lon
   return (int)(j % (P.D + 1));
 }
 
-// ----------------------------------------------------------------- GEMM
-__global__ void __launch_bounds__(GEMM_THREADS) bf16_gemm_kernel(const __grid_constant__ CUtensorMap tmA,
+// ----------------------------------------------------------------- GEMM (forward and backward-data products)
+// Persistent: one CTA per SM walks 128 x 256 output tiles (N fastest, so that
+// the CTAs running together share operand tiles in L2); tensor memory holds
+// two 256-column accumulators, so the eight epilogue warps drain tile i while
+// the producer and the MMA warp work on tile i+1.
+constexpr int GN = 256;                                  // N tile of this kernel
+constexpr int G_STAGE_BYTES = (BM + GN) * BK * 2;        // 48 KiB
+constexpr int G_STAGES = 4;
+constexpr int G_EPI_WARPS = 8;
+constexpr int G_THREADS = 64 + 32 * G_EPI_WARPS;
+constexpr uint32_t IDESC_G = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(GN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+__global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_constant__ CUtensorMap tmA,
                                                                  const __grid_constant__ CUtensorMap tmB,
                                                                  const Params P, const GemmB a) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
-  __shared__ uint64_t full_bar[MAX_STAGES], empty_bar[MAX_STAGES], accum_bar;
+  __shared__ uint64_t full_bar[G_STAGES], empty_bar[G_STAGES], tfull_bar[2], tempty_bar[2];
   __shared__ uint32_t tmem_base_sm;
   unsigned char* tiles = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int z = blockIdx.z, q = z / P.G, g = z - q * P.G;
-  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
   const int nkb = (a.K + BK - 1) / BK;
-  const int stages = a.stages;
+  const int tiles_n = (a.N + GN - 1) / GN, tiles_m = (a.M + BM - 1) / BM;
+  const int total_tiles = tiles_n * tiles_m * 2 * P.G;
   const long long k_it = P.st->k;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < stages; ++s) {
+    for (int s = 0; s < G_STAGES; ++s) {
       mbar_init(&full_bar[s], 1);
       mbar_init(&empty_bar[s], 1);
     }
-    mbar_init(&accum_bar, 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&tfull_bar[s], 1);
+      mbar_init(&tempty_bar[s], G_EPI_WARPS);
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) {  // TMEM: 128 lanes x BN fp32 columns
+  if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_sm)),
-                 "r"((uint32_t)BN)
+                 "r"(512u)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -194,75 +210,83 @@ __global__ void __launch_bounds__(GEMM_THREADS) bf16_gemm_kernel(const __grid_co
 
   if (warp == 0) {
     if (lane == 0) {
-      const int zA = a.a_shared ? g : z;
-      const int zB = a.zb_mode == ZB_RING ? ring_slot(P, g, q, k_it) : (a.zb_mode == ZB_GROUP ? g : z);
       bool ok = true;
-      for (int kb = 0; kb < nkb && ok; ++kb) {
-        const int s = kb % stages;
-        ok = mbar_wait_bounded(&empty_bar[s], (uint32_t)(((kb / stages) & 1) ^ 1));
-        if (!ok) break;
-        unsigned char* sa = tiles + (size_t)s * STAGE_BYTES;
-        mbar_expect_tx(&full_bar[s], STAGE_BYTES);
-        tma_load_3d(sa, &tmA, kb * BK, m0, zA, &full_bar[s]);
-        tma_load_3d(sa + BM * BK * 2, &tmB, kb * BK, n0, zB, &full_bar[s]);
+      int it = 0;
+      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        const int nt = t % tiles_n, mt = (t / tiles_n) % tiles_m, z = t / (tiles_n * tiles_m);
+        const int q = z / P.G, g = z - q * P.G;
+        const int zA = a.a_shared ? g : z;
+        const int zB = a.zb_mode == ZB_RING ? ring_slot(P, g, q, k_it) : (a.zb_mode == ZB_GROUP ? g : z);
+        for (int kb = 0; kb < nkb && ok; ++kb, ++it) {
+          const int s = it % G_STAGES;
+          ok = mbar_wait_bounded(&empty_bar[s], (uint32_t)(((it / G_STAGES) & 1) ^ 1));
+          if (!ok) break;
+          unsigned char* sa = tiles + (size_t)s * G_STAGE_BYTES;
+          mbar_expect_tx(&full_bar[s], G_STAGE_BYTES);
+          tma_load_3d(sa, &tmA, kb * BK, mt * BM, zA, &full_bar[s]);
+          tma_load_3d(sa + BM * BK * 2, &tmB, kb * BK, nt * GN, zB, &full_bar[s]);
+        }
       }
-      if (!ok) {
-        atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
-      }
+      if (!ok) atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
     }
   } else if (warp == 1) {
     if (lane == 0) {
       bool ok = true;
-      for (int kb = 0; kb < nkb && ok; ++kb) {
-        const int s = kb % stages;
-        ok = mbar_wait_bounded(&full_bar[s], (uint32_t)((kb / stages) & 1));
+      int it = 0, i = 0;
+      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++i) {
+        const int slot = i & 1;
+        ok = mbar_wait_bounded(&tempty_bar[slot], (uint32_t)(((i >> 1) & 1) ^ 1));
         if (!ok) break;
         tc_fence_after();
-        const uint32_t sa = smem_u32(tiles + (size_t)s * STAGE_BYTES);
-        const uint64_t da = make_desc(sa), db = make_desc(sa + BM * BK * 2);
+        for (int kb = 0; kb < nkb && ok; ++kb, ++it) {
+          const int s = it % G_STAGES;
+          ok = mbar_wait_bounded(&full_bar[s], (uint32_t)((it / G_STAGES) & 1));
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t sa = smem_u32(tiles + (size_t)s * G_STAGE_BYTES);
+          const uint64_t da = make_desc(sa), db = make_desc(sa + BM * BK * 2);
 #pragma unroll
-        for (int kk = 0; kk < BK / 16; ++kk)  // 16 bf16 = 32 bytes = 2 descriptor units per MMA
-          tc_mma_bf16(tmem_base, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), IDESC, (kb | kk) != 0 ? 1u : 0u);
-        tc_commit(&empty_bar[s]);  // frees the stage once these MMAs have read it
+          for (int kk = 0; kk < BK / 16; ++kk)  // 16 bf16 = 32 bytes = 2 descriptor units per MMA
+            tc_mma_bf16(tmem_base + (uint32_t)(slot * GN), da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), IDESC_G,
+                        (kb | kk) != 0 ? 1u : 0u);
+          tc_commit(&empty_bar[s]);  // frees the stage once these MMAs have read it
+        }
+        if (ok) tc_commit(&tfull_bar[slot]);
       }
-      if (ok) {
-        tc_commit(&accum_bar);
-      } else {
-        atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
-      }
+      if (!ok) atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
     }
   } else {
-    // epilogue: warp w may touch TMEM lanes 32*(w%4) .. +31
+    // epilogue: warp w may touch TMEM lanes 32*(w%4) .. +31; the two warps of a quadrant split the columns
+    const int ew = warp - 2;
     const int quad = warp & 3;
-    const int m = m0 + quad * 32 + lane;
-    bool ok = mbar_wait_bounded(&accum_bar, 0u);
-    ok = __all_sync(0xffffffffu, ok);
-    if (ok) {
+    const int half = ew >> 2;
+    bool ok = true;
+    int i = 0;
+    for (int t = blockIdx.x; t < total_tiles; t += gridDim.x, ++i) {
+      const int slot = i & 1;
+      const int nt = t % tiles_n, mt = (t / tiles_n) % tiles_m, z = t / (tiles_n * tiles_m);
+      const int q = z / P.G, g = z - q * P.G;
+      if (ok) {
+        ok = mbar_wait_bounded(&tfull_bar[slot], (uint32_t)((i >> 1) & 1));
+        ok = __all_sync(0xffffffffu, ok);
+      }
+      if (!ok) continue;
       tc_fence_after();
+      const int m = mt * BM + quad * 32 + lane;
+      const int n0 = nt * GN;
       const float* bias = nullptr;
       if (a.epi == EPI_HIDDEN || a.epi == EPI_SCORES)
         bias = a.bias_ring + (long long)ring_slot(P, g, q, k_it) * a.bias_slot + a.bias_pos;
+      const uint32_t tbase = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(slot * GN);
 #pragma unroll 1
-      for (int c = 0; c < BN; c += 32) {
-        uint32_t v[32];
-        tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)c, v);
+      for (int c = half * (GN / 2); c < (half + 1) * (GN / 2); c += 32) {
         const int nc = n0 + c;
-        if (nc >= a.N) break;  // uniform across the CTA
+        if (nc >= a.N) break;  // uniform across the warp
+        uint32_t v[32];
+        tc_ld32(tbase + (uint32_t)c, v);
         const bool row_ok = m < a.M;
         const bool full = nc + 32 <= a.N;
-        if (a.epi == EPI_DW) {
-          float* dst = (q == 0 ? P.fresh : P.stale) + (long long)g * P.p_pad + a.c_off + (long long)m * a.ldc + nc;
-          if (row_ok) {
-            if (full && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0)) {
-#pragma unroll
-              for (int j = 0; j < 32; j += 4)
-                *reinterpret_cast<float4*>(dst + j) = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
-                                                                  __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
-            } else {
-              for (int j = 0; j < 32 && nc + j < a.N; ++j) dst[j] = __uint_as_float(v[j]);
-            }
-          }
-        } else if (a.epi == EPI_SCORES) {
+        if (a.epi == EPI_SCORES) {
           float* dst = a.out_f32 + ((long long)z * a.M + m) * a.N + nc;
           if (row_ok)
             for (int j = 0; j < 32 && nc + j < a.N; ++j) dst[j] = __uint_as_float(v[j]) + bias[nc + j];
@@ -273,10 +297,25 @@ __global__ void __launch_bounds__(GEMM_THREADS) bf16_gemm_kernel(const __grid_co
             for (int j = 0; j < 32; ++j) f[j] = fmaxf(__uint_as_float(v[j]) + (nc + j < a.N ? bias[nc + j] : 0.f), 0.f);
           } else {  // EPI_DA: ReLU derivative of the layer below
             const __nv_bfloat16* mk = a.mask + (long long)z * a.z_stride_out + (long long)m * a.ldo + nc;
+            if (full && row_ok) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              const bool on = row_ok && nc + j < a.N && __bfloat162float(mk[j]) > 0.f;
-              f[j] = on ? __uint_as_float(v[j]) : 0.f;
+              for (int j = 0; j < 32; j += 8) {
+                const uint4 pk = *reinterpret_cast<const uint4*>(mk + j);
+                const uint32_t wds[4] = {pk.x, pk.y, pk.z, pk.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  // a bf16 is positive iff its bits are non-zero and its sign bit clear
+                  const uint32_t lo = wds[e] & 0xFFFFu, hi = wds[e] >> 16;
+                  f[j + 2 * e] = (lo != 0u && lo < 0x8000u) ? __uint_as_float(v[j + 2 * e]) : 0.f;
+                  f[j + 2 * e + 1] = (hi != 0u && hi < 0x8000u) ? __uint_as_float(v[j + 2 * e + 1]) : 0.f;
+                }
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                const bool on = row_ok && nc + j < a.N && __bfloat162float(mk[j]) > 0.f;
+                f[j] = on ? __uint_as_float(v[j]) : 0.f;
+              }
             }
           }
           if (row_ok) {
@@ -303,15 +342,17 @@ __global__ void __launch_bounds__(GEMM_THREADS) bf16_gemm_kernel(const __grid_co
           }
         }
       }
-    } else if (lane == 0) {
-      atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tempty_bar[slot]);
     }
+    if (!ok && lane == 0) atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
   }
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)BN) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
   }
 }
 
@@ -342,10 +383,6 @@ constexpr int DW_PITCH = 36;   // floats per staged row (16-byte aligned, confli
 constexpr int DW_EPI_WARPS = 8;
 constexpr int DW_THREADS = 64 + 32 * DW_EPI_WARPS;
 constexpr int DW_STAGE_FLOATS = DW_EPI_WARPS * 32 * DW_PITCH;
-
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
 
 __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_constant__ CUtensorMap tmA,
                                                                 const __grid_constant__ CUtensorMap tmB,
@@ -704,12 +741,12 @@ bool make_map(CUtensorMap* tm, const void* base, long long k_extent, long long r
 
 long long up(long long x, long long m) { return (x + m - 1) / m * m; }
 
-cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const Params& P, GemmB a, cudaStream_t st) {
-  const int nkb = (a.K + BK - 1) / BK;
-  a.stages = nkb < MAX_STAGES ? nkb : MAX_STAGES;
-  const size_t smem = (size_t)a.stages * STAGE_BYTES + 1024;
-  dim3 grid((a.N + BN - 1) / BN, (a.M + BM - 1) / BM, 2 * P.G);
-  bf16_gemm_kernel<<<grid, GEMM_THREADS, smem, st>>>(ta, tb, P, a);
+cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const Params& P, GemmB a, int sm_count,
+                        cudaStream_t st) {
+  a.stages = G_STAGES;
+  const long long tiles = (long long)((a.N + GN - 1) / GN) * ((a.M + BM - 1) / BM) * 2 * P.G;
+  const int ctas = (int)(tiles < sm_count ? tiles : sm_count);
+  bf16_gemm_kernel<<<ctas, G_THREADS, (size_t)G_STAGES * G_STAGE_BYTES + 1024, st>>>(ta, tb, P, a);
   return cudaGetLastError();
 }
 
@@ -788,10 +825,10 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
       ok &= make_map(&im->tm_fwd_a[l], im->xb, ni, Bp, G, im->ld[0], Bp * im->ld[0], BM);
     else
       ok &= make_map(&im->tm_fwd_a[l], im->act[l - 1], ni, Bp, 2LL * G, im->ld[l - 1], Bp * im->ld[l - 1], BM);
-    ok &= make_map(&im->tm_fwd_b[l], im->wb + im->w_pos[l], ni, no, D + 1, im->ld[l - 1], im->slot_elems, BN);
+    ok &= make_map(&im->tm_fwd_b[l], im->wb + im->w_pos[l], ni, no, D + 1, im->ld[l - 1], im->slot_elems, GN);
     // backward data: A = dz_l rows, B = W_l^T (ring)
     ok &= make_map(&im->tm_da_a[l], im->dz[l], no, Bp, 2LL * G, im->ld[l], Bp * im->ld[l], BM);
-    ok &= make_map(&im->tm_da_b[l], im->wb + im->wt_pos[l], no, ni, D + 1, im->ld[l], im->slot_elems, BN);
+    ok &= make_map(&im->tm_da_b[l], im->wb + im->wt_pos[l], no, ni, D + 1, im->ld[l], im->slot_elems, GN);
     // weight gradient: A = dz_l^T, B = a_{l-1}^T
     ok &= make_map(&im->tm_dw_a[l], im->dzT[l], Bp, no, 2LL * G, Bp, (long long)no * Bp, BM);
     if (l == 1)
@@ -804,7 +841,7 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
     return cudaSuccess;
   }
   cudaError_t e = cudaFuncSetAttribute(bf16_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       MAX_STAGES * STAGE_BYTES + 1024);
+                                       G_STAGES * G_STAGE_BYTES + 1024);
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(bf16_dw_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            4 * STAGE_BYTES + 1024 + DW_STAGE_FLOATS * 4);
@@ -867,7 +904,7 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
       a.epi = EPI_SCORES;
       a.out_f32 = im->scores;
     }
-    if ((e = launch_gemm(im->tm_fwd_a[l], im->tm_fwd_b[l], P, a, st)) != cudaSuccess) return e;
+    if ((e = launch_gemm(im->tm_fwd_a[l], im->tm_fwd_b[l], P, a, pl.sm_count, st)) != cudaSuccess) return e;
     ++n;
   }
   bf16_softmax_grad_kernel<<<(unsigned)((2 * rows * 32 + 255) / 256), 256, 0, st>>>(
@@ -911,7 +948,7 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
       d.ldt = Bp;
       d.z_stride_out = (long long)Bp * im->ld[l - 1];
       d.z_stride_outT = (long long)pl.dims[l - 1] * Bp;
-      if ((e = launch_gemm(im->tm_da_a[l], im->tm_da_b[l], P, d, st)) != cudaSuccess) return e;
+      if ((e = launch_gemm(im->tm_da_a[l], im->tm_da_b[l], P, d, pl.sm_count, st)) != cudaSuccess) return e;
       ++n;
     }
   }
