@@ -195,7 +195,8 @@ gcada_status gcada_get_debug(gcada_ctx *ctx, int what, void *out, long long byte
 gcada_status gcada_get_launch_count(gcada_ctx *ctx, unsigned long long *launches);
 
 /* With GCADA_OPT_TIMING on: mean device time in milliseconds of the three
- * phases of an iteration, ms[0] gradient kernels, ms[1] selection kernel,
+ * phases of an iteration, ms[0] gradient kernels (including any that run
+ * after the selection), ms[1] selection kernel,
  * ms[2] update kernel, over the (at most 512) most recent timed iterations,
  * whose number goes to *n_timed.  Synchronises the stream. */
 gcada_status gcada_get_kernel_times(gcada_ctx *ctx, double ms[3], int *n_timed);

@@ -62,7 +62,7 @@ struct gcada_ctx {
   cudaGraphExec_t graph1 = nullptr, graphN = nullptr;
   // optional per-phase timing
   int timing = 0;
-  std::vector<cudaEvent_t> events;  // TIMING_CAP * 4
+  std::vector<cudaEvent_t> events;  // TIMING_CAP * 5
   long long timed = 0;              // timed iterations so far
   bool capturing = false;
   std::string err;
@@ -255,10 +255,10 @@ gcada_status enqueue_iteration(gcada_ctx* ctx, const Params& P) {
   cudaEvent_t* ev = nullptr;
   if (ctx->timing && !ctx->capturing) {
     if (ctx->events.empty()) {
-      ctx->events.resize((size_t)TIMING_CAP * 4, nullptr);
+      ctx->events.resize((size_t)TIMING_CAP * 5, nullptr);
       for (auto& e : ctx->events) CK(cudaEventCreate(&e));
     }
-    ev = &ctx->events[(size_t)(ctx->timed % TIMING_CAP) * 4];
+    ev = &ctx->events[(size_t)(ctx->timed % TIMING_CAP) * 5];
     CK(cudaEventRecord(ev[0], ctx->stream));
   }
   if (is_linear(ctx)) {
@@ -272,9 +272,15 @@ gcada_status enqueue_iteration(gcada_ctx* ctx, const Params& P) {
   if (ev) CK(cudaEventRecord(ev[1], ctx->stream));
   CK(launch_select(P, ctx->tail, ctx->stream));
   if (ev) CK(cudaEventRecord(ev[2], ctx->stream));
+  if (!is_linear(ctx)) {  // gradient work that needs the selection (counted with the gradient phase)
+    int n = 0;
+    CK(launch_grad_mlp_post(P, ctx->mlp, ctx->stream, &n));
+    ctx->launches += (unsigned long long)n;
+  }
+  if (ev) CK(cudaEventRecord(ev[3], ctx->stream));
   CK(launch_update(P, ctx->tail, ctx->stream));
   if (ev) {
-    CK(cudaEventRecord(ev[3], ctx->stream));
+    CK(cudaEventRecord(ev[4], ctx->stream));
     ctx->timed += 1;
   }
   ctx->launches += 2;
@@ -302,7 +308,11 @@ gcada_status capture(gcada_ctx* ctx, int iters, cudaGraphExec_t* out) {
   return GCADA_OK;
 }
 
-int kernels_per_iteration(const gcada_ctx* ctx) { return 2 + (is_linear(ctx) ? 1 : ctx->mlp.launches_per_iter); }
+int kernels_per_iteration(const gcada_ctx* ctx) {
+  if (is_linear(ctx)) return 3;
+  const bool two_pass = ctx->compute == GCADA_COMPUTE_BF16 && !ctx->P.stale;
+  return 2 + ctx->mlp.launches_per_iter + (two_pass ? ctx->mlp.n_layers : 0);
+}
 
 gcada_status check_runnable(gcada_ctx* ctx, bool need_data) {
   if (!ctx->have_theta) return fail(ctx, GCADA_ESTATE, "gcada_set_theta has not been called");
@@ -718,11 +728,12 @@ gcada_status gcada_get_kernel_times(gcada_ctx* ctx, double ms[3], int* n_timed) 
   *n_timed = (int)n;
   if (n == 0) return GCADA_OK;
   for (long long i = 0; i < n; ++i) {
-    cudaEvent_t* ev = &ctx->events[(size_t)i * 4];
-    for (int j = 0; j < 3; ++j) {
+    cudaEvent_t* ev = &ctx->events[(size_t)i * 5];
+    const int phase_of[4] = {0, 1, 0, 2};  // gradient, selection, gradient (post-selection part), update
+    for (int j = 0; j < 4; ++j) {
       float t = 0.f;
       CK(cudaEventElapsedTime(&t, ev[j], ev[j + 1]));
-      ms[j] += t;
+      ms[phase_of[j]] += t;
     }
   }
   for (int j = 0; j < 3; ++j) ms[j] /= (double)n;

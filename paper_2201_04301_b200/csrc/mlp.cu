@@ -243,6 +243,12 @@ cudaError_t mlp_plan_create(const std::vector<int>& dims, int compute, int G, in
   return cudaSuccess;
 }
 
+cudaError_t launch_grad_mlp_post(const Params& P, const MlpPlan& pl, cudaStream_t st, int* n_launches) {
+  *n_launches = 0;
+  if (pl.compute == 1) return mlp_bf16_launch_post(P, pl, st, n_launches);
+  return cudaSuccess;
+}
+
 cudaError_t launch_grad_mlp(const Params& P, const MlpPlan& pl, cudaStream_t st, int* n_launches) {
   if (pl.compute == 1) return mlp_bf16_launch(P, pl, st, n_launches);
   const int L = pl.n_layers, G = P.G, B = P.B;

@@ -38,5 +38,7 @@ cudaError_t mlp_plan_create(const std::vector<int>& dims, int compute, int G, in
                             const char** why);
 // Enqueues the dual-point forward/backward of every group; writes P.fresh and P.stale.
 cudaError_t launch_grad_mlp(const Params& P, const MlpPlan& plan, cudaStream_t st, int* n_launches);
+// Gradient work that must follow the selection kernel (none for the fp32 path).
+cudaError_t launch_grad_mlp_post(const Params& P, const MlpPlan& plan, cudaStream_t st, int* n_launches);
 
 }  // namespace gcada

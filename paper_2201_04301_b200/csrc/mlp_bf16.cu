@@ -377,7 +377,11 @@ struct DwArgs {
   int tiles_m, tiles_n, total_tiles;
   long long c_off, ldc;   // position of W_l inside the gradient vector, row stride
   int part_base, n_parts; // this layer's first slot in lhs_part and slots per group
+  int mode;               // DW_BOTH: both points, norm, gradients written for every group;
+                          // DW_NORM: both points, norm only (nothing written but lhs_part);
+                          // DW_SELECTED: point 0 only, fresh gradient written for the groups selected this iteration
 };
+enum { DW_BOTH = 0, DW_NORM = 1, DW_SELECTED = 2 };
 
 constexpr int DW_PITCH = 36;   // floats per staged row (16-byte aligned, conflict-free 16-byte stores)
 constexpr int DW_EPI_WARPS = 8;
@@ -395,7 +399,8 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
   float* stage_all = reinterpret_cast<float*>(tiles + (size_t)a.stages * STAGE_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int stages = a.stages;
-  const int kb_per_tile = 2 * a.nkb;
+  const int kb_per_tile = a.mode == DW_SELECTED ? a.nkb : 2 * a.nkb;
+  const unsigned char* sel = a.mode == DW_SELECTED ? P.mask_cur : nullptr;  // tiles of unselected groups are skipped
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) {
@@ -425,6 +430,7 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
       int it = 0;
       for (int t = blockIdx.x; t < a.total_tiles && ok; t += gridDim.x) {
         const int nt = t % a.tiles_n, mt = (t / a.tiles_n) % a.tiles_m, g = t / (a.tiles_n * a.tiles_m);
+        if (sel && !sel[g]) continue;
         for (int j = 0; j < kb_per_tile && ok; ++j, ++it) {
           const int q = j / a.nkb, kb = j - q * a.nkb;
           const int s = it % stages;
@@ -442,7 +448,8 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
     if (lane == 0) {
       bool ok = true;
       int it = 0, i = 0;
-      for (int t = blockIdx.x; t < a.total_tiles && ok; t += gridDim.x, ++i) {
+      for (int t = blockIdx.x; t < a.total_tiles && ok; t += gridDim.x) {
+        if (sel && !sel[t / (a.tiles_n * a.tiles_m)]) continue;
         const int slot = i & 1;
         ok = mbar_wait_bounded(&tempty_bar[slot], (uint32_t)(((i >> 1) & 1) ^ 1));  // epilogue has drained the slot
         if (!ok) break;
@@ -462,6 +469,7 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
           tc_commit(&empty_bar[s]);
         }
         if (ok) tc_commit(&tfull_bar[slot]);
+        ++i;
       }
       if (!ok) atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
     }
@@ -474,36 +482,42 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
                         (P.p_pad & 3) == 0;
     bool ok = true;
     int i = 0;
-    for (int t = blockIdx.x; t < a.total_tiles; t += gridDim.x, ++i) {
-      const int slot = i & 1;
+    for (int t = blockIdx.x; t < a.total_tiles; t += gridDim.x) {
       const int nt = t % a.tiles_n, mt = (t / a.tiles_n) % a.tiles_m, g = t / (a.tiles_n * a.tiles_m);
+      if (sel && !sel[g]) continue;
+      const int slot = i & 1;
+      const int phase = (i >> 1) & 1;
+      ++i;
       double local = 0.0;
       if (ok) {
-        ok = mbar_wait_bounded(&tfull_bar[slot], (uint32_t)((i >> 1) & 1));
+        ok = mbar_wait_bounded(&tfull_bar[slot], (uint32_t)phase);
         ok = __all_sync(0xffffffffu, ok);
       }
       if (ok) {
         tc_fence_after();
         float* fresh = P.fresh + (long long)g * P.p_pad + a.c_off;
-        float* stale = P.stale ? P.stale + (long long)g * P.p_pad + a.c_off : nullptr;
+        float* stale = (a.mode == DW_BOTH && P.stale) ? P.stale + (long long)g * P.p_pad + a.c_off : nullptr;
+        const int n_pass = a.mode == DW_NORM ? 0 : (stale ? 2 : 1);
         const int mrow = mt * BM + quad * 32;
         const uint32_t tbase = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(slot * 2 * BN);
 #pragma unroll 1
         for (int c = half * 64; c < half * 64 + 64; c += 32) {
-          uint32_t v0[32], v1[32];
-          tc_ld32(tbase + (uint32_t)c, v0);
-          tc_ld32(tbase + (uint32_t)(BN + c), v1);
           const int nc = nt * BN + c;
           if (nc >= a.N) break;
-          const bool row_ok = mrow + lane < a.M;
-          float part = 0.f;
+          uint32_t v0[32], v1[32];
+          tc_ld32(tbase + (uint32_t)c, v0);
+          if (a.mode != DW_SELECTED) {
+            tc_ld32(tbase + (uint32_t)(BN + c), v1);
+            const bool row_ok = mrow + lane < a.M;
+            float part = 0.f;
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const float d = __uint_as_float(v0[j]) - __uint_as_float(v1[j]);
-            if (row_ok && nc + j < a.N) part += d * d;
+            for (int j = 0; j < 32; ++j) {
+              const float d = __uint_as_float(v0[j]) - __uint_as_float(v1[j]);
+              if (row_ok && nc + j < a.N) part += d * d;
+            }
+            local += (double)part;
           }
-          local += (double)part;
-          for (int pass = 0; pass < (stale ? 2 : 1); ++pass) {
+          for (int pass = 0; pass < n_pass; ++pass) {
             const uint32_t* v = pass == 0 ? v0 : v1;
             float* out = pass == 0 ? fresh : stale;
             __syncwarp();
@@ -537,7 +551,7 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
       local = warp_sum(local);
       if (lane == 0) norm_sm[slot][ew] = local;
       asm volatile("bar.sync 1, %0;" ::"n"(32 * DW_EPI_WARPS) : "memory");
-      if (ew == 0 && lane == 0) {
+      if (ew == 0 && lane == 0 && a.mode != DW_SELECTED) {
         double tsum = 0.0;
 #pragma unroll
         for (int w = 0; w < DW_EPI_WARPS; ++w) tsum += norm_sm[slot][w];
@@ -750,6 +764,28 @@ cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const Para
   return cudaGetLastError();
 }
 
+cudaError_t launch_dw(const Params& P, const MlpPlan& pl, const Bf16Impl* im, int l, int mode, cudaStream_t st) {
+  DwArgs w{};
+  w.M = pl.dims[l];
+  w.N = pl.dims[l - 1];
+  w.K = im->Bp;
+  w.b_shared = l == 1;
+  w.nkb = im->Bp / BK;
+  w.stages = 4;
+  w.tiles_m = (w.M + BM - 1) / BM;
+  w.tiles_n = (w.N + BN - 1) / BN;
+  w.total_tiles = w.tiles_m * w.tiles_n * P.G;
+  w.c_off = pl.w_off[l];
+  w.ldc = pl.dims[l - 1];
+  w.part_base = im->dw_part_base[l];
+  w.n_parts = im->n_parts;
+  w.mode = mode;
+  const int ctas = w.total_tiles < pl.sm_count ? w.total_tiles : pl.sm_count;
+  const size_t smem = (size_t)w.stages * STAGE_BYTES + 1024 + DW_STAGE_FLOATS * 4;
+  bf16_dw_kernel<<<ctas, DW_THREADS, smem, st>>>(im->tm_dw_a[l], im->tm_dw_b[l], P, w);
+  return cudaGetLastError();
+}
+
 }  // namespace
 
 const char* mlp_bf16_supported(const std::vector<int>& dims) {
@@ -911,27 +947,9 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
       P, im->scores, im->yb, im->dz[L], im->dzT[L], pl.dims[L], im->ld[L], Bp);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   ++n;
+  const int dw_mode = P.stale ? DW_BOTH : DW_NORM;  // gradients of every group are materialised only on request
   for (int l = L; l >= 1; --l) {
-    DwArgs w{};
-    w.M = pl.dims[l];
-    w.N = pl.dims[l - 1];
-    w.K = Bp;
-    w.b_shared = l == 1;
-    w.nkb = Bp / BK;
-    w.stages = 4;
-    w.tiles_m = (w.M + BM - 1) / BM;
-    w.tiles_n = (w.N + BN - 1) / BN;
-    w.total_tiles = w.tiles_m * w.tiles_n * G;
-    w.c_off = pl.w_off[l];
-    w.ldc = pl.dims[l - 1];
-    w.part_base = im->dw_part_base[l];
-    w.n_parts = im->n_parts;
-    {
-      const int ctas = w.total_tiles < pl.sm_count ? w.total_tiles : pl.sm_count;
-      const size_t smem = (size_t)w.stages * STAGE_BYTES + 1024 + DW_STAGE_FLOATS * 4;
-      bf16_dw_kernel<<<ctas, DW_THREADS, smem, st>>>(im->tm_dw_a[l], im->tm_dw_b[l], P, w);
-      if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    }
+    if ((e = launch_dw(P, pl, im, l, dw_mode, st)) != cudaSuccess) return e;
     ++n;
     if (l > 1) {
       GemmB d{};
@@ -970,4 +988,20 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
   return cudaSuccess;
 }
 
+}  // namespace gcada
+
+namespace gcada {
+// After the selection: weight gradients of the selected groups (the only ones
+// the server's aggregate needs, Eq. 3) are recomputed at theta^k and written.
+cudaError_t mlp_bf16_launch_post(const Params& P, const MlpPlan& pl, cudaStream_t st, int* n_launches) {
+  *n_launches = 0;
+  if (P.stale) return cudaSuccess;  // everything was materialised by the first pass
+  const Bf16Impl* im = static_cast<const Bf16Impl*>(pl.bf16_impl);
+  for (int l = pl.n_layers; l >= 1; --l) {
+    cudaError_t e = launch_dw(P, pl, im, l, DW_SELECTED, st);
+    if (e != cudaSuccess) return e;
+    ++*n_launches;
+  }
+  return cudaSuccess;
+}
 }  // namespace gcada

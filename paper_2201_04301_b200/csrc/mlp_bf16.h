@@ -6,4 +6,6 @@ namespace gcada {
 const char* mlp_bf16_supported(const std::vector<int>& dims);
 cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<void*>* owned, const char** why);
 cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& plan, cudaStream_t st, int* n_launches);
+// Work that has to follow the selection kernel (writes the selected groups' weight gradients).
+cudaError_t mlp_bf16_launch_post(const Params& P, const MlpPlan& plan, cudaStream_t st, int* n_launches);
 }  // namespace gcada

@@ -37,3 +37,23 @@ def test_deterministic_and_counts():
     assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
     up, comm, comp = outs[0][2]
     assert up == int(outs[0][1].sum()) and comm == 3 * up and comp == 2 * up and outs[0][1][0].all()
+
+
+def test_two_pass_weight_gradients_equal_materialised_ones():
+    """Without GCADA_OPT_KEEP_STALE the weight gradients are not written for every
+    group: a first pass only forms the innovation norms, and after the selection
+    the selected groups' gradients are recomputed and written.  Both ways must
+    give the same bits."""
+    w = to_cuda(make_workload("cfg5", rows=3000, dims=(64, 128, 40), M=6, M_G=2, D=4, batch=128, c=5.0))
+    a = binding.from_workload(w, stream=torch.cuda.Stream(), options={binding.OPT_KEEP_STALE: 1.0})
+    b = binding.from_workload(w, stream=torch.cuda.Stream())
+    for chunk in (1, 7, 17):
+        a.step(chunk)
+        b.step(chunk)
+        assert np.array_equal(a.get_theta(), b.get_theta())
+        assert np.array_equal(a.get_debug(binding.DBG_LHS), b.get_debug(binding.DBG_LHS))
+        assert np.array_equal(a.get_debug(binding.DBG_GLAST), b.get_debug(binding.DBG_GLAST))
+    ma, mb = a.get_selection_mask(0, 25), b.get_selection_mask(0, 25)
+    assert np.array_equal(ma, mb) and 0 < ma.sum() < ma.size          # some uploads were skipped
+    assert a.get_comm_count() == b.get_comm_count()
+    assert b.get_launch_count() > a.get_launch_count()                 # the second pass exists
