@@ -29,8 +29,7 @@ namespace gcada {
 namespace {
 
 constexpr int BM = 128, BN = 128, BK = 64;      // tile; BK * 2 bytes = one 128-byte swizzle row
-constexpr int MAX_STAGES = 6;
-constexpr int STAGE_BYTES = (BM + BN) * BK * 2;  // 32 KiB
+constexpr int MAX_STAGES = 8;
 
 enum { EPI_HIDDEN = 0, EPI_SCORES = 1, EPI_DA = 2, EPI_DW = 3 };
 enum { ZB_BATCH = 0, ZB_GROUP = 1, ZB_RING = 2 };
@@ -97,10 +96,30 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait for the single-thread producer / MMA loops: non-blocking polls, so that the thread
+// reacts within a few cycles of the phase flipping (try_wait may park the thread for a while).
+__device__ __forceinline__ bool mbar_spin_bounded(uint64_t* bar, uint32_t parity) {
+  for (uint32_t it = 0; it < (1u << 26); ++it)
+    if (mbar_test_wait(bar, parity)) return true;
+  return false;
+}
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
-  for (uint32_t it = 0; it < (1u << 22); ++it) {
+  // no back-off for the first polls: a sleeping producer or MMA thread adds its wake-up time to every
+  // pipeline step, which dominates when a tile has only a few steps
+  for (uint32_t it = 0; it < (1u << 24); ++it) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (it > 32) __nanosleep(64);
+    if (it > (1u << 16)) __nanosleep(128);
   }
   return false;
 }
@@ -126,18 +145,24 @@ __device__ __forceinline__ void tc_mma_bf16(uint32_t tmem_c, uint64_t da, uint64
       : "r"(tmem_c), "l"(da), "l"(db), "r"(idesc), "r"(accum), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
       : "memory");
 }
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+// Issues the load only; the registers are valid after tc_ld_wait().
+__device__ __forceinline__ void tc_ld32_issue(uint32_t taddr, uint32_t (&v)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n\t"
-      "tcgen05.wait::ld.sync.aligned;"
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
       : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
         "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
         "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
         "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
       : "r"(taddr)
       : "memory");
+}
+
+__device__ __forceinline__ void tc_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  tc_ld32_issue(taddr, v);
+  tc_ld_wait();
 }
 
 // Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes
@@ -149,7 +174,6 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr) {
          (2ull << 61);
 }
 // Instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, N >> 3 at bit 17, M >> 4 at bit 24.
-constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
 __device__ __forceinline__ int ring_slot(const Params& P, int g, int q, long long k) {
   long long j = q == 0 ? k : k - P.tau[g];
@@ -219,7 +243,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
         const int zB = a.zb_mode == ZB_RING ? ring_slot(P, g, q, k_it) : (a.zb_mode == ZB_GROUP ? g : z);
         for (int kb = 0; kb < nkb && ok; ++kb, ++it) {
           const int s = it % G_STAGES;
-          ok = mbar_wait_bounded(&empty_bar[s], (uint32_t)(((it / G_STAGES) & 1) ^ 1));
+          ok = mbar_spin_bounded(&empty_bar[s], (uint32_t)(((it / G_STAGES) & 1) ^ 1));
           if (!ok) break;
           unsigned char* sa = tiles + (size_t)s * G_STAGE_BYTES;
           mbar_expect_tx(&full_bar[s], G_STAGE_BYTES);
@@ -235,12 +259,12 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
       int it = 0, i = 0;
       for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++i) {
         const int slot = i & 1;
-        ok = mbar_wait_bounded(&tempty_bar[slot], (uint32_t)(((i >> 1) & 1) ^ 1));
+        ok = mbar_spin_bounded(&tempty_bar[slot], (uint32_t)(((i >> 1) & 1) ^ 1));
         if (!ok) break;
         tc_fence_after();
         for (int kb = 0; kb < nkb && ok; ++kb, ++it) {
           const int s = it % G_STAGES;
-          ok = mbar_wait_bounded(&full_bar[s], (uint32_t)((it / G_STAGES) & 1));
+          ok = mbar_spin_bounded(&full_bar[s], (uint32_t)((it / G_STAGES) & 1));
           if (!ok) break;
           tc_fence_after();
           const uint32_t sa = smem_u32(tiles + (size_t)s * G_STAGE_BYTES);
@@ -358,14 +382,18 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
 
 // ----------------------------------------------------------------- weight gradients, both points in one CTA
 // dW_l of one group at theta^k (accumulator 0) and at the stale iterate
-// (accumulator 1), 128 x 128 tiles.  The epilogue writes the fresh gradient
+// (accumulator 1), 128 x 256 tiles.  The epilogue writes the fresh gradient
 // (and the stale one only when it is kept for inspection), forms the squared
 // norm of their difference - the tile's share of the left side of Eq. (9) -
 // and stores it in the tile's own slot of lhs_part, so the per-group
 // gradients are never re-read to build the test.
 //
-// Persistent: one CTA per SM walks tiles t = blockIdx.x, + gridDim.x, ...;
-// tensor memory holds two accumulator pairs (2 x 256 columns) so that the
+// Persistent: one CTA per SM walks work units u = blockIdx.x, + gridDim.x,
+// ...; a unit is one (group, 128-row block of W_l) and its tiles are all the
+// column blocks.  The unit's A operand (dz_l^T at both points, 2 x K x 128
+// bf16) stays in shared memory for the whole unit and only B is streamed: with
+// K = 128 the product is bound by operand traffic from L2, and this halves it.
+// Tensor memory holds two accumulator pairs (2 x 256 columns) so that the
 // eight epilogue warps drain tile i while the producer and the MMA warp work
 // on tile i+1.  Rows reach global memory as full 128-byte lines through a
 // per-warp staging tile.
@@ -377,12 +405,14 @@ struct DwArgs {
   int tiles_m, tiles_n, total_tiles;
   long long c_off, ldc;   // position of W_l inside the gradient vector, row stride
   int part_base, n_parts; // this layer's first slot in lhs_part and slots per group
-  int mode;               // DW_BOTH: both points, norm, gradients written for every group;
-                          // DW_NORM: both points, norm only (nothing written but lhs_part);
+  int mode;               // DW_BOTH: both points in two accumulators, norm, gradients written for every group;
+                          // DW_NORM: one accumulator receives dW(theta^k) - dW(stale) (the second product enters
+                          //          negated), norm only, nothing written but lhs_part;
                           // DW_SELECTED: point 0 only, fresh gradient written for the groups selected this iteration
 };
 enum { DW_BOTH = 0, DW_NORM = 1, DW_SELECTED = 2 };
 
+constexpr int DW_BN = 256;     // N tile: the MMA issue rate, not the tensor pipe, limits 128-wide instructions
 constexpr int DW_PITCH = 36;   // floats per staged row (16-byte aligned, conflict-free 16-byte stores)
 constexpr int DW_EPI_WARPS = 8;
 constexpr int DW_THREADS = 64 + 32 * DW_EPI_WARPS;
@@ -392,11 +422,18 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
                                                                 const __grid_constant__ CUtensorMap tmB,
                                                                 const Params P, const DwArgs a) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
-  __shared__ uint64_t full_bar[MAX_STAGES], empty_bar[MAX_STAGES], tfull_bar[2], tempty_bar[2];
+  __shared__ uint64_t full_bar[MAX_STAGES], empty_bar[MAX_STAGES], tfull_bar[4], tempty_bar[4], afull_bar, aempty_bar;
   __shared__ uint32_t tmem_base_sm;
-  __shared__ double norm_sm[2][DW_EPI_WARPS];
-  unsigned char* tiles = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  float* stage_all = reinterpret_cast<float*>(tiles + (size_t)a.stages * STAGE_BYTES);
+  __shared__ double norm_sm[4][DW_EPI_WARPS];
+  // accumulator slots in the 512 columns of tensor memory: one pair, or two single accumulators
+  const int n_slots = a.mode == DW_BOTH ? 1 : 2;
+  const int slot_cols = a.mode == DW_BOTH ? 2 * DW_BN : DW_BN;
+  constexpr int BLK = BM * BK * 2;      // one 128 x 64 bf16 block of A, 16 KiB
+  constexpr int BBLK = DW_BN * BK * 2;  // one 256 x 64 bf16 block of B, 32 KiB
+  unsigned char* a_res = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  unsigned char* tiles = a_res + (size_t)2 * a.nkb * BLK;  // ring of B blocks
+  float* stage_all = reinterpret_cast<float*>(tiles + (size_t)a.stages * BBLK);
+  const int n_units = a.tiles_m * P.G;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int stages = a.stages;
   const int kb_per_tile = a.mode == DW_SELECTED ? a.nkb : 2 * a.nkb;
@@ -407,10 +444,12 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
       mbar_init(&full_bar[s], 1);
       mbar_init(&empty_bar[s], 1);
     }
-    for (int s = 0; s < 2; ++s) {
+    for (int s = 0; s < 4; ++s) {
       mbar_init(&tfull_bar[s], 1);
       mbar_init(&tempty_bar[s], DW_EPI_WARPS);
     }
+    mbar_init(&afull_bar, 1);
+    mbar_init(&aempty_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {  // all 512 columns: two slots of two fp32 accumulators
@@ -427,19 +466,28 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
   if (warp == 0) {
     if (lane == 0) {
       bool ok = true;
-      int it = 0;
-      for (int t = blockIdx.x; t < a.total_tiles && ok; t += gridDim.x) {
-        const int nt = t % a.tiles_n, mt = (t / a.tiles_n) % a.tiles_m, g = t / (a.tiles_n * a.tiles_m);
+      int it = 0, ui = 0;
+      for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+        const int mt = u % a.tiles_m, g = u / a.tiles_m;
         if (sel && !sel[g]) continue;
-        for (int j = 0; j < kb_per_tile && ok; ++j, ++it) {
+        // the unit's A blocks, once the MMAs of the previous unit have finished reading them
+        ok = mbar_spin_bounded(&aempty_bar, (uint32_t)((ui & 1) ^ 1));
+        if (!ok) break;
+        mbar_expect_tx(&afull_bar, (uint32_t)(kb_per_tile * BLK));
+        for (int j = 0; j < kb_per_tile; ++j) {
           const int q = j / a.nkb, kb = j - q * a.nkb;
-          const int s = it % stages;
-          ok = mbar_wait_bounded(&empty_bar[s], (uint32_t)(((it / stages) & 1) ^ 1));
-          if (!ok) break;
-          unsigned char* sa = tiles + (size_t)s * STAGE_BYTES;
-          mbar_expect_tx(&full_bar[s], STAGE_BYTES);
-          tma_load_3d(sa, &tmA, kb * BK, mt * BM, q * P.G + g, &full_bar[s]);
-          tma_load_3d(sa + BM * BK * 2, &tmB, kb * BK, nt * BN, a.b_shared ? g : q * P.G + g, &full_bar[s]);
+          tma_load_3d(a_res + (size_t)j * BLK, &tmA, kb * BK, mt * BM, q * P.G + g, &afull_bar);
+        }
+        ++ui;
+        for (int nt = 0; nt < a.tiles_n && ok; ++nt) {
+          for (int j = 0; j < kb_per_tile && ok; ++j, ++it) {
+            const int q = j / a.nkb, kb = j - q * a.nkb;
+            const int s = it % stages;
+            ok = mbar_spin_bounded(&empty_bar[s], (uint32_t)(((it / stages) & 1) ^ 1));
+            if (!ok) break;
+            mbar_expect_tx(&full_bar[s], BBLK);
+            tma_load_3d(tiles + (size_t)s * BBLK, &tmB, kb * BK, nt * DW_BN, a.b_shared ? g : q * P.G + g, &full_bar[s]);
+          }
         }
       }
       if (!ok) atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
@@ -447,46 +495,55 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
   } else if (warp == 1) {
     if (lane == 0) {
       bool ok = true;
-      int it = 0, i = 0;
-      for (int t = blockIdx.x; t < a.total_tiles && ok; t += gridDim.x) {
-        if (sel && !sel[t / (a.tiles_n * a.tiles_m)]) continue;
-        const int slot = i & 1;
-        ok = mbar_wait_bounded(&tempty_bar[slot], (uint32_t)(((i >> 1) & 1) ^ 1));  // epilogue has drained the slot
+      int it = 0, i = 0, ui = 0;
+      for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+        if (sel && !sel[u / a.tiles_m]) continue;
+        ok = mbar_spin_bounded(&afull_bar, (uint32_t)(ui & 1));
         if (!ok) break;
-        tc_fence_after();
-        for (int j = 0; j < kb_per_tile && ok; ++j, ++it) {
-          const int q = j / a.nkb, kb = j - q * a.nkb;
-          const int s = it % stages;
-          ok = mbar_wait_bounded(&full_bar[s], (uint32_t)((it / stages) & 1));
+        ++ui;
+        for (int nt = 0; nt < a.tiles_n && ok; ++nt, ++i) {
+          const int slot = i % n_slots;
+          ok = mbar_spin_bounded(&tempty_bar[slot], (uint32_t)(((i / n_slots) & 1) ^ 1));  // epilogue has drained the slot
           if (!ok) break;
           tc_fence_after();
-          const uint32_t sa = smem_u32(tiles + (size_t)s * STAGE_BYTES);
-          const uint64_t da = make_desc(sa), db = make_desc(sa + BM * BK * 2);
+          for (int j = 0; j < kb_per_tile && ok; ++j, ++it) {
+            const int q = j / a.nkb, kb = j - q * a.nkb;
+            const int s = it % stages;
+            ok = mbar_spin_bounded(&full_bar[s], (uint32_t)((it / stages) & 1));
+            if (!ok) break;
+            tc_fence_after();
+            const uint64_t da = make_desc(smem_u32(a_res + (size_t)j * BLK));
+            const uint64_t db = make_desc(smem_u32(tiles + (size_t)s * BBLK));
+            // DW_NORM: the stale-point product is subtracted in the same accumulator (A negated, bit 13)
+            const uint32_t idesc = (a.mode == DW_NORM && q == 1) ? (IDESC_G | (1u << 13)) : IDESC_G;
+            const uint32_t acc_col = (uint32_t)(slot * slot_cols + (a.mode == DW_BOTH ? q * DW_BN : 0));
 #pragma unroll
-          for (int kk = 0; kk < BK / 16; ++kk)
-            tc_mma_bf16(tmem_base + (uint32_t)(slot * 2 * BN + q * BN), da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2),
-                        IDESC, (kb | kk) != 0 ? 1u : 0u);
-          tc_commit(&empty_bar[s]);
+            for (int kk = 0; kk < BK / 16; ++kk)
+              tc_mma_bf16(tmem_base + acc_col, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc,
+                          ((a.mode == DW_NORM ? j : kb) | kk) != 0 ? 1u : 0u);
+            tc_commit(&empty_bar[s]);
+          }
+          if (ok) tc_commit(&tfull_bar[slot]);
         }
-        if (ok) tc_commit(&tfull_bar[slot]);
-        ++i;
+        if (ok) tc_commit(&aempty_bar);  // the A blocks may be overwritten once these MMAs are done
       }
       if (!ok) atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
     }
   } else {
     const int ew = warp - 2;           // 0..7
     const int quad = warp & 3;         // TMEM lanes this warp may read
-    const int half = ew >> 2;          // which 64 columns of the tile
+    const int half = ew >> 2;          // which 128 columns of the tile
     float* stg = stage_all + (size_t)ew * 32 * DW_PITCH;
     const bool vec_ok = ((a.c_off | a.ldc) & 3) == 0 && (reinterpret_cast<uintptr_t>(P.fresh) & 15) == 0 &&
                         (P.p_pad & 3) == 0;
     bool ok = true;
     int i = 0;
-    for (int t = blockIdx.x; t < a.total_tiles; t += gridDim.x) {
-      const int nt = t % a.tiles_n, mt = (t / a.tiles_n) % a.tiles_m, g = t / (a.tiles_n * a.tiles_m);
+    for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
+      const int mt = u % a.tiles_m, g = u / a.tiles_m;
       if (sel && !sel[g]) continue;
-      const int slot = i & 1;
-      const int phase = (i >> 1) & 1;
+      for (int nt = 0; nt < a.tiles_n; ++nt) {
+      const int slot = i % n_slots;
+      const int phase = (i / n_slots) & 1;
       ++i;
       double local = 0.0;
       if (ok) {
@@ -499,23 +556,26 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
         float* stale = (a.mode == DW_BOTH && P.stale) ? P.stale + (long long)g * P.p_pad + a.c_off : nullptr;
         const int n_pass = a.mode == DW_NORM ? 0 : (stale ? 2 : 1);
         const int mrow = mt * BM + quad * 32;
-        const uint32_t tbase = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(slot * 2 * BN);
+        const uint32_t tbase = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(slot * slot_cols);
 #pragma unroll 1
-        for (int c = half * 64; c < half * 64 + 64; c += 32) {
-          const int nc = nt * BN + c;
+        for (int c = half * (DW_BN / 2); c < (half + 1) * (DW_BN / 2); c += 32) {
+          const int nc = nt * DW_BN + c;
           if (nc >= a.N) break;
           uint32_t v0[32], v1[32];
-          tc_ld32(tbase + (uint32_t)c, v0);
+          tc_ld32_issue(tbase + (uint32_t)c, v0);
+          if (a.mode == DW_BOTH) tc_ld32_issue(tbase + (uint32_t)(DW_BN + c), v1);
+          tc_ld_wait();  // one wait for both accumulators
           if (a.mode != DW_SELECTED) {
-            tc_ld32(tbase + (uint32_t)(BN + c), v1);
             const bool row_ok = mrow + lane < a.M;
+            const bool interior = nc + 32 <= a.N;
             float part = 0.f;
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
-              const float d = __uint_as_float(v0[j]) - __uint_as_float(v1[j]);
-              if (row_ok && nc + j < a.N) part += d * d;
+              // DW_NORM: the accumulator already holds the difference
+              const float d = a.mode == DW_BOTH ? __uint_as_float(v0[j]) - __uint_as_float(v1[j]) : __uint_as_float(v0[j]);
+              if (interior || nc + j < a.N) part += d * d;
             }
-            local += (double)part;
+            if (row_ok) local += (double)part;
           }
           for (int pass = 0; pass < n_pass; ++pass) {
             const uint32_t* v = pass == 0 ? v0 : v1;
@@ -556,6 +616,7 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
 #pragma unroll
         for (int w = 0; w < DW_EPI_WARPS; ++w) tsum += norm_sm[slot][w];
         P.lhs_part[(long long)g * a.n_parts + a.part_base + mt * a.tiles_n + nt] = tsum;
+      }
       }
     }
     if (!ok && lane == 0) atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
@@ -771,17 +832,19 @@ cudaError_t launch_dw(const Params& P, const MlpPlan& pl, const Bf16Impl* im, in
   w.K = im->Bp;
   w.b_shared = l == 1;
   w.nkb = im->Bp / BK;
-  w.stages = 4;
+  w.stages = (11 - 2 * w.nkb) / 2;  // 32 KiB B blocks in the shared memory left beside the resident A blocks
+  if (w.stages < 1) w.stages = 1;
   w.tiles_m = (w.M + BM - 1) / BM;
-  w.tiles_n = (w.N + BN - 1) / BN;
+  w.tiles_n = (w.N + DW_BN - 1) / DW_BN;
   w.total_tiles = w.tiles_m * w.tiles_n * P.G;
   w.c_off = pl.w_off[l];
   w.ldc = pl.dims[l - 1];
   w.part_base = im->dw_part_base[l];
   w.n_parts = im->n_parts;
   w.mode = mode;
-  const int ctas = w.total_tiles < pl.sm_count ? w.total_tiles : pl.sm_count;
-  const size_t smem = (size_t)w.stages * STAGE_BYTES + 1024 + DW_STAGE_FLOATS * 4;
+  const int units = w.tiles_m * P.G;
+  const int ctas = units < pl.sm_count ? units : pl.sm_count;
+  const size_t smem = (size_t)(2 * w.nkb + 2 * w.stages) * (BM * BK * 2) + 1024 + DW_STAGE_FLOATS * 4;
   bf16_dw_kernel<<<ctas, DW_THREADS, smem, st>>>(im->tm_dw_a[l], im->tm_dw_b[l], P, w);
   return cudaGetLastError();
 }
@@ -795,6 +858,10 @@ const char* mlp_bf16_supported(const std::vector<int>& dims) {
 
 cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<void*>* owned, const char** why) {
   const int L = plan->n_layers, G = plan->G, B = plan->B, D = plan->D;
+  if (plan->B > 256) {
+    *why = "the bf16 MLP path supports minibatches of at most 256 rows per group";
+    return cudaSuccess;
+  }
   Bf16Impl* im = new Bf16Impl();
   plan->bf16_impl = im;  // lives as long as the process (a few hundred bytes per plan)
   im->Bp = (int)up(B, 128);
@@ -814,7 +881,7 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
   int parts = 0;
   for (int l = 1; l <= L; ++l) {
     im->dw_part_base[l] = parts;
-    parts += ((plan->dims[l] + BM - 1) / BM) * ((plan->dims[l - 1] + BN - 1) / BN);
+    parts += ((plan->dims[l] + BM - 1) / BM) * ((plan->dims[l - 1] + DW_BN - 1) / DW_BN);
   }
   for (int l = 1; l <= L; ++l) {
     im->bias_part_base[l] = parts;
@@ -868,9 +935,9 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
     // weight gradient: A = dz_l^T, B = a_{l-1}^T
     ok &= make_map(&im->tm_dw_a[l], im->dzT[l], Bp, no, 2LL * G, Bp, (long long)no * Bp, BM);
     if (l == 1)
-      ok &= make_map(&im->tm_dw_b[l], im->xbT, Bp, ni, G, Bp, (long long)ni * Bp, BN);
+      ok &= make_map(&im->tm_dw_b[l], im->xbT, Bp, ni, G, Bp, (long long)ni * Bp, DW_BN);
     else
-      ok &= make_map(&im->tm_dw_b[l], im->actT[l - 1], Bp, ni, 2LL * G, Bp, (long long)ni * Bp, BN);
+      ok &= make_map(&im->tm_dw_b[l], im->actT[l - 1], Bp, ni, 2LL * G, Bp, (long long)ni * Bp, DW_BN);
   }
   if (!ok) {
     *why = "tensor map creation failed for this MLP shape";
@@ -880,7 +947,7 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
                                        G_STAGES * G_STAGE_BYTES + 1024);
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(bf16_dw_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           4 * STAGE_BYTES + 1024 + DW_STAGE_FLOATS * 4);
+                           11 * (BM * BK * 2) + 1024 + DW_STAGE_FLOATS * 4);
   if (e != cudaSuccess) return e;
   plan->launches_per_iter = 3 + L + 1 + L + (L - 1);
   return cudaSuccess;

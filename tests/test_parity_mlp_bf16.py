@@ -41,19 +41,41 @@ def test_deterministic_and_counts():
 
 def test_two_pass_weight_gradients_equal_materialised_ones():
     """Without GCADA_OPT_KEEP_STALE the weight gradients are not written for every
-    group: a first pass only forms the innovation norms, and after the selection
-    the selected groups' gradients are recomputed and written.  Both ways must
-    give the same bits."""
+    group: a first pass only forms the innovation norms (from one accumulator
+    that receives the fresh product and, negated, the stale one), and after the
+    selection the selected groups' gradients are recomputed and written.  Given
+    the same selections the parameters must come out bit-identical; the norms
+    agree to accumulation order."""
     w = to_cuda(make_workload("cfg5", rows=3000, dims=(64, 128, 40), M=6, M_G=2, D=4, batch=128, c=5.0))
     a = binding.from_workload(w, stream=torch.cuda.Stream(), options={binding.OPT_KEEP_STALE: 1.0})
     b = binding.from_workload(w, stream=torch.cuda.Stream())
-    for chunk in (1, 7, 17):
-        a.step(chunk)
-        b.step(chunk)
+    K = 25
+    for k in range(K):
+        a.step(1)
+        b.step_forced(a.get_selection_mask(k, 1))
         assert np.array_equal(a.get_theta(), b.get_theta())
-        assert np.array_equal(a.get_debug(binding.DBG_LHS), b.get_debug(binding.DBG_LHS))
-        assert np.array_equal(a.get_debug(binding.DBG_GLAST), b.get_debug(binding.DBG_GLAST))
-    ma, mb = a.get_selection_mask(0, 25), b.get_selection_mask(0, 25)
-    assert np.array_equal(ma, mb) and 0 < ma.sum() < ma.size          # some uploads were skipped
+        la, lb = a.get_debug(binding.DBG_LHS), b.get_debug(binding.DBG_LHS)
+        assert np.allclose(la, lb, rtol=2e-3, atol=1e-10), (k, la, lb)   # exact zero vs fp32 residue at k = 0
+    assert np.array_equal(a.get_debug(binding.DBG_GLAST), b.get_debug(binding.DBG_GLAST))
+    ma = a.get_selection_mask(0, K)
+    assert 0 < ma.sum() < ma.size                                      # some uploads were skipped
     assert a.get_comm_count() == b.get_comm_count()
     assert b.get_launch_count() > a.get_launch_count()                 # the second pass exists
+
+
+def test_two_pass_norms_against_the_oracle():
+    """The production path's left side of the test (difference accumulated in
+    tensor memory) against the oracle, teacher-forced."""
+    from parity import make_oracle, TOL_BF16
+    w = make_workload("cfg5", rows=3000, dims=(64, 128, 96, 40), M=6, M_G=2, D=3, batch=128, c=0.3)
+    o = make_oracle(w)
+    g = binding.from_workload(to_cuda(w), stream=torch.cuda.Stream())
+    for k in range(9):
+        rec = o.step()
+        g.step_forced(rec["mask"][None, :])
+        lhs = g.get_debug(binding.DBG_LHS)
+        assert np.allclose(lhs, rec["lhs"], rtol=2 * TOL_BF16, atol=1e-12), (k, lhs, rec["lhs"])
+        fresh = g.get_debug(binding.DBG_FRESH)
+        for gi in np.nonzero(rec["mask"])[0]:          # only selected groups are written
+            assert np.linalg.norm(fresh[gi] - rec["fresh"][gi]) <= TOL_BF16 * np.linalg.norm(rec["fresh"][gi])
+    assert np.linalg.norm(g.get_theta() - o.theta) <= TOL_BF16 * np.linalg.norm(o.theta)
