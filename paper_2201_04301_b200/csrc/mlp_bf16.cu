@@ -28,7 +28,7 @@ namespace gcada {
 
 namespace {
 
-constexpr int BM = 128, BN = 128, BK = 64;      // tile; BK * 2 bytes = one 128-byte swizzle row
+constexpr int BM = 128, BK = 64;  // M tile; K block (BK * 2 bytes = one 128-byte swizzle row)
 constexpr int MAX_STAGES = 8;
 
 enum { EPI_HIDDEN = 0, EPI_SCORES = 1, EPI_DA = 2, EPI_DW = 3 };
@@ -673,10 +673,12 @@ __global__ void __launch_bounds__(256) bf16_convert_kernel(const Params P, const
 }
 
 // ----------------------------------------------------------------- gather (rows and their transpose)
-// Block = 32 consecutive rows of one group; features move through a 32 x 64 tile.
+// Block = 32 consecutive rows of one group; features move through a 32 x 256 tile: 16-byte loads and
+// row-major stores, 64-byte runs for the transposed copy.
+constexpr int GT_COLS = 256, GT_PITCH = GT_COLS + 2;  // pitch of 129 words: conflict-free column reads
 __global__ void __launch_bounds__(256) bf16_gather_kernel(const Params P, __nv_bfloat16* xb, __nv_bfloat16* xbT,
                                                           int* yb, int d, int ld0, int Bp) {
-  __shared__ __nv_bfloat16 tile[32][66];
+  __shared__ __nv_bfloat16 tile[32 * GT_PITCH];
   __shared__ long long rows_sm[32];
   const int g = blockIdx.y, rb = blockIdx.x * 32;
   const int tid = threadIdx.x;
@@ -689,63 +691,90 @@ __global__ void __launch_bounds__(256) bf16_gather_kernel(const Params P, __nv_b
   }
   __syncthreads();
   const __nv_bfloat16* X = reinterpret_cast<const __nv_bfloat16*>(P.X);
-  for (int c0 = 0; c0 < d; c0 += 64) {
-    for (int e = tid; e < 32 * 64; e += 256) {
-      const int r = e >> 6, c = e & 63;
-      const long long row = rows_sm[r];
-      __nv_bfloat16 v = __float2bfloat16_rn(0.f);
-      if (row >= 0 && c0 + c < d) v = X[row * P.ld + c0 + c];
-      tile[r][c] = v;
-      if (c0 + c < d) xb[((long long)g * Bp + rb + r) * ld0 + c0 + c] = v;
+  const bool vec = (P.ld & 7) == 0 && (reinterpret_cast<uintptr_t>(X) & 15) == 0 && (d & 7) == 0;
+  for (int c0 = 0; c0 < d; c0 += GT_COLS) {
+    if (vec) {
+      for (int e = tid; e < 32 * (GT_COLS / 8); e += 256) {
+        const int r = e / (GT_COLS / 8), c = (e - r * (GT_COLS / 8)) * 8;
+        const long long row = rows_sm[r];
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (c0 + c < d) {
+          if (row >= 0) v = *reinterpret_cast<const uint4*>(X + row * P.ld + c0 + c);
+          *reinterpret_cast<uint4*>(xb + ((long long)g * Bp + rb + r) * ld0 + c0 + c) = v;
+        }
+        uint32_t* t = reinterpret_cast<uint32_t*>(tile + r * GT_PITCH + c);
+        t[0] = v.x;
+        t[1] = v.y;
+        t[2] = v.z;
+        t[3] = v.w;
+      }
+    } else {
+      for (int e = tid; e < 32 * GT_COLS; e += 256) {
+        const int r = e / GT_COLS, c = e - r * GT_COLS;
+        const long long row = rows_sm[r];
+        __nv_bfloat16 v = __float2bfloat16_rn(0.f);
+        if (row >= 0 && c0 + c < d) v = X[row * P.ld + c0 + c];
+        tile[r * GT_PITCH + c] = v;
+        if (c0 + c < d) xb[((long long)g * Bp + rb + r) * ld0 + c0 + c] = v;
+      }
     }
     __syncthreads();
-    for (int e = tid; e < 64 * 32; e += 256) {
+    for (int e = tid; e < GT_COLS * 32; e += 256) {
       const int c = e >> 5, r = e & 31;
-      if (c0 + c < d) xbT[((long long)g * d + c0 + c) * Bp + rb + r] = tile[r][c];
+      if (c0 + c < d) xbT[((long long)g * d + c0 + c) * Bp + rb + r] = tile[r * GT_PITCH + c];
     }
     __syncthreads();
   }
 }
 
 // ----------------------------------------------------------------- loss gradient
-// Warp per (point, padded row): dz = (softmax(scores) - onehot(y)) * scale in both orientations;
-// padding rows (y < 0) get zeros.
+// dz = (softmax(scores) - onehot(y)) * scale in both orientations; padding rows (y < 0) get zeros.
+// Block = 32 consecutive rows of one (point, group); each of the 8 warps takes 4 rows; the bf16
+// results also go to a shared tile from which the transposed copy leaves in 64-byte runs.
 __global__ void __launch_bounds__(256) bf16_softmax_grad_kernel(const Params P, const float* scores, const int* yb,
                                                                 __nv_bfloat16* dz, __nv_bfloat16* dzT, int n_cls,
-                                                                int ldz, int Bp) {
+                                                                int ldz, int Bp, int pitch) {
+  extern __shared__ __nv_bfloat16 sm_tile[];  // [32][pitch]
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const long long rows = (long long)P.G * Bp;
-  const long long w = ((long long)blockIdx.x * 256 + threadIdx.x) >> 5;
-  const int lane = threadIdx.x & 31;
-  if (w >= 2 * rows) return;
-  const long long r = w % rows;
-  const int q = (int)(w / rows);
-  const int g = (int)(r / Bp), mrow = (int)(r - (long long)g * Bp);
-  const float* s = scores + w * n_cls;
-  __nv_bfloat16* o = dz + w * ldz;
-  __nv_bfloat16* oT = dzT + ((long long)(q * P.G + g) * n_cls) * Bp + mrow;
-  const int y = yb[r];
-  if (y < 0) {
-    for (int c = lane; c < n_cls; c += 32) {
-      o[c] = __float2bfloat16_rn(0.f);
-      oT[(long long)c * Bp] = __float2bfloat16_rn(0.f);
+  const long long w0 = (long long)blockIdx.x * 32;  // first (point, row) of the block
+  const int q = (int)(w0 / rows);
+  const long long r0 = w0 - (long long)q * rows;
+  const int g = (int)(r0 / Bp), m0 = (int)(r0 - (long long)g * Bp);
+  for (int i = 0; i < 4; ++i) {
+    const int lr = warp * 4 + i;
+    const long long w = w0 + lr;
+    const float* s = scores + w * n_cls;
+    __nv_bfloat16* o = dz + w * ldz;
+    __nv_bfloat16* t = sm_tile + lr * pitch;
+    const int y = yb[r0 + lr];
+    if (y < 0) {
+      for (int c = lane; c < n_cls; c += 32) {
+        o[c] = __float2bfloat16_rn(0.f);
+        t[c] = __float2bfloat16_rn(0.f);
+      }
+      continue;
     }
-    return;
-  }
-  float mx = -3.0e38f;
-  for (int c = lane; c < n_cls; c += 32) mx = fmaxf(mx, s[c]);
+    float mx = -3.0e38f;
+    for (int c = lane; c < n_cls; c += 32) mx = fmaxf(mx, s[c]);
 #pragma unroll
-  for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-  float others = 0.f;
-  for (int c = lane; c < n_cls; c += 32)
-    if (c != y) others += expf(s[c] - mx);
-  others = warp_sum(others);
-  const float inv = 1.0f / (others + expf(s[y] - mx));
-  for (int c = lane; c < n_cls; c += 32) {
-    const float v = (c == y ? -others * inv : expf(s[c] - mx) * inv) * P.scale;
-    const __nv_bfloat16 b = __float2bfloat16_rn(v);
-    o[c] = b;
-    oT[(long long)c * Bp] = b;
+    for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+    // p_y - 1 = -(sum of the other classes' exponentials) / sum, free of cancellation
+    float others = 0.f;
+    for (int c = lane; c < n_cls; c += 32)
+      if (c != y) others += expf(s[c] - mx);
+    others = warp_sum(others);
+    const float inv = 1.0f / (others + expf(s[y] - mx));
+    for (int c = lane; c < n_cls; c += 32) {
+      const float v = (c == y ? -others * inv : expf(s[c] - mx) * inv) * P.scale;
+      const __nv_bfloat16 b = __float2bfloat16_rn(v);
+      o[c] = b;
+      t[c] = b;
+    }
   }
+  __syncthreads();
+  __nv_bfloat16* oT = dzT + ((long long)(q * P.G + g) * n_cls) * Bp + m0;
+  for (int c = warp; c < n_cls; c += 8) oT[(long long)c * Bp + lane] = sm_tile[lane * pitch + c];
 }
 
 // ----------------------------------------------------------------- bias gradients
@@ -758,25 +787,49 @@ struct BiasArgsB {
   int part_base[MLP_MAX_LAYERS + 1];
   int n_parts;
 };
+// Block = 64 columns x 8 row slices: lane pairs of columns (bf16x2 loads), warp = row slice.
 __global__ void __launch_bounds__(256) bf16_bias_grad_kernel(const Params P, const BiasArgsB a, int Bp) {
+  __shared__ float red[2][8][64];
   __shared__ double scratch[40];
   const int l = blockIdx.z + 1;
-  if ((int)blockIdx.x * 256 >= a.n[l]) return;
-  const int n = blockIdx.x * 256 + threadIdx.x;
+  const int n_l = a.n[l];
+  if ((int)blockIdx.x * 64 >= n_l) return;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = blockIdx.y;
-  double d2 = 0.0;
-  if (n < a.n[l]) {
-    const long long rows = (long long)P.G * Bp;
-    const __nv_bfloat16* s0 = a.dz[l] + ((long long)g * Bp) * a.ld[l] + n;
-    const __nv_bfloat16* s1 = s0 + rows * a.ld[l];
-    float f = 0.f, s = 0.f;
-    for (int r = 0; r < Bp; ++r) {
-      f += __bfloat162float(s0[(long long)r * a.ld[l]]);
-      s += __bfloat162float(s1[(long long)r * a.ld[l]]);
+  const int n = blockIdx.x * 64 + 2 * lane;  // this lane's column pair (ld is even, so the pair is inside the row)
+  const long long rows = (long long)P.G * Bp;
+  float f0 = 0.f, f1 = 0.f, s0 = 0.f, s1 = 0.f;
+  if (n < n_l) {
+    const __nv_bfloat16* p0 = a.dz[l] + ((long long)g * Bp) * a.ld[l] + n;
+    const __nv_bfloat16* p1 = p0 + rows * a.ld[l];
+    for (int r = warp; r < Bp; r += 8) {
+      const __nv_bfloat162 u = *reinterpret_cast<const __nv_bfloat162*>(p0 + (long long)r * a.ld[l]);
+      const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(p1 + (long long)r * a.ld[l]);
+      f0 += __low2float(u);
+      f1 += __high2float(u);
+      s0 += __low2float(v);
+      s1 += __high2float(v);
     }
-    (P.fresh + (long long)g * P.p_pad + a.b_off[l])[n] = f;
-    if (P.stale) (P.stale + (long long)g * P.p_pad + a.b_off[l])[n] = s;
-    d2 = (double)(f - s) * (double)(f - s);
+  }
+  red[0][warp][2 * lane] = f0;
+  red[0][warp][2 * lane + 1] = f1;
+  red[1][warp][2 * lane] = s0;
+  red[1][warp][2 * lane + 1] = s1;
+  __syncthreads();
+  double d2 = 0.0;
+  if (threadIdx.x < 64) {
+    const int c = blockIdx.x * 64 + threadIdx.x;
+    if (c < n_l) {
+      float f = 0.f, sv = 0.f;
+#pragma unroll
+      for (int w = 0; w < 8; ++w) {
+        f += red[0][w][threadIdx.x];
+        sv += red[1][w][threadIdx.x];
+      }
+      (P.fresh + (long long)g * P.p_pad + a.b_off[l])[c] = f;
+      if (P.stale) (P.stale + (long long)g * P.p_pad + a.b_off[l])[c] = sv;
+      d2 = (double)(f - sv) * (double)(f - sv);
+    }
   }
   d2 = block_sum(d2, scratch);
   if (threadIdx.x == 0) P.lhs_part[(long long)g * a.n_parts + a.part_base[l] + blockIdx.x] = d2;
@@ -862,6 +915,10 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
     *why = "the bf16 MLP path supports minibatches of at most 256 rows per group";
     return cudaSuccess;
   }
+  if (plan->dims[L] > 3500) {
+    *why = "the bf16 MLP path supports at most 3500 classes";
+    return cudaSuccess;
+  }
   Bf16Impl* im = new Bf16Impl();
   plan->bf16_impl = im;  // lives as long as the process (a few hundred bytes per plan)
   im->Bp = (int)up(B, 128);
@@ -885,7 +942,7 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
   }
   for (int l = 1; l <= L; ++l) {
     im->bias_part_base[l] = parts;
-    parts += (plan->dims[l] + 255) / 256;
+    parts += (plan->dims[l] + 63) / 64;
   }
   im->n_parts = parts;
   plan->norm_parts = parts;
@@ -945,6 +1002,9 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
   }
   cudaError_t e = cudaFuncSetAttribute(bf16_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        G_STAGES * G_STAGE_BYTES + 1024);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(bf16_softmax_grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           32 * (plan->dims[L] + 4) * 2);
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(bf16_dw_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            11 * (BM * BK * 2) + 1024 + DW_STAGE_FLOATS * 4);
@@ -1010,8 +1070,11 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
     if ((e = launch_gemm(im->tm_fwd_a[l], im->tm_fwd_b[l], P, a, pl.sm_count, st)) != cudaSuccess) return e;
     ++n;
   }
-  bf16_softmax_grad_kernel<<<(unsigned)((2 * rows * 32 + 255) / 256), 256, 0, st>>>(
-      P, im->scores, im->yb, im->dz[L], im->dzT[L], pl.dims[L], im->ld[L], Bp);
+  {
+    const int pitch = pl.dims[L] + 2 + (pl.dims[L] & 1);  // even, and an odd number of 32-bit words when possible
+    bf16_softmax_grad_kernel<<<(unsigned)(2 * rows / 32), 256, (size_t)32 * pitch * 2, st>>>(
+        P, im->scores, im->yb, im->dz[L], im->dzT[L], pl.dims[L], im->ld[L], Bp, pitch);
+  }
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   ++n;
   const int dw_mode = P.stale ? DW_BOTH : DW_NORM;  // gradients of every group are materialised only on request
@@ -1048,7 +1111,7 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
     if (pl.dims[l] > maxn) maxn = pl.dims[l];
   }
   ba.n_parts = im->n_parts;
-  bf16_bias_grad_kernel<<<dim3((maxn + 255) / 256, G, L), 256, 0, st>>>(P, ba, Bp);
+  bf16_bias_grad_kernel<<<dim3((maxn + 63) / 64, G, L), 256, 0, st>>>(P, ba, Bp);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   ++n;
   *n_launches = n;
