@@ -92,19 +92,26 @@ class ClockSampler(threading.Thread):
                 "reasons": sorted(self.reasons), "samples": len(s)}
 
 
-def _dist_setup(n_gpus):
+def _dist_setup(n_gpus, backend="nccl"):
+    """One process per GPU (replicas only: no collective on the data path).  Reads RANK / LOCAL_RANK /
+    WORLD_SIZE / MASTER_* from the environment; `backend="gloo"` runs the same host logic on CPU."""
     import torch
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
-    torch.cuda.set_device(local)
+    if backend == "nccl":
+        torch.cuda.set_device(local)
     if world > 1:
         import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        if backend == "nccl":
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        else:
+            dist.init_process_group(backend)
     return rank, local, world
 
 
 def _barrier_max(world, value_ms, device):
+    """Max over ranks of a per-rank time (the job is as slow as its slowest replica)."""
     import torch
     if world == 1:
         return value_ms
@@ -119,7 +126,13 @@ def _barrier(world):
     if world > 1:
         import torch.distributed as dist
         dist.barrier()
-    torch.cuda.synchronize()
+    if torch.cuda.is_available():
+        torch.cuda.synchronize()
+
+
+def aggregate_value(world, steps, ms):
+    """Whole-job iterations per second: every rank ran `steps` iterations in at most `ms`."""
+    return world * steps / (ms * 1e-3)
 
 
 def algorithmic_bytes_per_launch(w):
@@ -182,7 +195,7 @@ def run_ours(args):
     sampler.join()
     ms = _barrier_max(world, e0.elapsed_time(e1), dev)
     launches = g.get_launch_count() - l0
-    value = world * args.steps / (ms * 1e-3)
+    value = aggregate_value(world, args.steps, ms)
 
     # --- per-kernel times (plain launches bracketed by events) -------------------
     g.set_option(binding.OPT_TIMING, 1)

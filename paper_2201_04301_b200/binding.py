@@ -54,6 +54,7 @@ SIGNATURES = {
     "gcada_get_wallclock": (C.c_int, [_VP, C.POINTER(C.c_double), C.POINTER(C.c_double)]),
     "gcada_get_iteration": (C.c_int, [_VP, C.POINTER(_LL)]),
     "gcada_get_debug": (C.c_int, [_VP, C.c_int, _VP, _LL]),
+    "gcada_get_group_gradient": (C.c_int, [_VP, C.c_int, C.c_int, _VP, _LL]),
     "gcada_get_launch_count": (C.c_int, [_VP, _ULLP]),
     "gcada_get_kernel_times": (C.c_int, [_VP, C.POINTER(C.c_double), C.POINTER(C.c_int)]),
     "gcada_innovation_norms_noalloc": (C.c_int, [_VP, _VP, C.c_int, _LL, _LL, _VP, _VP, C.c_char_p, C.c_size_t]),
@@ -198,6 +199,11 @@ class GCada:
         n = C.c_ulonglong()
         self._ck(self.lib.gcada_get_launch_count(self.h, C.byref(n)))
         return n.value
+
+    def get_group_gradient(self, what, g):
+        out = np.empty(self.p, dtype=np.float32)
+        self._ck(self.lib.gcada_get_group_gradient(self.h, int(what), int(g), _VP(out.ctypes.data), self.p))
+        return out
 
     def get_kernel_times(self):
         """(ms_gradient, ms_select, ms_update), n_timed: see GCADA_OPT_TIMING."""

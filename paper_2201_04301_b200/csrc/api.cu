@@ -713,6 +713,26 @@ gcada_status gcada_get_debug(gcada_ctx* ctx, int what, void* out, long long byte
   return GCADA_OK;
 }
 
+gcada_status gcada_get_group_gradient(gcada_ctx* ctx, int what, int g, float* out, long long p) {
+  if (!ctx) return GCADA_EINVAL;
+  if (!out || p != ctx->p) return fail(ctx, GCADA_EINVAL, "need a buffer of p = %lld floats", ctx->p);
+  if (g < 0 || g >= ctx->G) return fail(ctx, GCADA_EINVAL, "group %d out of range", g);
+  if (!ctx->have_theta) return fail(ctx, GCADA_ESTATE, "gcada_set_theta has not been called");
+  DeviceGuard dg(ctx->device);
+  DevState s;
+  TRY(read_state(ctx, &s));
+  const float* src = nullptr;
+  switch (what) {
+    case GCADA_DBG_FRESH: src = ctx->P.fresh; break;
+    case GCADA_DBG_STALE: src = ctx->P.stale; break;
+    case GCADA_DBG_GLAST: src = ctx->P.g_last; break;
+    default: return fail(ctx, GCADA_EINVAL, "item %d is not a per-group gradient", what);
+  }
+  if (!src) return fail(ctx, GCADA_ESTATE, "stale gradients are not kept: set GCADA_OPT_KEEP_STALE");
+  CK(cudaMemcpy(out, src + (long long)g * ctx->p_pad, sizeof(float) * (size_t)p, cudaMemcpyDeviceToHost));
+  return GCADA_OK;
+}
+
 gcada_status gcada_get_launch_count(gcada_ctx* ctx, unsigned long long* launches) {
   if (!ctx || !launches) return GCADA_EINVAL;
   *launches = ctx->launches;

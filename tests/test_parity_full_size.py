@@ -1,0 +1,76 @@
+"""Parity at the full workload sizes, in the launch configuration the benchmark
+times (graph replay on a stream): the CUDA path runs free, then sampled groups'
+gradients are recomputed by the CPU oracle from the CUDA path's own iterate and
+the rows it must have sampled, and properties that hold at any size are checked."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import philox
+from oracle.models import make_model
+from paper_2201_04301_b200 import binding
+from paper_2201_04301_b200.workloads import make_workload
+
+from parity import TOL_BF16, TOL_FP32, rel_l2
+
+pytestmark = pytest.mark.gpu
+
+
+def _group_batch(w, k, g, G):
+    n_g = w["X"].shape[0] // G
+    idx = philox.batch_indices(w["seed"], k, g, w["batch"], n_g)
+    t = torch.as_tensor(idx, device=w["X"].device)
+    d = w["dims"][0]
+    return w["X"].index_select(0, t)[:, :d].float().cpu().numpy().astype(np.float64), w["y"].index_select(0, t).cpu().numpy()
+
+
+def test_cfg3_full_size_sampled_groups():
+    """d = 4096, N = 2,000,000 (32.8 GB resident), 64 groups x 512 rows."""
+    w = make_workload("cfg3", device="cuda")
+    G = w["M"] // w["M_G"]
+    g = binding.from_workload(w, stream=torch.cuda.Stream())
+    model = make_model("logistic", w["dims"])
+    K = 24
+    for k in range(K):
+        theta = g.get_theta().astype(np.float64)
+        g.step(1)
+        if k in (0, 7, 23):
+            for gi in (0, 31, 63):
+                Xb, yb = _group_batch(w, k, gi, G)
+                want = model.grad(theta, Xb, yb, "mean")
+                assert rel_l2(g.get_group_gradient(binding.DBG_FRESH, gi), want) <= TOL_FP32
+    masks = g.get_selection_mask(0, K)
+    up, comm, comp = g.get_comm_count()
+    assert masks[0].all() and up == int(masks.sum()) and comm == (w["M_G"] + 1) * up and comp == w["M_G"] * up
+    # no group goes D iterations without an upload
+    for gi in range(G):
+        gaps = np.diff(np.nonzero(masks[:, gi])[0])
+        assert gaps.size == 0 or gaps.max() <= w["D"]
+    # the aggregate equals the sum of the last uploaded gradients (Eq. 3)
+    agg = g.get_debug(binding.DBG_AGG).astype(np.float64)
+    assert rel_l2(agg, g.get_debug(binding.DBG_GLAST).astype(np.float64).sum(axis=0)) <= 1e-6
+    g.step(200)                       # replayed graphs, 16 iterations each
+    assert g.get_iteration() == K + 200 and np.isfinite(g.get_theta()).all()
+
+
+def test_cfg5_full_size_sampled_groups():
+    """1024-4096-4096-1000, bf16 operands, 256 groups x 128 rows: the first iteration selects every
+    group, so every fresh gradient is written; two of them are recomputed by the oracle."""
+    w = make_workload("cfg5", device="cuda")
+    G = w["M"] // w["M_G"]
+    g = binding.from_workload(w, stream=torch.cuda.Stream())
+    model = make_model("mlp", w["dims"], bf16=True)
+    theta = g.get_theta().astype(np.float64)
+    g.step(1)
+    assert g.get_selection_mask(0, 1).all()
+    for gi in (3, 200):
+        Xb, yb = _group_batch(w, 0, gi, G)
+        want = model.grad(theta, Xb, yb, "mean")
+        got = g.get_group_gradient(binding.DBG_FRESH, gi)
+        assert rel_l2(got, want) <= TOL_BF16
+        assert np.array_equal(got, g.get_group_gradient(binding.DBG_GLAST, gi))
+    g.step(12)
+    masks = g.get_selection_mask(0, 13)
+    up, comm, comp = g.get_comm_count()
+    assert up == int(masks.sum()) and comm == 5 * up and comp == 4 * up
+    assert np.isfinite(g.get_theta()).all()
