@@ -147,7 +147,11 @@ gcada_status gcada_set_delay_model(gcada_ctx *ctx, double shift, double rate);
 
 gcada_status gcada_set_option(gcada_ctx *ctx, int key, double value);
 
-/* Smoothness constants L_g (host, G doubles) for rule PS (Eq. 9 as printed). */
+/* Smoothness constants L_g >= 0 (host, G doubles; copied) for rule PS, the left side of Eq. (9) as
+ * printed: L_g^2 ||theta^k - theta^{k-tau_g}||^2, evaluated from the ring of the last D+1 iterates.  Set
+ * them before the first step; stepping with GCADA_OPT_RULE = 1 and no constants gives GCADA_ESTATE.  In this
+ * build the gradients of every group are still evaluated each iteration (at both points); only the test and
+ * therefore the selection, the aggregate and the counters follow the printed rule. */
 gcada_status gcada_set_smoothness(gcada_ctx *ctx, const double *L, int G);
 
 /* Run n_iters iterations of Algorithm 1 on the stream (asynchronous).

@@ -246,7 +246,7 @@ def innovation_norms_noalloc(fresh, stale, lhs_out, stream=None):
         raise GCadaError(st, buf.value.decode())
 
 
-def from_workload(w, stream=None, options=None):
+def from_workload(w, stream=None, options=None, smoothness=None):
     """Context for a dict made by workloads.make_workload (tensors on CUDA)."""
     g = GCada(w["kind"], w["dims"], w["M"], w["M_G"], w["D"], w["c"], w["alpha"], w["beta1"], w["beta2"],
               w["eps"], compute=w["compute"], stream=stream)
@@ -254,6 +254,8 @@ def from_workload(w, stream=None, options=None):
     g.set_delay_model(w["shift"], w["rate"])
     for key, val in (options or {}).items():
         g.set_option(key, val)
+    if smoothness is not None:
+        g.set_smoothness(smoothness)
     g.set_data(w["X"], w["y"], w["batch"], ld=w["ld"])
     g.set_theta(w["theta0"])
     return g

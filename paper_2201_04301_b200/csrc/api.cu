@@ -48,6 +48,7 @@ struct gcada_ctx {
   unsigned long long launches = 0;
   // device memory
   std::vector<void*> owned;
+  std::vector<double> L2;  // squared smoothness constants (rule PS)
   DevState* st = nullptr;
   Params P{};
   LinearPlan lin{};
@@ -246,6 +247,16 @@ gcada_status make_plans(gcada_ctx* ctx) {
       TRY(dev_alloc(ctx, &P.lhs_part, (size_t)ctx->G * ctx->mlp.norm_parts));
     }
   }
+  if (ctx->rule == 1) {
+    double* l2 = nullptr;
+    TRY(dev_alloc(ctx, &l2, (size_t)ctx->G));
+    CK(cudaMemcpyAsync(l2, ctx->L2.data(), sizeof(double) * ctx->G, cudaMemcpyHostToDevice, ctx->stream));
+    P.ps_L2 = l2;
+    TRY(dev_alloc(ctx, &P.ps_lhs, (size_t)ctx->G));
+    TRY(dev_alloc(ctx, &P.ps_part, (size_t)ctx->D * ctx->tail.ps_blocks));
+  } else {
+    P.ps_L2 = nullptr;
+  }
   CK(cudaStreamSynchronize(ctx->stream));
   ctx->ready = true;
   return GCADA_OK;
@@ -270,6 +281,10 @@ gcada_status enqueue_iteration(gcada_ctx* ctx, const Params& P) {
     ctx->launches += (unsigned long long)n;
   }
   if (ev) CK(cudaEventRecord(ev[1], ctx->stream));
+  if (P.ps_L2) {
+    CK(launch_ps_lhs(P, ctx->tail, ctx->stream));
+    ctx->launches += 1;
+  }
   CK(launch_select(P, ctx->tail, ctx->stream));
   if (ev) CK(cudaEventRecord(ev[2], ctx->stream));
   if (!is_linear(ctx)) {  // gradient work that needs the selection (counted with the gradient phase)
@@ -309,16 +324,17 @@ gcada_status capture(gcada_ctx* ctx, int iters, cudaGraphExec_t* out) {
 }
 
 int kernels_per_iteration(const gcada_ctx* ctx) {
-  if (is_linear(ctx)) return 3;
+  if (is_linear(ctx)) return 3 + (ctx->rule == 1 ? 1 : 0);
   const bool two_pass = ctx->compute == GCADA_COMPUTE_BF16 && !ctx->P.stale;
-  return 2 + ctx->mlp.launches_per_iter + (two_pass ? ctx->mlp.n_layers : 0);
+  return 2 + ctx->mlp.launches_per_iter + (two_pass ? ctx->mlp.n_layers : 0) + (ctx->rule == 1 ? 1 : 0);
 }
 
 gcada_status check_runnable(gcada_ctx* ctx, bool need_data) {
   if (!ctx->have_theta) return fail(ctx, GCADA_ESTATE, "gcada_set_theta has not been called");
   if (need_data && !ctx->have_data) return fail(ctx, GCADA_ESTATE, "gcada_set_data has not been called");
   if (ctx->B <= 0) return fail(ctx, GCADA_ESTATE, "no minibatch size: call gcada_set_data or gcada_set_batch");
-  if (ctx->rule != 0) return fail(ctx, GCADA_EINVAL, "rule PS is not available in this build");
+  if (ctx->rule != 0 && ctx->L2.empty())
+    return fail(ctx, GCADA_ESTATE, "rule PS needs the smoothness constants: call gcada_set_smoothness");
   return GCADA_OK;
 }
 
@@ -485,7 +501,6 @@ gcada_status gcada_set_option(gcada_ctx* ctx, int key, double value) {
   switch (key) {
     case GCADA_OPT_RULE:
       if (value != 0 && value != 1) return fail(ctx, GCADA_EINVAL, "rule must be 0 (INNOV) or 1 (PS)");
-      if (value == 1) return fail(ctx, GCADA_EINVAL, "rule PS is not available in this build");
       ctx->rule = (int)value;
       break;
     case GCADA_OPT_REDUCTION:
@@ -524,7 +539,14 @@ gcada_status gcada_set_option(gcada_ctx* ctx, int key, double value) {
 gcada_status gcada_set_smoothness(gcada_ctx* ctx, const double* L, int G) {
   if (!ctx) return GCADA_EINVAL;
   if (!L || G != ctx->G) return fail(ctx, GCADA_EINVAL, "need G = %d smoothness constants", ctx->G);
-  return fail(ctx, GCADA_EINVAL, "rule PS is not available in this build");
+  for (int g = 0; g < G; ++g)
+    if (!(L[g] >= 0)) return fail(ctx, GCADA_EINVAL, "smoothness constants must be non-negative");
+  if (ctx->k_host > 0) return fail(ctx, GCADA_ESTATE, "the smoothness constants are fixed once stepping has begun");
+  ctx->L2.resize(G);
+  for (int g = 0; g < G; ++g) ctx->L2[g] = L[g] * L[g];
+  ctx->ready = false;  // the device copy is made with the plans
+  drop_graphs(ctx);
+  return GCADA_OK;
 }
 
 static gcada_status run_iterations(gcada_ctx* ctx, int n_iters, const unsigned char* mask) {

@@ -79,6 +79,10 @@ struct Params {
   long long hist_cap;
   const unsigned char* forced;  // [n][G] or null
   long long forced_base;        // iteration of forced row 0
+  // rule PS (the left side of Eq. (9) as printed): L_g^2 ||theta^k - theta^{k-tau_g}||^2
+  const double* ps_L2;          // [G] squared smoothness constants, or null (rule INNOV)
+  double* ps_lhs;               // [G] the printed left side, written by ps_lhs_kernel
+  double* ps_part;              // [D][blocks] partial sums of ||theta^k - theta^{k-d}||^2
 };
 
 // ---------------------------------------------------------------------------

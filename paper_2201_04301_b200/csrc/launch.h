@@ -31,8 +31,11 @@ struct TailPlan {
   int select_cols4_per_block;  // float4 columns per block of the selection kernel
   int select_blocks_x;         // blocks per group
   int update_blocks;
+  int ps_blocks;               // column blocks of ps_lhs_kernel
 };
 void plan_tail(long long p_pad, int G, int sm_count, TailPlan* plan);
+// Rule PS only: the printed left side of Eq. (9) for every group (run before the selection kernel).
+cudaError_t launch_ps_lhs(const Params& P, const TailPlan& plan, cudaStream_t st);
 cudaError_t launch_select(const Params& P, const TailPlan& plan, cudaStream_t st);
 cudaError_t launch_update(const Params& P, const TailPlan& plan, cudaStream_t st);
 

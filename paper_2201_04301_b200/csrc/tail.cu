@@ -147,6 +147,7 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
       }
     }
     if (have) {
+      if (P.ps_L2) lhs = P.ps_lhs[gg];  // rule PS: the test uses the printed left side, not the measured innovation
       const bool sel = P.forced ? sel_forced : ((tau >= P.D) || (lhs > rhs));
       P.lhs[gg] = lhs;
       P.t_g[gg] = t;
@@ -334,6 +335,52 @@ __global__ void __launch_bounds__(256) update_kernel(const Params P) {
   }
 }
 
+// Rule PS: left side of Eq. (9) exactly as printed, L_g^2 ||theta^k - theta^{k-tau_g}||^2, from the
+// iterate ring.  Grid (column blocks, D): block (b, d-1) sums its slice of ||theta^k - theta^{k-d}||^2
+// (theta^j = theta^0 for j < 0); the last block adds the slices in a fixed order and scales by L_g^2.
+__global__ void __launch_bounds__(256) ps_lhs_kernel(const Params P) {
+  __shared__ double scratch[40];
+  __shared__ bool is_last;
+  const int tid = threadIdx.x;
+  const int d = blockIdx.y + 1;
+  const long long cols4 = P.p_pad >> 2;
+  const long long k = P.st->k;
+  const int ring = P.D + 1;
+  long long j = k - d;
+  if (j < 0) j = 0;
+  const float* a = P.theta_ring + (k % ring) * P.p_pad;
+  const float* b = P.theta_ring + (j % ring) * P.p_pad;
+  double local = 0.0;
+  for (long long i4 = (long long)blockIdx.x * 256 + tid; i4 < cols4; i4 += (long long)gridDim.x * 256) {
+    const float4 x = ld4(a + i4 * 4), y = ld4(b + i4 * 4);
+    const float dx = x.x - y.x, dy = x.y - y.y, dz = x.z - y.z, dw = x.w - y.w;
+    local += (double)dx * dx + (double)dy * dy + (double)dz * dz + (double)dw * dw;
+  }
+  const double tot = block_sum(local, scratch);
+  if (tid == 0) {
+    P.ps_part[(long long)(d - 1) * gridDim.x + blockIdx.x] = tot;
+    __threadfence();
+    is_last = atomicAdd(&P.st->ticket_aux, 1u) == gridDim.x * gridDim.y - 1u;
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  const volatile double* parts = P.ps_part;
+  for (int g = tid; g < P.G; g += 256) {
+    const int tau = P.tau[g];
+    const int dd = tau < 1 ? 1 : (tau > P.D ? P.D : tau);
+    double s = 0.0;
+    for (unsigned int bb = 0; bb < gridDim.x; ++bb) s += parts[(long long)(dd - 1) * gridDim.x + bb];
+    P.ps_lhs[g] = P.ps_L2[g] * s;
+  }
+  if (tid == 0) P.st->ticket_aux = 0u;
+}
+
+cudaError_t launch_ps_lhs(const Params& P, const TailPlan& plan, cudaStream_t st) {
+  ps_lhs_kernel<<<dim3(plan.ps_blocks, P.D), 256, 0, st>>>(P);
+  return cudaGetLastError();
+}
+
 void plan_tail(long long p_pad, int G, int sm_count, TailPlan* plan) {
   (void)G;
   (void)sm_count;
@@ -342,6 +389,8 @@ void plan_tail(long long p_pad, int G, int sm_count, TailPlan* plan) {
   plan->select_cols4_per_block = 256 * U;
   plan->select_blocks_x = (int)((cols4 + 256 * U - 1) / (256 * U));
   plan->update_blocks = (int)((cols4 + 31) / 32);
+  long long pb = (cols4 + 256 * 8 - 1) / (256 * 8);  // about eight float4 per thread
+  plan->ps_blocks = (int)(pb < 1 ? 1 : (pb > 1024 ? 1024 : pb));
 }
 
 cudaError_t launch_select(const Params& P, const TailPlan& plan, cudaStream_t st) {

@@ -80,15 +80,17 @@ def _kink_match(o, got, theta, Xb, yb, reduction, tol, kink_tol):
 
 
 def forced_parity(w, K, tol=TOL_FP32, stream=None, reduction="mean", check_stale=True, kink_tol=2e-6,
-                  margin=MARGIN, rhs_tol=1e-4):
+                  margin=MARGIN, rhs_tol=1e-4, L=None):
     """Run the oracle free for K steps and the CUDA path teacher-forced with the
     oracle's masks; compare every step.  Returns the number of steps at which
     the CUDA path's own test outcome differed from the oracle's (only allowed
     within MARGIN)."""
-    o = make_oracle(w, reduction=reduction)
+    o = make_oracle(w, reduction=reduction, **({"rule": "ps", "L": L} if L is not None else {}))
     wc = to_cuda(w)
     opts = {binding.OPT_KEEP_STALE: 1.0, binding.OPT_REDUCTION: 0.0 if reduction == "mean" else 1.0}
-    g = binding.from_workload(wc, stream=stream, options=opts)
+    if L is not None:
+        opts[binding.OPT_RULE] = 1.0
+    g = binding.from_workload(wc, stream=stream, options=opts, smoothness=L)
     flips = 0
     worst = dict(fresh=0.0, stale=0.0, theta=0.0, lhs=0.0, kinks=0)
     is_mlp = w["kind"] == "mlp"

@@ -151,3 +151,28 @@ def test_state_errors_and_history_window():
     assert g.get_launch_count() == 60
     g.set_theta(w["theta0"])                       # restart
     assert g.get_iteration() == 0 and g.get_comm_count() == (0, 0, 0)
+
+
+def test_rule_ps_printed_left_side():
+    """GCADA_OPT_RULE = 1: the test uses L_g^2 ||theta^k - theta^{k-tau_g}||^2 (Eq. 9 as printed)."""
+    w = make_workload("cfg1", rows=3000, D=5, c=0.4)
+    L = [0.9, 1.4, 2.0]
+    flips, worst = forced_parity(w, 40, stream=_stream(), L=L)
+    print("rule PS worst", worst, "flips", flips)
+    # free-running: masks equal the oracle's (up to near-ties) and uploads are skipped
+    o = make_oracle(w, rule="ps", L=L)
+    g = binding.from_workload(to_cuda(w), stream=_stream(), options={binding.OPT_RULE: 1.0}, smoothness=L)
+    g.step(40)
+    got = g.get_selection_mask(0, 40)
+    for k in range(40):
+        rec = o.step()
+        if not np.array_equal(got[k], rec["mask"]):
+            for gi in np.nonzero(got[k] != rec["mask"])[0]:
+                assert abs(rec["lhs"][gi] - rec["rhs"]) / max(rec["lhs"][gi], rec["rhs"]) < MARGIN
+            break
+    assert 0 < got.sum() < got.size
+    # without constants the rule cannot run
+    h = binding.from_workload(to_cuda(w), options={binding.OPT_RULE: 1.0})
+    with pytest.raises(binding.GCadaError) as e:
+        h.step(1)
+    assert e.value.status == binding.ESTATE
