@@ -92,6 +92,9 @@ template <int THREADS, int CPT, int R, int MINB, bool QUAD, bool FULL>
 __global__ void __launch_bounds__(THREADS, MINB) grad_linear_large_kernel(const Params P, int nslot) {
   constexpr int V = 2 * R;
   constexpr int NW = THREADS / 32;
+  // the copies are issued by lane 0 of the last warp: the first R warps are on the critical path of every
+  // batch (they turn the dot products into coefficients), the last one is not
+  constexpr int ISSUER = THREADS - 32;
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int d = P.d;
@@ -192,7 +195,7 @@ __global__ void __launch_bounds__(THREADS, MINB) grad_linear_large_kernel(const 
     }
     __syncthreads();
     int issued = 0;
-    if (tid == 0) {
+    if (tid == ISSUER) {
       const int n0 = nrows < nslot ? nrows : nslot;
       for (; issued < n0; ++issued) {
         int s = cslot + issued;
@@ -273,7 +276,7 @@ __global__ void __launch_bounds__(THREADS, MINB) grad_linear_large_kernel(const 
       for (int v = 0; v < V; ++v) part[v * THREADS + tid] = pz[v];
       failed = __syncthreads_or(failed);  // (A) rows are in registers: their slots are free
       if (failed) break;
-      if (tid == 0) {
+      if (tid == ISSUER) {
         for (int r = 0; r < nb && issued < nrows; ++r, ++issued) {
           int s = cslot + r;  // slot of a row consumed just now
           if (s >= nslot) s -= nslot;
@@ -339,7 +342,7 @@ __global__ void __launch_bounds__(THREADS, MINB) grad_linear_large_kernel(const 
     }
     if (failed) {
       // give copies already in flight a bounded chance to land before leaving
-      if (tid == 0) {
+      if (tid == ISSUER) {
         atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
         for (int j = consumed; j < issued; ++j) {
           int s = cslot + (j - consumed);
