@@ -175,8 +175,8 @@ gcada_status make_ready(gcada_ctx* ctx, const float* theta0, int on_device) {
   TRY(dev_alloc(ctx, &P.vhat, (size_t)pp));
   TRY(dev_alloc(ctx, &P.agg_hi, (size_t)pp));
   TRY(dev_alloc(ctx, &P.agg_lo, (size_t)pp));
-  TRY(dev_alloc(ctx, &P.g_last, (size_t)G * pp));
-  TRY(dev_alloc(ctx, &P.fresh, (size_t)G * pp));
+  TRY(dev_alloc(ctx, &P.gbuf, (size_t)2 * G * pp));
+  TRY(dev_alloc(ctx, &P.cur, (size_t)G));
   // the fp32 MLP kernels hand over both gradients; the others keep the stale one only on request
   if (ctx->keep_stale || (!is_linear(ctx) && ctx->compute == GCADA_COMPUTE_FP32))
     TRY(dev_alloc(ctx, &P.stale, (size_t)G * pp));
@@ -336,6 +336,15 @@ gcada_status check_runnable(gcada_ctx* ctx, bool need_data) {
   if (ctx->rule != 0 && ctx->L2.empty())
     return fail(ctx, GCADA_ESTATE, "rule PS needs the smoothness constants: call gcada_set_smoothness");
   return GCADA_OK;
+}
+
+// Device row holding group g's fresh gradient of the last iteration (what = 0) or its last uploaded
+// gradient (what = 1), given host copies of cur[] and of the last selection mask.
+const float* group_row(const gcada_ctx* ctx, int what, int g, const std::vector<unsigned char>& cur,
+                       const std::vector<unsigned char>& mask) {
+  int buf = cur[g];
+  if (what == 0 && !mask[g]) buf = 1 - buf;  // an unselected group's fresh gradient sits in the other row
+  return ctx->P.gbuf + ((long long)buf * ctx->G + g) * ctx->p_pad;
 }
 
 gcada_status read_state(gcada_ctx* ctx, DevState* out) {
@@ -711,12 +720,13 @@ gcada_status gcada_get_debug(gcada_ctx* ctx, int what, void* out, long long byte
   const long long G = ctx->G, p = ctx->p, pp = ctx->p_pad;
   const void* src = nullptr;
   long long rows = 1, row_bytes = 0, src_pitch = 0;
+  int per_group = -1;
   switch (what) {
-    case GCADA_DBG_FRESH: src = P.fresh; rows = G; row_bytes = p * 4; src_pitch = pp * 4; break;
+    case GCADA_DBG_FRESH: per_group = 0; break;
     case GCADA_DBG_STALE:
       if (!P.stale) return fail(ctx, GCADA_ESTATE, "stale gradients are not kept: set GCADA_OPT_KEEP_STALE");
       src = P.stale; rows = G; row_bytes = p * 4; src_pitch = pp * 4; break;
-    case GCADA_DBG_GLAST: src = P.g_last; rows = G; row_bytes = p * 4; src_pitch = pp * 4; break;
+    case GCADA_DBG_GLAST: per_group = 1; break;
     case GCADA_DBG_LHS: src = P.lhs; row_bytes = G * 8; break;
     case GCADA_DBG_RHS: src = &ctx->st->rhs; row_bytes = 8; break;
     case GCADA_DBG_TAU: src = P.tau; row_bytes = G * 4; break;
@@ -726,6 +736,16 @@ gcada_status gcada_get_debug(gcada_ctx* ctx, int what, void* out, long long byte
     case GCADA_DBG_TGROUP: src = P.t_g; row_bytes = G * 8; break;
     case GCADA_DBG_SRING: src = P.s_ring; row_bytes = (long long)ctx->D * 8; break;
     default: return fail(ctx, GCADA_EINVAL, "unknown debug item %d", what);
+  }
+  if (per_group >= 0) {
+    if (bytes != G * p * 4) return fail(ctx, GCADA_EINVAL, "item %d has %lld bytes, buffer has %lld", what, G * p * 4, bytes);
+    std::vector<unsigned char> cur((size_t)G), mask((size_t)G);
+    CK(cudaMemcpy(cur.data(), P.cur, (size_t)G, cudaMemcpyDeviceToHost));
+    CK(cudaMemcpy(mask.data(), P.mask_cur, (size_t)G, cudaMemcpyDeviceToHost));
+    for (int g = 0; g < (int)G; ++g)
+      CK(cudaMemcpy(static_cast<float*>(out) + (long long)g * p, group_row(ctx, per_group, g, cur, mask),
+                    (size_t)p * 4, cudaMemcpyDeviceToHost));
+    return GCADA_OK;
   }
   if (bytes != rows * row_bytes) return fail(ctx, GCADA_EINVAL, "item %d has %lld bytes, buffer has %lld", what, rows * row_bytes, bytes);
   if (rows == 1)
@@ -744,14 +764,18 @@ gcada_status gcada_get_group_gradient(gcada_ctx* ctx, int what, int g, float* ou
   DevState s;
   TRY(read_state(ctx, &s));
   const float* src = nullptr;
-  switch (what) {
-    case GCADA_DBG_FRESH: src = ctx->P.fresh; break;
-    case GCADA_DBG_STALE: src = ctx->P.stale; break;
-    case GCADA_DBG_GLAST: src = ctx->P.g_last; break;
-    default: return fail(ctx, GCADA_EINVAL, "item %d is not a per-group gradient", what);
+  if (what == GCADA_DBG_STALE) {
+    if (!ctx->P.stale) return fail(ctx, GCADA_ESTATE, "stale gradients are not kept: set GCADA_OPT_KEEP_STALE");
+    src = ctx->P.stale + (long long)g * ctx->p_pad;
+  } else if (what == GCADA_DBG_FRESH || what == GCADA_DBG_GLAST) {
+    std::vector<unsigned char> cur((size_t)ctx->G), mask((size_t)ctx->G);
+    CK(cudaMemcpy(cur.data(), ctx->P.cur, (size_t)ctx->G, cudaMemcpyDeviceToHost));
+    CK(cudaMemcpy(mask.data(), ctx->P.mask_cur, (size_t)ctx->G, cudaMemcpyDeviceToHost));
+    src = group_row(ctx, what == GCADA_DBG_GLAST ? 1 : 0, g, cur, mask);
+  } else {
+    return fail(ctx, GCADA_EINVAL, "item %d is not a per-group gradient", what);
   }
-  if (!src) return fail(ctx, GCADA_ESTATE, "stale gradients are not kept: set GCADA_OPT_KEEP_STALE");
-  CK(cudaMemcpy(out, src + (long long)g * ctx->p_pad, sizeof(float) * (size_t)p, cudaMemcpyDeviceToHost));
+  CK(cudaMemcpy(out, src, sizeof(float) * (size_t)p, cudaMemcpyDeviceToHost));
   return GCADA_OK;
 }
 

@@ -62,8 +62,10 @@ struct Params {
   float* vhat;
   float* agg_hi;        // lazily aggregated gradient, Eq. (3), as an unevaluated sum hi + lo
   float* agg_lo;
-  float* g_last;        // [G] last uploaded gradient
-  float* fresh;         // [G] gradient at theta^k
+  // Two gradient buffers per group: buffer cur[g] holds the group's last uploaded gradient, the other one
+  // receives this iteration's fresh gradient; selecting the group flips cur[g], so nothing is copied.
+  float* gbuf;          // [2][G] rows of p_pad floats
+  unsigned char* cur;   // [G]
   float* stale;         // [G] gradient at the stale iterate (optional, may be null)
   float* partial;       // [slots][2] partial sums of (fresh, stale)
   PartialMap pm;
@@ -113,6 +115,19 @@ __device__ __forceinline__ long long batch_row(const Params& P, uint32_t k, int 
   if (P.identity_batch) return (long long)g * P.B + j;
   const uint32_t w = philox_word((uint32_t)j, (uint32_t)g, k, 0u, P.seed_lo, P.seed_hi);
   return (long long)g * P.n_g + (long long)(((unsigned long long)w * (unsigned long long)P.n_g) >> 32);
+}
+
+// Row that receives group g's gradient at theta^k BEFORE this iteration's selection has flipped cur[g].
+__device__ __forceinline__ float* fresh_row(const Params& P, int g) {
+  return P.gbuf + ((long long)(1 - P.cur[g]) * P.G + g) * P.p_pad;
+}
+// Row holding the last uploaded gradient of group g (for a group selected this iteration, after the flip,
+// that is its fresh gradient) and the other row (for such a group: the gradient it replaces).
+__device__ __forceinline__ float* last_row(const Params& P, int g) {
+  return P.gbuf + ((long long)P.cur[g] * P.G + g) * P.p_pad;
+}
+__device__ __forceinline__ float* other_row(const Params& P, int g) {
+  return P.gbuf + ((long long)(1 - P.cur[g]) * P.G + g) * P.p_pad;
 }
 
 // Computing time of worker m at iteration k (Section II-B).

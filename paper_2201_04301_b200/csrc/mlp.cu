@@ -120,7 +120,7 @@ __global__ void __launch_bounds__(256) mlp_sgemm_kernel(const Params P, const Ge
 
   float* Cb;
   if (a.c_grad)
-    Cb = (q == 0 ? P.fresh : P.stale) + (long long)g * P.p_pad + a.c_off;
+    Cb = (q == 0 ? fresh_row(P, g) : P.stale + (long long)g * P.p_pad) + a.c_off;
   else
     Cb = a.C + g * a.c_zg + q * a.c_zq;
   const float* Mb = a.mask ? a.mask + g * a.c_zg + q * a.c_zq : nullptr;
@@ -187,7 +187,7 @@ __global__ void __launch_bounds__(256) mlp_bias_grad_kernel(const Params P, cons
   const float* src = a.dz[l] + ((long long)z * P.B) * a.n[l] + n;
   float s = 0.f;
   for (int r = 0; r < P.B; ++r) s += src[(long long)r * a.n[l]];
-  ((q == 0 ? P.fresh : P.stale) + (long long)g * P.p_pad + a.b_off[l])[n] = s;
+  ((q == 0 ? fresh_row(P, g) : P.stale + (long long)g * P.p_pad) + a.b_off[l])[n] = s;
 }
 
 cudaError_t launch_gemm(const Params& P, const GemmArgs& a, cudaStream_t st) {

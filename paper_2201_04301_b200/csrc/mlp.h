@@ -36,7 +36,7 @@ const char* mlp_supported(const std::vector<int>& dims, int compute);
 cudaError_t mlp_plan_create(const std::vector<int>& dims, int compute, int G, int B, int D, long long p_pad,
                             int sm_count, cudaStream_t st, MlpPlan* plan, std::vector<void*>* owned,
                             const char** why);
-// Enqueues the dual-point forward/backward of every group; writes P.fresh and P.stale.
+// Enqueues the dual-point forward/backward of every group; writes each group's fresh-gradient row and P.stale.
 cudaError_t launch_grad_mlp(const Params& P, const MlpPlan& plan, cudaStream_t st, int* n_launches);
 // Gradient work that must follow the selection kernel (none for the fp32 path).
 cudaError_t launch_grad_mlp_post(const Params& P, const MlpPlan& plan, cudaStream_t st, int* n_launches);

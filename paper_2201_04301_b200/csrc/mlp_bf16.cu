@@ -534,7 +534,7 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
     const int quad = warp & 3;         // TMEM lanes this warp may read
     const int half = ew >> 2;          // which 128 columns of the tile
     float* stg = stage_all + (size_t)ew * 32 * DW_PITCH;
-    const bool vec_ok = ((a.c_off | a.ldc) & 3) == 0 && (reinterpret_cast<uintptr_t>(P.fresh) & 15) == 0 &&
+    const bool vec_ok = ((a.c_off | a.ldc) & 3) == 0 && (reinterpret_cast<uintptr_t>(P.gbuf) & 15) == 0 &&
                         (P.p_pad & 3) == 0;
     bool ok = true;
     int i = 0;
@@ -552,7 +552,9 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
       }
       if (ok) {
         tc_fence_after();
-        float* fresh = P.fresh + (long long)g * P.p_pad + a.c_off;
+        // before the selection the fresh gradient goes to the row that is not the last uploaded one; the
+        // post-selection pass runs on selected groups only, whose cur[g] already points at that same row
+        float* fresh = (a.mode == DW_SELECTED ? last_row(P, g) : fresh_row(P, g)) + a.c_off;
         float* stale = (a.mode == DW_BOTH && P.stale) ? P.stale + (long long)g * P.p_pad + a.c_off : nullptr;
         const int n_pass = a.mode == DW_NORM ? 0 : (stale ? 2 : 1);
         const int mrow = mt * BM + quad * 32;
@@ -826,7 +828,7 @@ __global__ void __launch_bounds__(256) bf16_bias_grad_kernel(const Params P, con
         f += red[0][w][threadIdx.x];
         sv += red[1][w][threadIdx.x];
       }
-      (P.fresh + (long long)g * P.p_pad + a.b_off[l])[c] = f;
+      (fresh_row(P, g) + a.b_off[l])[c] = f;
       if (P.stale) (P.stale + (long long)g * P.p_pad + a.b_off[l])[c] = sv;
       d2 = (double)(f - sv) * (double)(f - sv);
     }
@@ -885,7 +887,12 @@ cudaError_t launch_dw(const Params& P, const MlpPlan& pl, const Bf16Impl* im, in
   w.K = im->Bp;
   w.b_shared = l == 1;
   w.nkb = im->Bp / BK;
-  w.stages = (11 - 2 * w.nkb) / 2;  // 32 KiB B blocks in the shared memory left beside the resident A blocks
+  // 32 KiB B blocks in whatever shared memory is left beside the resident A blocks (and the staging tile of
+  // the modes that write gradients): the B stream is bound by bytes in flight, so every stage counts
+  const long long stage_bytes = mode == DW_NORM ? 0 : (long long)DW_STAGE_FLOATS * 4;
+  const long long room = 232448 - 4096 - 1024 - (long long)2 * w.nkb * (BM * BK * 2) - stage_bytes;
+  w.stages = (int)(room / (DW_BN * BK * 2));
+  if (w.stages > MAX_STAGES) w.stages = MAX_STAGES;
   if (w.stages < 1) w.stages = 1;
   w.tiles_m = (w.M + BM - 1) / BM;
   w.tiles_n = (w.N + DW_BN - 1) / DW_BN;
@@ -897,7 +904,7 @@ cudaError_t launch_dw(const Params& P, const MlpPlan& pl, const Bf16Impl* im, in
   w.mode = mode;
   const int units = w.tiles_m * P.G;
   const int ctas = units < pl.sm_count ? units : pl.sm_count;
-  const size_t smem = (size_t)(2 * w.nkb + 2 * w.stages) * (BM * BK * 2) + 1024 + DW_STAGE_FLOATS * 4;
+  const size_t smem = (size_t)(2 * w.nkb + 2 * w.stages) * (BM * BK * 2) + 1024 + (size_t)stage_bytes;
   bf16_dw_kernel<<<ctas, DW_THREADS, smem, st>>>(im->tm_dw_a[l], im->tm_dw_b[l], P, w);
   return cudaGetLastError();
 }
@@ -1006,8 +1013,7 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
   e = cudaFuncSetAttribute(bf16_softmax_grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            32 * (plan->dims[L] + 4) * 2);
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(bf16_dw_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           11 * (BM * BK * 2) + 1024 + DW_STAGE_FLOATS * 4);
+  e = cudaFuncSetAttribute(bf16_dw_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 4096);  // the rest is static
   if (e != cudaSuccess) return e;
   plan->launches_per_iter = 3 + L + 1 + L + (L - 1);
   return cudaSuccess;

@@ -37,6 +37,7 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
   // ---- phase 1: partial sums -> fresh_g (and stale_g), innovation norm
   // (skipped when the gradient kernels have already delivered the norm partial sums)
   if (P.pm.n_cta >= 0) {
+    float* fresh_g = fresh_row(P, g);
     int c_lo = 0, c_hi = -1;
     const long long Rtot = (long long)P.G * P.pm.rows_per_group;
     const int n = P.pm.n_cta;
@@ -76,11 +77,11 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
           }
         }
         // second slot half = innovation; the stale-point gradient is fresh - innovation
-        st4(P.fresh + (long long)g * P.p_pad + i4 * 4, f);
+        st4(fresh_g + i4 * 4, f);
         if (P.stale)
           st4(P.stale + (long long)g * P.p_pad + i4 * 4, make_float4(f.x - s.x, f.y - s.y, f.z - s.z, f.w - s.w));
       } else {
-        f = ld4(P.fresh + (long long)g * P.p_pad + i4 * 4);
+        f = ld4(fresh_g + i4 * 4);
         s = ld4(P.stale + (long long)g * P.p_pad + i4 * 4);
         s = make_float4(f.x - s.x, f.y - s.y, f.z - s.z, f.w - s.w);
       }
@@ -154,6 +155,7 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
       P.mask_cur[gg] = sel ? 1 : 0;
       P.hist[(k % P.hist_cap) * P.G + gg] = sel ? 1 : 0;
       P.tau[gg] = sel ? 1 : tau + 1;
+      if (sel) P.cur[gg] ^= 1;  // the fresh gradient's row becomes the last uploaded one
       if (sel) {
         ++nsel;
         tmax = fmax(tmax, t);
@@ -244,20 +246,17 @@ __global__ void __launch_bounds__(256) update_kernel(const Params P) {
   if (active) {
     for (int j0 = warp; j0 < n_sel; j0 += 32) {  // four groups of this warp per round, loads first
       float4 f[4], l[4];
-      long long go[4];
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         const int j = j0 + 8 * u;
         if (j < n_sel) {
-          go[u] = (long long)sel_list[j] * P.p_pad + o;
-          f[u] = ld4(P.fresh + go[u]);
-          l[u] = ld4(P.g_last + go[u]);
+          f[u] = ld4(last_row(P, sel_list[j]) + o);   // selected: cur[g] already points at the fresh gradient
+          l[u] = ld4(other_row(P, sel_list[j]) + o);  // the gradient it replaces
         }
       }
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         if (j0 + 8 * u < n_sel) {
-          st4(P.g_last + go[u], f[u]);
           fold(hi.x, lo.x, f[u].x, l[u].x);
           fold(hi.y, lo.y, f[u].y, l[u].y);
           fold(hi.z, lo.z, f[u].z, l[u].z);

@@ -1,0 +1,79 @@
+"""Degenerate and boundary shapes through the C ABI, against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2201_04301_b200 import binding
+from paper_2201_04301_b200.workloads import make_workload
+
+from parity import forced_parity, to_cuda
+
+pytestmark = pytest.mark.gpu
+
+
+def _stream():
+    return torch.cuda.Stream()
+
+
+def test_single_sample_batches_and_one_row_shards():
+    # batch of one row per group; shards of exactly one row (every draw is that row)
+    w = make_workload("cfg1", rows=3, dims=(9,), M=3, M_G=1, D=2, batch=1)
+    forced_parity(w, 8, stream=_stream())
+    w = make_workload("cfg1", rows=50, dims=(300,), M=2, M_G=1, D=2, batch=1)
+    forced_parity(w, 6, stream=_stream())
+
+
+def test_widest_supported_linear_model_and_the_first_unsupported():
+    w = make_workload("cfg1", rows=200, dims=(4096,), M=4, M_G=2, D=2, batch=9)
+    forced_parity(w, 5, stream=_stream())
+    with pytest.raises(binding.GCadaError) as e:
+        binding.GCada("logistic", (4097,), 4, 2, 2, 1.0, 0.01, 0.9, 0.99, 1e-8)
+    assert e.value.status == binding.EINVAL
+
+
+def test_misaligned_wide_rows_are_rejected_not_misread():
+    w = to_cuda(make_workload("cfg1", rows=100, dims=(512,), M=2, M_G=1, D=2, batch=4))
+    g = binding.GCada("logistic", (512,), 2, 1, 2, 1.0, 0.01, 0.9, 0.99, 1e-8)
+    Xp = torch.zeros(100, 514, device="cuda")
+    Xp[:, :512] = w["X"]
+    with pytest.raises(binding.GCadaError) as e:
+        g.set_data(Xp, w["y"], 4, ld=514)              # row stride not a multiple of 4 floats
+    assert e.value.status == binding.EINVAL
+    with pytest.raises(binding.GCadaError) as e:
+        g.set_data(w["X"], w["y"], 4, ld=511)          # stride smaller than d
+    assert e.value.status == binding.EINVAL
+    with pytest.raises(binding.GCadaError) as e:
+        g.set_data(w["X"][:1], w["y"][:1], 4)           # fewer rows than groups
+    assert e.value.status == binding.EINVAL
+
+
+def test_many_groups_and_workers_per_group():
+    # 300 groups (more than one 256-group pass of the scheduling phase), 5 workers each; D = 1: everyone, always
+    w = make_workload("cfg1", rows=300 * 4, dims=(6,), M=1500, M_G=5, D=1, batch=2)
+    forced_parity(w, 4, stream=_stream())
+    g = binding.from_workload(to_cuda(w), stream=_stream())
+    g.step(5)
+    assert g.get_selection_mask(0, 5).all()
+    up, comm, comp = g.get_comm_count()
+    assert (up, comm, comp) == (1500, 1500 * 6, 1500 * 5)
+
+
+def test_zero_iterations_and_getters_before_stepping():
+    w = to_cuda(make_workload("cfg1", rows=600))
+    g = binding.from_workload(w, stream=_stream())
+    g.step(0)
+    assert g.get_iteration() == 0 and g.get_wallclock() == (0.0, 0.0) and g.get_comm_count() == (0, 0, 0)
+    assert np.array_equal(g.get_theta(), w["theta0"].cpu().numpy())
+    with pytest.raises(binding.GCadaError):
+        g.get_selection_mask(0, 1)
+
+
+def test_mlp_batch_not_a_multiple_of_the_tile_and_single_class_margin():
+    w = make_workload("cfg4", rows=400, dims=(20, 3), M=2, M_G=1, D=2, batch=65, alpha=0.01)
+    forced_parity(w, 6, stream=_stream())
+    w = make_workload("cfg5", rows=900, dims=(24, 40, 8), M=3, M_G=1, D=2, batch=200)   # padded to 256 rows
+    forced_parity(w, 5, tol=2e-2, stream=_stream(), margin=None, rhs_tol=2e-2)
+    with pytest.raises(binding.GCadaError) as e:                                        # beyond the bf16 path's limit
+        h = binding.from_workload(to_cuda(make_workload("cfg5", rows=900, dims=(24, 8), M=3, M_G=1, D=2, batch=300)))
+        h.step(1)
+    assert e.value.status == binding.EINVAL
