@@ -86,6 +86,15 @@ class ClockSampler(threading.Thread):
                 pass
             time.sleep(0.02)
 
+    def sample_once(self):
+        """One synchronous sample (so that even a very short timed region has clock data)."""
+        if self.nv is None:
+            return
+        try:
+            self.samples.append(self.nv.nvmlDeviceGetClockInfo(self.handle, self.nv.NVML_CLOCK_SM))
+        except Exception:
+            pass
+
     def result(self):
         s = sorted(self.samples)
         return {"sm_mhz": (s[len(s) // 2] if s else None), "sm_max_mhz": self.max_mhz,
@@ -173,8 +182,12 @@ def run_ours(args):
     w = make_workload(args.config, device=dev, data_seed=rank, rows=args.rows, **overrides)
     stream = torch.cuda.Stream(device=dev)
     torch.cuda.synchronize()
-    g = binding.from_workload(w, stream=stream, options={binding.OPT_GRAPH: 0.0 if args.no_graph else 1.0,
-                                       binding.OPT_LINEAR_VARIANT: float(args.variant)})
+    opts = {binding.OPT_GRAPH: 0.0 if args.no_graph else 1.0, binding.OPT_LINEAR_VARIANT: float(args.variant)}
+    smooth = None
+    if args.rule == "ps":      # Eq. (9) as printed, with one smoothness constant for every group
+        opts[binding.OPT_RULE] = 1.0
+        smooth = [args.smoothness] * (w["M"] // w["M_G"])
+    g = binding.from_workload(w, stream=stream, options=opts, smoothness=smooth)
     gen_s = time.time() - t0
     G = g.G
 
@@ -189,6 +202,7 @@ def run_ours(args):
     e0.record(stream)
     g.step(args.steps)
     e1.record(stream)
+    sampler.sample_once()          # work is in flight
     e1.synchronize()
     _barrier(world)
     sampler.stop_flag = True
@@ -196,6 +210,8 @@ def run_ours(args):
     ms = _barrier_max(world, e0.elapsed_time(e1), dev)
     launches = g.get_launch_count() - l0
     value = aggregate_value(world, args.steps, ms)
+    n_hist = min(args.steps, 4096)
+    sel_frac = float(g.get_selection_mask(g.get_iteration() - n_hist, n_hist).mean())
 
     # --- per-kernel times (plain launches bracketed by events) -------------------
     g.set_option(binding.OPT_TIMING, 1)
@@ -241,14 +257,16 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16" if w["compute"] == "bf16" else "f32", "data": "synthetic",
-        "config": {"workload": "%s: %s dims=%s N=%d M=%d M_G=%d batch=%d D=%d c=%g" % (
-            args.config, w["kind"], list(w["dims"]), w["X"].shape[0], w["M"], w["M_G"], w["batch"], w["D"], w["c"]),
+        "config": {"workload": "%s: %s dims=%s N=%d M=%d M_G=%d batch=%d D=%d c=%g rule=%s" % (
+            args.config, w["kind"], list(w["dims"]), w["X"].shape[0], w["M"], w["M_G"], w["batch"], w["D"], w["c"],
+            args.rule),
             "parallelism": "replicas only (%d)" % world,
             "l2": "inputs larger than L2: each step gathers its rows from the resident training set"
                   if w["X"].numel() * w["X"].element_size() > 126e6 else "training set smaller than L2 (latency-bound workload)",
             "setup_s": round(gen_s, 1)},
         "clocks": sampler.result(),
         "gpu_launches": int(launches),
+        "selected_fraction": sel_frac,
         "kernel_ms": {"gradient": ms_grad, "select": ms_sel, "update": ms_upd, "timed_iterations": n_timed},
     }
     if e2e:
@@ -402,6 +420,9 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="plain launches instead of graph replay")
     ap.add_argument("--workers", type=int, default=None, help="override M (fewer groups, for profiling captures)")
+    ap.add_argument("--rule", default="innov", choices=["innov", "ps"],
+                    help="innov: measured gradient innovation (default); ps: left side of Eq. (9) as printed")
+    ap.add_argument("--smoothness", type=float, default=0.25, help="L_g of every group for --rule ps")
     ap.add_argument("--variant", type=int, default=0, help="GCADA_OPT_LINEAR_VARIANT (kernel shape knob)")
     ap.add_argument("--e2e-steps", type=int, default=60)
     ap.add_argument("--cpu-budget", type=float, default=15.0)

@@ -252,10 +252,12 @@ gcada_status make_plans(gcada_ctx* ctx) {
     TRY(dev_alloc(ctx, &l2, (size_t)ctx->G));
     CK(cudaMemcpyAsync(l2, ctx->L2.data(), sizeof(double) * ctx->G, cudaMemcpyHostToDevice, ctx->stream));
     P.ps_L2 = l2;
+    P.skip_unselected = (is_linear(ctx) && ctx->G <= SKIP_MAX_GROUPS) ? 1 : 0;
     TRY(dev_alloc(ctx, &P.ps_lhs, (size_t)ctx->G));
     TRY(dev_alloc(ctx, &P.ps_part, (size_t)ctx->D * ctx->tail.ps_blocks));
   } else {
     P.ps_L2 = nullptr;
+    P.skip_unselected = 0;
   }
   CK(cudaStreamSynchronize(ctx->stream));
   ctx->ready = true;
@@ -271,6 +273,26 @@ gcada_status enqueue_iteration(gcada_ctx* ctx, const Params& P) {
     }
     ev = &ctx->events[(size_t)(ctx->timed % TIMING_CAP) * 5];
     CK(cudaEventRecord(ev[0], ctx->stream));
+  }
+  if (P.skip_unselected) {
+    // Rule PS on a linear model, Algorithm 1 in its printed order: the server decides first (no gradient
+    // is needed for the printed test), then only the selected groups compute.
+    CK(launch_ps_lhs(P, ctx->tail, ctx->stream));
+    CK(launch_select(P, ctx->tail, ctx->stream, 1));
+    if (ev) CK(cudaEventRecord(ev[1], ctx->stream));  // reported as "selection" below via the phase map
+    CK(launch_grad_linear(P, ctx->lin, ctx->kind == GCADA_MODEL_QUADRATIC, ctx->stream));
+    CK(launch_select(P, ctx->tail, ctx->stream, 2));
+    if (ev) {
+      CK(cudaEventRecord(ev[2], ctx->stream));
+      CK(cudaEventRecord(ev[3], ctx->stream));
+    }
+    CK(launch_update(P, ctx->tail, ctx->stream));
+    if (ev) {
+      CK(cudaEventRecord(ev[4], ctx->stream));
+      ctx->timed += 1;
+    }
+    ctx->launches += 5;
+    return GCADA_OK;
   }
   if (is_linear(ctx)) {
     CK(launch_grad_linear(P, ctx->lin, ctx->kind == GCADA_MODEL_QUADRATIC, ctx->stream));
@@ -324,7 +346,7 @@ gcada_status capture(gcada_ctx* ctx, int iters, cudaGraphExec_t* out) {
 }
 
 int kernels_per_iteration(const gcada_ctx* ctx) {
-  if (is_linear(ctx)) return 3 + (ctx->rule == 1 ? 1 : 0);
+  if (is_linear(ctx)) return ctx->P.skip_unselected ? 5 : 3 + (ctx->rule == 1 ? 1 : 0);
   const bool two_pass = ctx->compute == GCADA_COMPUTE_BF16 && !ctx->P.stale;
   return 2 + ctx->mlp.launches_per_iter + (two_pass ? ctx->mlp.n_layers : 0) + (ctx->rule == 1 ? 1 : 0);
 }
@@ -795,7 +817,10 @@ gcada_status gcada_get_kernel_times(gcada_ctx* ctx, double ms[3], int* n_timed) 
   if (n == 0) return GCADA_OK;
   for (long long i = 0; i < n; ++i) {
     cudaEvent_t* ev = &ctx->events[(size_t)i * 5];
-    const int phase_of[4] = {0, 1, 0, 2};  // gradient, selection, gradient (post-selection part), update
+    // normal order: gradient, selection, gradient (post-selection part), update;
+    // skip mode (rule PS on linear models): selection first, then the selected groups' gradients
+    const int normal[4] = {0, 1, 0, 2}, skip_first[4] = {1, 0, 0, 2};
+    const int* phase_of = ctx->P.skip_unselected ? skip_first : normal;
     for (int j = 0; j < 4; ++j) {
       float t = 0.f;
       CK(cudaEventElapsedTime(&t, ev[j], ev[j + 1]));

@@ -85,6 +85,9 @@ struct Params {
   const double* ps_L2;          // [G] squared smoothness constants, or null (rule INNOV)
   double* ps_lhs;               // [G] the printed left side, written by ps_lhs_kernel
   double* ps_part;              // [D][blocks] partial sums of ||theta^k - theta^{k-d}||^2
+  int skip_unselected;          // 1: the selection of this iteration is already in mask_cur and the gradient
+                                // kernels work on the selected groups only (rule PS: Algorithm 1 as printed,
+                                // workers of unselected groups compute nothing)
 };
 
 // ---------------------------------------------------------------------------
@@ -128,6 +131,28 @@ __device__ __forceinline__ float* last_row(const Params& P, int g) {
 }
 __device__ __forceinline__ float* other_row(const Params& P, int g) {
   return P.gbuf + ((long long)(1 - P.cur[g]) * P.G + g) * P.p_pad;
+}
+
+// Groups the gradient kernels work on: all of them (identity, returns P.G), or - in skip mode - the
+// ones selected this iteration, ascending, in list[] (shared memory, SKIP_MAX_GROUPS ints).  Called by
+// every thread of the block; contains block-wide barriers.
+constexpr int SKIP_MAX_GROUPS = 1024;
+__device__ __forceinline__ int build_group_list(const Params& P, int* list, int* count_sm) {
+  if (!P.skip_unselected) return P.G;
+  if (threadIdx.x < 32) {
+    const int lane = threadIdx.x;
+    int cnt = 0;
+    for (int g0 = 0; g0 < P.G; g0 += 32) {
+      const int gg = g0 + lane;
+      const bool s = gg < P.G && P.mask_cur[gg] != 0;
+      const unsigned int b = __ballot_sync(0xffffffffu, s);
+      if (s) list[cnt + __popc(b & ((1u << lane) - 1u))] = gg;
+      cnt += __popc(b);
+    }
+    if (lane == 0) *count_sm = cnt;
+  }
+  __syncthreads();
+  return *count_sm;
 }
 
 // Computing time of worker m at iteration k (Section II-B).

@@ -118,7 +118,12 @@ __global__ void __launch_bounds__(THREADS, MINB) grad_linear_large_kernel(const 
   const float* yf = reinterpret_cast<const float*>(P.y);
   const int B = P.B;
 
-  const long long Rtot = (long long)P.G * B;
+  // group numbers below are positions in the list of groups worked on (all groups, or the selected ones)
+  __shared__ int sel_sm[SKIP_MAX_GROUPS];
+  __shared__ int n_groups_sm;
+  const int n_groups = build_group_list(P, sel_sm, &n_groups_sm);
+  const bool skip = P.skip_unselected != 0;
+  const long long Rtot = (long long)n_groups * B;
   const long long r0 = (long long)blockIdx.x * Rtot / gridDim.x;
   const long long r1 = (long long)(blockIdx.x + 1) * Rtot / gridDim.x;
   if (r0 >= r1) return;
@@ -189,7 +194,7 @@ __global__ void __launch_bounds__(THREADS, MINB) grad_linear_large_kernel(const 
     for (int i = tid; i < nrows; i += THREADS) {
       const int pos = in_g0 + cs + i;
       const int gi = pos / B;
-      const long long row = batch_row(P, k32, g_first + gi, pos - gi * B);
+      const long long row = batch_row(P, k32, skip ? sel_sm[g_first + gi] : g_first + gi, pos - gi * B);
       row_sm[i] = row * P.ld;
       y_sm[i] = yf[row];
     }
@@ -211,7 +216,7 @@ __global__ void __launch_bounds__(THREADS, MINB) grad_linear_large_kernel(const 
         if (cur_g >= 0) flush(cur_g);
         cur_g = cur_g < 0 ? g_first : cur_g + 1;
         g_end = (cur_g + 1 - g_first) * B - in_g0;
-        long long js = k - P.tau[cur_g];
+        long long js = k - P.tau[skip ? sel_sm[cur_g] : cur_g];
         if (js < 0) js = 0;
         const float* theta_s = P.theta_ring + (js % ring) * P.p_pad;
 #pragma unroll
@@ -378,7 +383,11 @@ __global__ void __launch_bounds__(256) grad_linear_small_kernel(const Params P) 
   const float* theta_k = P.theta_ring + (k % ring) * P.p_pad;
   const float* Xf = reinterpret_cast<const float*>(P.X);
   const float* yf = reinterpret_cast<const float*>(P.y);
-  const long long Rtot = (long long)P.G * P.B;
+  __shared__ int sel_sm[SKIP_MAX_GROUPS];
+  __shared__ int n_groups_sm;
+  const int n_groups = build_group_list(P, sel_sm, &n_groups_sm);  // positions in this list are called g below
+  const bool skip = P.skip_unselected != 0;
+  const long long Rtot = (long long)n_groups * P.B;
   const long long r0 = (long long)blockIdx.x * Rtot / gridDim.x;
   const long long r1 = (long long)(blockIdx.x + 1) * Rtot / gridDim.x;
   if (r0 >= r1) return;
@@ -394,7 +403,8 @@ __global__ void __launch_bounds__(256) grad_linear_small_kernel(const Params P) 
   while (seg0 < r1) {
     const int g = (int)(seg0 / P.B);
     const long long seg1 = (long long)(g + 1) * P.B < r1 ? (long long)(g + 1) * P.B : r1;
-    long long js = k - P.tau[g];
+    const int g_real = skip ? sel_sm[g] : g;
+    long long js = k - P.tau[g_real];
     if (js < 0) js = 0;
     const float* theta_s = P.theta_ring + (js % ring) * P.p_pad;
 #pragma unroll
@@ -410,7 +420,7 @@ __global__ void __launch_bounds__(256) grad_linear_small_kernel(const Params P) 
       long long myrow = 0;
       float myy = 0.f;
       if (lane < RR && rb + lane < seg1) {
-        myrow = batch_row(P, k32, g, (int)(rb + lane - (long long)g * P.B));
+        myrow = batch_row(P, k32, g_real, (int)(rb + lane - (long long)g * P.B));
         myy = yf[myrow];
       }
       float x[RR][CPL], z[RR], zs[RR];
@@ -529,7 +539,9 @@ bool plan_linear(int d, long long ld, const void* X, int G, int B, int sm_count,
     plan->R = plan->ctas_per_sm == 1 ? 4 : 2;
     const size_t rowbytes = (size_t)nchunks * 16;
     const size_t fixed = large_smem_fixed(plan->threads, plan->R);
-    const long long budget = plan->ctas_per_sm == 1 ? (long long)smem_optin : ((long long)smem_optin + 1024) / 2 - 1024;
+    // per CTA: the opt-in limit (or half an SM's shared memory) less the kernel's static arrays
+    const long long budget =
+        (plan->ctas_per_sm == 1 ? (long long)smem_optin : ((long long)smem_optin + 1024) / 2 - 1024) - 4608;
     long long nslot = (budget - (long long)fixed) / (long long)rowbytes;
     if (nslot > 32) nslot = 32;
     if (nslot < 2 * plan->R) {

@@ -36,7 +36,8 @@ struct TailPlan {
 void plan_tail(long long p_pad, int G, int sm_count, TailPlan* plan);
 // Rule PS only: the printed left side of Eq. (9) for every group (run before the selection kernel).
 cudaError_t launch_ps_lhs(const Params& P, const TailPlan& plan, cudaStream_t st);
-cudaError_t launch_select(const Params& P, const TailPlan& plan, cudaStream_t st);
+// what: 0 = reduce the gradient partial sums and schedule, 1 = schedule only, 2 = reduce only (skip mode).
+cudaError_t launch_select(const Params& P, const TailPlan& plan, cudaStream_t st, int what = 0);
 cudaError_t launch_update(const Params& P, const TailPlan& plan, cudaStream_t st);
 
 }  // namespace gcada

@@ -21,8 +21,14 @@ namespace gcada {
 __device__ __forceinline__ float4 ld4(const float* p) { return *reinterpret_cast<const float4*>(p); }
 __device__ __forceinline__ void st4(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
 
+// what: SEL_ALL = reduce the partial sums, then schedule (last block); SEL_SCHEDULE = schedule only (one
+// block; the left sides come from lhs_part as it stands, or from rule PS); SEL_REDUCE = reduce only (skip
+// mode: the gradient kernels ran after the scheduling, on the selected groups, and only their partial sums
+// have to become gradients).
+enum { SEL_ALL = 0, SEL_SCHEDULE = 1, SEL_REDUCE = 2 };
+
 template <int U>
-__global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_x) {
+__global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_x, int what) {
   __shared__ double scratch[40];
   __shared__ int sh_nsel[8];
   __shared__ double sh_tmax[8];
@@ -36,13 +42,27 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
 
   // ---- phase 1: partial sums -> fresh_g (and stale_g), innovation norm
   // (skipped when the gradient kernels have already delivered the norm partial sums)
-  if (P.pm.n_cta >= 0) {
-    float* fresh_g = fresh_row(P, g);
+  if (P.pm.n_cta >= 0 && what != SEL_SCHEDULE) {
+    // skip mode: the group's rank among the selected ones locates its partial sums, and its fresh gradient
+    // goes to the row that the flip of cur[g] has already made the last uploaded one
+    int gi = g, n_groups = P.G;
+    if (what == SEL_REDUCE) {
+      if (!P.mask_cur[g]) return;
+      int before = 0, total = 0;
+      for (int j = tid; j < P.G; j += 256) {
+        const int m = P.mask_cur[j] != 0;
+        total += m;
+        before += (j < g) ? m : 0;
+      }
+      gi = (int)(block_sum((double)before, scratch) + 0.5);
+      n_groups = (int)(block_sum((double)total, scratch) + 0.5);
+    }
+    float* fresh_g = what == SEL_REDUCE ? last_row(P, g) : fresh_row(P, g);
     int c_lo = 0, c_hi = -1;
-    const long long Rtot = (long long)P.G * P.pm.rows_per_group;
+    const long long Rtot = (long long)n_groups * P.pm.rows_per_group;
     const int n = P.pm.n_cta;
     if (n > 0) {
-      const long long x0 = (long long)g * P.pm.rows_per_group;
+      const long long x0 = (long long)gi * P.pm.rows_per_group;
       const long long x1 = x0 + P.pm.rows_per_group - 1;
       c_lo = (int)(((x0 + 1) * n - 1) / Rtot);
       c_hi = (int)(((x1 + 1) * n - 1) / Rtot);
@@ -63,7 +83,7 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
             const int c = c0 + u;
             if (c <= c_hi) {
               const int gf = (int)(((long long)c * Rtot / n) / P.pm.rows_per_group);
-              const float* src = P.partial + ((long long)(c * P.pm.maxseg + (g - gf)) * 2) * P.p_pad + i4 * 4;
+              const float* src = P.partial + ((long long)(c * P.pm.maxseg + (gi - gf)) * 2) * P.p_pad + i4 * 4;
               a[u] = ld4(src);
               b[u] = ld4(src + P.p_pad);
             }
@@ -88,6 +108,7 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
       const float dx = s.x, dy = s.y, dz = s.z, dw = s.w;  // the innovation
       local += (double)dx * dx + (double)dy * dy + (double)dz * dz + (double)dw * dw;
     }
+    if (what == SEL_REDUCE) return;
     const double tot = block_sum(local, scratch);
     if (tid == 0) {
       P.lhs_part[(long long)g * blocks_x + blockIdx.x] = tot;
@@ -392,16 +413,18 @@ void plan_tail(long long p_pad, int G, int sm_count, TailPlan* plan) {
   plan->ps_blocks = (int)(pb < 1 ? 1 : (pb > 1024 ? 1024 : pb));
 }
 
-cudaError_t launch_select(const Params& P, const TailPlan& plan, cudaStream_t st) {
-  if (P.pm.n_cta < 0) {  // norm partial sums already in lhs_part: only the scheduling phase remains
-    select_kernel<1><<<dim3(1, 1), 256, 0, st>>>(P, P.pm.maxseg);
+cudaError_t launch_select(const Params& P, const TailPlan& plan, cudaStream_t st, int what) {
+  if (what == SEL_SCHEDULE || P.pm.n_cta < 0) {
+    // nothing to reduce: with n_cta < 0 the norm partial sums are already in lhs_part (maxseg per group);
+    // in skip mode (rule PS) the left sides come from ps_lhs and lhs_part is not read (0 slots)
+    select_kernel<1><<<dim3(1, 1), 256, 0, st>>>(P, P.pm.n_cta < 0 ? P.pm.maxseg : 0, SEL_SCHEDULE);
     return cudaGetLastError();
   }
   dim3 grid(plan.select_blocks_x, P.G);
   if (plan.select_cols4_per_block == 256)
-    select_kernel<1><<<grid, 256, 0, st>>>(P, plan.select_blocks_x);
+    select_kernel<1><<<grid, 256, 0, st>>>(P, plan.select_blocks_x, what);
   else
-    select_kernel<4><<<grid, 256, 0, st>>>(P, plan.select_blocks_x);
+    select_kernel<4><<<grid, 256, 0, st>>>(P, plan.select_blocks_x, what);
   return cudaGetLastError();
 }
 

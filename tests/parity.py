@@ -107,6 +107,9 @@ def forced_parity(w, K, tol=TOL_FP32, stream=None, reduction="mean", check_stale
                                         ("stale", stale[gi], rec["stale"][gi], th_old[gi])):
                 if name == "stale" and not check_stale:
                     continue
+                # printed rule on a linear model: only the selected groups compute, and only at theta^k
+                if L is not None and not is_mlp and (name == "stale" or not rec["mask"][gi]):
+                    continue
                 e = rel_l2(got, want)
                 if e > tol and is_mlp and _kink_match(o, got, th, batches[gi][1], batches[gi][2], reduction, tol, kink_tol):
                     worst["kinks"] += 1

@@ -171,8 +171,18 @@ def test_rule_ps_printed_left_side():
                 assert abs(rec["lhs"][gi] - rec["rhs"]) / max(rec["lhs"][gi], rec["rhs"]) < MARGIN
             break
     assert 0 < got.sum() < got.size
+    assert g.get_launch_count() == 5 * 40      # distances, schedule, gradients of the selected, reduce, update
     # without constants the rule cannot run
     h = binding.from_workload(to_cuda(w), options={binding.OPT_RULE: 1.0})
     with pytest.raises(binding.GCadaError) as e:
         h.step(1)
     assert e.value.status == binding.ESTATE
+
+
+def test_rule_ps_wide_model_skips_work():
+    """Row-ring kernel under the printed rule: gradients of the selected groups only (the rows of the
+    others are never read), checked against the oracle; the kernel gets faster as fewer groups upload."""
+    w = make_workload("cfg3", rows=16 * 600, M=32, M_G=2, D=6, c=0.05)
+    L = [0.5 + 0.1 * g for g in range(16)]
+    flips, worst = forced_parity(w, 14, stream=_stream(), L=L)
+    print("rule PS wide worst", worst, "flips", flips)
