@@ -149,9 +149,12 @@ gcada_status gcada_set_option(gcada_ctx *ctx, int key, double value);
 
 /* Smoothness constants L_g >= 0 (host, G doubles; copied) for rule PS, the left side of Eq. (9) as
  * printed: L_g^2 ||theta^k - theta^{k-tau_g}||^2, evaluated from the ring of the last D+1 iterates.  Set
- * them before the first step; stepping with GCADA_OPT_RULE = 1 and no constants gives GCADA_ESTATE.  In this
- * build the gradients of every group are still evaluated each iteration (at both points); only the test and
- * therefore the selection, the aggregate and the counters follow the printed rule. */
+ * them before the first step; stepping with GCADA_OPT_RULE = 1 and no constants gives GCADA_ESTATE.  The
+ * printed test needs no gradient, so for logistic / quadratic models (up to 1024 groups) an iteration runs in
+ * Algorithm 1's order: test, selection, then gradients at theta^k for the selected groups only (the cost of
+ * an iteration scales with the number of uploads; GCADA_DBG_FRESH / _STALE / _LHS-by-innovation of
+ * unselected groups are then not produced).  For MLPs the rule decides the selection, but both gradients of
+ * every group are still evaluated. */
 gcada_status gcada_set_smoothness(gcada_ctx *ctx, const double *L, int G);
 
 /* Run n_iters iterations of Algorithm 1 on the stream (asynchronous).
@@ -244,6 +247,13 @@ gcada_status gcada_get_kernel_times(gcada_ctx *ctx, double ms[3], int *n_timed);
 gcada_status gcada_innovation_norms_noalloc(const float *fresh_dev, const float *stale_dev, int G,
                                             long long p, long long ld, double *lhs_dev,
                                             void *cuda_stream, char *errbuf, size_t errbuf_len);
+
+/* Measurement aid: enqueue the gradient kernel(s) of the current iteration `reps` times back to back on the
+ * stream, bracketed by ONE pair of CUDA events, and return the mean device time per repetition in
+ * milliseconds (per-launch event brackets, as GCADA_OPT_TIMING uses, add the launch gaps of each bracket to
+ * a kernel that lasts tens of microseconds).  The repetitions recompute the same gradients and change no
+ * state that an iteration reads.  Synchronises the stream before and after. */
+gcada_status gcada_time_gradient(gcada_ctx *ctx, int reps, double *ms_per_rep);
 
 /* Text of the last error of this context ("" if none); valid until the next
  * call on the context.  ctx == NULL returns the text of the last failed

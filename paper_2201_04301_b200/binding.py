@@ -58,6 +58,7 @@ SIGNATURES = {
     "gcada_get_launch_count": (C.c_int, [_VP, _ULLP]),
     "gcada_get_kernel_times": (C.c_int, [_VP, C.POINTER(C.c_double), C.POINTER(C.c_int)]),
     "gcada_innovation_norms_noalloc": (C.c_int, [_VP, _VP, C.c_int, _LL, _LL, _VP, _VP, C.c_char_p, C.c_size_t]),
+    "gcada_time_gradient": (C.c_int, [_VP, C.c_int, C.POINTER(C.c_double)]),
     "gcada_last_error": (C.c_char_p, [_VP]),
     "gcada_destroy": (None, [_VP]),
 }
@@ -204,6 +205,12 @@ class GCada:
         out = np.empty(self.p, dtype=np.float32)
         self._ck(self.lib.gcada_get_group_gradient(self.h, int(what), int(g), _VP(out.ctypes.data), self.p))
         return out
+
+    def time_gradient(self, reps):
+        """Mean device time (ms) of the gradient kernel(s) over `reps` back-to-back repetitions."""
+        ms = C.c_double()
+        self._ck(self.lib.gcada_time_gradient(self.h, int(reps), C.byref(ms)))
+        return ms.value
 
     def get_kernel_times(self):
         """(ms_gradient, ms_select, ms_update), n_timed: see GCADA_OPT_TIMING."""

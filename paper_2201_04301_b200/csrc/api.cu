@@ -831,6 +831,38 @@ gcada_status gcada_get_kernel_times(gcada_ctx* ctx, double ms[3], int* n_timed) 
   return GCADA_OK;
 }
 
+gcada_status gcada_time_gradient(gcada_ctx* ctx, int reps, double* ms_per_rep) {
+  if (!ctx || !ms_per_rep || reps < 1) return GCADA_EINVAL;
+  TRY(check_runnable(ctx, true));
+  DeviceGuard dg(ctx->device);
+  TRY(make_plans(ctx));
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  CK(cudaEventCreate(&e0));
+  CK(cudaEventCreate(&e1));
+  Params P = ctx->P;
+  P.skip_unselected = 0;  // every group, as in the default rule
+  CK(cudaStreamSynchronize(ctx->stream));
+  CK(cudaEventRecord(e0, ctx->stream));
+  for (int r = 0; r < reps; ++r) {
+    if (is_linear(ctx)) {
+      CK(launch_grad_linear(P, ctx->lin, ctx->kind == GCADA_MODEL_QUADRATIC, ctx->stream));
+      ctx->launches += 1;
+    } else {
+      int n = 0;
+      CK(launch_grad_mlp(P, ctx->mlp, ctx->stream, &n));
+      ctx->launches += (unsigned long long)n;
+    }
+  }
+  CK(cudaEventRecord(e1, ctx->stream));
+  CK(cudaEventSynchronize(e1));
+  float ms = 0.f;
+  CK(cudaEventElapsedTime(&ms, e0, e1));
+  cudaEventDestroy(e0);
+  cudaEventDestroy(e1);
+  *ms_per_rep = (double)ms / reps;
+  return GCADA_OK;
+}
+
 const char* gcada_last_error(const gcada_ctx* ctx) { return ctx ? ctx->err.c_str() : g_create_error.c_str(); }
 
 void gcada_destroy(gcada_ctx* ctx) {
