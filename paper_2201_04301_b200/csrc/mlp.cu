@@ -33,7 +33,22 @@ __global__ void __launch_bounds__(256) mlp_gather_kernel(const Params P, float* 
   const long long row = batch_row(P, (uint32_t)P.st->k, g, j);
   const float* src = reinterpret_cast<const float*>(P.X) + row * P.ld;
   float* dst = xb + (long long)warp * d;
-  for (int c = lane; c < d; c += 32) dst[c] = src[c];
+  if (((d | P.ld) & 3) == 0 && ((reinterpret_cast<uintptr_t>(P.X) | reinterpret_cast<uintptr_t>(xb)) & 15) == 0) {
+    const float4* s4 = reinterpret_cast<const float4*>(src);
+    float4* d4 = reinterpret_cast<float4*>(dst);
+    const int n4 = d >> 2;
+    for (int c0 = 0; c0 < n4; c0 += 256) {  // eight 16-byte loads in flight per lane
+      float4 v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        if (c0 + lane + 32 * u < n4) v[u] = s4[c0 + lane + 32 * u];
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        if (c0 + lane + 32 * u < n4) d4[c0 + lane + 32 * u] = v[u];
+    }
+  } else {
+    for (int c = lane; c < d; c += 32) dst[c] = src[c];
+  }
   if (lane == 0) yb[warp] = reinterpret_cast<const int*>(P.y)[row];
 }
 
