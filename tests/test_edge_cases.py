@@ -77,3 +77,26 @@ def test_mlp_batch_not_a_multiple_of_the_tile_and_single_class_margin():
         h = binding.from_workload(to_cuda(make_workload("cfg5", rows=900, dims=(24, 8), M=3, M_G=1, D=2, batch=300)))
         h.step(1)
     assert e.value.status == binding.EINVAL
+
+
+def test_special_cases_distributed_adam_and_cada():
+    """c = 0: every group uploads every iteration (the 'distributed Adam' of Section V); M_G = 1: groups are
+    single workers and the scheme is CADA (Section III).  Both against the oracle, and the mean simulated
+    wall-clock of the first against the order-statistics formula (Eq. 10): with G groups of M_G workers,
+    shift 1 and rate 1 the server waits 1 + H_G / M_G per iteration on average."""
+    w = make_workload("cfg1", rows=3000, c=0.0)
+    forced_parity(w, 30, stream=_stream())
+    g = binding.from_workload(to_cuda(make_workload("cfg1", c=0.0)), stream=_stream())
+    K = 6000
+    g.step(K)
+    assert g.get_selection_mask(K - 50, 50).all()
+    assert g.get_comm_count() == (3 * K, 3 * 3 * K, 3 * 2 * K)
+    mean = g.get_wallclock()[0] / K
+    want = 1.0 + (1 + 1 / 2 + 1 / 3) / 2
+    assert abs(mean - want) < 5 * 0.45 / np.sqrt(K), (mean, want)      # sd of the max of three Exp(2) is < 0.45
+    w = make_workload("cfg1", rows=3000, M=5, M_G=1, c=2.0)
+    forced_parity(w, 30, stream=_stream())
+    h = binding.from_workload(to_cuda(w), stream=_stream())
+    h.step(100)
+    up, comm, comp = h.get_comm_count()
+    assert comm == 2 * up and comp == up and 0 < up < 500               # Eqs. (18), (21) with equality
