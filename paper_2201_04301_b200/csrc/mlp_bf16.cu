@@ -186,11 +186,12 @@ __device__ __forceinline__ int ring_slot(const Params& P, int g, int q, long lon
 // the CTAs running together share operand tiles in L2); tensor memory holds
 // two 256-column accumulators, so the eight epilogue warps drain tile i while
 // the producer and the MMA warp work on tile i+1.
-constexpr int GN = 256;                                  // N tile of this kernel
+constexpr int GN = 256;                                  // N tile of this kernel (the epilogue assumes 2 x 4 chunks of 32)
 constexpr int G_STAGE_BYTES = (BM + GN) * BK * 2;        // 48 KiB
 constexpr int G_STAGES = 4;
 constexpr int G_EPI_WARPS = 8;
 constexpr int G_THREADS = 64 + 32 * G_EPI_WARPS;
+constexpr int G_TR_BYTES = G_EPI_WARPS * 32 * 17 * 4;  // per-warp transposition tiles of the epilogue
 constexpr uint32_t IDESC_G = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(GN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
@@ -284,6 +285,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
     const int ew = warp - 2;
     const int quad = warp & 3;
     const int half = ew >> 2;
+    uint32_t* tr = reinterpret_cast<uint32_t*>(tiles + (size_t)G_STAGES * G_STAGE_BYTES) + ew * (32 * 17);
     bool ok = true;
     int i = 0;
     for (int t = blockIdx.x; t < total_tiles; t += gridDim.x, ++i) {
@@ -302,18 +304,25 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
       if (a.epi == EPI_HIDDEN || a.epi == EPI_SCORES)
         bias = a.bias_ring + (long long)ring_slot(P, g, q, k_it) * a.bias_slot + a.bias_pos;
       const uint32_t tbase = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(slot * GN);
-#pragma unroll 1
-      for (int c = half * (GN / 2); c < (half + 1) * (GN / 2); c += 32) {
+      // one 32-column chunk of this thread's row
+      auto chunk = [&](const uint32_t (&v)[32], int c) {
         const int nc = n0 + c;
-        if (nc >= a.N) break;  // uniform across the warp
-        uint32_t v[32];
-        tc_ld32(tbase + (uint32_t)c, v);
+        if (nc >= a.N) return;  // uniform across the warp
         const bool row_ok = m < a.M;
         const bool full = nc + 32 <= a.N;
         if (a.epi == EPI_SCORES) {
           float* dst = a.out_f32 + ((long long)z * a.M + m) * a.N + nc;
-          if (row_ok)
-            for (int j = 0; j < 32 && nc + j < a.N; ++j) dst[j] = __uint_as_float(v[j]) + bias[nc + j];
+          if (row_ok) {
+            if (full && (a.N & 3) == 0) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 4)
+                *reinterpret_cast<float4*>(dst + j) =
+                    make_float4(__uint_as_float(v[j]) + bias[nc + j], __uint_as_float(v[j + 1]) + bias[nc + j + 1],
+                                __uint_as_float(v[j + 2]) + bias[nc + j + 2], __uint_as_float(v[j + 3]) + bias[nc + j + 3]);
+            } else {
+              for (int j = 0; j < 32 && nc + j < a.N; ++j) dst[j] = __uint_as_float(v[j]) + bias[nc + j];
+            }
+          }
         } else {
           float f[32];
           if (a.epi == EPI_HIDDEN) {
@@ -342,29 +351,63 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
               }
             }
           }
+          // bf16 pairs of this thread's row
+          uint32_t h[16];
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) {
+            __nv_bfloat162 t2 = __floats2bfloat162_rn(f[j], f[j + 1]);
+            h[j >> 1] = *reinterpret_cast<uint32_t*>(&t2);
+          }
           if (row_ok) {
             __nv_bfloat16* dst = a.out + (long long)z * a.z_stride_out + (long long)m * a.ldo + nc;
             if (full) {
 #pragma unroll
-              for (int j = 0; j < 32; j += 8) {
-                __nv_bfloat162 h0 = __floats2bfloat162_rn(f[j], f[j + 1]), h1 = __floats2bfloat162_rn(f[j + 2], f[j + 3]);
-                __nv_bfloat162 h2 = __floats2bfloat162_rn(f[j + 4], f[j + 5]), h3 = __floats2bfloat162_rn(f[j + 6], f[j + 7]);
-                uint4 pk;
-                pk.x = *reinterpret_cast<uint32_t*>(&h0);
-                pk.y = *reinterpret_cast<uint32_t*>(&h1);
-                pk.z = *reinterpret_cast<uint32_t*>(&h2);
-                pk.w = *reinterpret_cast<uint32_t*>(&h3);
-                *reinterpret_cast<uint4*>(dst + j) = pk;
-              }
+              for (int j = 0; j < 16; j += 4)
+                *reinterpret_cast<uint4*>(dst + 2 * j) = make_uint4(h[j], h[j + 1], h[j + 2], h[j + 3]);
             } else {
               for (int j = 0; j < 32 && nc + j < a.N; ++j) dst[j] = __float2bfloat16_rn(f[j]);
             }
-            __nv_bfloat16* dstT = a.outT + (long long)z * a.z_stride_outT + (long long)nc * a.ldt + m;
+          }
+          // transposed copy: the warp's 32 x 32 block goes through shared memory (rows of 17 words, free
+          // of bank conflicts both ways) so that lane n writes 64 contiguous bytes of output row nc + n
+          __syncwarp();
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (nc + j < a.N) dstT[(long long)j * a.ldt] = __float2bfloat16_rn(f[j]);
+          for (int j = 0; j < 16; ++j) tr[lane * 17 + j] = h[j];
+          __syncwarp();
+          if (nc + lane < a.N) {
+            uint32_t o[16];
+#pragma unroll
+            for (int r = 0; r < 32; r += 2) {
+              const uint32_t w0 = tr[r * 17 + (lane >> 1)], w1 = tr[(r + 1) * 17 + (lane >> 1)];
+              const uint32_t e0 = (lane & 1) ? (w0 >> 16) : (w0 & 0xFFFFu);
+              const uint32_t e1 = (lane & 1) ? (w1 >> 16) : (w1 & 0xFFFFu);
+              o[r >> 1] = e0 | (e1 << 16);
+            }
+            __nv_bfloat16* dstT = a.outT + (long long)z * a.z_stride_outT + (long long)(nc + lane) * a.ldt +
+                                  (mt * BM + quad * 32);
+#pragma unroll
+            for (int j = 0; j < 16; j += 4)
+              *reinterpret_cast<uint4*>(dstT + 2 * j) = make_uint4(o[j], o[j + 1], o[j + 2], o[j + 3]);
           }
         }
+      };
+      // The four chunks of this warp, software-pipelined: the tensor-memory load of the next chunk is in
+      // flight while the current one is converted and stored (a load takes far longer than its issue).
+      {
+        const int cb = half * (GN / 2);
+        uint32_t va[32], vb[32];
+        tc_ld32_issue(tbase + (uint32_t)cb, va);
+        tc_ld_wait();
+        tc_ld32_issue(tbase + (uint32_t)(cb + 32), vb);
+        chunk(va, cb);
+        tc_ld_wait();
+        tc_ld32_issue(tbase + (uint32_t)(cb + 64), va);
+        chunk(vb, cb + 32);
+        tc_ld_wait();
+        tc_ld32_issue(tbase + (uint32_t)(cb + 96), vb);
+        chunk(va, cb + 64);
+        tc_ld_wait();
+        chunk(vb, cb + 96);
       }
       tc_fence_before();
       __syncwarp();
@@ -876,7 +919,7 @@ cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const Para
   a.stages = G_STAGES;
   const long long tiles = (long long)((a.N + GN - 1) / GN) * ((a.M + BM - 1) / BM) * 2 * P.G;
   const int ctas = (int)(tiles < sm_count ? tiles : sm_count);
-  bf16_gemm_kernel<<<ctas, G_THREADS, (size_t)G_STAGES * G_STAGE_BYTES + 1024, st>>>(ta, tb, P, a);
+  bf16_gemm_kernel<<<ctas, G_THREADS, (size_t)G_STAGES * G_STAGE_BYTES + 1024 + G_TR_BYTES, st>>>(ta, tb, P, a);
   return cudaGetLastError();
 }
 
@@ -1008,7 +1051,7 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
     return cudaSuccess;
   }
   cudaError_t e = cudaFuncSetAttribute(bf16_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       G_STAGES * G_STAGE_BYTES + 1024);
+                                       G_STAGES * G_STAGE_BYTES + 1024 + G_TR_BYTES);
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(bf16_softmax_grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            32 * (plan->dims[L] + 4) * 2);
