@@ -198,8 +198,10 @@ gcada_status gcada_get_iteration(gcada_ctx *ctx, long long *k);
 /* Internal quantities (GCADA_DBG_*); `bytes` must equal the item's size. */
 gcada_status gcada_get_debug(gcada_ctx *ctx, int what, void *out, long long bytes);
 /* One group's row of GCADA_DBG_FRESH / GCADA_DBG_STALE / GCADA_DBG_GLAST (p floats to the host), for models
- * whose [G][p] arrays are too large to copy whole.  With the bf16 MLP and GCADA_OPT_KEEP_STALE off, the fresh
- * gradient of a group is only written in iterations that select the group. */
+ * whose [G][p] arrays are too large to copy whole.  With the bf16 MLP and GCADA_OPT_KEEP_STALE off no
+ * per-group gradient vector exists on the device: each upload is kept as the two bf16 factors of every
+ * layer's weight gradient, GCADA_DBG_GLAST rebuilds the group's last uploaded gradient from them on demand,
+ * and GCADA_DBG_FRESH returns the same (a fresh gradient survives only as an upload). */
 gcada_status gcada_get_group_gradient(gcada_ctx *ctx, int what, int g, float *out, long long p);
 /* Number of kernel launches enqueued by this context so far (graph replays
  * count the kernels they contain). */

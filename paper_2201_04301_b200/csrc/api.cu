@@ -59,6 +59,7 @@ struct gcada_ctx {
   void* stage_x = nullptr;
   void* stage_y = nullptr;
   long long stage_ld = 0;
+  float* row_scratch = nullptr;  // one p-vector for getters that rebuild a group's gradient on demand
   // graphs (free-running resident-data mode only)
   cudaGraphExec_t graph1 = nullptr, graphN = nullptr;
   // optional per-phase timing
@@ -123,6 +124,7 @@ void free_all(gcada_ctx* ctx) {
   if (ctx->stage_x) cudaFree(ctx->stage_x);
   if (ctx->stage_y) cudaFree(ctx->stage_y);
   ctx->stage_x = ctx->stage_y = nullptr;
+  ctx->row_scratch = nullptr;  // was in `owned`
   ctx->st = nullptr;
   ctx->ready = false;
 }
@@ -145,6 +147,9 @@ gcada_status dev_alloc(gcada_ctx* ctx, T** out, size_t count) {
   } while (0)
 
 bool is_linear(const gcada_ctx* ctx) { return ctx->kind != GCADA_MODEL_MLP; }
+// bf16 MLP: the aggregate is formed from the stored factors of the last uploads; per-group gradient
+// vectors exist only when they are kept for inspection
+bool factored(const gcada_ctx* ctx) { return !is_linear(ctx) && ctx->compute == GCADA_COMPUTE_BF16; }
 
 // (Re)build device state and plans once model, data shape and theta^0 are known.
 gcada_status make_ready(gcada_ctx* ctx, const float* theta0, int on_device) {
@@ -175,7 +180,8 @@ gcada_status make_ready(gcada_ctx* ctx, const float* theta0, int on_device) {
   TRY(dev_alloc(ctx, &P.vhat, (size_t)pp));
   TRY(dev_alloc(ctx, &P.agg_hi, (size_t)pp));
   TRY(dev_alloc(ctx, &P.agg_lo, (size_t)pp));
-  TRY(dev_alloc(ctx, &P.gbuf, (size_t)2 * G * pp));
+  P.agg_direct = factored(ctx) ? 1 : 0;
+  if (!factored(ctx) || ctx->keep_stale) TRY(dev_alloc(ctx, &P.gbuf, (size_t)2 * G * pp));
   TRY(dev_alloc(ctx, &P.cur, (size_t)G));
   // the fp32 MLP kernels hand over both gradients; the others keep the stale one only on request
   if (ctx->keep_stale || (!is_linear(ctx) && ctx->compute == GCADA_COMPUTE_FP32))
@@ -309,7 +315,7 @@ gcada_status enqueue_iteration(gcada_ctx* ctx, const Params& P) {
   }
   CK(launch_select(P, ctx->tail, ctx->stream));
   if (ev) CK(cudaEventRecord(ev[2], ctx->stream));
-  if (!is_linear(ctx)) {  // gradient work that needs the selection (counted with the gradient phase)
+  if (!is_linear(ctx)) {  // bf16 MLP: the uploads are kept and the aggregate is formed (counted with the update phase)
     int n = 0;
     CK(launch_grad_mlp_post(P, ctx->mlp, ctx->stream, &n));
     ctx->launches += (unsigned long long)n;
@@ -347,8 +353,7 @@ gcada_status capture(gcada_ctx* ctx, int iters, cudaGraphExec_t* out) {
 
 int kernels_per_iteration(const gcada_ctx* ctx) {
   if (is_linear(ctx)) return ctx->P.skip_unselected ? 5 : 3 + (ctx->rule == 1 ? 1 : 0);
-  const bool two_pass = ctx->compute == GCADA_COMPUTE_BF16 && !ctx->P.stale;
-  return 2 + ctx->mlp.launches_per_iter + (two_pass ? ctx->mlp.n_layers : 0) + (ctx->rule == 1 ? 1 : 0);
+  return 2 + ctx->mlp.launches_per_iter + ctx->mlp.post_launches + (ctx->rule == 1 ? 1 : 0);
 }
 
 gcada_status check_runnable(gcada_ctx* ctx, bool need_data) {
@@ -367,6 +372,26 @@ const float* group_row(const gcada_ctx* ctx, int what, int g, const std::vector<
   int buf = cur[g];
   if (what == 0 && !mask[g]) buf = 1 - buf;  // an unselected group's fresh gradient sits in the other row
   return ctx->P.gbuf + ((long long)buf * ctx->G + g) * ctx->p_pad;
+}
+
+// Device pointer to group g's row for a getter.  Where per-group gradients are not materialised (bf16 MLP
+// without GCADA_OPT_KEEP_STALE) the last uploaded gradient is rebuilt from its stored factors into a
+// scratch row; the fresh gradient of a group is then only available as its last upload.
+gcada_status group_row_dev(gcada_ctx* ctx, int what, int g, const std::vector<unsigned char>& cur,
+                           const std::vector<unsigned char>& mask, const float** out) {
+  if (ctx->P.gbuf) {
+    *out = group_row(ctx, what, g, cur, mask);
+    return GCADA_OK;
+  }
+  if (!ctx->ready) return fail(ctx, GCADA_ESTATE, "no iteration has run yet");
+  if (!ctx->row_scratch) {
+    TRY(dev_alloc(ctx, &ctx->row_scratch, (size_t)ctx->p_pad));
+  }
+  CK(cudaMemsetAsync(ctx->row_scratch, 0, sizeof(float) * (size_t)ctx->p_pad, ctx->stream));
+  CK(mlp_group_gradient(ctx->P, ctx->mlp, g, ctx->row_scratch, ctx->stream));
+  CK(cudaStreamSynchronize(ctx->stream));
+  *out = ctx->row_scratch;
+  return GCADA_OK;
 }
 
 gcada_status read_state(gcada_ctx* ctx, DevState* out) {
@@ -764,9 +789,11 @@ gcada_status gcada_get_debug(gcada_ctx* ctx, int what, void* out, long long byte
     std::vector<unsigned char> cur((size_t)G), mask((size_t)G);
     CK(cudaMemcpy(cur.data(), P.cur, (size_t)G, cudaMemcpyDeviceToHost));
     CK(cudaMemcpy(mask.data(), P.mask_cur, (size_t)G, cudaMemcpyDeviceToHost));
-    for (int g = 0; g < (int)G; ++g)
-      CK(cudaMemcpy(static_cast<float*>(out) + (long long)g * p, group_row(ctx, per_group, g, cur, mask),
-                    (size_t)p * 4, cudaMemcpyDeviceToHost));
+    for (int g = 0; g < (int)G; ++g) {
+      const float* row = nullptr;
+      TRY(group_row_dev(ctx, per_group, g, cur, mask, &row));
+      CK(cudaMemcpy(static_cast<float*>(out) + (long long)g * p, row, (size_t)p * 4, cudaMemcpyDeviceToHost));
+    }
     return GCADA_OK;
   }
   if (bytes != rows * row_bytes) return fail(ctx, GCADA_EINVAL, "item %d has %lld bytes, buffer has %lld", what, rows * row_bytes, bytes);
@@ -793,7 +820,7 @@ gcada_status gcada_get_group_gradient(gcada_ctx* ctx, int what, int g, float* ou
     std::vector<unsigned char> cur((size_t)ctx->G), mask((size_t)ctx->G);
     CK(cudaMemcpy(cur.data(), ctx->P.cur, (size_t)ctx->G, cudaMemcpyDeviceToHost));
     CK(cudaMemcpy(mask.data(), ctx->P.mask_cur, (size_t)ctx->G, cudaMemcpyDeviceToHost));
-    src = group_row(ctx, what == GCADA_DBG_GLAST ? 1 : 0, g, cur, mask);
+    TRY(group_row_dev(ctx, what == GCADA_DBG_GLAST ? 1 : 0, g, cur, mask, &src));
   } else {
     return fail(ctx, GCADA_EINVAL, "item %d is not a per-group gradient", what);
   }
@@ -819,8 +846,8 @@ gcada_status gcada_get_kernel_times(gcada_ctx* ctx, double ms[3], int* n_timed) 
     cudaEvent_t* ev = &ctx->events[(size_t)i * 5];
     // normal order: gradient, selection, gradient (post-selection part), update;
     // skip mode (rule PS on linear models): selection first, then the selected groups' gradients
-    const int normal[4] = {0, 1, 0, 2}, skip_first[4] = {1, 0, 0, 2};
-    const int* phase_of = ctx->P.skip_unselected ? skip_first : normal;
+    const int normal[4] = {0, 1, 0, 2}, skip_first[4] = {1, 0, 0, 2}, agg_after[4] = {0, 1, 2, 2};
+    const int* phase_of = ctx->P.skip_unselected ? skip_first : (ctx->P.agg_direct ? agg_after : normal);
     for (int j = 0; j < 4; ++j) {
       float t = 0.f;
       CK(cudaEventElapsedTime(&t, ev[j], ev[j + 1]));

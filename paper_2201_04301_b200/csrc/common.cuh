@@ -62,9 +62,11 @@ struct Params {
   float* vhat;
   float* agg_hi;        // lazily aggregated gradient, Eq. (3), as an unevaluated sum hi + lo
   float* agg_lo;
+  int agg_direct;       // 1: agg_hi already holds this iteration's aggregate when the update kernel runs (it was
+                        // formed from the stored factors of the last uploads); nothing is folded in from gbuf
   // Two gradient buffers per group: buffer cur[g] holds the group's last uploaded gradient, the other one
   // receives this iteration's fresh gradient; selecting the group flips cur[g], so nothing is copied.
-  float* gbuf;          // [2][G] rows of p_pad floats
+  float* gbuf;          // [2][G] rows of p_pad floats (null when per-group gradients are not materialised)
   unsigned char* cur;   // [G]
   float* stale;         // [G] gradient at the stale iterate (optional, may be null)
   float* partial;       // [slots][2] partial sums of (fresh, stale)

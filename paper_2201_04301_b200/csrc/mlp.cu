@@ -264,6 +264,11 @@ cudaError_t launch_grad_mlp_post(const Params& P, const MlpPlan& pl, cudaStream_
   return cudaSuccess;
 }
 
+cudaError_t mlp_group_gradient(const Params& P, const MlpPlan& pl, int g, float* row, cudaStream_t st) {
+  if (pl.compute != 1) return cudaErrorNotSupported;
+  return mlp_bf16_group_gradient(P, pl, g, row, st);
+}
+
 cudaError_t launch_grad_mlp(const Params& P, const MlpPlan& pl, cudaStream_t st, int* n_launches) {
   if (pl.compute == 1) return mlp_bf16_launch(P, pl, st, n_launches);
   const int L = pl.n_layers, G = P.G, B = P.B;

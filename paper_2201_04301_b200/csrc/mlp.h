@@ -13,6 +13,7 @@ constexpr int MLP_MAX_LAYERS = 15;
 struct MlpPlan {
   int n_layers = 0;           // L
   int launches_per_iter = 0;
+  int post_launches = 0;      // kernels that follow the selection kernel (bf16 path: upload + aggregate)
   int compute = 0;            // 0 fp32, 1 bf16 operands
   int G = 0, B = 0, D = 0;
   long long p_pad = 0;
@@ -38,7 +39,10 @@ cudaError_t mlp_plan_create(const std::vector<int>& dims, int compute, int G, in
                             const char** why);
 // Enqueues the dual-point forward/backward of every group; writes each group's fresh-gradient row and P.stale.
 cudaError_t launch_grad_mlp(const Params& P, const MlpPlan& plan, cudaStream_t st, int* n_launches);
-// Gradient work that must follow the selection kernel (none for the fp32 path).
+// Work that must follow the selection kernel (none for the fp32 path; bf16: the selected groups' uploads
+// are kept and the aggregate of Eq. (3) is formed).
 cudaError_t launch_grad_mlp_post(const Params& P, const MlpPlan& plan, cudaStream_t st, int* n_launches);
+// bf16 path without kept per-group gradients: group g's last uploaded gradient rebuilt into `row` (device).
+cudaError_t mlp_group_gradient(const Params& P, const MlpPlan& plan, int g, float* row, cudaStream_t st);
 
 }  // namespace gcada

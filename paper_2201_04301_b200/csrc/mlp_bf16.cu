@@ -2,13 +2,17 @@
 // gradient step for every group at theta^k and at theta^{k-tau_g}).
 //
 // Operands are bf16 (features as stored; weights rounded from the fp32 master
-// iterate once per iteration), accumulation is fp32 in tensor memory, the
-// per-group weight gradients are written in fp32 straight into the gradient
-// vectors.  Every product is an "NT" GEMM  C[M x N] = A[M x K] * B[N x K]^T
+// iterate once per iteration), accumulation is fp32 in tensor memory.  Per-group
+// weight gradients are never materialised on the production path: a first pass
+// forms only the squared innovation norms, and the server's aggregate (Eq. 3,
+// the sum over groups of each group's last uploaded gradient) is one product per
+// layer over the stored factors (dz_l^T, a_{l-1}^T) of every group's last
+// upload, with K running over all groups' rows.  Every product is an "NT" GEMM  C[M x N] = A[M x K] * B[N x K]^T
 // with both operands K-major, so one kernel serves all of them:
 //     forward   z_l   = a_{l-1} W_l^T        A = a_{l-1} [rows][n_{l-1}],  B = W_l   [n_l][n_{l-1}]
 //     backward  da    = dz_l W_l             A = dz_l    [rows][n_l],      B = W_l^T [n_{l-1}][n_l]
 //     weights   dW_l  = dz_l^T a_{l-1}       A = dz_l^T  [n_l][rows],      B = a_{l-1}^T [n_{l-1}][rows]
+//     aggregate sum_g dW_l(last upload of g) the same with rows = all groups' rows of their last uploads
 // which is why activations, dz and the weights are kept in both orientations
 // (the epilogues write the second orientation for free).
 //
@@ -31,7 +35,7 @@ namespace {
 constexpr int BM = 128, BK = 64;  // M tile; K block (BK * 2 bytes = one 128-byte swizzle row)
 constexpr int MAX_STAGES = 8;
 
-enum { EPI_HIDDEN = 0, EPI_SCORES = 1, EPI_DA = 2, EPI_DW = 3 };
+enum { EPI_HIDDEN = 0, EPI_SCORES = 1, EPI_DA = 2, EPI_AGG = 3 };
 enum { ZB_BATCH = 0, ZB_GROUP = 1, ZB_RING = 2 };
 
 struct Bf16Impl {
@@ -52,11 +56,19 @@ struct Bf16Impl {
   __nv_bfloat16* dz[MLP_MAX_LAYERS + 1] = {nullptr};
   __nv_bfloat16* dzT[MLP_MAX_LAYERS + 1] = {nullptr};
   float* scores = nullptr;       // [2][G*Bp][n_L]
+  // factors of each group's last uploaded weight gradient, dW_l = lastA[l][g] * lastB[l][g]^T
+  __nv_bfloat16* lastA[MLP_MAX_LAYERS + 1] = {nullptr};  // [G][n_l][Bp]      dz_l^T at the upload
+  __nv_bfloat16* lastB[MLP_MAX_LAYERS + 1] = {nullptr};  // [G][n_{l-1}][Bp]  a_{l-1}^T at the upload
+  int nbias = 0;                                         // bias entries of all layers
+  int bias_loc[MLP_MAX_LAYERS + 2] = {0};                // first entry of layer l in the compact bias arrays
+  float* db_fresh = nullptr;     // [G][nbias] bias gradients at theta^k, this iteration
+  float* db_last = nullptr;      // [G][nbias] bias gradients of each group's last upload
   int dw_part_base[MLP_MAX_LAYERS + 1] = {0}, bias_part_base[MLP_MAX_LAYERS + 1] = {0};
   int n_parts = 0;               // innovation-norm partial sums per group
   CUtensorMap tm_fwd_a[MLP_MAX_LAYERS + 1], tm_fwd_b[MLP_MAX_LAYERS + 1];
   CUtensorMap tm_da_a[MLP_MAX_LAYERS + 1], tm_da_b[MLP_MAX_LAYERS + 1];
   CUtensorMap tm_dw_a[MLP_MAX_LAYERS + 1], tm_dw_b[MLP_MAX_LAYERS + 1];
+  CUtensorMap tm_agg_a[MLP_MAX_LAYERS + 1], tm_agg_b[MLP_MAX_LAYERS + 1];
 };
 
 struct GemmB {
@@ -65,6 +77,8 @@ struct GemmB {
   int zb_mode;       // ZB_*
   int epi;           // EPI_*
   int stages;
+  int k_batched;     // 1: one output [M][N]; K runs over the batch entries of both operands (kpg K blocks each)
+  int kpg, n_batch;
   // epilogue operands
   __nv_bfloat16* out;    // row-major bf16 [z][M][ldo]
   __nv_bfloat16* outT;   // transposed bf16 [z][N][ldt]
@@ -74,7 +88,7 @@ struct GemmB {
   long long bias_slot, bias_pos;
   long long ldo, ldt;
   long long z_stride_out, z_stride_outT;
-  long long c_off, ldc;       // EPI_DW: offset inside the gradient vector, row stride
+  long long c_off, ldc;       // EPI_AGG: offset inside out_f32 (a p-vector), row stride
 };
 
 // ----------------------------------------------------------------- PTX helpers
@@ -160,10 +174,6 @@ __device__ __forceinline__ void tc_ld32_issue(uint32_t taddr, uint32_t (&v)[32])
 }
 
 __device__ __forceinline__ void tc_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
-  tc_ld32_issue(taddr, v);
-  tc_ld_wait();
-}
 
 // Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes
 // (64 bf16) under the 128-byte swizzle: 8-row atoms of 1024 bytes, start
@@ -206,9 +216,9 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
   __shared__ uint32_t tmem_base_sm;
   unsigned char* tiles = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int nkb = (a.K + BK - 1) / BK;
+  const int nkb = a.k_batched ? a.kpg * a.n_batch : (a.K + BK - 1) / BK;
   const int tiles_n = (a.N + GN - 1) / GN, tiles_m = (a.M + BM - 1) / BM;
-  const int total_tiles = tiles_n * tiles_m * 2 * P.G;
+  const int total_tiles = a.k_batched ? tiles_n * tiles_m : tiles_n * tiles_m * 2 * P.G;
   const long long k_it = P.st->k;
 
   if (threadIdx.x == 0) {
@@ -240,16 +250,26 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
       for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
         const int nt = t % tiles_n, mt = (t / tiles_n) % tiles_m, z = t / (tiles_n * tiles_m);
         const int q = z / P.G, g = z - q * P.G;
-        const int zA = a.a_shared ? g : z;
-        const int zB = a.zb_mode == ZB_RING ? ring_slot(P, g, q, k_it) : (a.zb_mode == ZB_GROUP ? g : z);
+        int zA = 0, zB = 0;
+        if (!a.k_batched) {
+          zA = a.a_shared ? g : z;
+          zB = a.zb_mode == ZB_RING ? ring_slot(P, g, q, k_it) : (a.zb_mode == ZB_GROUP ? g : z);
+        }
+        int kin = 0;  // K block inside the current batch entry (k_batched)
         for (int kb = 0; kb < nkb && ok; ++kb, ++it) {
           const int s = it % G_STAGES;
           ok = mbar_spin_bounded(&empty_bar[s], (uint32_t)(((it / G_STAGES) & 1) ^ 1));
           if (!ok) break;
           unsigned char* sa = tiles + (size_t)s * G_STAGE_BYTES;
           mbar_expect_tx(&full_bar[s], G_STAGE_BYTES);
-          tma_load_3d(sa, &tmA, kb * BK, mt * BM, zA, &full_bar[s]);
-          tma_load_3d(sa + BM * BK * 2, &tmB, kb * BK, nt * GN, zB, &full_bar[s]);
+          const int kc = (a.k_batched ? kin : kb) * BK;
+          tma_load_3d(sa, &tmA, kc, mt * BM, zA, &full_bar[s]);
+          tma_load_3d(sa + BM * BK * 2, &tmB, kc, nt * GN, zB, &full_bar[s]);
+          if (a.k_batched && ++kin == a.kpg) {
+            kin = 0;
+            ++zA;
+            ++zB;
+          }
         }
       }
       if (!ok) atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
@@ -310,7 +330,19 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
         if (nc >= a.N) return;  // uniform across the warp
         const bool row_ok = m < a.M;
         const bool full = nc + 32 <= a.N;
-        if (a.epi == EPI_SCORES) {
+        if (a.epi == EPI_AGG) {  // a block of the aggregated weight gradient, straight into the p-vector
+          float* dst = a.out_f32 + a.c_off + (long long)m * a.ldc + nc;
+          if (row_ok) {
+            if (full && ((a.c_off | a.ldc) & 3) == 0) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 4)
+                *reinterpret_cast<float4*>(dst + j) = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
+                                                                  __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+            } else {
+              for (int j = 0; j < 32 && nc + j < a.N; ++j) dst[j] = __uint_as_float(v[j]);
+            }
+          }
+        } else if (a.epi == EPI_SCORES) {
           float* dst = a.out_f32 + ((long long)z * a.M + m) * a.N + nc;
           if (row_ok) {
             if (full && (a.N & 3) == 0) {
@@ -425,11 +457,10 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
 
 // ----------------------------------------------------------------- weight gradients, both points in one CTA
 // dW_l of one group at theta^k (accumulator 0) and at the stale iterate
-// (accumulator 1), 128 x 256 tiles.  The epilogue writes the fresh gradient
-// (and the stale one only when it is kept for inspection), forms the squared
-// norm of their difference - the tile's share of the left side of Eq. (9) -
-// and stores it in the tile's own slot of lhs_part, so the per-group
-// gradients are never re-read to build the test.
+// (accumulator 1), 128 x 256 tiles.  The epilogue forms the squared norm of
+// their difference - the tile's share of the left side of Eq. (9) - and stores
+// it in the tile's own slot of lhs_part; the gradients themselves are written
+// only when they are kept for inspection.
 //
 // Persistent: one CTA per SM walks work units u = blockIdx.x, + gridDim.x,
 // ...; a unit is one (group, 128-row block of W_l) and its tiles are all the
@@ -451,9 +482,12 @@ struct DwArgs {
   int mode;               // DW_BOTH: both points in two accumulators, norm, gradients written for every group;
                           // DW_NORM: one accumulator receives dW(theta^k) - dW(stale) (the second product enters
                           //          negated), norm only, nothing written but lhs_part;
-                          // DW_SELECTED: point 0 only, fresh gradient written for the groups selected this iteration
+                          // DW_ONE: one group's last uploaded gradient rebuilt from its stored factors (the
+                          //          operands are the last-upload stores) and written to out_row; used by getters
+  int g_only;             // DW_ONE: the group
+  float* out_row;         // DW_ONE: a p-vector
 };
-enum { DW_BOTH = 0, DW_NORM = 1, DW_SELECTED = 2 };
+enum { DW_BOTH = 0, DW_NORM = 1, DW_ONE = 2 };
 
 constexpr int DW_BN = 256;     // N tile: the MMA issue rate, not the tensor pipe, limits 128-wide instructions
 constexpr int DW_PITCH = 36;   // floats per staged row (16-byte aligned, conflict-free 16-byte stores)
@@ -476,11 +510,10 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
   unsigned char* a_res = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   unsigned char* tiles = a_res + (size_t)2 * a.nkb * BLK;  // ring of B blocks
   float* stage_all = reinterpret_cast<float*>(tiles + (size_t)a.stages * BBLK);
-  const int n_units = a.tiles_m * P.G;
+  const int n_units = a.mode == DW_ONE ? a.tiles_m : a.tiles_m * P.G;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int stages = a.stages;
-  const int kb_per_tile = a.mode == DW_SELECTED ? a.nkb : 2 * a.nkb;
-  const unsigned char* sel = a.mode == DW_SELECTED ? P.mask_cur : nullptr;  // tiles of unselected groups are skipped
+  const int kb_per_tile = a.mode == DW_ONE ? a.nkb : 2 * a.nkb;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) {
@@ -511,8 +544,7 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
       bool ok = true;
       int it = 0, ui = 0;
       for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-        const int mt = u % a.tiles_m, g = u / a.tiles_m;
-        if (sel && !sel[g]) continue;
+        const int mt = u % a.tiles_m, g = a.mode == DW_ONE ? a.g_only : u / a.tiles_m;
         // the unit's A blocks, once the MMAs of the previous unit have finished reading them
         ok = mbar_spin_bounded(&aempty_bar, (uint32_t)((ui & 1) ^ 1));
         if (!ok) break;
@@ -540,7 +572,6 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
       bool ok = true;
       int it = 0, i = 0, ui = 0;
       for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-        if (sel && !sel[u / a.tiles_m]) continue;
         ok = mbar_spin_bounded(&afull_bar, (uint32_t)(ui & 1));
         if (!ok) break;
         ++ui;
@@ -577,13 +608,12 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
     const int quad = warp & 3;         // TMEM lanes this warp may read
     const int half = ew >> 2;          // which 128 columns of the tile
     float* stg = stage_all + (size_t)ew * 32 * DW_PITCH;
-    const bool vec_ok = ((a.c_off | a.ldc) & 3) == 0 && (reinterpret_cast<uintptr_t>(P.gbuf) & 15) == 0 &&
-                        (P.p_pad & 3) == 0;
+    const bool vec_ok = ((a.c_off | a.ldc) & 3) == 0 && (P.p_pad & 3) == 0 &&
+                        (reinterpret_cast<uintptr_t>(a.mode == DW_ONE ? a.out_row : P.gbuf) & 15) == 0;
     bool ok = true;
     int i = 0;
     for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
-      const int mt = u % a.tiles_m, g = u / a.tiles_m;
-      if (sel && !sel[g]) continue;
+      const int mt = u % a.tiles_m, g = a.mode == DW_ONE ? a.g_only : u / a.tiles_m;
       for (int nt = 0; nt < a.tiles_n; ++nt) {
       const int slot = i % n_slots;
       const int phase = (i / n_slots) & 1;
@@ -595,9 +625,8 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
       }
       if (ok) {
         tc_fence_after();
-        // before the selection the fresh gradient goes to the row that is not the last uploaded one; the
-        // post-selection pass runs on selected groups only, whose cur[g] already points at that same row
-        float* fresh = (a.mode == DW_SELECTED ? last_row(P, g) : fresh_row(P, g)) + a.c_off;
+        // kept for inspection: the fresh gradient goes to the row that is not the last uploaded one
+        float* fresh = a.mode == DW_NORM ? nullptr : (a.mode == DW_ONE ? a.out_row : fresh_row(P, g)) + a.c_off;
         float* stale = (a.mode == DW_BOTH && P.stale) ? P.stale + (long long)g * P.p_pad + a.c_off : nullptr;
         const int n_pass = a.mode == DW_NORM ? 0 : (stale ? 2 : 1);
         const int mrow = mt * BM + quad * 32;
@@ -610,7 +639,7 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
           tc_ld32_issue(tbase + (uint32_t)c, v0);
           if (a.mode == DW_BOTH) tc_ld32_issue(tbase + (uint32_t)(DW_BN + c), v1);
           tc_ld_wait();  // one wait for both accumulators
-          if (a.mode != DW_SELECTED) {
+          if (a.mode != DW_ONE) {
             const bool row_ok = mrow + lane < a.M;
             const bool interior = nc + 32 <= a.N;
             float part = 0.f;
@@ -656,7 +685,7 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
       local = warp_sum(local);
       if (lane == 0) norm_sm[slot][ew] = local;
       asm volatile("bar.sync 1, %0;" ::"n"(32 * DW_EPI_WARPS) : "memory");
-      if (ew == 0 && lane == 0 && a.mode != DW_SELECTED) {
+      if (ew == 0 && lane == 0 && a.mode != DW_ONE) {
         double tsum = 0.0;
 #pragma unroll
         for (int w = 0; w < DW_EPI_WARPS; ++w) tsum += norm_sm[slot][w];
@@ -831,6 +860,9 @@ struct BiasArgsB {
   long long b_off[MLP_MAX_LAYERS + 1];
   int part_base[MLP_MAX_LAYERS + 1];
   int n_parts;
+  float* db_fresh;                    // [G][nbias]
+  int bias_loc[MLP_MAX_LAYERS + 1];   // first entry of layer l in a db row
+  int nbias;
 };
 // Block = 64 columns x 8 row slices: lane pairs of columns (bf16x2 loads), warp = row slice.
 __global__ void __launch_bounds__(256) bf16_bias_grad_kernel(const Params P, const BiasArgsB a, int Bp) {
@@ -871,13 +903,65 @@ __global__ void __launch_bounds__(256) bf16_bias_grad_kernel(const Params P, con
         f += red[0][w][threadIdx.x];
         sv += red[1][w][threadIdx.x];
       }
-      (fresh_row(P, g) + a.b_off[l])[c] = f;
+      a.db_fresh[(long long)g * a.nbias + a.bias_loc[l] + c] = f;
+      if (P.gbuf) (fresh_row(P, g) + a.b_off[l])[c] = f;  // kept for inspection
       if (P.stale) (P.stale + (long long)g * P.p_pad + a.b_off[l])[c] = sv;
       d2 = (double)(f - sv) * (double)(f - sv);
     }
   }
   d2 = block_sum(d2, scratch);
   if (threadIdx.x == 0) P.lhs_part[(long long)g * a.n_parts + a.part_base[l] + blockIdx.x] = d2;
+}
+
+// ----------------------------------------------------------------- upload: keep the selected groups' factors
+// A selected group's upload replaces its last uploaded gradient (Eq. 3).  The weight gradient is kept as its
+// two factors (dz_l^T and a_{l-1}^T at theta^k, bf16), the bias gradient as it is.  Grid (slices, G).
+struct KeepArgs {
+  const __nv_bfloat16* src[2 * MLP_MAX_LAYERS];
+  __nv_bfloat16* dst[2 * MLP_MAX_LAYERS];
+  long long elems[2 * MLP_MAX_LAYERS];  // per group; a multiple of 8
+  int n_seg;
+  const float* db_fresh;
+  float* db_last;
+  int nbias;
+};
+__global__ void __launch_bounds__(256) bf16_keep_kernel(const Params P, const KeepArgs a) {
+  const int g = blockIdx.y;
+  if (!P.mask_cur[g]) return;
+  for (int s = 0; s < a.n_seg; ++s) {
+    const uint4* src = reinterpret_cast<const uint4*>(a.src[s] + (long long)g * a.elems[s]);
+    uint4* dst = reinterpret_cast<uint4*>(a.dst[s] + (long long)g * a.elems[s]);
+    const long long n16 = a.elems[s] >> 3;
+    for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < n16; i += (long long)gridDim.x * 256) dst[i] = src[i];
+  }
+  for (int i = blockIdx.x * 256 + threadIdx.x; i < a.nbias; i += gridDim.x * 256)
+    a.db_last[(long long)g * a.nbias + i] = a.db_fresh[(long long)g * a.nbias + i];
+}
+
+// Bias part of the aggregate: sum over groups (ascending) of the last uploaded bias gradients.
+struct BiasAggArgs {
+  const float* db_last;
+  int nbias, n_layers;
+  int bias_loc[MLP_MAX_LAYERS + 2];
+  long long b_off[MLP_MAX_LAYERS + 1];
+};
+__global__ void __launch_bounds__(256) bf16_bias_agg_kernel(const Params P, const BiasAggArgs a, float* agg) {
+  const int i = blockIdx.x * 256 + threadIdx.x;
+  if (i >= a.nbias) return;
+  float s = 0.f;
+  for (int g = 0; g < P.G; ++g) s += a.db_last[(long long)g * a.nbias + i];
+  int l = 1;
+  while (l < a.n_layers && i >= a.bias_loc[l + 1]) ++l;
+  agg[a.b_off[l] + (i - a.bias_loc[l])] = s;
+}
+
+// One group's bias gradient of its last upload into a p-vector (getters).
+__global__ void __launch_bounds__(256) bf16_bias_row_kernel(const BiasAggArgs a, int g, float* row) {
+  const int i = blockIdx.x * 256 + threadIdx.x;
+  if (i >= a.nbias) return;
+  int l = 1;
+  while (l < a.n_layers && i >= a.bias_loc[l + 1]) ++l;
+  row[a.b_off[l] + (i - a.bias_loc[l])] = a.db_last[(long long)g * a.nbias + i];
 }
 
 // ----------------------------------------------------------------- host
@@ -917,18 +1001,21 @@ long long up(long long x, long long m) { return (x + m - 1) / m * m; }
 cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const Params& P, GemmB a, int sm_count,
                         cudaStream_t st) {
   a.stages = G_STAGES;
-  const long long tiles = (long long)((a.N + GN - 1) / GN) * ((a.M + BM - 1) / BM) * 2 * P.G;
+  const long long tiles = (long long)((a.N + GN - 1) / GN) * ((a.M + BM - 1) / BM) * (a.k_batched ? 1 : 2 * P.G);
   const int ctas = (int)(tiles < sm_count ? tiles : sm_count);
   bf16_gemm_kernel<<<ctas, G_THREADS, (size_t)G_STAGES * G_STAGE_BYTES + 1024 + G_TR_BYTES, st>>>(ta, tb, P, a);
   return cudaGetLastError();
 }
 
-cudaError_t launch_dw(const Params& P, const MlpPlan& pl, const Bf16Impl* im, int l, int mode, cudaStream_t st) {
+cudaError_t launch_dw(const Params& P, const MlpPlan& pl, const Bf16Impl* im, int l, int mode, cudaStream_t st,
+                      int g_only = 0, float* out_row = nullptr) {
   DwArgs w{};
+  w.g_only = g_only;
+  w.out_row = out_row;
   w.M = pl.dims[l];
   w.N = pl.dims[l - 1];
   w.K = im->Bp;
-  w.b_shared = l == 1;
+  w.b_shared = (l == 1 || mode == DW_ONE) ? 1 : 0;  // the last-upload stores have one entry per group
   w.nkb = im->Bp / BK;
   // 32 KiB B blocks in whatever shared memory is left beside the resident A blocks (and the staging tile of
   // the modes that write gradients): the B stream is bound by bytes in flight, so every stage counts
@@ -945,10 +1032,13 @@ cudaError_t launch_dw(const Params& P, const MlpPlan& pl, const Bf16Impl* im, in
   w.part_base = im->dw_part_base[l];
   w.n_parts = im->n_parts;
   w.mode = mode;
-  const int units = w.tiles_m * P.G;
+  const int units = mode == DW_ONE ? w.tiles_m : w.tiles_m * P.G;
   const int ctas = units < pl.sm_count ? units : pl.sm_count;
   const size_t smem = (size_t)(2 * w.nkb + 2 * w.stages) * (BM * BK * 2) + 1024 + (size_t)stage_bytes;
-  bf16_dw_kernel<<<ctas, DW_THREADS, smem, st>>>(im->tm_dw_a[l], im->tm_dw_b[l], P, w);
+  if (mode == DW_ONE)
+    bf16_dw_kernel<<<ctas, DW_THREADS, smem, st>>>(im->tm_agg_a[l], im->tm_agg_b[l], P, w);
+  else
+    bf16_dw_kernel<<<ctas, DW_THREADS, smem, st>>>(im->tm_dw_a[l], im->tm_dw_b[l], P, w);
   return cudaGetLastError();
 }
 
@@ -996,6 +1086,8 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
   }
   im->n_parts = parts;
   plan->norm_parts = parts;
+  for (int l = 1; l <= L; ++l) im->bias_loc[l + 1] = im->bias_loc[l] + plan->dims[l];
+  im->nbias = im->bias_loc[L + 1];
   auto alloc = [&](void** q, size_t bytes) -> cudaError_t {
     cudaError_t e = cudaMalloc(q, bytes);
     if (e != cudaSuccess) return e;
@@ -1021,6 +1113,12 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
     A_(im->dzT[l], 2LL * G * plan->dims[l] * im->Bp, __nv_bfloat16);
   }
   A_(im->scores, 2 * rows * plan->dims[L], float);
+  for (int l = 1; l <= L; ++l) {
+    A_(im->lastA[l], (long long)G * plan->dims[l] * im->Bp, __nv_bfloat16);
+    A_(im->lastB[l], (long long)G * plan->dims[l - 1] * im->Bp, __nv_bfloat16);
+  }
+  A_(im->db_fresh, (long long)G * im->nbias, float);
+  A_(im->db_last, (long long)G * im->nbias, float);
 #undef A_
   if (!encode_fn()) {
     *why = "cuTensorMapEncodeTiled is not available from this driver";
@@ -1045,6 +1143,9 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
       ok &= make_map(&im->tm_dw_b[l], im->xbT, Bp, ni, G, Bp, (long long)ni * Bp, DW_BN);
     else
       ok &= make_map(&im->tm_dw_b[l], im->actT[l - 1], Bp, ni, 2LL * G, Bp, (long long)ni * Bp, DW_BN);
+    // aggregate: the same two operands, taken from the last-upload stores (one entry per group)
+    ok &= make_map(&im->tm_agg_a[l], im->lastA[l], Bp, no, G, Bp, (long long)no * Bp, BM);
+    ok &= make_map(&im->tm_agg_b[l], im->lastB[l], Bp, ni, G, Bp, (long long)ni * Bp, GN);
   }
   if (!ok) {
     *why = "tensor map creation failed for this MLP shape";
@@ -1059,6 +1160,7 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
   e = cudaFuncSetAttribute(bf16_dw_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 4096);  // the rest is static
   if (e != cudaSuccess) return e;
   plan->launches_per_iter = 3 + L + 1 + L + (L - 1);
+  plan->post_launches = L + 2;
   return cudaSuccess;
 }
 
@@ -1157,9 +1259,12 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
     ba.ld[l] = im->ld[l];
     ba.b_off[l] = pl.b_off[l];
     ba.part_base[l] = im->bias_part_base[l];
+    ba.bias_loc[l] = im->bias_loc[l];
     if (pl.dims[l] > maxn) maxn = pl.dims[l];
   }
   ba.n_parts = im->n_parts;
+  ba.db_fresh = im->db_fresh;
+  ba.nbias = im->nbias;
   bf16_bias_grad_kernel<<<dim3((maxn + 63) / 64, G, L), 256, 0, st>>>(P, ba, Bp);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   ++n;
@@ -1170,17 +1275,71 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
 }  // namespace gcada
 
 namespace gcada {
-// After the selection: weight gradients of the selected groups (the only ones
-// the server's aggregate needs, Eq. 3) are recomputed at theta^k and written.
+namespace {
+BiasAggArgs bias_agg_args(const MlpPlan& pl, const Bf16Impl* im) {
+  BiasAggArgs b{};
+  b.db_last = im->db_last;
+  b.nbias = im->nbias;
+  b.n_layers = pl.n_layers;
+  for (int l = 1; l <= pl.n_layers + 1; ++l) b.bias_loc[l] = im->bias_loc[l];
+  for (int l = 1; l <= pl.n_layers; ++l) b.b_off[l] = pl.b_off[l];
+  return b;
+}
+}  // namespace
+
+// After the selection, the server's side of Eq. (3): the selected groups' uploads replace their last
+// uploaded gradients (kept as factors), and the aggregate - the sum over ALL groups of the last uploaded
+// gradients - is formed anew as one product per layer whose K dimension runs over every group's rows.
+// Nothing is accumulated across iterations, so the aggregate carries no drift.
 cudaError_t mlp_bf16_launch_post(const Params& P, const MlpPlan& pl, cudaStream_t st, int* n_launches) {
   *n_launches = 0;
-  if (P.stale) return cudaSuccess;  // everything was materialised by the first pass
   const Bf16Impl* im = static_cast<const Bf16Impl*>(pl.bf16_impl);
-  for (int l = pl.n_layers; l >= 1; --l) {
-    cudaError_t e = launch_dw(P, pl, im, l, DW_SELECTED, st);
-    if (e != cudaSuccess) return e;
+  const int L = pl.n_layers, G = P.G, Bp = im->Bp;
+  cudaError_t e;
+  KeepArgs k{};
+  for (int l = 1; l <= L; ++l) {
+    k.src[k.n_seg] = im->dzT[l];
+    k.dst[k.n_seg] = im->lastA[l];
+    k.elems[k.n_seg++] = (long long)pl.dims[l] * Bp;
+    k.src[k.n_seg] = l == 1 ? im->xbT : im->actT[l - 1];
+    k.dst[k.n_seg] = im->lastB[l];
+    k.elems[k.n_seg++] = (long long)pl.dims[l - 1] * Bp;
+  }
+  k.db_fresh = im->db_fresh;
+  k.db_last = im->db_last;
+  k.nbias = im->nbias;
+  bf16_keep_kernel<<<dim3(64, G), 256, 0, st>>>(P, k);
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  ++*n_launches;
+  for (int l = L; l >= 1; --l) {
+    GemmB a{};
+    a.M = pl.dims[l];
+    a.N = pl.dims[l - 1];
+    a.K = G * Bp;
+    a.k_batched = 1;
+    a.kpg = Bp / BK;
+    a.n_batch = G;
+    a.epi = EPI_AGG;
+    a.out_f32 = P.agg_hi;
+    a.c_off = pl.w_off[l];
+    a.ldc = pl.dims[l - 1];
+    if ((e = launch_gemm(im->tm_agg_a[l], im->tm_agg_b[l], P, a, pl.sm_count, st)) != cudaSuccess) return e;
     ++*n_launches;
   }
+  bf16_bias_agg_kernel<<<(im->nbias + 255) / 256, 256, 0, st>>>(P, bias_agg_args(pl, im), P.agg_hi);
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  ++*n_launches;
   return cudaSuccess;
+}
+
+// Group g's last uploaded gradient, rebuilt from its stored factors into `row` (a p-vector on the device).
+cudaError_t mlp_bf16_group_gradient(const Params& P, const MlpPlan& pl, int g, float* row, cudaStream_t st) {
+  const Bf16Impl* im = static_cast<const Bf16Impl*>(pl.bf16_impl);
+  for (int l = pl.n_layers; l >= 1; --l) {
+    cudaError_t e = launch_dw(P, pl, im, l, DW_ONE, st, g, row);
+    if (e != cudaSuccess) return e;
+  }
+  bf16_bias_row_kernel<<<(im->nbias + 255) / 256, 256, 0, st>>>(bias_agg_args(pl, im), g, row);
+  return cudaGetLastError();
 }
 }  // namespace gcada

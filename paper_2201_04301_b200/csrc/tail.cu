@@ -355,6 +355,61 @@ __global__ void __launch_bounds__(256) update_kernel(const Params P) {
   }
 }
 
+// Eq. (8a)-(8c) when the aggregate has already been formed in agg_hi (P.agg_direct): one float4 per thread.
+__global__ void __launch_bounds__(256) update_direct_kernel(const Params P) {
+  __shared__ double scratch[40];
+  __shared__ bool is_last;
+  const int tid = threadIdx.x;
+  const long long cols4 = P.p_pad >> 2;
+  const long long k = P.st->k;
+  const int ring = P.D + 1;
+  const long long i4 = (long long)blockIdx.x * 256 + tid;
+  double local = 0.0;
+  if (i4 < cols4) {
+    const long long o = i4 * 4;
+    const float4 ahi = ld4(P.agg_hi + o);
+    float4 h = ld4(P.h + o), vh = ld4(P.vhat + o);
+    const float4 th = ld4(P.theta_ring + (k % ring) * P.p_pad + o);
+    float4 tn;
+#define GCADA_AMSGRAD(c)                                   \
+  {                                                        \
+    const float gr = ahi.c;                                \
+    h.c = P.beta1 * h.c + P.omb1 * gr;                     \
+    const float v = P.beta2 * vh.c + P.omb2 * (gr * gr);   \
+    vh.c = fmaxf(vh.c, v);                                 \
+    const float up = P.alpha * h.c / sqrtf(P.eps + vh.c);  \
+    tn.c = th.c - up;                                      \
+    local += (double)up * (double)up;                      \
+  }
+    GCADA_AMSGRAD(x)
+    GCADA_AMSGRAD(y)
+    GCADA_AMSGRAD(z)
+    GCADA_AMSGRAD(w)
+#undef GCADA_AMSGRAD
+    st4(P.h + o, h);
+    st4(P.vhat + o, vh);
+    st4(P.theta_ring + ((k + 1) % ring) * P.p_pad + o, tn);
+  }
+  const double tot = block_sum(local, scratch);
+  if (tid == 0) {
+    P.upd_part[blockIdx.x] = tot;
+    __threadfence();
+    is_last = atomicAdd(&P.st->ticket_update, 1u) == gridDim.x - 1u;
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  const volatile double* parts = P.upd_part;
+  double s = 0.0;
+  for (unsigned int b = tid; b < gridDim.x; b += 256) s += parts[b];
+  s = block_sum(s, scratch);
+  if (tid == 0) {
+    P.s_ring[k % P.D] = s;
+    P.st->k = k + 1;
+    P.st->ticket_update = 0u;
+  }
+}
+
 // Rule PS: left side of Eq. (9) exactly as printed, L_g^2 ||theta^k - theta^{k-tau_g}||^2, from the
 // iterate ring.  Grid (column blocks, D): block (b, d-1) sums its slice of ||theta^k - theta^{k-d}||^2
 // (theta^j = theta^0 for j < 0); the last block adds the slices in a fixed order and scales by L_g^2.
@@ -429,6 +484,10 @@ cudaError_t launch_select(const Params& P, const TailPlan& plan, cudaStream_t st
 }
 
 cudaError_t launch_update(const Params& P, const TailPlan& plan, cudaStream_t st) {
+  if (P.agg_direct) {
+    update_direct_kernel<<<(plan.update_blocks + 7) / 8, 256, 0, st>>>(P);
+    return cudaGetLastError();
+  }
   update_kernel<<<plan.update_blocks, 256, (size_t)P.G * sizeof(int), st>>>(P);
   return cudaGetLastError();
 }

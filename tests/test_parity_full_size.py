@@ -54,23 +54,30 @@ def test_cfg3_full_size_sampled_groups():
 
 
 def test_cfg5_full_size_sampled_groups():
-    """1024-4096-4096-1000, bf16 operands, 256 groups x 128 rows: the first iteration selects every
-    group, so every fresh gradient is written; two of them are recomputed by the oracle."""
+    """1024-4096-4096-1000, bf16 operands, 256 groups x 128 rows.  The first iteration is forced to
+    upload eight groups only: two of their gradients (rebuilt from the kept factors) are recomputed by
+    the oracle, and the aggregate must be the sum of the eight (Eq. 3)."""
     w = make_workload("cfg5", device="cuda")
     G = w["M"] // w["M_G"]
     g = binding.from_workload(w, stream=torch.cuda.Stream())
     model = make_model("mlp", w["dims"], bf16=True)
     theta = g.get_theta().astype(np.float64)
-    g.step(1)
-    assert g.get_selection_mask(0, 1).all()
-    for gi in (3, 200):
-        Xb, yb = _group_batch(w, 0, gi, G)
-        want = model.grad(theta, Xb, yb, "mean")
-        got = g.get_group_gradient(binding.DBG_FRESH, gi)
-        assert rel_l2(got, want) <= TOL_BF16
-        assert np.array_equal(got, g.get_group_gradient(binding.DBG_GLAST, gi))
+    chosen = (3, 40, 77, 100, 131, 200, 201, 255)
+    mask0 = np.zeros((1, G), dtype=np.uint8)
+    mask0[0, list(chosen)] = 1
+    g.step_forced(mask0)
+    total = np.zeros(g.p, dtype=np.float64)
+    for gi in chosen:
+        got = g.get_group_gradient(binding.DBG_GLAST, gi)
+        total += got
+        if gi in (3, 200):
+            Xb, yb = _group_batch(w, 0, gi, G)
+            assert rel_l2(got, model.grad(theta, Xb, yb, "mean")) <= TOL_BF16
+    assert rel_l2(g.get_debug(binding.DBG_AGG), total) <= 1e-5
+    assert not g.get_group_gradient(binding.DBG_GLAST, 0).any()      # never uploaded
     g.step(12)
     masks = g.get_selection_mask(0, 13)
+    assert masks[1, np.setdiff1d(np.arange(G), chosen)].all()        # the others' age passed D: selected by the age rule
     up, comm, comp = g.get_comm_count()
     assert up == int(masks.sum()) and comm == 5 * up and comp == 4 * up
     assert np.isfinite(g.get_theta()).all()
