@@ -145,6 +145,31 @@ gcada_status gcada_set_seed(gcada_ctx *ctx, unsigned long long seed);
  * shift 0, rate 1/eta.  GCADA_EINVAL unless shift >= 0 and rate > 0. */
 gcada_status gcada_set_delay_model(gcada_ctx *ctx, double shift, double rate);
 
+/* Law of the computing times.  Section II-B takes them exponential; the analysis of Section V only uses
+ * that they are i.i.d., so two more laws are offered, with the (shift, rate) of gcada_set_delay_model:
+ * GCADA_DELAY_EXP      T = shift - ln(1-u)/rate           (default)
+ * GCADA_DELAY_PARETO   T = shift * (1-u)^(-1/rate)        heavy tail, P(T > t) = (shift/t)^rate, shift > 0
+ * GCADA_DELAY_UNIFORM  T = shift + u/rate                 bounded */
+#define GCADA_DELAY_EXP 0
+#define GCADA_DELAY_PARETO 1
+#define GCADA_DELAY_UNIFORM 2
+gcada_status gcada_set_delay_law(gcada_ctx *ctx, int law);
+
+/* Per-lag constants {c_d} (host, D doubles >= 0; copied) of Algorithm 1's input list: the right side of
+ * the test becomes sum_{d=1..D} c_d ||theta^{k+1-d} - theta^{k-d}||^2.  NULL restores c_d = c, which is
+ * Eq. (9) as printed.  Set before the first step (GCADA_ESTATE afterwards). */
+gcada_status gcada_set_lag_weights(gcada_ctx *ctx, const double *c_d, int D);
+
+/* Step size alpha^k of Eq. (2) / Eq. (8c), alpha being gcada_create's:
+ * GCADA_SCHEDULE_CONST  alpha^k = alpha                          (default; a, b ignored)
+ * GCADA_SCHEDULE_POLY   alpha^k = alpha / (1 + k/a)^b            a > 0, b >= 0
+ * GCADA_SCHEDULE_STEP   alpha^k = alpha * b^floor(k/a)           integer a >= 1, b > 0
+ * k counts from 0.  May be changed between steps. */
+#define GCADA_SCHEDULE_CONST 0
+#define GCADA_SCHEDULE_POLY 1
+#define GCADA_SCHEDULE_STEP 2
+gcada_status gcada_set_step_schedule(gcada_ctx *ctx, int kind, double a, double b);
+
 gcada_status gcada_set_option(gcada_ctx *ctx, int key, double value);
 
 /* Smoothness constants L_g >= 0 (host, G doubles; copied) for rule PS, the left side of Eq. (9) as
@@ -256,6 +281,21 @@ gcada_status gcada_innovation_norms_noalloc(const float *fresh_dev, const float 
  * a kernel that lasts tens of microseconds).  The repetitions recompute the same gradients and change no
  * state that an iteration reads.  Synchronises the stream before and after. */
 gcada_status gcada_time_gradient(gcada_ctx *ctx, int reps, double *ms_per_rep);
+
+/*
+ * Checkpoints (the paper has no counterpart).  A checkpoint is everything an iteration inherits from
+ * earlier ones: iteration counter, counters and wall-clock, the last D+1 iterates, h, v-hat, the
+ * aggregate, every group's last uploaded gradient (or its factors), ages, the ring of squared step norms
+ * and the mask history.  It does NOT hold the constructor arguments, seed, delay model, options or the
+ * training set: load into a context created and configured like the one that saved (gcada_create, options,
+ * gcada_set_data or gcada_set_batch, gcada_set_theta with any theta), otherwise GCADA_EINVAL and nothing is
+ * changed.  After a load the run continues bit-for-bit as the saved one would have.
+ * gcada_checkpoint_size gives the byte count for this context; save / load need a host buffer of exactly
+ * that size.  All three synchronise the stream.
+ */
+gcada_status gcada_checkpoint_size(gcada_ctx *ctx, unsigned long long *bytes);
+gcada_status gcada_checkpoint_save(gcada_ctx *ctx, void *host_buf, unsigned long long bytes);
+gcada_status gcada_checkpoint_load(gcada_ctx *ctx, const void *host_buf, unsigned long long bytes);
 
 /* Text of the last error of this context ("" if none); valid until the next
  * call on the context.  ctx == NULL returns the text of the last failed

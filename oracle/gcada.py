@@ -35,6 +35,12 @@ constant c; minibatch = `batch` uniform draws with replacement from the
 group's shard, shared by the workers of the group; computing time
 T = shift - ln(1-u)/rate (shift 0, rate 1/eta is the paper's exponential).
 
+Optional generalisations the paper names without using them: per-lag constants
+{c_d} (Algorithm 1's input list) weight the D terms of the right side of
+Eq. (9) individually; the step size alpha^k (Eq. 2, Eq. 8c) may follow a
+schedule; computing times may follow another law than the exponential of
+Section II-B (the analysis of Section V only needs i.i.d. times).
+
 parity unpinned: free-running trajectories longer than the pinned special
 cases (near-ties in the selection test may legitimately flip).
 """
@@ -46,7 +52,8 @@ from . import philox
 class GCadaOracle:
     def __init__(self, model, M, M_G, D, c, alpha, beta1, beta2, eps, *,
                  X, y, batch, theta0, seed=0, shift=1.0, rate=1.0,
-                 rule="innov", reduction="mean", L=None):
+                 rule="innov", reduction="mean", L=None, c_d=None, schedule=("const",),
+                 delay_law="exp"):
         if M <= 0 or M_G <= 0 or M % M_G or D < 1 or c < 0 or alpha <= 0 \
                 or not (0 < beta1 < 1) or not (0 < beta2 < 1) or eps <= 0:
             raise ValueError("invalid G-CADA parameters")
@@ -61,6 +68,10 @@ class GCadaOracle:
         self.seed, self.shift, self.rate = seed, float(shift), float(rate)
         self.rule, self.reduction = rule, reduction
         self.L = None if L is None else np.asarray(L, dtype=np.float64)
+        # c_d[d-1] multiplies ||theta^{k+1-d} - theta^{k-d}||^2; the printed Eq. (9) has c_d = c for all d
+        self.c_d = np.full(D, self.c) if c_d is None else np.asarray(c_d, dtype=np.float64).reshape(D)
+        self.schedule = tuple(schedule)
+        self.delay_law = delay_law
         p = model.p
         self.thetas = [np.array(theta0, dtype=np.float64).reshape(p)]   # theta^0..theta^k
         self.h = np.zeros(p)
@@ -80,14 +91,28 @@ class GCadaOracle:
         return self.thetas[max(j, 0)]
 
     def rhs(self):
-        """c * sum_{d=1..D} ||theta^{k+1-d} - theta^{k-d}||^2  (Eq. 9, right side)."""
+        """sum_{d=1..D} c_d ||theta^{k+1-d} - theta^{k-d}||^2  (Eq. 9, right side; c_d = c as printed)."""
         k, total = self.k, 0.0
         for d in range(1, self.D + 1):
             if k - d < 0:
                 continue
             diff = self.thetas[k + 1 - d] - self.thetas[k - d]
-            total += float(diff @ diff)
-        return self.c * total
+            total += self.c_d[d - 1] * float(diff @ diff)
+        return total
+
+    def step_size(self, k):
+        """alpha^k of Eq. (8c).  ("const",): alpha;  ("poly", t0, q): alpha / (1 + k/t0)^q;
+        ("step", every, factor): alpha * factor^floor(k / every)."""
+        kind = self.schedule[0]
+        if kind == "const":
+            return self.alpha
+        if kind == "poly":
+            _, t0, q = self.schedule
+            return self.alpha / (1.0 + k / float(t0)) ** float(q)
+        if kind == "step":
+            _, every, factor = self.schedule
+            return self.alpha * float(factor) ** (k // int(every))
+        raise ValueError(kind)
 
     def minibatch(self, g):
         idx = philox.batch_indices(self.seed, self.k, g, self.batch, self.n_g)
@@ -98,7 +123,13 @@ class GCadaOracle:
     def delays(self):
         """T_m^k for all M workers (Section II-B)."""
         u = philox.uniform01(self.seed, self.k, np.arange(self.M))
-        return self.shift - np.log1p(-u) / self.rate
+        if self.delay_law == "exp":         # Section II-B (shift 0): exponential with mean 1/rate
+            return self.shift - np.log1p(-u) / self.rate
+        if self.delay_law == "pareto":      # heavy tail: P(T > t) = (shift/t)^rate for t >= shift
+            return self.shift * np.exp(-np.log1p(-u) / self.rate)
+        if self.delay_law == "uniform":     # bounded: uniform on [shift, shift + 1/rate]
+            return self.shift + u / self.rate
+        raise ValueError(self.delay_law)
 
     @staticmethod
     def wallclock_increment(T, mask, M_G):
@@ -149,7 +180,7 @@ class GCadaOracle:
         agg = self.g_last.sum(axis=0)
         theta_next, self.h, self.vhat = self.amsgrad(
             theta_k, self.h, self.vhat, agg,
-            self.alpha, self.beta1, self.beta2, self.eps)
+            self.step_size(k), self.beta1, self.beta2, self.eps)
         self.thetas.append(theta_next)
         tau_used = self.tau.copy()
         self.tau = np.where(mask, 1, self.tau + 1)

@@ -20,6 +20,8 @@ OPT_RULE, OPT_REDUCTION, OPT_HISTORY, OPT_KEEP_STALE, OPT_GRAPH, OPT_TIMING, OPT
  DBG_SRING) = range(11)
 MODEL_KINDS = {"logistic": MODEL_LOGISTIC, "mlp": MODEL_MLP, "quadratic": MODEL_QUADRATIC}
 COMPUTE_KINDS = {"fp32": COMPUTE_FP32, "bf16": COMPUTE_BF16}
+DELAY_LAWS = {"exp": 0, "pareto": 1, "uniform": 2}
+SCHEDULES = {"const": 0, "poly": 1, "step": 2}
 
 
 class Model(C.Structure):
@@ -43,6 +45,9 @@ SIGNATURES = {
     "gcada_set_seed": (C.c_int, [_VP, C.c_ulonglong]),
     "gcada_set_delay_model": (C.c_int, [_VP, C.c_double, C.c_double]),
     "gcada_set_option": (C.c_int, [_VP, C.c_int, C.c_double]),
+    "gcada_set_delay_law": (C.c_int, [_VP, C.c_int]),
+    "gcada_set_lag_weights": (C.c_int, [_VP, C.POINTER(C.c_double), C.c_int]),
+    "gcada_set_step_schedule": (C.c_int, [_VP, C.c_int, C.c_double, C.c_double]),
     "gcada_set_smoothness": (C.c_int, [_VP, C.POINTER(C.c_double), C.c_int]),
     "gcada_step": (C.c_int, [_VP, C.c_int]),
     "gcada_step_forced": (C.c_int, [_VP, C.c_int, _VP]),
@@ -59,6 +64,9 @@ SIGNATURES = {
     "gcada_get_kernel_times": (C.c_int, [_VP, C.POINTER(C.c_double), C.POINTER(C.c_int)]),
     "gcada_innovation_norms_noalloc": (C.c_int, [_VP, _VP, C.c_int, _LL, _LL, _VP, _VP, C.c_char_p, C.c_size_t]),
     "gcada_time_gradient": (C.c_int, [_VP, C.c_int, C.POINTER(C.c_double)]),
+    "gcada_checkpoint_size": (C.c_int, [_VP, _ULLP]),
+    "gcada_checkpoint_save": (C.c_int, [_VP, _VP, C.c_ulonglong]),
+    "gcada_checkpoint_load": (C.c_int, [_VP, _VP, C.c_ulonglong]),
     "gcada_last_error": (C.c_char_p, [_VP]),
     "gcada_destroy": (None, [_VP]),
 }
@@ -152,6 +160,19 @@ class GCada:
     def set_option(self, key, value):
         self._ck(self.lib.gcada_set_option(self.h, int(key), float(value)))
 
+    def set_delay_law(self, law):
+        self._ck(self.lib.gcada_set_delay_law(self.h, DELAY_LAWS.get(law, law)))
+
+    def set_lag_weights(self, c_d):
+        if c_d is None:
+            self._ck(self.lib.gcada_set_lag_weights(self.h, None, 0))
+        else:
+            a = (C.c_double * len(c_d))(*[float(v) for v in c_d])
+            self._ck(self.lib.gcada_set_lag_weights(self.h, a, len(c_d)))
+
+    def set_step_schedule(self, kind, a=1.0, b=0.0):
+        self._ck(self.lib.gcada_set_step_schedule(self.h, SCHEDULES.get(kind, kind), float(a), float(b)))
+
     def set_smoothness(self, L):
         a = (C.c_double * len(L))(*[float(v) for v in L])
         self._ck(self.lib.gcada_set_smoothness(self.h, a, len(L)))
@@ -219,6 +240,18 @@ class GCada:
         self._ck(self.lib.gcada_get_kernel_times(self.h, ms, C.byref(n)))
         return (ms[0], ms[1], ms[2]), n.value
 
+    def checkpoint_save(self):
+        """The run's state as a numpy byte array (see gcada_checkpoint_save)."""
+        n = C.c_ulonglong()
+        self._ck(self.lib.gcada_checkpoint_size(self.h, C.byref(n)))
+        buf = np.empty(n.value, dtype=np.uint8)
+        self._ck(self.lib.gcada_checkpoint_save(self.h, _VP(buf.ctypes.data), n.value))
+        return buf
+
+    def checkpoint_load(self, buf):
+        buf = np.ascontiguousarray(buf, dtype=np.uint8)
+        self._ck(self.lib.gcada_checkpoint_load(self.h, _VP(buf.ctypes.data), buf.size))
+
     def get_debug(self, what):
         G, p, D = self.G, self.p, self.D
         shape, dt = {
@@ -253,7 +286,7 @@ def innovation_norms_noalloc(fresh, stale, lhs_out, stream=None):
         raise GCadaError(st, buf.value.decode())
 
 
-def from_workload(w, stream=None, options=None, smoothness=None):
+def from_workload(w, stream=None, options=None, smoothness=None, c_d=None, schedule=None, delay_law=None):
     """Context for a dict made by workloads.make_workload (tensors on CUDA)."""
     g = GCada(w["kind"], w["dims"], w["M"], w["M_G"], w["D"], w["c"], w["alpha"], w["beta1"], w["beta2"],
               w["eps"], compute=w["compute"], stream=stream)
@@ -263,6 +296,12 @@ def from_workload(w, stream=None, options=None, smoothness=None):
         g.set_option(key, val)
     if smoothness is not None:
         g.set_smoothness(smoothness)
+    if c_d is not None:
+        g.set_lag_weights(c_d)
+    if schedule is not None:
+        g.set_step_schedule(*schedule)
+    if delay_law is not None:
+        g.set_delay_law(delay_law)
     g.set_data(w["X"], w["y"], w["batch"], ld=w["ld"])
     g.set_theta(w["theta0"])
     return g

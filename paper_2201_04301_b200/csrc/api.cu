@@ -49,6 +49,10 @@ struct gcada_ctx {
   // device memory
   std::vector<void*> owned;
   std::vector<double> L2;  // squared smoothness constants (rule PS)
+  std::vector<double> c_d; // per-lag constants of Eq. (9)'s right side (empty: c for every lag)
+  int sched_kind = 0;
+  double sched_a = 1.0, sched_b = 0.0;
+  int delay_law = 0;
   DevState* st = nullptr;
   Params P{};
   LinearPlan lin{};
@@ -59,6 +63,7 @@ struct gcada_ctx {
   void* stage_x = nullptr;
   void* stage_y = nullptr;
   long long stage_ld = 0;
+  std::vector<std::pair<void*, size_t>> state;  // device buffers a checkpoint holds (besides the plan's)
   float* row_scratch = nullptr;  // one p-vector for getters that rebuild a group's gradient on demand
   // graphs (free-running resident-data mode only)
   cudaGraphExec_t graph1 = nullptr, graphN = nullptr;
@@ -125,6 +130,7 @@ void free_all(gcada_ctx* ctx) {
   if (ctx->stage_y) cudaFree(ctx->stage_y);
   ctx->stage_x = ctx->stage_y = nullptr;
   ctx->row_scratch = nullptr;  // was in `owned`
+  ctx->state.clear();
   ctx->st = nullptr;
   ctx->ready = false;
 }
@@ -165,6 +171,10 @@ gcada_status make_ready(gcada_ctx* ctx, const float* theta0, int on_device) {
   P.d = ctx->dims[0];
   P.c = ctx->c;
   P.alpha = (float)ctx->alpha;
+  P.alpha_d = ctx->alpha;
+  P.sched_kind = ctx->sched_kind;
+  P.sched_a = ctx->sched_a;
+  P.sched_b = ctx->sched_b;
   P.beta1 = (float)ctx->beta1;
   P.beta2 = (float)ctx->beta2;
   P.omb1 = (float)(1.0 - ctx->beta1);
@@ -195,6 +205,24 @@ gcada_status make_ready(gcada_ctx* ctx, const float* theta0, int on_device) {
   plan_tail(pp, G, ctx->sm_count, &ctx->tail);
   TRY(dev_alloc(ctx, &P.lhs_part, (size_t)G * ctx->tail.select_blocks_x));
   TRY(dev_alloc(ctx, &P.upd_part, (size_t)ctx->tail.update_blocks));
+  // everything an iteration inherits from earlier ones
+  {
+    auto& S = ctx->state;
+    S.emplace_back(ctx->st, sizeof(DevState));
+    S.emplace_back(P.theta_ring, sizeof(float) * (size_t)(D + 1) * pp);
+    S.emplace_back(P.h, sizeof(float) * (size_t)pp);
+    S.emplace_back(P.vhat, sizeof(float) * (size_t)pp);
+    S.emplace_back(P.agg_hi, sizeof(float) * (size_t)pp);
+    S.emplace_back(P.agg_lo, sizeof(float) * (size_t)pp);
+    if (P.gbuf) S.emplace_back(P.gbuf, sizeof(float) * (size_t)2 * G * pp);
+    S.emplace_back(P.cur, (size_t)G);
+    S.emplace_back(P.tau, sizeof(int) * (size_t)G);
+    S.emplace_back(P.s_ring, sizeof(double) * (size_t)D);
+    S.emplace_back(P.mask_cur, (size_t)G);
+    S.emplace_back(P.hist, (size_t)ctx->hist_cap * G);
+    S.emplace_back(P.lhs, sizeof(double) * (size_t)G);
+    S.emplace_back(P.t_g, sizeof(double) * (size_t)G);
+  }
   // tau_g^0 = D: the first iteration selects every group
   {
     std::vector<int> tau0(G, D);
@@ -219,6 +247,14 @@ gcada_status make_plans(gcada_ctx* ctx) {
   P.seed_hi = (uint32_t)(ctx->seed >> 32);
   P.shift = ctx->shift;
   P.inv_rate = 1.0 / ctx->rate;
+  P.delay_law = ctx->delay_law;
+  P.c_d = nullptr;
+  if (!ctx->c_d.empty()) {
+    double* cd = nullptr;
+    TRY(dev_alloc(ctx, &cd, (size_t)ctx->D));
+    CK(cudaMemcpyAsync(cd, ctx->c_d.data(), sizeof(double) * ctx->D, cudaMemcpyHostToDevice, ctx->stream));
+    P.c_d = cd;
+  }
   P.X = ctx->X;
   P.y = ctx->y;
   P.ld = ctx->ld;
@@ -541,6 +577,53 @@ gcada_status gcada_set_delay_model(gcada_ctx* ctx, double shift, double rate) {
   ctx->rate = rate;
   ctx->P.shift = shift;
   ctx->P.inv_rate = 1.0 / rate;
+  drop_graphs(ctx);
+  return GCADA_OK;
+}
+
+gcada_status gcada_set_delay_law(gcada_ctx* ctx, int law) {
+  if (!ctx) return GCADA_EINVAL;
+  if (law < 0 || law > 2) return fail(ctx, GCADA_EINVAL, "unknown delay law %d", law);
+  ctx->delay_law = law;
+  ctx->P.delay_law = law;
+  drop_graphs(ctx);
+  return GCADA_OK;
+}
+
+gcada_status gcada_set_lag_weights(gcada_ctx* ctx, const double* c_d, int D) {
+  if (!ctx) return GCADA_EINVAL;
+  if (ctx->k_host > 0) return fail(ctx, GCADA_ESTATE, "the lag weights are fixed once stepping has begun");
+  if (!c_d) {
+    ctx->c_d.clear();
+  } else {
+    if (D != ctx->D) return fail(ctx, GCADA_EINVAL, "need D = %d lag weights", ctx->D);
+    for (int d = 0; d < D; ++d)
+      if (!(c_d[d] >= 0)) return fail(ctx, GCADA_EINVAL, "lag weights must be non-negative");
+    ctx->c_d.assign(c_d, c_d + D);
+  }
+  ctx->ready = false;  // the device copy is made with the plans
+  drop_graphs(ctx);
+  return GCADA_OK;
+}
+
+gcada_status gcada_set_step_schedule(gcada_ctx* ctx, int kind, double a, double b) {
+  if (!ctx) return GCADA_EINVAL;
+  if (kind == GCADA_SCHEDULE_CONST) {
+    a = 1.0;
+    b = 0.0;
+  } else if (kind == GCADA_SCHEDULE_POLY) {
+    if (!(a > 0) || !(b >= 0)) return fail(ctx, GCADA_EINVAL, "polynomial decay needs a > 0 and b >= 0");
+  } else if (kind == GCADA_SCHEDULE_STEP) {
+    if (!(a >= 1) || a != (double)(long long)a || !(b > 0)) return fail(ctx, GCADA_EINVAL, "step decay needs an integer a >= 1 and b > 0");
+  } else {
+    return fail(ctx, GCADA_EINVAL, "unknown schedule %d", kind);
+  }
+  ctx->sched_kind = kind;
+  ctx->sched_a = a;
+  ctx->sched_b = b;
+  ctx->P.sched_kind = kind;
+  ctx->P.sched_a = a;
+  ctx->P.sched_b = b;
   drop_graphs(ctx);
   return GCADA_OK;
 }
@@ -887,6 +970,107 @@ gcada_status gcada_time_gradient(gcada_ctx* ctx, int reps, double* ms_per_rep) {
   cudaEventDestroy(e0);
   cudaEventDestroy(e1);
   *ms_per_rep = (double)ms / reps;
+  return GCADA_OK;
+}
+
+namespace {
+struct CkptHeader {
+  char magic[8];
+  long long kind, compute, n_dims, dims[MLP_MAX_LAYERS + 1], M, M_G, D, B, p, hist_cap, keep_stale, n_seg, total;
+};
+constexpr char CKPT_MAGIC[8] = {'G', 'C', 'A', 'D', 'A', 'C', 'K', '1'};
+
+gcada_status checkpoint_layout(gcada_ctx* ctx, CkptHeader* h, std::vector<std::pair<void*, size_t>>* segs) {
+  TRY(check_runnable(ctx, false));
+  TRY(make_plans(ctx));
+  *segs = ctx->state;
+  if (!is_linear(ctx)) segs->insert(segs->end(), ctx->mlp.state.begin(), ctx->mlp.state.end());
+  memset(h, 0, sizeof *h);
+  memcpy(h->magic, CKPT_MAGIC, 8);
+  h->kind = ctx->kind;
+  h->compute = ctx->compute;
+  h->n_dims = (long long)ctx->dims.size();
+  for (size_t i = 0; i < ctx->dims.size(); ++i) h->dims[i] = ctx->dims[i];
+  h->M = ctx->M;
+  h->M_G = ctx->M_G;
+  h->D = ctx->D;
+  h->B = ctx->B;
+  h->p = ctx->p;
+  h->hist_cap = ctx->hist_cap;
+  h->keep_stale = ctx->keep_stale;
+  h->n_seg = (long long)segs->size();
+  size_t total = sizeof(CkptHeader) + sizeof(unsigned long long) * segs->size();
+  for (auto& s : *segs) total += s.second;
+  h->total = (long long)total;
+  return GCADA_OK;
+}
+}  // namespace
+
+gcada_status gcada_checkpoint_size(gcada_ctx* ctx, unsigned long long* bytes) {
+  if (!ctx || !bytes) return GCADA_EINVAL;
+  DeviceGuard dg(ctx->device);
+  CkptHeader h;
+  std::vector<std::pair<void*, size_t>> segs;
+  TRY(checkpoint_layout(ctx, &h, &segs));
+  *bytes = (unsigned long long)h.total;
+  return GCADA_OK;
+}
+
+gcada_status gcada_checkpoint_save(gcada_ctx* ctx, void* host_buf, unsigned long long bytes) {
+  if (!ctx) return GCADA_EINVAL;
+  if (!host_buf) return fail(ctx, GCADA_EINVAL, "host_buf is NULL");
+  DeviceGuard dg(ctx->device);
+  CkptHeader h;
+  std::vector<std::pair<void*, size_t>> segs;
+  TRY(checkpoint_layout(ctx, &h, &segs));
+  if (bytes != (unsigned long long)h.total)
+    return fail(ctx, GCADA_EINVAL, "a checkpoint of this context has %lld bytes, the buffer has %llu", h.total, bytes);
+  DevState s;
+  TRY(read_state(ctx, &s));  // synchronises the stream and refuses to save after a device-side error
+  unsigned char* out = static_cast<unsigned char*>(host_buf);
+  memcpy(out, &h, sizeof h);
+  out += sizeof h;
+  for (auto& sg : segs) {
+    const unsigned long long n = sg.second;
+    memcpy(out, &n, sizeof n);
+    out += sizeof n;
+  }
+  for (auto& sg : segs) {
+    CK(cudaMemcpy(out, sg.first, sg.second, cudaMemcpyDeviceToHost));
+    out += sg.second;
+  }
+  return GCADA_OK;
+}
+
+gcada_status gcada_checkpoint_load(gcada_ctx* ctx, const void* host_buf, unsigned long long bytes) {
+  if (!ctx) return GCADA_EINVAL;
+  if (!host_buf) return fail(ctx, GCADA_EINVAL, "host_buf is NULL");
+  DeviceGuard dg(ctx->device);
+  CkptHeader h;
+  std::vector<std::pair<void*, size_t>> segs;
+  TRY(checkpoint_layout(ctx, &h, &segs));
+  if (bytes < sizeof(CkptHeader)) return fail(ctx, GCADA_EINVAL, "buffer too small for a checkpoint");
+  CkptHeader in;
+  memcpy(&in, host_buf, sizeof in);
+  if (memcmp(in.magic, CKPT_MAGIC, 8) != 0) return fail(ctx, GCADA_EINVAL, "not a checkpoint of this library");
+  if (memcmp(&in, &h, sizeof h) != 0 || bytes != (unsigned long long)h.total)
+    return fail(ctx, GCADA_EINVAL,
+                "the checkpoint was saved by a context with another model, grouping, D, batch size or options");
+  const unsigned char* src = static_cast<const unsigned char*>(host_buf) + sizeof h;
+  for (auto& sg : segs) {
+    unsigned long long n;
+    memcpy(&n, src, sizeof n);
+    src += sizeof n;
+    if (n != sg.second) return fail(ctx, GCADA_EINVAL, "checkpoint segment sizes do not match this context");
+  }
+  CK(cudaStreamSynchronize(ctx->stream));
+  for (auto& sg : segs) {
+    CK(cudaMemcpy(sg.first, src, sg.second, cudaMemcpyHostToDevice));
+    src += sg.second;
+  }
+  DevState s;
+  TRY(read_state(ctx, &s));
+  ctx->k_host = s.k;
   return GCADA_OK;
 }
 

@@ -52,7 +52,12 @@ struct Params {
   int identity_batch;   // 1: minibatch of group g = rows g*B .. of X (host-fed step)
   // constants
   double c;
+  const double* c_d;    // [D] per-lag constants of the right side of Eq. (9), or null: c_d = c as printed
   float alpha, beta1, beta2, omb1, omb2, eps;
+  double alpha_d;       // alpha in double, for the step-size schedule
+  int sched_kind;       // 0: alpha^k = alpha; 1: alpha / (1 + k/a)^b; 2: alpha * b^floor(k/a)
+  double sched_a, sched_b;
+  int delay_law;        // 0: shift - ln(1-u)/rate; 1: Pareto shift*(1-u)^(-1/rate); 2: uniform shift + u/rate
   float scale;          // 1/B (mean) or 1 (sum)
   uint32_t seed_lo, seed_hi;
   double shift, inv_rate;
@@ -161,7 +166,16 @@ __device__ __forceinline__ int build_group_list(const Params& P, int* list, int*
 __device__ __forceinline__ double worker_time(const Params& P, uint32_t k, int m) {
   const uint32_t w = philox_word((uint32_t)m, 0u, k, 1u, P.seed_lo, P.seed_hi);
   const double u = ((double)w + 0.5) * 2.3283064365386963e-10;  // 2^-32
+  if (P.delay_law == 1) return P.shift * exp(-log1p(-u) * P.inv_rate);
+  if (P.delay_law == 2) return P.shift + u * P.inv_rate;
   return P.shift - log1p(-u) * P.inv_rate;
+}
+
+// Step size alpha^k of Eq. (8c).
+__device__ __forceinline__ float step_size(const Params& P, long long k) {
+  if (P.sched_kind == 1) return (float)(P.alpha_d / pow(1.0 + (double)k / P.sched_a, P.sched_b));
+  if (P.sched_kind == 2) return (float)(P.alpha_d * pow(P.sched_b, (double)(k / (long long)P.sched_a)));
+  return P.alpha;
 }
 
 // ---------------------------------------------------------------------------

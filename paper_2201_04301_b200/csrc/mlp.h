@@ -2,6 +2,7 @@
 #pragma once
 #include <cuda_runtime.h>
 
+#include <utility>
 #include <vector>
 
 #include "common.cuh"
@@ -27,6 +28,7 @@ struct MlpPlan {
   float* act[MLP_MAX_LAYERS + 1] = {nullptr}; // act[l], 1 <= l < L: [2][G*B][dims[l]] after ReLU; act[L]: class scores
   float* dz[MLP_MAX_LAYERS + 1] = {nullptr};  // dz[l], 1 <= l <= L: [2][G*B][dims[l]] gradient w.r.t. z_l
   void* bf16_impl = nullptr;                  // opaque state of the bf16 tensor-core path
+  std::vector<std::pair<void*, size_t>> state;  // device buffers that carry state across iterations (checkpoints)
   int norm_parts = 0;                         // > 0: the gradient kernels themselves deliver this many partial sums
                                               // of ||fresh_g - stale_g||^2 per group in Params::lhs_part
 };

@@ -1120,6 +1120,15 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
   A_(im->db_fresh, (long long)G * im->nbias, float);
   A_(im->db_last, (long long)G * im->nbias, float);
 #undef A_
+  // what an iteration reads from earlier ones: the bf16 copies of the last D+1 iterates and every group's last upload
+  plan->state.clear();
+  plan->state.emplace_back(im->wb, sizeof(__nv_bfloat16) * (size_t)(D + 1) * im->slot_elems);
+  plan->state.emplace_back(im->bias, sizeof(float) * (size_t)(D + 1) * im->bias_slot);
+  for (int l = 1; l <= L; ++l) {
+    plan->state.emplace_back(im->lastA[l], sizeof(__nv_bfloat16) * (size_t)G * plan->dims[l] * im->Bp);
+    plan->state.emplace_back(im->lastB[l], sizeof(__nv_bfloat16) * (size_t)G * plan->dims[l - 1] * im->Bp);
+  }
+  plan->state.emplace_back(im->db_last, sizeof(float) * (size_t)G * im->nbias);
   if (!encode_fn()) {
     *why = "cuTensorMapEncodeTiled is not available from this driver";
     return cudaSuccess;

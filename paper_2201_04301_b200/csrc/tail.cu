@@ -125,8 +125,8 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
   // One thread per group, 256 groups at a time; everything a group needs is
   // fetched in one round of independent loads.
   double rhs = 0.0;
-  for (int i = 0; i < P.D; ++i) rhs += P.s_ring[i];
-  rhs *= P.c;
+  for (int d = 1; d <= P.D && k - d >= 0; ++d)  // ||theta^{k+1-d} - theta^{k-d}||^2 sits in slot (k-d) mod D
+    rhs += (P.c_d ? P.c_d[d - 1] : P.c) * P.s_ring[(k - d) % P.D];
   const uint32_t k32 = (uint32_t)k;
   const volatile double* parts = P.lhs_part;
   int nsel = 0;
@@ -245,6 +245,7 @@ __global__ void __launch_bounds__(256) update_kernel(const Params P) {
   const long long cols4 = P.p_pad >> 2;
   const long long k = P.st->k;
   const int ring = P.D + 1;
+  const float alpha_k = step_size(P, k);
 
   if (warp == 0) {
     int cnt = 0;
@@ -321,7 +322,7 @@ __global__ void __launch_bounds__(256) update_kernel(const Params P) {
     h.c = P.beta1 * h.c + P.omb1 * gr;                     \
     const float v = P.beta2 * vh.c + P.omb2 * (gr * gr);   \
     vh.c = fmaxf(vh.c, v);                                 \
-    const float up = P.alpha * h.c / sqrtf(P.eps + vh.c);  \
+    const float up = alpha_k * h.c / sqrtf(P.eps + vh.c);   \
     tn.c = th.c - up;                                      \
     local += (double)up * (double)up;                      \
   }
@@ -363,6 +364,7 @@ __global__ void __launch_bounds__(256) update_direct_kernel(const Params P) {
   const long long cols4 = P.p_pad >> 2;
   const long long k = P.st->k;
   const int ring = P.D + 1;
+  const float alpha_k = step_size(P, k);
   const long long i4 = (long long)blockIdx.x * 256 + tid;
   double local = 0.0;
   if (i4 < cols4) {
@@ -377,7 +379,7 @@ __global__ void __launch_bounds__(256) update_direct_kernel(const Params P) {
     h.c = P.beta1 * h.c + P.omb1 * gr;                     \
     const float v = P.beta2 * vh.c + P.omb2 * (gr * gr);   \
     vh.c = fmaxf(vh.c, v);                                 \
-    const float up = P.alpha * h.c / sqrtf(P.eps + vh.c);  \
+    const float up = alpha_k * h.c / sqrtf(P.eps + vh.c);   \
     tn.c = th.c - up;                                      \
     local += (double)up * (double)up;                      \
   }

@@ -80,17 +80,25 @@ def _kink_match(o, got, theta, Xb, yb, reduction, tol, kink_tol):
 
 
 def forced_parity(w, K, tol=TOL_FP32, stream=None, reduction="mean", check_stale=True, kink_tol=2e-6,
-                  margin=MARGIN, rhs_tol=1e-4, L=None):
+                  margin=MARGIN, rhs_tol=1e-4, L=None, c_d=None, schedule=None, delay_law=None):
     """Run the oracle free for K steps and the CUDA path teacher-forced with the
     oracle's masks; compare every step.  Returns the number of steps at which
     the CUDA path's own test outcome differed from the oracle's (only allowed
     within MARGIN)."""
-    o = make_oracle(w, reduction=reduction, **({"rule": "ps", "L": L} if L is not None else {}))
+    extra = {"rule": "ps", "L": L} if L is not None else {}
+    if c_d is not None:
+        extra["c_d"] = c_d
+    if schedule is not None:
+        extra["schedule"] = schedule
+    if delay_law is not None:
+        extra["delay_law"] = delay_law
+    o = make_oracle(w, reduction=reduction, **extra)
     wc = to_cuda(w)
     opts = {binding.OPT_KEEP_STALE: 1.0, binding.OPT_REDUCTION: 0.0 if reduction == "mean" else 1.0}
     if L is not None:
         opts[binding.OPT_RULE] = 1.0
-    g = binding.from_workload(wc, stream=stream, options=opts, smoothness=L)
+    g = binding.from_workload(wc, stream=stream, options=opts, smoothness=L, c_d=c_d, schedule=schedule,
+                              delay_law=delay_law)
     flips = 0
     worst = dict(fresh=0.0, stale=0.0, theta=0.0, lhs=0.0, kinks=0)
     is_mlp = w["kind"] == "mlp"

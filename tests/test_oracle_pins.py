@@ -308,6 +308,68 @@ def test_scalar_trajectory_by_hand():
     assert sum(int(m.sum()) for m in o.masks) < 60
 
 
+@pytest.mark.parametrize("schedule", [("poly", 5.0, 0.5), ("step", 4, 0.5)])
+def test_scalar_trajectory_by_hand_with_lag_weights_and_step_schedule(schedule):
+    """The same scalar recursion with the two generalisations the paper names:
+    per-lag constants c_d on the right side of Eq. (9) (Algorithm 1's input
+    list) and a step size alpha^k that depends on k (Eq. 2, Eq. 8c)."""
+    N = 20
+    X = np.ones((N, 1))
+    y = np.concatenate([np.ones(10), -np.ones(10)])
+    D, alpha, b1, b2, eps = 3, 0.1, 0.9, 0.99, 1e-8
+    c_d = [0.9, 0.3, 0.05]
+    o = GCadaOracle(Quadratic(1), 2, 1, D, 123.0, alpha, b1, b2, eps, X=X, y=y, batch=3,
+                    theta0=np.array([0.25]), seed=0, c_d=c_d, schedule=schedule)
+    th = [0.25]
+    h = vh = 0.0
+    tau = [D, D]
+    last = [0.0, 0.0]
+    off = [-1.0, 1.0]
+    for k in range(30):
+        rhs = sum(c_d[d - 1] * (th[k + 1 - d] - th[k - d]) ** 2 for d in range(1, D + 1) if k - d >= 0)
+        sel = []
+        for g in range(2):
+            old = th[max(k - tau[g], 0)]
+            sel.append(tau[g] >= D or ((th[k] + off[g]) - (old + off[g])) ** 2 > rhs)
+        for g in range(2):
+            if sel[g]:
+                last[g], tau[g] = th[k] + off[g], 1
+            else:
+                tau[g] += 1
+        agg = last[0] + last[1]
+        h = b1 * h + (1 - b1) * agg
+        vh = max(vh, b2 * vh + (1 - b2) * agg * agg)
+        a_k = alpha / math.sqrt(1 + k / 5.0) if schedule[0] == "poly" else alpha * 0.5 ** (k // 4)
+        th.append(th[k] - a_k * h / math.sqrt(eps + vh))
+        rec = o.step()
+        assert list(rec["mask"]) == [int(v) for v in sel]
+        assert rec["rhs"] == pytest.approx(rhs, rel=1e-12, abs=1e-300)
+        assert o.theta[0] == pytest.approx(th[-1], rel=1e-12)
+
+
+def test_equal_lag_weights_and_constant_schedule_are_the_printed_method():
+    a, b = _toy_oracle(c=0.7), _toy_oracle(c=0.7, c_d=[0.7] * 4, schedule=("poly", 1.0, 0.0))
+    for _ in range(25):
+        ra, rb = a.step(), b.step()
+        assert np.array_equal(ra["mask"], rb["mask"]) and np.array_equal(ra["theta"], rb["theta"])
+
+
+@pytest.mark.parametrize("law", ["pareto", "uniform"])
+def test_other_delay_laws(law):
+    from scipy import stats
+    o = _toy_oracle(M=8, M_G=2, shift=2.0, rate=3.0, delay_law=law)
+    T = []
+    for k in range(600):
+        o.k = k
+        T.append(o.delays())
+    T = np.concatenate(T)
+    if law == "pareto":     # P(T > t) = (shift / t)^rate
+        assert T.min() >= 2.0 and stats.kstest(T, "pareto", args=(3.0, 0, 2.0)).pvalue > 1e-3
+    else:                   # uniform on [shift, shift + 1/rate]
+        assert T.min() >= 2.0 and T.max() <= 2.0 + 1 / 3.0
+        assert stats.kstest(T, "uniform", args=(2.0, 1 / 3.0)).pvalue > 1e-3
+
+
 def test_c_zero_is_synchronous_distributed_adam():
     """c = 0: every group with a non-zero innovation violates Eq. (9) (and at
     k = 0 all are forced), so the run is the 'distributed Adam' of Section V:
