@@ -282,6 +282,12 @@ gcada_status gcada_innovation_norms_noalloc(const float *fresh_dev, const float 
  * state that an iteration reads.  Synchronises the stream before and after. */
 gcada_status gcada_time_gradient(gcada_ctx *ctx, int reps, double *ms_per_rep);
 
+/* Reporting aid (not a step of Algorithm 1): the mean per-sample loss of the current iterate over rows
+ * first_row .. first_row + n_rows - 1 of the resident training set, i.e. the objective of Eq. (1) restricted
+ * to those rows, in double precision, to *mean_loss (host).  Logistic and quadratic models only
+ * (GCADA_EINVAL for an MLP).  Synchronises the stream. */
+gcada_status gcada_eval_loss(gcada_ctx *ctx, long long first_row, long long n_rows, double *mean_loss);
+
 /*
  * Checkpoints (the paper has no counterpart).  A checkpoint is everything an iteration inherits from
  * earlier ones: iteration counter, counters and wall-clock, the last D+1 iterates, h, v-hat, the

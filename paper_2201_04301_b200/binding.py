@@ -64,6 +64,7 @@ SIGNATURES = {
     "gcada_get_kernel_times": (C.c_int, [_VP, C.POINTER(C.c_double), C.POINTER(C.c_int)]),
     "gcada_innovation_norms_noalloc": (C.c_int, [_VP, _VP, C.c_int, _LL, _LL, _VP, _VP, C.c_char_p, C.c_size_t]),
     "gcada_time_gradient": (C.c_int, [_VP, C.c_int, C.POINTER(C.c_double)]),
+    "gcada_eval_loss": (C.c_int, [_VP, _LL, _LL, C.POINTER(C.c_double)]),
     "gcada_checkpoint_size": (C.c_int, [_VP, _ULLP]),
     "gcada_checkpoint_save": (C.c_int, [_VP, _VP, C.c_ulonglong]),
     "gcada_checkpoint_load": (C.c_int, [_VP, _VP, C.c_ulonglong]),
@@ -239,6 +240,12 @@ class GCada:
         n = C.c_int()
         self._ck(self.lib.gcada_get_kernel_times(self.h, ms, C.byref(n)))
         return (ms[0], ms[1], ms[2]), n.value
+
+    def eval_loss(self, first_row, n_rows):
+        """Mean loss of the current iterate over a range of training rows (linear models)."""
+        v = C.c_double()
+        self._ck(self.lib.gcada_eval_loss(self.h, int(first_row), int(n_rows), C.byref(v)))
+        return v.value
 
     def checkpoint_save(self):
         """The run's state as a numpy byte array (see gcada_checkpoint_save)."""

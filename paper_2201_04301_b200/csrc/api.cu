@@ -64,6 +64,7 @@ struct gcada_ctx {
   void* stage_y = nullptr;
   long long stage_ld = 0;
   std::vector<std::pair<void*, size_t>> state;  // device buffers a checkpoint holds (besides the plan's)
+  double* eval_scratch = nullptr;
   float* row_scratch = nullptr;  // one p-vector for getters that rebuild a group's gradient on demand
   // graphs (free-running resident-data mode only)
   cudaGraphExec_t graph1 = nullptr, graphN = nullptr;
@@ -130,6 +131,7 @@ void free_all(gcada_ctx* ctx) {
   if (ctx->stage_y) cudaFree(ctx->stage_y);
   ctx->stage_x = ctx->stage_y = nullptr;
   ctx->row_scratch = nullptr;  // was in `owned`
+  ctx->eval_scratch = nullptr;
   ctx->state.clear();
   ctx->st = nullptr;
   ctx->ready = false;
@@ -970,6 +972,27 @@ gcada_status gcada_time_gradient(gcada_ctx* ctx, int reps, double* ms_per_rep) {
   cudaEventDestroy(e0);
   cudaEventDestroy(e1);
   *ms_per_rep = (double)ms / reps;
+  return GCADA_OK;
+}
+
+gcada_status gcada_eval_loss(gcada_ctx* ctx, long long first_row, long long n_rows, double* mean_loss) {
+  if (!ctx) return GCADA_EINVAL;
+  if (!mean_loss) return fail(ctx, GCADA_EINVAL, "mean_loss is NULL");
+  if (!is_linear(ctx)) return fail(ctx, GCADA_EINVAL, "gcada_eval_loss supports logistic and quadratic models only");
+  TRY(check_runnable(ctx, true));
+  if (first_row < 0 || n_rows < 1 || first_row + n_rows > ctx->N)
+    return fail(ctx, GCADA_EINVAL, "rows [%lld, %lld) are outside the training set of %lld rows", first_row,
+                first_row + n_rows, ctx->N);
+  DeviceGuard dg(ctx->device);
+  TRY(make_plans(ctx));
+  if (!ctx->eval_scratch) TRY(dev_alloc(ctx, &ctx->eval_scratch, (size_t)eval_loss_scratch_doubles()));
+  DevState s;
+  TRY(read_state(ctx, &s));
+  const float* theta = ctx->P.theta_ring + (s.k % (ctx->D + 1)) * ctx->p_pad;
+  CK(launch_eval_loss_linear(ctx->P, theta, ctx->kind == GCADA_MODEL_QUADRATIC, first_row, n_rows, ctx->eval_scratch,
+                             ctx->stream));
+  CK(cudaStreamSynchronize(ctx->stream));
+  CK(cudaMemcpy(mean_loss, ctx->eval_scratch, sizeof(double), cudaMemcpyDeviceToHost));
   return GCADA_OK;
 }
 

@@ -40,4 +40,10 @@ cudaError_t launch_ps_lhs(const Params& P, const TailPlan& plan, cudaStream_t st
 cudaError_t launch_select(const Params& P, const TailPlan& plan, cudaStream_t st, int what = 0);
 cudaError_t launch_update(const Params& P, const TailPlan& plan, cudaStream_t st);
 
+// Mean loss of a logistic / quadratic model over rows [first, first + n) of the resident training set at
+// `theta` (device, d floats); result in scratch[0].  `scratch` holds eval_loss_scratch_doubles() doubles.
+int eval_loss_scratch_doubles();
+cudaError_t launch_eval_loss_linear(const Params& P, const float* theta, bool quad, long long first, long long n,
+                                    double* scratch, cudaStream_t st);
+
 }  // namespace gcada
