@@ -304,6 +304,8 @@ def run_ours(args):
                            "frac_of_nominal_8TBs": achieved / 8000.0 if achieved else None}
     else:
         flops = mlp_flops_per_iteration(w)
+        if args.rule == "ps":     # only the selected groups compute, at theta^k only
+            flops = flops / 2 * sel_frac
         achieved = flops / (ms_grad * 1e-3) / 1e12 if ms_grad > 0 else None
         out["roofline"] = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_sustained"],
                            "unit": "TFLOP/s", "frac": achieved / peaks["bf16_sustained"] if achieved else None,

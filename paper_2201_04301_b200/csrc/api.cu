@@ -203,6 +203,8 @@ gcada_status make_ready(gcada_ctx* ctx, const float* theta0, int on_device) {
   TRY(dev_alloc(ctx, &P.t_g, (size_t)G));
   TRY(dev_alloc(ctx, &P.s_ring, (size_t)D));
   TRY(dev_alloc(ctx, &P.mask_cur, (size_t)G));
+  TRY(dev_alloc(ctx, &P.sel_list, (size_t)G));
+  TRY(dev_alloc(ctx, &P.sel_count, (size_t)1));
   TRY(dev_alloc(ctx, &P.hist, (size_t)ctx->hist_cap * G));
   plan_tail(pp, G, ctx->sm_count, &ctx->tail);
   TRY(dev_alloc(ctx, &P.lhs_part, (size_t)G * ctx->tail.select_blocks_x));
@@ -296,7 +298,9 @@ gcada_status make_plans(gcada_ctx* ctx) {
     TRY(dev_alloc(ctx, &l2, (size_t)ctx->G));
     CK(cudaMemcpyAsync(l2, ctx->L2.data(), sizeof(double) * ctx->G, cudaMemcpyHostToDevice, ctx->stream));
     P.ps_L2 = l2;
-    P.skip_unselected = (is_linear(ctx) && ctx->G <= SKIP_MAX_GROUPS) ? 1 : 0;
+    // the printed test needs no gradient: only the selected groups compute (Algorithm 1's own order).  The bf16
+    // MLP does so unless per-group gradients are kept for inspection; the fp32 MLP evaluates every group.
+    P.skip_unselected = ((is_linear(ctx) && ctx->G <= SKIP_MAX_GROUPS) || (factored(ctx) && !ctx->keep_stale)) ? 1 : 0;
     TRY(dev_alloc(ctx, &P.ps_lhs, (size_t)ctx->G));
     TRY(dev_alloc(ctx, &P.ps_part, (size_t)ctx->D * ctx->tail.ps_blocks));
   } else {
@@ -324,18 +328,24 @@ gcada_status enqueue_iteration(gcada_ctx* ctx, const Params& P) {
     CK(launch_ps_lhs(P, ctx->tail, ctx->stream));
     CK(launch_select(P, ctx->tail, ctx->stream, 1));
     if (ev) CK(cudaEventRecord(ev[1], ctx->stream));  // reported as "selection" below via the phase map
-    CK(launch_grad_linear(P, ctx->lin, ctx->kind == GCADA_MODEL_QUADRATIC, ctx->stream));
-    CK(launch_select(P, ctx->tail, ctx->stream, 2));
-    if (ev) {
-      CK(cudaEventRecord(ev[2], ctx->stream));
-      CK(cudaEventRecord(ev[3], ctx->stream));
+    if (is_linear(ctx)) {
+      CK(launch_grad_linear(P, ctx->lin, ctx->kind == GCADA_MODEL_QUADRATIC, ctx->stream));
+      CK(launch_select(P, ctx->tail, ctx->stream, 2));
+      if (ev) CK(cudaEventRecord(ev[2], ctx->stream));
+      ctx->launches += 5;
+    } else {
+      int n = 0, m = 0;
+      CK(launch_grad_mlp(P, ctx->mlp, ctx->stream, &n));
+      if (ev) CK(cudaEventRecord(ev[2], ctx->stream));
+      CK(launch_grad_mlp_post(P, ctx->mlp, ctx->stream, &m));
+      ctx->launches += (unsigned long long)(3 + n + m);
     }
+    if (ev) CK(cudaEventRecord(ev[3], ctx->stream));
     CK(launch_update(P, ctx->tail, ctx->stream));
     if (ev) {
       CK(cudaEventRecord(ev[4], ctx->stream));
       ctx->timed += 1;
     }
-    ctx->launches += 5;
     return GCADA_OK;
   }
   if (is_linear(ctx)) {
@@ -391,6 +401,7 @@ gcada_status capture(gcada_ctx* ctx, int iters, cudaGraphExec_t* out) {
 
 int kernels_per_iteration(const gcada_ctx* ctx) {
   if (is_linear(ctx)) return ctx->P.skip_unselected ? 5 : 3 + (ctx->rule == 1 ? 1 : 0);
+  if (ctx->P.skip_unselected) return 3 + ctx->mlp.skip_launches + ctx->mlp.post_launches;
   return 2 + ctx->mlp.launches_per_iter + ctx->mlp.post_launches + (ctx->rule == 1 ? 1 : 0);
 }
 
@@ -931,7 +942,7 @@ gcada_status gcada_get_kernel_times(gcada_ctx* ctx, double ms[3], int* n_timed) 
     cudaEvent_t* ev = &ctx->events[(size_t)i * 5];
     // normal order: gradient, selection, gradient (post-selection part), update;
     // skip mode (rule PS on linear models): selection first, then the selected groups' gradients
-    const int normal[4] = {0, 1, 0, 2}, skip_first[4] = {1, 0, 0, 2}, agg_after[4] = {0, 1, 2, 2};
+    const int normal[4] = {0, 1, 0, 2}, skip_first[4] = {1, 0, 2, 2}, agg_after[4] = {0, 1, 2, 2};
     const int* phase_of = ctx->P.skip_unselected ? skip_first : (ctx->P.agg_direct ? agg_after : normal);
     for (int j = 0; j < 4; ++j) {
       float t = 0.f;

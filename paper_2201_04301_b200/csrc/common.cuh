@@ -92,6 +92,8 @@ struct Params {
   const double* ps_L2;          // [G] squared smoothness constants, or null (rule INNOV)
   double* ps_lhs;               // [G] the printed left side, written by ps_lhs_kernel
   double* ps_part;              // [D][blocks] partial sums of ||theta^k - theta^{k-d}||^2
+  int* sel_list;                // [G] groups selected this iteration, ascending (written with the mask)
+  int* sel_count;               // [1] how many
   int skip_unselected;          // 1: the selection of this iteration is already in mask_cur and the gradient
                                 // kernels work on the selected groups only (rule PS: Algorithm 1 as printed,
                                 // workers of unselected groups compute nothing)

@@ -14,6 +14,7 @@ constexpr int MLP_MAX_LAYERS = 15;
 struct MlpPlan {
   int n_layers = 0;           // L
   int launches_per_iter = 0;
+  int skip_launches = 0;      // kernels before the update when only the selected groups compute (rule PS)
   int post_launches = 0;      // kernels that follow the selection kernel (bf16 path: upload + aggregate)
   int compute = 0;            // 0 fp32, 1 bf16 operands
   int G = 0, B = 0, D = 0;

@@ -218,7 +218,10 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nkb = a.k_batched ? a.kpg * a.n_batch : (a.K + BK - 1) / BK;
   const int tiles_n = (a.N + GN - 1) / GN, tiles_m = (a.M + BM - 1) / BM;
-  const int total_tiles = a.k_batched ? tiles_n * tiles_m : tiles_n * tiles_m * 2 * P.G;
+  // batch entries: (point, group) for every group, or - when only the selected groups compute (rule PS:
+  // Algorithm 1's own order, the selection is already known) - the selected groups at theta^k only
+  const int n_grp = P.skip_unselected ? P.sel_count[0] : P.G;
+  const int total_tiles = a.k_batched ? tiles_n * tiles_m : tiles_n * tiles_m * (P.skip_unselected ? 1 : 2) * n_grp;
   const long long k_it = P.st->k;
 
   if (threadIdx.x == 0) {
@@ -248,8 +251,10 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
       bool ok = true;
       int it = 0;
       for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-        const int nt = t % tiles_n, mt = (t / tiles_n) % tiles_m, z = t / (tiles_n * tiles_m);
-        const int q = z / P.G, g = z - q * P.G;
+        const int nt = t % tiles_n, mt = (t / tiles_n) % tiles_m, zi = t / (tiles_n * tiles_m);
+        const int q = a.k_batched ? 0 : zi / n_grp;
+        const int g = a.k_batched ? 0 : (P.skip_unselected ? P.sel_list[zi - q * n_grp] : zi - q * n_grp);
+        const int z = q * P.G + g;
         int zA = 0, zB = 0;
         if (!a.k_batched) {
           zA = a.a_shared ? g : z;
@@ -310,8 +315,10 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
     int i = 0;
     for (int t = blockIdx.x; t < total_tiles; t += gridDim.x, ++i) {
       const int slot = i & 1;
-      const int nt = t % tiles_n, mt = (t / tiles_n) % tiles_m, z = t / (tiles_n * tiles_m);
-      const int q = z / P.G, g = z - q * P.G;
+      const int nt = t % tiles_n, mt = (t / tiles_n) % tiles_m, zi = t / (tiles_n * tiles_m);
+      const int q = a.k_batched ? 0 : zi / n_grp;
+      const int g = a.k_batched ? 0 : (P.skip_unselected ? P.sel_list[zi - q * n_grp] : zi - q * n_grp);
+      const int z = q * P.G + g;
       if (ok) {
         ok = mbar_wait_bounded(&tfull_bar[slot], (uint32_t)((i >> 1) & 1));
         ok = __all_sync(0xffffffffu, ok);
@@ -756,6 +763,7 @@ __global__ void __launch_bounds__(256) bf16_gather_kernel(const Params P, __nv_b
   __shared__ long long rows_sm[32];
   const int g = blockIdx.y, rb = blockIdx.x * 32;
   const int tid = threadIdx.x;
+  if (P.skip_unselected && !P.mask_cur[g]) return;
   if (tid < 32) {
     const int j = rb + tid;
     long long row = -1;
@@ -815,6 +823,7 @@ __global__ void __launch_bounds__(256) bf16_softmax_grad_kernel(const Params P, 
   const int q = (int)(w0 / rows);
   const long long r0 = w0 - (long long)q * rows;
   const int g = (int)(r0 / Bp), m0 = (int)(r0 - (long long)g * Bp);
+  if (P.skip_unselected && (q != 0 || !P.mask_cur[g])) return;
   for (int i = 0; i < 4; ++i) {
     const int lr = warp * 4 + i;
     const long long w = w0 + lr;
@@ -873,6 +882,7 @@ __global__ void __launch_bounds__(256) bf16_bias_grad_kernel(const Params P, con
   if ((int)blockIdx.x * 64 >= n_l) return;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = blockIdx.y;
+  if (P.skip_unselected && !P.mask_cur[g]) return;  // (its stale-point sums below are then unused)
   const int n = blockIdx.x * 64 + 2 * lane;  // this lane's column pair (ld is even, so the pair is inside the row)
   const long long rows = (long long)P.G * Bp;
   float f0 = 0.f, f1 = 0.f, s0 = 0.f, s1 = 0.f;
@@ -1170,6 +1180,7 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
   if (e != cudaSuccess) return e;
   plan->launches_per_iter = 3 + L + 1 + L + (L - 1);
   plan->post_launches = L + 2;
+  plan->skip_launches = 2 + L + 1 + (L - 1) + 1;
   return cudaSuccess;
 }
 
@@ -1239,8 +1250,10 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
   ++n;
   const int dw_mode = P.stale ? DW_BOTH : DW_NORM;  // gradients of every group are materialised only on request
   for (int l = L; l >= 1; --l) {
-    if ((e = launch_dw(P, pl, im, l, dw_mode, st)) != cudaSuccess) return e;
-    ++n;
+    if (!P.skip_unselected) {  // the innovation norms; not needed when the printed test has already decided
+      if ((e = launch_dw(P, pl, im, l, dw_mode, st)) != cudaSuccess) return e;
+      ++n;
+    }
     if (l > 1) {
       GemmB d{};
       d.M = Bp;

@@ -31,6 +31,7 @@ template <int U>
 __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_x, int what) {
   __shared__ double scratch[40];
   __shared__ int sh_nsel[8];
+  __shared__ int sh_cnt[8];
   __shared__ double sh_tmax[8];
   __shared__ double tw_sm[1024];
   __shared__ double lhs_sm[256];
@@ -130,6 +131,7 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
   const uint32_t k32 = (uint32_t)k;
   const volatile double* parts = P.lhs_part;
   int nsel = 0;
+  int listed = 0;  // selected groups of earlier chunks (the same in every thread)
   double tmax = 0.0;
   for (int gc = 0; gc < P.G; gc += 256) {
     const int gg = gc + tid;
@@ -168,9 +170,10 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
         for (long long m = lo; m < hi; ++m) t = fmin(t, tw_sm[m - m0]);
       }
     }
+    bool sel = false;
     if (have) {
       if (P.ps_L2) lhs = P.ps_lhs[gg];  // rule PS: the test uses the printed left side, not the measured innovation
-      const bool sel = P.forced ? sel_forced : ((tau >= P.D) || (lhs > rhs));
+      sel = P.forced ? sel_forced : ((tau >= P.D) || (lhs > rhs));
       P.lhs[gg] = lhs;
       P.t_g[gg] = t;
       P.mask_cur[gg] = sel ? 1 : 0;
@@ -182,7 +185,22 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
         tmax = fmax(tmax, t);
       }
     }
+    // ascending list of the selected groups (for kernels that work on the selected groups only)
+    {
+      const unsigned int b = __ballot_sync(0xffffffffu, sel);
+      __syncthreads();
+      if (lane == 0) sh_cnt[warp] = __popc(b);
+      __syncthreads();
+      int base = listed, all = 0;
+      for (int w = 0; w < 8; ++w) {
+        if (w < warp) base += sh_cnt[w];
+        all += sh_cnt[w];
+      }
+      if (sel) P.sel_list[base + __popc(b & ((1u << lane) - 1u))] = gg;
+      listed += all;
+    }
   }
+  if (tid == 0) P.sel_count[0] = listed;
   // block-wide count and maximum
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
