@@ -178,10 +178,9 @@ gcada_status gcada_set_option(gcada_ctx *ctx, int key, double value);
  * printed test needs no gradient, so for logistic / quadratic models (up to 1024 groups) an iteration runs in
  * Algorithm 1's order: test, selection, then gradients at theta^k for the selected groups only (the cost of
  * an iteration scales with the number of uploads; GCADA_DBG_FRESH / _STALE / _LHS-by-innovation of
- * unselected groups are then not produced).  The bf16 MLP runs in the same order (forward and backward pass
+ * unselected groups are then not produced).  The MLPs run in the same order (forward and backward pass
  * of the selected groups at theta^k only; no stale-point pass, no innovation norms) unless
- * GCADA_OPT_KEEP_STALE is set.  For the fp32 MLP the rule decides the selection, but both gradients of every
- * group are still evaluated. */
+ * GCADA_OPT_KEEP_STALE is set, in which case both gradients of every group are still evaluated. */
 gcada_status gcada_set_smoothness(gcada_ctx *ctx, const double *L, int G);
 
 /* Run n_iters iterations of Algorithm 1 on the stream (asynchronous).

@@ -298,9 +298,9 @@ gcada_status make_plans(gcada_ctx* ctx) {
     TRY(dev_alloc(ctx, &l2, (size_t)ctx->G));
     CK(cudaMemcpyAsync(l2, ctx->L2.data(), sizeof(double) * ctx->G, cudaMemcpyHostToDevice, ctx->stream));
     P.ps_L2 = l2;
-    // the printed test needs no gradient: only the selected groups compute (Algorithm 1's own order).  The bf16
-    // MLP does so unless per-group gradients are kept for inspection; the fp32 MLP evaluates every group.
-    P.skip_unselected = ((is_linear(ctx) && ctx->G <= SKIP_MAX_GROUPS) || (factored(ctx) && !ctx->keep_stale)) ? 1 : 0;
+    // the printed test needs no gradient: only the selected groups compute (Algorithm 1's own order).  The
+    // MLPs do so unless per-group gradients are kept for inspection.
+    P.skip_unselected = ((is_linear(ctx) && ctx->G <= SKIP_MAX_GROUPS) || (!is_linear(ctx) && !ctx->keep_stale)) ? 1 : 0;
     TRY(dev_alloc(ctx, &P.ps_lhs, (size_t)ctx->G));
     TRY(dev_alloc(ctx, &P.ps_part, (size_t)ctx->D * ctx->tail.ps_blocks));
   } else {

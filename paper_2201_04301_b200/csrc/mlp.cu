@@ -30,6 +30,7 @@ __global__ void __launch_bounds__(256) mlp_gather_kernel(const Params P, float* 
   const long long rows = (long long)P.G * P.B;
   if (warp >= rows) return;
   const int g = warp / P.B, j = warp - g * P.B;
+  if (P.skip_unselected && !P.mask_cur[g]) return;  // rule PS: only the selected groups compute
   const long long row = batch_row(P, (uint32_t)P.st->k, g, j);
   const float* src = reinterpret_cast<const float*>(P.X) + row * P.ld;
   float* dst = xb + (long long)warp * d;
@@ -82,6 +83,8 @@ __global__ void __launch_bounds__(256) mlp_sgemm_kernel(const Params P, const Ge
   __shared__ float Bs[TK][TN + 4];
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   const int z = blockIdx.z, q = z / P.G, g = z - q * P.G;
+  // rule PS (the selection is already known): selected groups at theta^k only
+  if (P.skip_unselected && (q != 0 || !P.mask_cur[g])) return;
   const int m0 = blockIdx.y * TM, n0 = blockIdx.x * TN;
   const long long k_it = P.st->k;
   const float* Ab = a.A.ring ? ring_ptr(P, g, q, k_it) + a.A.off : a.A.base + g * a.A.zg + q * a.A.zq;
@@ -134,8 +137,8 @@ __global__ void __launch_bounds__(256) mlp_sgemm_kernel(const Params P, const Ge
   }
 
   float* Cb;
-  if (a.c_grad)
-    Cb = (q == 0 ? fresh_row(P, g) : P.stale + (long long)g * P.p_pad) + a.c_off;
+  if (a.c_grad)  // (after the selection the flip of cur[g] has made the target row the last uploaded one)
+    Cb = (q == 0 ? (P.skip_unselected ? last_row(P, g) : fresh_row(P, g)) : P.stale + (long long)g * P.p_pad) + a.c_off;
   else
     Cb = a.C + g * a.c_zg + q * a.c_zq;
   const float* Mb = a.mask ? a.mask + g * a.c_zg + q * a.c_zq : nullptr;
@@ -167,6 +170,7 @@ __global__ void __launch_bounds__(256) mlp_softmax_grad_kernel(const Params P, c
   const int lane = threadIdx.x & 31;
   if (w >= 2 * rows) return;
   const long long r = w % rows;
+  if (P.skip_unselected && (w >= rows || !P.mask_cur[r / P.B])) return;
   const float* s = scores + w * n_cls;
   float* o = dz + w * n_cls;
   float mx = -3.0e38f;
@@ -199,10 +203,11 @@ __global__ void __launch_bounds__(256) mlp_bias_grad_kernel(const Params P, cons
   const int n = blockIdx.x * 256 + threadIdx.x;
   if (n >= a.n[l]) return;
   const int z = blockIdx.y, q = z / P.G, g = z - q * P.G;
+  if (P.skip_unselected && (q != 0 || !P.mask_cur[g])) return;
   const float* src = a.dz[l] + ((long long)z * P.B) * a.n[l] + n;
   float s = 0.f;
   for (int r = 0; r < P.B; ++r) s += src[(long long)r * a.n[l]];
-  ((q == 0 ? fresh_row(P, g) : P.stale + (long long)g * P.p_pad) + a.b_off[l])[n] = s;
+  ((q == 0 ? (P.skip_unselected ? last_row(P, g) : fresh_row(P, g)) : P.stale + (long long)g * P.p_pad) + a.b_off[l])[n] = s;
 }
 
 cudaError_t launch_gemm(const Params& P, const GemmArgs& a, cudaStream_t st) {
@@ -255,6 +260,7 @@ cudaError_t mlp_plan_create(const std::vector<int>& dims, int compute, int G, in
     if ((e = alloc(reinterpret_cast<void**>(&plan->dz[l]), sizeof(float) * 2 * rows * dims[l])) != cudaSuccess) return e;
   }
   plan->launches_per_iter = 3 * L + 2;
+  plan->skip_launches = 3 * L + 2;  // the same kernels; blocks of unselected groups and of the stale point exit at once
   return cudaSuccess;
 }
 

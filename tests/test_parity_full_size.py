@@ -81,3 +81,32 @@ def test_cfg5_full_size_sampled_groups():
     up, comm, comp = g.get_comm_count()
     assert up == int(masks.sum()) and comm == 5 * up and comp == 4 * up
     assert np.isfinite(g.get_theta()).all()
+
+
+@pytest.mark.parametrize("name,tol", [("cfg1", TOL_FP32), ("cfg2", TOL_FP32), ("cfg4", TOL_FP32)])
+def test_small_workloads_at_full_size(name, tol):
+    """The latency-bound workloads at their full sizes, free-running under graph replay: every group's
+    fresh gradient at sampled iterations against the oracle's gradient at the CUDA path's own iterate on
+    the rows it must have drawn; counters and Eq. (3) throughout."""
+    w = make_workload(name, device="cuda")
+    G = w["M"] // w["M_G"]
+    g = binding.from_workload(w, stream=torch.cuda.Stream())
+    model = make_model(w["kind"], w["dims"])
+    K = 40
+    for k in range(K):
+        theta = g.get_theta().astype(np.float64)
+        g.step(1)
+        if k in (0, 11, 39):
+            for gi in range(G):
+                Xb, yb = _group_batch(w, k, gi, G)
+                want = model.grad(theta, Xb, yb, "mean")
+                got = g.get_group_gradient(binding.DBG_FRESH, gi)
+                kinks = w["kind"] == "mlp" and model.near_kinks(theta, Xb, 2e-6)
+                assert rel_l2(got, want) <= (tol if not kinks else 1e-3), (k, gi)
+    masks = g.get_selection_mask(0, K)
+    up, comm, comp = g.get_comm_count()
+    assert masks[0].all() and up == int(masks.sum()) and comm == (w["M_G"] + 1) * up and comp == w["M_G"] * up
+    agg = g.get_debug(binding.DBG_AGG).astype(np.float64)
+    assert rel_l2(agg, g.get_debug(binding.DBG_GLAST).astype(np.float64).sum(axis=0)) <= 1e-6
+    g.step(w["K"] - K)                # the rest of the workload's run, 16 iterations per replayed graph
+    assert g.get_iteration() == w["K"] and np.isfinite(g.get_theta()).all()

@@ -43,3 +43,36 @@ def test_cfg4_free_running_counts_and_determinism():
     up, comm, comp = outs[0][2]
     assert up == int(outs[0][1].sum()) and comm == 3 * up and comp == 2 * up
     assert outs[0][1][0].all() and up < 50 * 5
+
+
+def test_printed_rule_computes_only_the_selected_groups():
+    """Rule PS on the fp32 MLP: selection first, then only the selected groups run, at theta^k only.  The
+    free-running masks equal the oracle's, the uploaded gradients equal the oracle's gradient at the CUDA
+    path's own iterate, and the aggregate is the sum of the last uploads (Eq. 3)."""
+    import numpy as np
+    import torch
+    from paper_2201_04301_b200 import binding
+    from parity import make_oracle, rel_l2, to_cuda
+    w = make_workload("cfg4", rows=5 * 400, D=5, c=1.0)
+    G = 5
+    L = [2.0, 0.1, 0.7, 0.02, 1.3]      # none with L_g^2 = c: at k = 1 the test is L_g^2 > c exactly
+    o = make_oracle(w, rule="ps", L=L)
+    g = binding.from_workload(to_cuda(w), stream=torch.cuda.Stream(), options={binding.OPT_RULE: 1.0}, smoothness=L)
+    K = 20
+    for k in range(K):
+        theta_gpu = g.get_theta().astype(np.float64)
+        batches = [o.minibatch(gi) for gi in range(G)]
+        rec = o.step()
+        g.step(1)
+        mask = g.get_selection_mask(k, 1)[0]
+        assert np.array_equal(mask, rec["mask"]), (k, mask, rec["mask"])
+        assert np.allclose(g.get_debug(binding.DBG_LHS), rec["lhs"], rtol=1e-4, atol=1e-30)
+        last = g.get_debug(binding.DBG_GLAST)
+        for gi in np.nonzero(mask)[0]:
+            want = o.model.grad(theta_gpu, batches[gi][1], batches[gi][2], "mean")
+            assert rel_l2(last[gi], want) <= 5e-5, (k, gi)      # an occasional ReLU unit on its kink
+        assert rel_l2(g.get_debug(binding.DBG_AGG), last.astype(np.float64).sum(axis=0)) <= 1e-6
+        assert rel_l2(g.get_theta(), rec["theta"]) <= 1e-4
+    masks = g.get_selection_mask(0, K)
+    assert masks[0].all() and 0 < masks.sum() < masks.size
+    assert g.get_comm_count() == (o.uploads, o.comm, o.comp)

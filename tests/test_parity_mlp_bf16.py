@@ -107,7 +107,7 @@ def test_printed_rule_computes_only_the_selected_groups():
     from parity import make_oracle
     w = make_workload("cfg5", rows=6 * 800, dims=(64, 128, 96, 40), M=12, M_G=2, D=5, batch=128, c=1.0, alpha=1e-3)
     G = 6
-    L = [3.0, 0.2, 1.0, 0.05, 2.0, 0.5]
+    L = [3.0, 0.2, 1.4, 0.05, 2.0, 0.5]   # none with L_g^2 = c: at k = 1 the test is L_g^2 > c exactly
     o = make_oracle(w, rule="ps", L=L)
     g = binding.from_workload(to_cuda(w), stream=torch.cuda.Stream(), options={binding.OPT_RULE: 1.0}, smoothness=L)
     K = 24
