@@ -189,7 +189,9 @@ gcada_status gcada_step(gcada_ctx *ctx, int n_iters);
 
 /* As gcada_step, but the selected set of iteration i is mask[i*G + g] != 0
  * (host, n_iters*G bytes, copied before return) instead of the test's
- * outcome.  LHS, RHS and every other quantity are still computed. */
+ * outcome.  LHS, RHS and every other quantity are still computed.  The
+ * method's own rule never lets an age exceed D; if a forced mask does, the
+ * group's stale iterate is theta^{k-D}, the oldest one kept. */
 gcada_status gcada_step_forced(gcada_ctx *ctx, int n_iters, const unsigned char *mask);
 
 /*

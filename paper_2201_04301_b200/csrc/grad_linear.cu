@@ -217,6 +217,7 @@ __global__ void __launch_bounds__(THREADS, MINB) grad_linear_large_kernel(const 
         cur_g = cur_g < 0 ? g_first : cur_g + 1;
         g_end = (cur_g + 1 - g_first) * B - in_g0;
         long long js = k - P.tau[skip ? sel_sm[cur_g] : cur_g];
+        if (js < k - P.D) js = k - P.D;  // ages beyond D only arise under forced masks: oldest kept iterate
         if (js < 0) js = 0;
         const float* theta_s = P.theta_ring + (js % ring) * P.p_pad;
 #pragma unroll
@@ -405,6 +406,7 @@ __global__ void __launch_bounds__(256) grad_linear_small_kernel(const Params P) 
     const long long seg1 = (long long)(g + 1) * P.B < r1 ? (long long)(g + 1) * P.B : r1;
     const int g_real = skip ? sel_sm[g] : g;
     long long js = k - P.tau[g_real];
+    if (js < k - P.D) js = k - P.D;  // ages beyond D only arise under forced masks: oldest kept iterate
     if (js < 0) js = 0;
     const float* theta_s = P.theta_ring + (js % ring) * P.p_pad;
 #pragma unroll

@@ -19,6 +19,7 @@ namespace {
 
 __device__ __forceinline__ const float* ring_ptr(const Params& P, int g, int q, long long k) {
   long long j = q == 0 ? k : k - P.tau[g];
+  if (j < k - P.D) j = k - P.D;  // ages beyond D only arise under forced masks: oldest kept iterate
   if (j < 0) j = 0;
   return P.theta_ring + (j % (P.D + 1)) * P.p_pad;
 }

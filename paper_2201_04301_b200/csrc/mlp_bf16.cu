@@ -187,6 +187,7 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr) {
 
 __device__ __forceinline__ int ring_slot(const Params& P, int g, int q, long long k) {
   long long j = q == 0 ? k : k - P.tau[g];
+  if (j < k - P.D) j = k - P.D;  // ages beyond D only arise under forced masks: oldest kept iterate
   if (j < 0) j = 0;
   return (int)(j % (P.D + 1));
 }

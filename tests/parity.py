@@ -106,7 +106,7 @@ def forced_parity(w, K, tol=TOL_FP32, stream=None, reduction="mean", check_stale
         tau_before = g.get_debug(binding.DBG_TAU)
         batches = [o.minibatch(gi) for gi in range(o.G)] if is_mlp else None
         th_now = o.thetas[o.k]
-        th_old = [o.theta_at(o.k - int(o.tau[gi])) for gi in range(o.G)]
+        th_old = [o.theta_at(o.k - min(int(o.tau[gi]), o.D)) for gi in range(o.G)]
         rec = o.step()
         g.step_forced(rec["mask"][None, :])
         fresh, stale = g.get_debug(binding.DBG_FRESH), g.get_debug(binding.DBG_STALE)

@@ -100,3 +100,28 @@ def test_special_cases_distributed_adam_and_cada():
     h.step(100)
     up, comm, comp = h.get_comm_count()
     assert comm == 2 * up and comp == up and 0 < up < 500               # Eqs. (18), (21) with equality
+
+
+def test_forced_masks_that_starve_a_group_beyond_the_maximum_delay():
+    """The rule itself never lets an age exceed D.  A forced mask can: the stale iterate is then the oldest
+    one kept, theta^{k-D}, in the oracle and in every CUDA path (linear, wide linear, both MLPs)."""
+    import numpy as np
+    from parity import TOL_BF16, TOL_FP32, make_oracle, rel_l2
+    cases = [(make_workload("cfg1", rows=3000, D=3), TOL_FP32),
+             (make_workload("cfg3", rows=3 * 300, M=6, M_G=2, D=3, batch=40), TOL_FP32),
+             (make_workload("cfg4", rows=3 * 300, dims=(30, 16, 5), M=6, M_G=2, D=3, batch=24), 1e-4),
+             (make_workload("cfg5", rows=3 * 300, dims=(64, 72, 10), M=6, M_G=2, D=3, batch=128), TOL_BF16)]
+    for w, tol in cases:
+        o = make_oracle(w)
+        g = binding.from_workload(to_cuda(w), stream=_stream(), options={binding.OPT_KEEP_STALE: 1.0})
+        masks = np.ones((12, 3), dtype=np.uint8)
+        masks[1:10, 1] = 0                       # group 1 is not selected for nine iterations, D = 3
+        for k in range(12):
+            rec = o.step(forced_mask=masks[k])
+            g.step_forced(masks[k][None, :])
+            assert np.array_equal(g.get_debug(binding.DBG_TAU), o.tau)
+            stale = g.get_debug(binding.DBG_STALE)
+            assert rel_l2(stale[1], rec["stale"][1]) <= tol, (w["name"], k)
+            assert abs(g.get_debug(binding.DBG_LHS)[1] - rec["lhs"][1]) <= 2 * tol * max(rec["lhs"][1], 1e-30) + 1e-30
+        assert rel_l2(g.get_theta(), o.theta) <= tol
+        g.close()
