@@ -286,6 +286,16 @@ def run_ours(args):
                            "frac": achieved / peak if achieved else None, "traffic": None,
                            "kernel": "gradient (all launches of one iteration; latency-bound at this size)",
                            "peak_source": "derived: SMs x 128 lanes x 2 x max SM clock", "flops_per_iteration": flops}
+    elif launches == 1:
+        # narrow model: the whole timed region was ONE launch of the cluster kernel (all iterations inside it)
+        bytes_launch = algorithmic_bytes_per_launch(w) * args.steps
+        achieved = bytes_launch / (ms * 1e-3) / 1e9
+        out["roofline"] = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm"], "unit": "GB/s",
+                           "frac": achieved / peaks["hbm"], "traffic": None,
+                           "kernel": "linear_cluster_kernel (one launch = all %d iterations; latency-bound workload: "
+                                     "%.0f KB per iteration)" % (args.steps, algorithmic_bytes_per_launch(w) / 1e3),
+                           "peak_source": peaks["source"], "duration_ms": ms,
+                           "algorithmic_bytes_per_launch": bytes_launch}
     elif w["kind"] != "mlp":
         bytes_launch = algorithmic_bytes_per_launch(w)
         achieved = bytes_launch / (ms_grad_b2b * 1e-3) / 1e9 if ms_grad_b2b > 0 else None

@@ -83,6 +83,13 @@ typedef struct {
                                       SM with 4-row batches, 2 = two CTAs per SM with 2-row batches; results
                                       differ only in summation order */
 
+#define GCADA_OPT_PERSISTENT 7     /* 1 (default) = logistic / quadratic models with d <= 256, at most 64 groups and
+                                      1024 workers run free-running steps of the default rule as ONE launch of a
+                                      single thread-block cluster per gcada_step call, whatever n_iters is (the
+                                      whole iteration stays on chip; one cluster barrier per iteration);
+                                      0 = always the chain of kernels.  Both give the same results up to summation
+                                      order; forced, host-fed, timed and rule-PS steps always use the chain */
+
 /* Items for gcada_get_debug.  Sizes are in elements of the stated type. */
 #define GCADA_DBG_FRESH 0   /* float [G][p]: gradient of each group at theta^k, last iteration run */
 #define GCADA_DBG_STALE 1   /* float [G][p]: gradient at the stale iterate (needs GCADA_OPT_KEEP_STALE) */

@@ -15,7 +15,8 @@ LIB_PATH = os.path.join(HERE, "libgcada.so")
 OK, EINVAL, ENOMEM, ECUDA, ESTATE, ETIMEOUT = range(6)
 MODEL_LOGISTIC, MODEL_MLP, MODEL_QUADRATIC = 0, 1, 2
 COMPUTE_FP32, COMPUTE_BF16 = 0, 1
-OPT_RULE, OPT_REDUCTION, OPT_HISTORY, OPT_KEEP_STALE, OPT_GRAPH, OPT_TIMING, OPT_LINEAR_VARIANT = range(7)
+(OPT_RULE, OPT_REDUCTION, OPT_HISTORY, OPT_KEEP_STALE, OPT_GRAPH, OPT_TIMING, OPT_LINEAR_VARIANT,
+ OPT_PERSISTENT) = range(8)
 (DBG_FRESH, DBG_STALE, DBG_LHS, DBG_RHS, DBG_TAU, DBG_AGG, DBG_H, DBG_VHAT, DBG_TGROUP, DBG_GLAST,
  DBG_SRING) = range(11)
 MODEL_KINDS = {"logistic": MODEL_LOGISTIC, "mlp": MODEL_MLP, "quadratic": MODEL_QUADRATIC}

@@ -12,7 +12,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libgcada.so")
-SOURCES = ["api.cu", "grad_linear.cu", "tail.cu", "mlp.cu", "mlp_bf16.cu", "noalloc.cu", "eval.cu"]
+SOURCES = ["api.cu", "grad_linear.cu", "tail.cu", "mlp.cu", "mlp_bf16.cu", "noalloc.cu", "eval.cu", "linear_cluster.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC,-Wall,-Wno-unused-function", "--expt-relaxed-constexpr"]
 

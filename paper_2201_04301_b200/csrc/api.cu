@@ -36,7 +36,8 @@ struct gcada_ctx {
   double c = 0, alpha = 0, beta1 = 0, beta2 = 0, eps = 0;
   unsigned long long seed = 0;
   double shift = 1.0, rate = 1.0;
-  int rule = 0, reduction = 0, keep_stale = 0, use_graph = 1, linear_variant = 0;
+  int rule = 0, reduction = 0, keep_stale = 0, use_graph = 1, linear_variant = 0, persistent = 1;
+  ClusterPlan cluster{};
   long long hist_cap = 65536;
   // data
   const void* X = nullptr;
@@ -272,6 +273,10 @@ gcada_status make_plans(gcada_ctx* ctx) {
                      &ctx->lin, &why))
       return fail(ctx, GCADA_EINVAL, "%s", why);
     CK(prepare_grad_linear(ctx->lin, ctx->kind == GCADA_MODEL_QUADRATIC));
+    // narrow models with few groups: whole iterations inside one thread-block cluster
+    ctx->cluster.usable = false;
+    if (ctx->persistent && ctx->have_data && ctx->rule == 0 && !ctx->keep_stale)
+      plan_linear_cluster(ctx->dims[0], ctx->G, ctx->M, ctx->D, ctx->B, ctx->p_pad, ctx->smem_optin, &ctx->cluster);
     P.pm.n_cta = ctx->lin.n_cta;
     P.pm.maxseg = ctx->lin.maxseg;
     P.pm.rows_per_group = ctx->B;
@@ -670,6 +675,9 @@ gcada_status gcada_set_option(gcada_ctx* ctx, int key, double value) {
     case GCADA_OPT_KEEP_STALE:
       ctx->keep_stale = value != 0;
       break;
+    case GCADA_OPT_PERSISTENT:
+      ctx->persistent = value != 0;
+      break;
     case GCADA_OPT_GRAPH:
       ctx->use_graph = value != 0;
       drop_graphs(ctx);
@@ -726,6 +734,16 @@ static gcada_status run_iterations(gcada_ctx* ctx, int n_iters, const unsigned c
     return GCADA_OK;
   }
   int left = n_iters;
+  if (is_linear(ctx) && ctx->cluster.usable && !ctx->timing) {
+    cudaError_t e = launch_linear_cluster(ctx->P, ctx->cluster, ctx->kind == GCADA_MODEL_QUADRATIC, n_iters, ctx->stream);
+    if (e == cudaSuccess) {
+      ctx->launches += 1;
+      ctx->k_host += n_iters;
+      return GCADA_OK;
+    }
+    cudaGetLastError();            // this device does not take the cluster launch: the kernel chain does the work
+    ctx->cluster.usable = false;
+  }
   if (ctx->use_graph && ctx->stream != nullptr && !ctx->timing) {
     if (!ctx->graph1) TRY(capture(ctx, 1, &ctx->graph1));
     if (!ctx->graphN && n_iters >= GRAPH_CHAIN) TRY(capture(ctx, GRAPH_CHAIN, &ctx->graphN));

@@ -40,6 +40,16 @@ cudaError_t launch_ps_lhs(const Params& P, const TailPlan& plan, cudaStream_t st
 cudaError_t launch_select(const Params& P, const TailPlan& plan, cudaStream_t st, int what = 0);
 cudaError_t launch_update(const Params& P, const TailPlan& plan, cudaStream_t st);
 
+// Narrow linear models, free-running default rule: any number of iterations in one launch of a single
+// thread-block cluster (see linear_cluster.cu).
+struct ClusterPlan {
+  bool usable = false;
+  int cpl = 1, rr = 8, n_cta = 1;
+  size_t smem_bytes = 0;
+};
+bool plan_linear_cluster(int d, int G, int M, int D, int B, long long p_pad, size_t smem_optin, ClusterPlan* plan);
+cudaError_t launch_linear_cluster(const Params& P, const ClusterPlan& plan, bool quad, int n_iters, cudaStream_t st);
+
 // Mean loss of a logistic / quadratic model over rows [first, first + n) of the resident training set at
 // `theta` (device, d floats); result in scratch[0].  `scratch` holds eval_loss_scratch_doubles() doubles.
 int eval_loss_scratch_doubles();
