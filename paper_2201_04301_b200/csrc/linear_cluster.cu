@@ -62,9 +62,42 @@ __device__ __forceinline__ void fold2(float& hi, float& lo, float f, float l) {
   lo += e1 + e2;
 }
 
+// Sums V values over the 32 lanes with V-1 + log2(32/V) shuffles instead of 5 V: at each of the first
+// log2(V) steps a lane keeps half of its values and hands the other half to its partner.  On return
+// v[0] of lane l is the total of value number (l * V) / 32 (so 32 / V consecutive lanes hold the same one).
+template <int V>
+__device__ __forceinline__ void reduce_spread(float (&v)[V], int lane) {
+  static_assert(V == 8 || V == 4, "8 or 4 values");
+  const unsigned int full = 0xffffffffu;
+  if (V == 8) {
+    const bool up = lane & 16;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float send = up ? v[i] : v[i + 4], keep = up ? v[i + 4] : v[i];
+      v[i] = keep + __shfl_xor_sync(full, send, 16);
+    }
+  }
+  constexpr int W1 = V == 8 ? 8 : 16;  // lane bit of the step that halves four values to two
+  {
+    const bool up = lane & W1;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const float send = up ? v[i] : v[i + 2], keep = up ? v[i + 2] : v[i];
+      v[i] = keep + __shfl_xor_sync(full, send, W1);
+    }
+  }
+  {
+    const bool up = lane & (W1 >> 1);
+    const float send = up ? v[0] : v[1], keep = up ? v[1] : v[0];
+    v[0] = keep + __shfl_xor_sync(full, send, W1 >> 1);
+  }
+#pragma unroll
+  for (int w = W1 >> 2; w >= 1; w >>= 1) v[0] += __shfl_xor_sync(full, v[0], w);
+}
+
 struct Carve {
   float *ring, *h, *vhat, *agg_hi, *agg_lo, *glast, *fresh, *innov, *part, *accw;
-  double *s_ring, *lhs, *tg, *tw, *red;
+  double *s_ring, *lhs, *tg, *tw, *red, *lhsp;
   int* tau;
   unsigned char* mask;
 };
@@ -82,7 +115,8 @@ __host__ __device__ inline size_t carve(unsigned char* base, int G, int M, int D
                o_ah = take(4 * (size_t)pp), o_al = take(4 * (size_t)pp), o_gl = take(4 * gp), o_fr = take(4 * gp),
                o_in = take(4 * gp), o_pa = take(4 * 2 * 2 * gp), o_aw = take(4 * (size_t)LC_WARPS * 2 * gp),
                o_sr = take(8 * (size_t)D), o_lhs = take(8 * (size_t)G), o_tg = take(8 * (size_t)G), o_tw = take(8 * (size_t)M),
-               o_red = take(8 * 40), o_tau = take(4 * (size_t)G), o_mask = take((size_t)G);
+               o_red = take(8 * 40), o_lhsp = take(8 * (size_t)G * 8), o_tau = take(4 * (size_t)G),
+               o_mask = take((size_t)G);
   if (c) {
     c->ring = reinterpret_cast<float*>(base + o_ring);
     c->h = reinterpret_cast<float*>(base + o_h);
@@ -99,6 +133,7 @@ __host__ __device__ inline size_t carve(unsigned char* base, int G, int M, int D
     c->tg = reinterpret_cast<double*>(base + o_tg);
     c->tw = reinterpret_cast<double*>(base + o_tw);
     c->red = reinterpret_cast<double*>(base + o_red);
+    c->lhsp = reinterpret_cast<double*>(base + o_lhsp);
     c->tau = reinterpret_cast<int*>(base + o_tau);
     c->mask = base + o_mask;
   }
@@ -142,7 +177,9 @@ __global__ void __launch_bounds__(LC_THREADS, 1) linear_cluster_kernel(const Par
 
   const int nb_g = (B + RR - 1) / RR;          // batches of RR rows per group
   const int n_batches = G * nb_g;
-  const int wg = cta * LC_WARPS + warp, nw_tot = C * LC_WARPS;
+  // batches are dealt warp-major, so that the last warp of every CTA has the fewest (it also forms the
+  // right side of Eq. (9) while the others fetch their first rows)
+  const int wg = warp * C + cta, nw_tot = C * LC_WARPS;
   // ring positions are kept as small counters (no 64-bit division inside the loop)
   int kslot = (int)(st.k % ring), dslot = (int)(st.k % D), hslot = (int)(st.k % P.hist_cap);
   // computing times of the first iteration (those of iteration k+1 are drawn while iteration k updates)
@@ -158,12 +195,51 @@ __global__ void __launch_bounds__(LC_THREADS, 1) linear_cluster_kernel(const Par
     for (int e = lane; e < gp2; e += 32) accw_w[e] = 0.f;  // groups this warp does not visit contribute zero
     __syncwarp();
 
-    // ---- gradients: this warp's batches (ascending, so its groups come in one run each)
+    // the last warp forms the right side of Eq. (9) (it depends on earlier iterations only)
+    if (warp == LC_WARPS - 1 && lane == 0) {
+      double rhs = 0.0;
+      for (int dd = 1; dd <= kfill; ++dd) {  // ||theta^{k+1-dd} - theta^{k-dd}||^2 sits in slot (k-dd) mod D
+        int sl = dslot - dd;
+        if (sl < 0) sl += D;
+        rhs += (P.c_d ? P.c_d[dd - 1] : P.c) * S.s_ring[sl];
+      }
+      S.red[39] = rhs;
+    }
+
+    // ---- gradients: this warp's batches (ascending, so its groups come in one run each); the rows of
+    // the next batch are fetched before the current one is worked on
     float th[CPL], ths[CPL], acc0[CPL], acc1[CPL];
 #pragma unroll
     for (int i = 0; i < CPL; ++i) th[i] = lane + 32 * i < pp ? theta_k[lane + 32 * i] : 0.f;  // (the pad of a p-vector is zero)
     int cur_g = -1;
-    for (int b = wg; b < n_batches; b += nw_tot) {
+    constexpr int SPREAD = 32 / RR;  // lanes that end up holding the same row's dot products
+    auto fetch = [&](int b, float& yy, float (&x)[RR][CPL]) {
+      const int g = b / nb_g, rb = (b - g * nb_g) * RR;
+      long long myrow = 0;
+      yy = 0.f;
+      if (lane < RR && rb + lane < B) {
+        myrow = batch_row(P, k32, g, rb + lane);
+        yy = yf[myrow];
+      }
+#pragma unroll
+      for (int r = 0; r < RR; ++r) {
+        const long long row = __shfl_sync(0xffffffffu, myrow, r);
+        const bool valid = rb + r < B;
+#pragma unroll
+        for (int i = 0; i < CPL; ++i) {
+          const int c = lane + 32 * i;
+          x[r][i] = (valid && c < d) ? Xf[row * P.ld + c] : 0.f;
+        }
+      }
+    };
+    float xc[RR][CPL], yc = 0.f;
+    int b = wg;
+    if (b < n_batches) fetch(b, yc, xc);
+    while (b < n_batches) {
+      const int bn = b + nw_tot;
+      float xn[RR][CPL], yn = 0.f;
+      constexpr bool PREFETCH = RR * CPL <= 16;  // wider rows would not fit two batches in registers
+      if (PREFETCH && bn < n_batches) fetch(bn, yn, xn);
       const int g = b / nb_g, rb = (b - g * nb_g) * RR;
       if (g != cur_g) {
         if (cur_g >= 0) {
@@ -187,45 +263,43 @@ __global__ void __launch_bounds__(LC_THREADS, 1) linear_cluster_kernel(const Par
           acc1[i] = 0.f;
         }
       }
-      long long myrow = 0;
-      float myy = 0.f;
-      if (lane < RR && rb + lane < B) {
-        myrow = batch_row(P, k32, g, rb + lane);
-        myy = yf[myrow];
-      }
-      float x[RR][CPL], z[RR], zs[RR];
+      float z[RR], zs[RR];
 #pragma unroll
       for (int r = 0; r < RR; ++r) {
-        const long long row = __shfl_sync(0xffffffffu, myrow, r);
-        const bool valid = rb + r < B;
         z[r] = 0.f;
         zs[r] = 0.f;
 #pragma unroll
         for (int i = 0; i < CPL; ++i) {
-          const int c = lane + 32 * i;
-          x[r][i] = (valid && c < d) ? Xf[row * P.ld + c] : 0.f;
-          z[r] += x[r][i] * th[i];
-          zs[r] += x[r][i] * ths[i];
+          z[r] += xc[r][i] * th[i];
+          zs[r] += xc[r][i] * ths[i];
         }
       }
+      reduce_spread<RR>(z, lane);
+      reduce_spread<RR>(zs, lane);
+      // lane l now holds both dot products of row l / SPREAD and turns them into that row's two coefficients
+      // (every lane used to repeat this for all RR rows)
+      const int my_r = lane / SPREAD;
+      const float my_y = __shfl_sync(0xffffffffu, yc, my_r);
+      float my_a = 0.f, my_e = 0.f;
+      if (rb + my_r < B) residuals<QUAD>(z[0], zs[0], my_y, my_a, my_e);
+      my_a *= P.scale;
+      my_e *= P.scale;
 #pragma unroll
       for (int r = 0; r < RR; ++r) {
-        z[r] = warp_sum(z[r]);
-        zs[r] = warp_sum(zs[r]);
-      }
-#pragma unroll
-      for (int r = 0; r < RR; ++r) {
-        const float yy = __shfl_sync(0xffffffffu, myy, r);
-        float a = 0.f, e = 0.f;
-        if (rb + r < B) residuals<QUAD>(z[r], zs[r], yy, a, e);
-        a *= P.scale;
-        e *= P.scale;
+        const float a = __shfl_sync(0xffffffffu, my_a, r * SPREAD), e = __shfl_sync(0xffffffffu, my_e, r * SPREAD);
 #pragma unroll
         for (int i = 0; i < CPL; ++i) {
-          acc0[i] += a * x[r][i];
-          acc1[i] += e * x[r][i];
+          acc0[i] += a * xc[r][i];
+          acc1[i] += e * xc[r][i];
         }
       }
+      if (!PREFETCH && bn < n_batches) fetch(bn, yn, xn);
+      b = bn;
+      yc = yn;
+#pragma unroll
+      for (int r = 0; r < RR; ++r)
+#pragma unroll
+        for (int i = 0; i < CPL; ++i) xc[r][i] = xn[r][i];
     }
     if (cur_g >= 0) {
 #pragma unroll
@@ -247,29 +321,23 @@ __global__ void __launch_bounds__(LC_THREADS, 1) linear_cluster_kernel(const Par
     }
     cluster.sync();  // the one cluster-wide barrier of the iteration
 
-    // ---- CTA partials -> every group's gradient and innovation, in every CTA (CTA order); a warp takes
-    // whole (group, point) rows, so the warp that sums an innovation also forms its squared norm
-    for (int gq = warp; gq < 2 * G; gq += LC_WARPS) {
-      const int g = gq >> 1;
-      double nrm = 0.0;
-      for (int c = lane; c < pp; c += 32) {
-        const int e = gq * pp + c;
-        float v[16];  // all remote loads in flight before the first add
+    // ---- CTA partials -> every group's gradient and innovation, in every CTA (CTA order).  One element per
+    // thread; the 32 elements of a warp lie in one (group, point) row, so the warp also forms its share of
+    // the squared innovation norm
+    for (int e = tid; e < gp2; e += LC_THREADS) {
+      float v[16];  // all remote loads in flight before the first add
 #pragma unroll
-        for (int r = 0; r < 16; ++r) v[r] = r < C ? cluster.map_shared_rank(part, r)[e] : 0.f;
-        float s = 0.f;
+      for (int r = 0; r < 16; ++r) v[r] = r < C ? cluster.map_shared_rank(part, r)[e] : 0.f;
+      float s = 0.f;
 #pragma unroll
-        for (int r = 0; r < 16; ++r) s += v[r];
-        if (gq & 1) {
-          S.innov[g * pp + c] = s;
-          nrm += (double)s * (double)s;
-        } else {
-          S.fresh[g * pp + c] = s;
-        }
-      }
-      if (gq & 1) {  // LHS_g = ||innovation_g||^2
-        nrm = warp_sum(nrm);
-        if (lane == 0) S.lhs[g] = nrm;
+      for (int r = 0; r < 16; ++r) s += v[r];
+      const int gq = e / pp, c = e - gq * pp, g = gq >> 1;
+      if (gq & 1) {
+        S.innov[g * pp + c] = s;
+        const double nrm = warp_sum((double)s * (double)s);
+        if (lane == 0) S.lhsp[g * 8 + (c >> 5)] = nrm;
+      } else {
+        S.fresh[g * pp + c] = s;
       }
     }
     __syncthreads();
@@ -277,20 +345,17 @@ __global__ void __launch_bounds__(LC_THREADS, 1) linear_cluster_kernel(const Par
     // ---- the server's decision (Eq. 9, the age rule), ages, clock and counters
     if (tid < G) {
       const int g = tid, tau = S.tau[g];
-      double rhs = 0.0;
-      for (int dd = 1; dd <= kfill; ++dd) {  // ||theta^{k+1-dd} - theta^{k-dd}||^2 sits in slot (k-dd) mod D
-        int sl = dslot - dd;
-        if (sl < 0) sl += D;
-        rhs += (P.c_d ? P.c_d[dd - 1] : P.c) * S.s_ring[sl];
-      }
+      const double rhs = S.red[39];
+      double lhs = 0.0;
+      for (int ch = 0; ch < (pp >> 5); ++ch) lhs += S.lhsp[g * 8 + ch];  // LHS_g = ||innovation_g||^2
+      S.lhs[g] = lhs;
       double t = 1.0e300;
       for (int m = g * P.M_G; m < (g + 1) * P.M_G; ++m) t = fmin(t, S.tw[m]);
-      const bool sel = (tau >= D) || (S.lhs[g] > rhs);
+      const bool sel = (tau >= D) || (lhs > rhs);
       S.tg[g] = t;
       S.mask[g] = sel ? 1 : 0;
       S.tau[g] = sel ? 1 : tau + 1;
       if (cta == 0) P.hist[(long long)hslot * G + g] = sel ? 1 : 0;
-      if (g == 0) S.red[39] = rhs;
     }
     __syncthreads();
     int nsel = 0;
