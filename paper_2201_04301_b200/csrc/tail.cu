@@ -62,11 +62,18 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
     int c_lo = 0, c_hi = -1;
     const long long Rtot = (long long)n_groups * P.pm.rows_per_group;
     const int n = P.pm.n_cta;
+    // CTA c of the gradient kernel owns rows [c*Rtot/n, (c+1)*Rtot/n); 32-bit arithmetic where the products fit
+    const bool small = (Rtot + 1) * (long long)(n + 1) < 0x7fffffffLL;
     if (n > 0) {
       const long long x0 = (long long)gi * P.pm.rows_per_group;
       const long long x1 = x0 + P.pm.rows_per_group - 1;
-      c_lo = (int)(((x0 + 1) * n - 1) / Rtot);
-      c_hi = (int)(((x1 + 1) * n - 1) / Rtot);
+      if (small) {
+        c_lo = (int)(((unsigned)(x0 + 1) * (unsigned)n - 1u) / (unsigned)Rtot);
+        c_hi = (int)(((unsigned)(x1 + 1) * (unsigned)n - 1u) / (unsigned)Rtot);
+      } else {
+        c_lo = (int)(((x0 + 1) * n - 1) / Rtot);
+        c_hi = (int)(((x1 + 1) * n - 1) / Rtot);
+      }
     }
     double local = 0.0;
   #pragma unroll
@@ -83,7 +90,8 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
           for (int u = 0; u < 4; ++u) {
             const int c = c0 + u;
             if (c <= c_hi) {
-              const int gf = (int)(((long long)c * Rtot / n) / P.pm.rows_per_group);
+              const int gf = small ? (int)(((unsigned)c * (unsigned)Rtot / (unsigned)n) / (unsigned)P.pm.rows_per_group)
+                                   : (int)(((long long)c * Rtot / n) / P.pm.rows_per_group);
               const float* src = P.partial + ((long long)(c * P.pm.maxseg + (gi - gf)) * 2) * P.p_pad + i4 * 4;
               a[u] = ld4(src);
               b[u] = ld4(src + P.p_pad);
@@ -125,9 +133,16 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
   // ---- phase 2 (last block only): the server's scheduling decision.
   // One thread per group, 256 groups at a time; everything a group needs is
   // fetched in one round of independent loads.
+  // Everything below is one dependency chain in one block, so all loads are issued before the arithmetic
+  // that does not need them (the computing times) and consumed after it.
+  // Right side of Eq. (9).  With one constant c it is c times the sum of the ring of squared step norms
+  // (slots of steps that have not happened yet hold zero), which needs no slot arithmetic.
+  constexpr int RING_REGS = 16;
+  const bool ring_in_regs = !P.c_d && P.D <= RING_REGS;
+  double sv[RING_REGS];
+#pragma unroll
+  for (int i = 0; i < RING_REGS; ++i) sv[i] = (ring_in_regs && i < P.D) ? P.s_ring[i] : 0.0;
   double rhs = 0.0;
-  for (int d = 1; d <= P.D && k - d >= 0; ++d)  // ||theta^{k+1-d} - theta^{k-d}||^2 sits in slot (k-d) mod D
-    rhs += (P.c_d ? P.c_d[d - 1] : P.c) * P.s_ring[(k - d) % P.D];
   const uint32_t k32 = (uint32_t)k;
   const volatile double* parts = P.lhs_part;
   int nsel = 0;
@@ -142,7 +157,12 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
     bool sel_forced = false;
     if (have && P.forced) sel_forced = P.forced[(k - P.forced_base) * P.G + gg] != 0;
     double lhs = 0.0;
-    if (blocks_x <= 64) {
+    constexpr int PART_REGS = 8;
+    double pv[PART_REGS];
+    if (blocks_x <= PART_REGS) {  // issued now, added (in block order) after the computing times
+#pragma unroll
+      for (int b = 0; b < PART_REGS; ++b) pv[b] = (have && b < blocks_x) ? parts[(long long)gg * blocks_x + b] : 0.0;
+    } else if (blocks_x <= 64) {
       if (have)
         for (int b = 0; b < blocks_x; ++b) lhs += parts[(long long)gg * blocks_x + b];
     } else {
@@ -171,6 +191,24 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
       }
     }
     bool sel = false;
+    if (blocks_x <= PART_REGS) {
+#pragma unroll
+      for (int b = 0; b < PART_REGS; ++b) lhs += pv[b];
+    }
+    if (gc == 0) {
+      if (ring_in_regs) {
+#pragma unroll
+        for (int i = 0; i < RING_REGS; ++i) rhs += sv[i];
+        rhs *= P.c;
+      } else {
+        int slot = (int)(k % P.D);  // ||theta^{k+1-d} - theta^{k-d}||^2 sits in slot (k-d) mod D
+        const int terms = k < P.D ? (int)k : P.D;
+        for (int d = 1; d <= terms; ++d) {
+          if (--slot < 0) slot = P.D - 1;
+          rhs += (P.c_d ? P.c_d[d - 1] : P.c) * P.s_ring[slot];
+        }
+      }
+    }
     if (have) {
       if (P.ps_L2) lhs = P.ps_lhs[gg];  // rule PS: the test uses the printed left side, not the measured innovation
       sel = P.forced ? sel_forced : ((tau >= P.D) || (lhs > rhs));
@@ -255,7 +293,7 @@ __device__ __forceinline__ void renorm(float& hi, float& lo) {
 // partial sum; the eight partial sums are then added to the aggregate in warp
 // order, so the result does not depend on timing.
 __global__ void __launch_bounds__(256) update_kernel(const Params P) {
-  extern __shared__ int sel_list[];  // selected groups, ascending
+  extern __shared__ int sel_list[];  // selected groups, ascending; bit 30 set = the group's cur[] is 1
   __shared__ int n_sel_sh;
   __shared__ float4 wsum_hi[8][32], wsum_lo[8][32];
   __shared__ bool is_last;
@@ -270,18 +308,28 @@ __global__ void __launch_bounds__(256) update_kernel(const Params P) {
     for (int g0 = 0; g0 < P.G; g0 += 32) {
       const int gg = g0 + lane;
       const bool s = gg < P.G && P.mask_cur[gg] != 0;
+      const int cur = gg < P.G ? P.cur[gg] : 0;  // read with the mask, so that the fold need not wait for it
       const unsigned int b = __ballot_sync(0xffffffffu, s);
-      if (s) sel_list[cnt + __popc(b & ((1u << lane) - 1u))] = gg;
+      if (s) sel_list[cnt + __popc(b & ((1u << lane) - 1u))] = gg | (cur << 30);
       cnt += __popc(b);
     }
     if (lane == 0) n_sel_sh = cnt;
   }
-  __syncthreads();
-  const int n_sel = n_sel_sh;
-
   const long long i4 = (long long)blockIdx.x * 32 + lane;
   const bool active = i4 < cols4;
   const long long o = i4 * 4;
+  // the vectors Eq. (8) needs do not depend on the selection: fetched now, used after the fold
+  float4 ahi = make_float4(0.f, 0.f, 0.f, 0.f), alo = ahi, h = ahi, vh = ahi, th = ahi;
+  if (warp == 0 && active) {
+    ahi = ld4(P.agg_hi + o);
+    alo = ld4(P.agg_lo + o);
+    h = ld4(P.h + o);
+    vh = ld4(P.vhat + o);
+    th = ld4(P.theta_ring + (k % ring) * P.p_pad + o);
+  }
+  __syncthreads();
+  const int n_sel = n_sel_sh;
+
   float4 hi = make_float4(0.f, 0.f, 0.f, 0.f), lo = hi;
   if (active) {
     for (int j0 = warp; j0 < n_sel; j0 += 32) {  // four groups of this warp per round, loads first
@@ -290,8 +338,9 @@ __global__ void __launch_bounds__(256) update_kernel(const Params P) {
       for (int u = 0; u < 4; ++u) {
         const int j = j0 + 8 * u;
         if (j < n_sel) {
-          f[u] = ld4(last_row(P, sel_list[j]) + o);   // selected: cur[g] already points at the fresh gradient
-          l[u] = ld4(other_row(P, sel_list[j]) + o);  // the gradient it replaces
+          const int e = sel_list[j], g = e & 0x3fffffff, cur = e >> 30;
+          f[u] = ld4(P.gbuf + ((long long)cur * P.G + g) * P.p_pad + o);        // selected: cur[g] already points at the fresh gradient
+          l[u] = ld4(P.gbuf + ((long long)(1 - cur) * P.G + g) * P.p_pad + o);  // the gradient it replaces
         }
       }
 #pragma unroll
@@ -311,7 +360,6 @@ __global__ void __launch_bounds__(256) update_kernel(const Params P) {
   if (warp == 0) {
     double local = 0.0;
     if (active) {
-      float4 ahi = ld4(P.agg_hi + o), alo = ld4(P.agg_lo + o);
 #pragma unroll
       for (int w = 0; w < 8; ++w) {
         const float4 h2 = wsum_hi[w][lane], l2 = wsum_lo[w][lane];
@@ -331,8 +379,6 @@ __global__ void __launch_bounds__(256) update_kernel(const Params P) {
       st4(P.agg_hi + o, ahi);
       st4(P.agg_lo + o, alo);
       // Eq. (8a)-(8c)
-      float4 h = ld4(P.h + o), vh = ld4(P.vhat + o);
-      const float4 th = ld4(P.theta_ring + (k % ring) * P.p_pad + o);
       float4 tn;
 #define GCADA_AMSGRAD(c)                                   \
   {                                                        \
