@@ -311,7 +311,10 @@ def run_ours(args):
                            "duration_ms": ms_grad_b2b, "duration_how": "200 back-to-back launches, one CUDA-event pair",
                            "achieved_from_bracketed_launches": bytes_launch / (ms_grad * 1e-3) / 1e9 if ms_grad > 0 else None,
                            "algorithmic_bytes_per_launch": bytes_launch,
-                           "frac_of_nominal_8TBs": achieved / 8000.0 if achieved else None}
+                           "frac_of_nominal_8TBs": achieved / 8000.0 if achieved else None,
+                           # the same bytes over the whole timed step (gradient + selection + update kernels)
+                           "whole_step_gbs": bytes_launch / (ms / args.steps * 1e-3) / 1e9,
+                           "whole_step_frac": bytes_launch / (ms / args.steps * 1e-3) / 1e9 / peaks["hbm"]}
     else:
         flops = mlp_flops_per_iteration(w)
         if args.rule == "ps":     # only the selected groups compute, at theta^k only
