@@ -861,6 +861,68 @@ __global__ void __launch_bounds__(256) bf16_softmax_grad_kernel(const Params P, 
   for (int c = warp; c < n_cls; c += 8) oT[(long long)c * Bp + lane] = sm_tile[lane * pitch + c];
 }
 
+// The same for an even number of classes up to 64 * NP: a lane keeps its NP class pairs of a row in registers,
+// so the scores are read once (8-byte loads), every exponential is taken once, and the results leave as bf16
+// pairs.
+template <int NP>
+__global__ void __launch_bounds__(256) bf16_softmax_grad_pairs_kernel(const Params P, const float* scores, const int* yb,
+                                                                      __nv_bfloat16* dz, __nv_bfloat16* dzT, int n_cls,
+                                                                      int ldz, int Bp, int pitch) {
+  extern __shared__ __nv_bfloat16 sm_tile[];  // [32][pitch]
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const long long rows = (long long)P.G * Bp;
+  const long long w0 = (long long)blockIdx.x * 32;  // first (point, row) of the block
+  const int q = (int)(w0 / rows);
+  const long long r0 = w0 - (long long)q * rows;
+  const int g = (int)(r0 / Bp), m0 = (int)(r0 - (long long)g * Bp);
+  if (P.skip_unselected && (q != 0 || !P.mask_cur[g])) return;
+  for (int i = 0; i < 4; ++i) {
+    const int lr = warp * 4 + i;
+    const long long w = w0 + lr;
+    const float* s = scores + w * n_cls;
+    __nv_bfloat16* o = dz + w * ldz;
+    __nv_bfloat16* t = sm_tile + lr * pitch;
+    const int y = yb[r0 + lr];
+    float2 v[NP];
+    float mx = -3.0e38f;
+#pragma unroll
+    for (int j = 0; j < NP; ++j) {
+      const int c = 2 * lane + 64 * j;
+      v[j] = (y >= 0 && c < n_cls) ? *reinterpret_cast<const float2*>(s + c) : make_float2(-3.0e38f, -3.0e38f);
+      mx = fmaxf(mx, fmaxf(v[j].x, v[j].y));
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+    // p_y - 1 = -(sum of the other classes' exponentials) / sum, free of cancellation
+    float others = 0.f, ey = 0.f;
+#pragma unroll
+    for (int j = 0; j < NP; ++j) {
+      const int c = 2 * lane + 64 * j;
+      v[j].x = expf(v[j].x - mx);  // classes beyond n_cls: exp of a huge negative number, zero
+      v[j].y = expf(v[j].y - mx);
+      if (c == y) ey = v[j].x; else others += v[j].x;
+      if (c + 1 == y) ey = v[j].y; else others += v[j].y;
+    }
+    others = warp_sum(others);
+    ey = warp_sum(ey);
+    const float inv = y >= 0 ? 1.0f / (others + ey) : 0.f;
+#pragma unroll
+    for (int j = 0; j < NP; ++j) {
+      const int c = 2 * lane + 64 * j;
+      if (c < n_cls) {
+        const float a = y < 0 ? 0.f : (c == y ? -others * inv : v[j].x * inv) * P.scale;
+        const float b = y < 0 ? 0.f : (c + 1 == y ? -others * inv : v[j].y * inv) * P.scale;
+        const __nv_bfloat162 pr = __floats2bfloat162_rn(a, b);
+        *reinterpret_cast<__nv_bfloat162*>(o + c) = pr;
+        *reinterpret_cast<__nv_bfloat162*>(t + c) = pr;
+      }
+    }
+  }
+  __syncthreads();
+  __nv_bfloat16* oT = dzT + ((long long)(q * P.G + g) * n_cls) * Bp + m0;
+  for (int c = warp; c < n_cls; c += 8) oT[(long long)c * Bp + lane] = sm_tile[lane * pitch + c];
+}
+
 // ----------------------------------------------------------------- bias gradients
 // db_l at both points (column sums of dz_l over the group's rows), their
 // squared difference summed per block into the block's lhs_part slot.
@@ -1177,6 +1239,12 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
   e = cudaFuncSetAttribute(bf16_softmax_grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            32 * (plan->dims[L] + 4) * 2);
   if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(bf16_softmax_grad_pairs_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 32 * (256 + 4) * 2);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(bf16_softmax_grad_pairs_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 32 * (512 + 4) * 2);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(bf16_softmax_grad_pairs_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 32 * (1024 + 4) * 2);
+  if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(bf16_dw_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 4096);  // the rest is static
   if (e != cudaSuccess) return e;
   plan->launches_per_iter = 3 + L + 1 + L + (L - 1);
@@ -1244,8 +1312,19 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
   }
   {
     const int pitch = pl.dims[L] + 2 + (pl.dims[L] & 1);  // even, and an odd number of 32-bit words when possible
-    bf16_softmax_grad_kernel<<<(unsigned)(2 * rows / 32), 256, (size_t)32 * pitch * 2, st>>>(
-        P, im->scores, im->yb, im->dz[L], im->dzT[L], pl.dims[L], im->ld[L], Bp, pitch);
+    const int nc = pl.dims[L];
+    const unsigned blocks = (unsigned)(2 * rows / 32);
+    const size_t sm = (size_t)32 * pitch * 2;
+    if ((nc & 1) == 0 && nc <= 1024) {  // class pairs in registers
+      if (nc <= 256)
+        bf16_softmax_grad_pairs_kernel<4><<<blocks, 256, sm, st>>>(P, im->scores, im->yb, im->dz[L], im->dzT[L], nc, im->ld[L], Bp, pitch);
+      else if (nc <= 512)
+        bf16_softmax_grad_pairs_kernel<8><<<blocks, 256, sm, st>>>(P, im->scores, im->yb, im->dz[L], im->dzT[L], nc, im->ld[L], Bp, pitch);
+      else
+        bf16_softmax_grad_pairs_kernel<16><<<blocks, 256, sm, st>>>(P, im->scores, im->yb, im->dz[L], im->dzT[L], nc, im->ld[L], Bp, pitch);
+    } else {
+      bf16_softmax_grad_kernel<<<blocks, 256, sm, st>>>(P, im->scores, im->yb, im->dz[L], im->dzT[L], nc, im->ld[L], Bp, pitch);
+    }
   }
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   ++n;
