@@ -619,14 +619,14 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
     const bool vec_ok = ((a.c_off | a.ldc) & 3) == 0 && (P.p_pad & 3) == 0 &&
                         (reinterpret_cast<uintptr_t>(a.mode == DW_ONE ? a.out_row : P.gbuf) & 15) == 0;
     bool ok = true;
-    int i = 0;
-    for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
+    int i = 0, ui = 0;
+    for (int u = blockIdx.x; u < n_units; u += gridDim.x, ++ui) {
       const int mt = u % a.tiles_m, g = a.mode == DW_ONE ? a.g_only : u / a.tiles_m;
+      double local = 0.0;  // this warp's share of the unit's squared innovation norm (all its column tiles)
       for (int nt = 0; nt < a.tiles_n; ++nt) {
       const int slot = i % n_slots;
       const int phase = (i / n_slots) & 1;
       ++i;
-      double local = 0.0;
       if (ok) {
         ok = mbar_wait_bounded(&tfull_bar[slot], (uint32_t)phase);
         ok = __all_sync(0xffffffffu, ok);
@@ -639,6 +639,31 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
         const int n_pass = a.mode == DW_NORM ? 0 : (stale ? 2 : 1);
         const int mrow = mt * BM + quad * 32;
         const uint32_t tbase = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(slot * slot_cols);
+        if (a.mode == DW_NORM) {
+          // Norm only.  Rows and columns outside the matrix were zero-filled by the copies, so the whole
+          // 128 x 256 accumulator is summed without predicates; the four tensor-memory loads of this warp
+          // are pipelined (a load takes far longer than its issue).
+          const uint32_t cb = (uint32_t)(half * (DW_BN / 2));
+          uint32_t va[32], vb[32];
+          auto sq = [&](const uint32_t(&v)[32]) {
+            float part = 0.f;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) part += __uint_as_float(v[j]) * __uint_as_float(v[j]);
+            local += (double)part;
+          };
+          tc_ld32_issue(tbase + cb, va);
+          tc_ld_wait();
+          tc_ld32_issue(tbase + cb + 32, vb);
+          sq(va);
+          tc_ld_wait();
+          tc_ld32_issue(tbase + cb + 64, va);
+          sq(vb);
+          tc_ld_wait();
+          tc_ld32_issue(tbase + cb + 96, vb);
+          sq(va);
+          tc_ld_wait();
+          sq(vb);
+        } else
 #pragma unroll 1
         for (int c = half * (DW_BN / 2); c < (half + 1) * (DW_BN / 2); c += 32) {
           const int nc = nt * DW_BN + c;
@@ -690,15 +715,17 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
         __syncwarp();
         if (lane == 0) mbar_arrive(&tempty_bar[slot]);  // this warp is done with the slot's tensor memory
       }
+      }
+      // one partial sum per unit (the eight warps in warp order); the buffer alternates between units, so a
+      // warp that runs ahead cannot overwrite values that thread 0 of the first warp is still adding
       local = warp_sum(local);
-      if (lane == 0) norm_sm[slot][ew] = local;
+      if (lane == 0) norm_sm[ui & 1][ew] = local;
       asm volatile("bar.sync 1, %0;" ::"n"(32 * DW_EPI_WARPS) : "memory");
       if (ew == 0 && lane == 0 && a.mode != DW_ONE) {
         double tsum = 0.0;
 #pragma unroll
-        for (int w = 0; w < DW_EPI_WARPS; ++w) tsum += norm_sm[slot][w];
-        P.lhs_part[(long long)g * a.n_parts + a.part_base + mt * a.tiles_n + nt] = tsum;
-      }
+        for (int w = 0; w < DW_EPI_WARPS; ++w) tsum += norm_sm[ui & 1][w];
+        P.lhs_part[(long long)g * a.n_parts + a.part_base + mt] = tsum;
       }
     }
     if (!ok && lane == 0) atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
@@ -1151,7 +1178,7 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
   int parts = 0;
   for (int l = 1; l <= L; ++l) {
     im->dw_part_base[l] = parts;
-    parts += ((plan->dims[l] + BM - 1) / BM) * ((plan->dims[l - 1] + DW_BN - 1) / DW_BN);
+    parts += (plan->dims[l] + BM - 1) / BM;  // one per (group, 128-row block of W_l)
   }
   for (int l = 1; l <= L; ++l) {
     im->bias_part_base[l] = parts;
