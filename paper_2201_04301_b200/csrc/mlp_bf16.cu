@@ -1120,7 +1120,7 @@ cudaError_t launch_dw(const Params& P, const MlpPlan& pl, const Bf16Impl* im, in
   // 32 KiB B blocks in whatever shared memory is left beside the resident A blocks (and the staging tile of
   // the modes that write gradients): the B stream is bound by bytes in flight, so every stage counts
   const long long stage_bytes = mode == DW_NORM ? 0 : (long long)DW_STAGE_FLOATS * 4;
-  const long long room = 232448 - 4096 - 1024 - (long long)2 * w.nkb * (BM * BK * 2) - stage_bytes;
+  const long long room = 232448 - 1024 - 1024 - (long long)2 * w.nkb * (BM * BK * 2) - stage_bytes;
   w.stages = (int)(room / (DW_BN * BK * 2));
   if (w.stages > MAX_STAGES) w.stages = MAX_STAGES;
   if (w.stages < 1) w.stages = 1;
@@ -1272,7 +1272,7 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(bf16_softmax_grad_pairs_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 32 * (1024 + 4) * 2);
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(bf16_dw_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 4096);  // the rest is static
+  e = cudaFuncSetAttribute(bf16_dw_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024);  // the kernel's static arrays take under 1 KiB
   if (e != cudaSuccess) return e;
   plan->launches_per_iter = 3 + L + 1 + L + (L - 1);
   plan->post_launches = L + 2;
