@@ -320,14 +320,43 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
       const int q = a.k_batched ? 0 : zi / n_grp;
       const int g = a.k_batched ? 0 : (P.skip_unselected ? P.sel_list[zi - q * n_grp] : zi - q * n_grp);
       const int z = q * P.G + g;
+      const int m = mt * BM + quad * 32 + lane;
+      const int n0 = nt * GN;
+      // EPI_DA: the ReLU mask of this thread's row does not depend on the accumulator, so it is fetched (one
+      // bit per column, four words for the four chunks) while the MMAs of the tile are still running
+      uint32_t mbits[4] = {0u, 0u, 0u, 0u};
+      const bool mask_in_regs = a.epi == EPI_DA && m < a.M;
+      if (mask_in_regs) {
+        const __nv_bfloat16* mk = a.mask + (long long)z * a.z_stride_out + (long long)m * a.ldo;
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+          const int nc = n0 + half * (GN / 2) + ch * 32;
+          if (nc + 32 <= a.N) {
+            uint4 pk[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) pk[j] = *reinterpret_cast<const uint4*>(mk + nc + 8 * j);
+            uint32_t bits = 0u;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const uint32_t wds[4] = {pk[j].x, pk[j].y, pk[j].z, pk[j].w};
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                // a bf16 is positive iff its bits are non-zero and its sign bit clear
+                const uint32_t lo = wds[e] & 0xFFFFu, hi = wds[e] >> 16;
+                bits |= (uint32_t)(lo != 0u && lo < 0x8000u) << (8 * j + 2 * e);
+                bits |= (uint32_t)(hi != 0u && hi < 0x8000u) << (8 * j + 2 * e + 1);
+              }
+            }
+            mbits[ch] = bits;
+          }
+        }
+      }
       if (ok) {
         ok = mbar_wait_bounded(&tfull_bar[slot], (uint32_t)((i >> 1) & 1));
         ok = __all_sync(0xffffffffu, ok);
       }
       if (!ok) continue;
       tc_fence_after();
-      const int m = mt * BM + quad * 32 + lane;
-      const int n0 = nt * GN;
       const float* bias = nullptr;
       if (a.epi == EPI_HIDDEN || a.epi == EPI_SCORES)
         bias = a.bias_ring + (long long)ring_slot(P, g, q, k_it) * a.bias_slot + a.bias_pos;
@@ -371,18 +400,9 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
           } else {  // EPI_DA: ReLU derivative of the layer below
             const __nv_bfloat16* mk = a.mask + (long long)z * a.z_stride_out + (long long)m * a.ldo + nc;
             if (full && row_ok) {
+              const uint32_t bits = mbits[(c - half * (GN / 2)) >> 5];
 #pragma unroll
-              for (int j = 0; j < 32; j += 8) {
-                const uint4 pk = *reinterpret_cast<const uint4*>(mk + j);
-                const uint32_t wds[4] = {pk.x, pk.y, pk.z, pk.w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                  // a bf16 is positive iff its bits are non-zero and its sign bit clear
-                  const uint32_t lo = wds[e] & 0xFFFFu, hi = wds[e] >> 16;
-                  f[j + 2 * e] = (lo != 0u && lo < 0x8000u) ? __uint_as_float(v[j + 2 * e]) : 0.f;
-                  f[j + 2 * e + 1] = (hi != 0u && hi < 0x8000u) ? __uint_as_float(v[j + 2 * e + 1]) : 0.f;
-                }
-              }
+              for (int j = 0; j < 32; ++j) f[j] = ((bits >> j) & 1u) ? __uint_as_float(v[j]) : 0.f;
             } else {
 #pragma unroll
               for (int j = 0; j < 32; ++j) {
@@ -398,22 +418,44 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
             __nv_bfloat162 t2 = __floats2bfloat162_rn(f[j], f[j + 1]);
             h[j >> 1] = *reinterpret_cast<uint32_t*>(&t2);
           }
-          if (row_ok) {
-            __nv_bfloat16* dst = a.out + (long long)z * a.z_stride_out + (long long)m * a.ldo + nc;
-            if (full) {
-#pragma unroll
-              for (int j = 0; j < 16; j += 4)
-                *reinterpret_cast<uint4*>(dst + 2 * j) = make_uint4(h[j], h[j + 1], h[j + 2], h[j + 3]);
-            } else {
-              for (int j = 0; j < 32 && nc + j < a.N; ++j) dst[j] = __float2bfloat16_rn(f[j]);
-            }
-          }
-          // transposed copy: the warp's 32 x 32 block goes through shared memory (rows of 17 words, free
-          // of bank conflicts both ways) so that lane n writes 64 contiguous bytes of output row nc + n
+          // The warp's 32 x 32 block goes through shared memory (rows of 17 words) for both copies, so that
+          // every store instruction writes whole 32-byte sectors: a lane that stored 16 bytes of its own row
+          // touched half a sector, and the L2 counted twice the sectors the data needs.
           __syncwarp();
 #pragma unroll
           for (int j = 0; j < 16; ++j) tr[lane * 17 + j] = h[j];
           __syncwarp();
+          const int rows_here = a.M - (mt * BM + quad * 32);  // valid rows of this warp's block (>= 32 inside)
+          if (full && rows_here >= 32) {
+            // row-major copy: lanes 4r..4r+3 write the 64 bytes of row r, eight rows per instruction
+            __nv_bfloat16* dst0 = a.out + (long long)z * a.z_stride_out + (long long)(mt * BM + quad * 32) * a.ldo + nc;
+#pragma unroll
+            for (int it = 0; it < 4; ++it) {
+              const int r = it * 8 + (lane >> 2), qd = lane & 3;
+              const uint32_t* src = tr + r * 17 + qd * 4;
+              *reinterpret_cast<uint4*>(dst0 + (long long)r * a.ldo + qd * 8) = make_uint4(src[0], src[1], src[2], src[3]);
+            }
+            // transposed copy: lanes 4n..4n+3 write the 64 bytes (32 rows) of output row nc + n
+            __nv_bfloat16* dstT0 = a.outT + (long long)z * a.z_stride_outT + (long long)nc * a.ldt + (mt * BM + quad * 32);
+#pragma unroll
+            for (int it = 0; it < 4; ++it) {
+              const int n = it * 8 + (lane >> 2), qd = lane & 3;
+              uint32_t o4[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const uint32_t w0 = tr[(qd * 8 + 2 * e) * 17 + (n >> 1)], w1 = tr[(qd * 8 + 2 * e + 1) * 17 + (n >> 1)];
+                const uint32_t e0 = (n & 1) ? (w0 >> 16) : (w0 & 0xFFFFu);
+                const uint32_t e1 = (n & 1) ? (w1 >> 16) : (w1 & 0xFFFFu);
+                o4[e] = e0 | (e1 << 16);
+              }
+              *reinterpret_cast<uint4*>(dstT0 + (long long)n * a.ldt + qd * 8) = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+            }
+            return;
+          }
+          if (row_ok) {
+            __nv_bfloat16* dst = a.out + (long long)z * a.z_stride_out + (long long)m * a.ldo + nc;
+            for (int j = 0; j < 32 && nc + j < a.N; ++j) dst[j] = __float2bfloat16_rn(f[j]);
+          }
           if (nc + lane < a.N) {
             uint32_t o[16];
 #pragma unroll
