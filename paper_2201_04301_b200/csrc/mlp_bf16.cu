@@ -1206,7 +1206,8 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
   im->Bp = (int)up(B, 128);
   const long long rows = (long long)G * im->Bp;
   long long pos = 0, bpos = 0;
-  for (int l = 0; l <= L; ++l) im->ld[l] = (int)up(plan->dims[l], 8);
+  // row strides of whole 128-byte lines: a K-major row that starts inside a line costs the copies two lines per box row
+  for (int l = 0; l <= L; ++l) im->ld[l] = (int)up(plan->dims[l], 64);
   for (int l = 1; l <= L; ++l) {
     im->w_pos[l] = pos;
     pos += up((long long)plan->dims[l] * im->ld[l - 1], 64);
