@@ -102,7 +102,10 @@ def test_graph_replay_equals_plain_launches_bitwise():
 
 @pytest.mark.parametrize("name,rows,over", [("cfg1", None, {}), ("cfg2", 60000, {}),
                                             ("cfg1", 9000, dict(dims=(200,), M=12, M_G=4, batch=50, D=4)),
-                                            ("cfg1", 3000, dict(kind="quadratic", alpha=0.002, dims=(70,), batch=33))])
+                                            ("cfg1", 3000, dict(kind="quadratic", alpha=0.002, dims=(70,), batch=33)),
+                                            ("cfg1", 3200, dict(dims=(7,), M=512, M_G=16, batch=1, D=1)),       # 32 groups of 16 workers
+                                            ("cfg1", 2000, dict(dims=(256,), M=4, M_G=2, batch=97, D=2, c=0.2)),
+                                            ("cfg1", 5000, dict(dims=(33,), M=10, M_G=1, batch=300, D=7, c=3.0))])
 def test_cluster_kernel_equals_the_kernel_chain(name, rows, over):
     """Narrow models run whole iterations inside one thread-block cluster (any number per launch).  The
     result must not depend on how the iterations are cut into launches (bitwise), and must agree with the
