@@ -236,14 +236,15 @@ def run_ours(args):
         h.set_batch(w["batch"])
         h.set_theta(w["theta0"])
         n_e2e = max(3, min(args.steps, args.e2e_steps))
+        theta_host = torch.empty(g.p, dtype=torch.float32).pin_memory()   # the step's result lands here
         for _ in range(3):
             h.step_host_batch(Xb, yb)
-            h.get_theta()
+            h.get_theta(out=theta_host)
         _barrier(world)
         t_a = time.perf_counter()
         for _ in range(n_e2e):
             h.step_host_batch(Xb, yb)
-            h.get_theta()
+            h.get_theta(out=theta_host)
         torch.cuda.synchronize()
         dt = time.perf_counter() - t_a
         _barrier(world)
@@ -324,9 +325,46 @@ def run_ours(args):
                            "unit": "TFLOP/s", "frac": achieved / peaks["bf16_sustained"] if achieved else None,
                            "traffic": None, "kernel": "gradient (all GEMM launches of one iteration)",
                            "peak_source": peaks["source"] + " (sustained)", "flops_per_iteration": flops}
+    if world == 1 and not (args.no_others or args.no_e2e or args.no_cpu):   # any --no-* switch: a short / profiling run
+        # the remaining workloads of the statement, each for its own number of iterations (device-resident,
+        # same protocol: warm-up, one CUDA-event pair around gcada_step); parity cases elsewhere, here for context
+        g.close()
+        del g, w
+        torch.cuda.empty_cache()
+        out["other_workloads"] = other_workloads(args.config, dev, stream)
     if world == 1 and not args.no_cpu:
         out["cpu_baseline"] = cpu_baseline(args.config, budget_s=args.cpu_budget)
     print(json.dumps(out), flush=True)
+
+
+def other_workloads(skip, dev, stream):
+    """Iterations per second of every other named workload, timed like the main one."""
+    import torch
+    from paper_2201_04301_b200 import binding
+    from paper_2201_04301_b200.workloads import CONFIGS, make_workload
+    res = {}
+    for name in ("cfg1", "cfg2", "cfg3", "cfg4", "cfg5"):
+        if name == skip:
+            continue
+        w = make_workload(name, device=dev)
+        g = binding.from_workload(w, stream=stream, options={binding.OPT_GRAPH: 1.0})
+        K = int(CONFIGS[name]["K"])
+        g.step(max(3, min(20, K // 10)))
+        torch.cuda.synchronize()
+        l0 = g.get_launch_count()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        g.step(K)
+        e1.record(stream)
+        e1.synchronize()
+        ms = e0.elapsed_time(e1)
+        res[name] = {"value": K / (ms * 1e-3), "unit": UNIT, "steps": K, "ms_per_step": ms / K,
+                     "gpu_launches": int(g.get_launch_count() - l0),
+                     "selected_fraction": float(g.get_selection_mask(g.get_iteration() - K, K).mean())}
+        g.close()
+        del g, w
+        torch.cuda.empty_cache()
+    return res
 
 
 # ------------------------------------------------------------------------------
@@ -438,6 +476,8 @@ def main():
     ap.add_argument("--rows", type=int, default=None, help="cut the training set to this many rows")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-others", action="store_true",
+                    help="do not time the other named workloads after the main one (1 GPU; a few seconds)")
     ap.add_argument("--no-graph", action="store_true", help="plain launches instead of graph replay")
     ap.add_argument("--workers", type=int, default=None, help="override M (fewer groups, for profiling captures)")
     ap.add_argument("--rule", default="innov", choices=["innov", "ps"],

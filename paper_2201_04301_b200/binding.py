@@ -194,9 +194,17 @@ class GCada:
         self._ck(self.lib.gcada_step_host_batch(self.h, _VP(xp), _VP(yp)))
 
     # -- getters -----------------------------------------------------------
-    def get_theta(self):
-        out = np.empty(self.p, dtype=np.float32)
-        self._ck(self.lib.gcada_get_theta(self.h, _VP(out.ctypes.data), self.p))
+    def get_theta(self, out=None):
+        """theta^k as p floats on the host.  `out`: an optional float32 host buffer of p elements to fill
+        (a numpy array or a CPU torch tensor; a pinned one is copied into without a staging pass)."""
+        if out is None:
+            out = np.empty(self.p, dtype=np.float32)
+        n = out.numel() if hasattr(out, "numel") else out.size
+        contiguous = out.is_contiguous() if hasattr(out, "is_contiguous") else out.flags["C_CONTIGUOUS"]
+        if n != self.p or "float32" not in str(out.dtype) or not contiguous or getattr(out, "is_cuda", False):
+            raise ValueError("get_theta: out must be a contiguous host buffer of p = %d float32 values" % self.p)
+        ptr = out.data_ptr() if hasattr(out, "data_ptr") else out.ctypes.data
+        self._ck(self.lib.gcada_get_theta(self.h, _VP(ptr), self.p))
         return out
 
     def get_selection_mask(self, first_iter, n_iters):
