@@ -14,7 +14,9 @@
 //   * warps are combined inside a CTA through shared memory, CTAs through
 //     distributed shared memory after ONE hardware cluster barrier per
 //     iteration (the exchange buffer is double-buffered, so no second barrier
-//     is needed), always in a fixed order;
+//     is needed), always in a fixed order; a CTA works on a contiguous range
+//     of batches, so a group's sum is read only from the CTAs that hold a
+//     share of it;
 //   * every CTA then holds every group's gradient and innovation norm and
 //     redundantly evaluates Eq. (9), the age rule, the computing times and
 //     wall-clock (Section II-B), the aggregate (Eq. 3) and Eq. (8a)-(8c) on
@@ -177,9 +179,15 @@ __global__ void __launch_bounds__(LC_THREADS, 1) linear_cluster_kernel(const Par
 
   const int nb_g = (B + RR - 1) / RR;          // batches of RR rows per group
   const int n_batches = G * nb_g;
-  // batches are dealt warp-major, so that the last warp of every CTA has the fewest (it also forms the
-  // right side of Eq. (9) while the others fetch their first rows)
-  const int wg = warp * C + cta, nw_tot = C * LC_WARPS;
+  // every CTA takes a contiguous range of batches, hence of groups: only the CTAs that worked on a group
+  // hold a partial sum of it, and the exchange below reads only those.  Inside the CTA batches are dealt
+  // warp-major, so that the last warp has the fewest (it also forms the right side of Eq. (9) while the
+  // others fetch their first rows)
+  const int bpc = (n_batches + C - 1) / C;
+  const int b_lo = cta * bpc < n_batches ? cta * bpc : n_batches, b_hi = b_lo + bpc < n_batches ? b_lo + bpc : n_batches;
+  const int wg = b_lo + warp, nw_tot = LC_WARPS;
+  // (group, point, column) elements of this CTA's groups: [e_lo, e_hi)
+  const int e_lo = b_lo < b_hi ? (b_lo / nb_g) * 2 * pp : 0, e_hi = b_lo < b_hi ? ((b_hi - 1) / nb_g + 1) * 2 * pp : 0;
   // ring positions are kept as small counters (no 64-bit division inside the loop)
   int kslot = (int)(st.k % ring), dslot = (int)(st.k % D), hslot = (int)(st.k % P.hist_cap);
   // computing times of the first iteration (those of iteration k+1 are drawn while iteration k updates)
@@ -192,7 +200,7 @@ __global__ void __launch_bounds__(LC_THREADS, 1) linear_cluster_kernel(const Par
     const int kfill = k < D ? (int)k : D;       // how many earlier iterates exist, up to D
     const float* theta_k = S.ring + kslot * pp;
     float* accw_w = S.accw + (size_t)warp * gp2;
-    for (int e = lane; e < gp2; e += 32) accw_w[e] = 0.f;  // groups this warp does not visit contribute zero
+    for (int e = e_lo + lane; e < e_hi; e += 32) accw_w[e] = 0.f;  // groups this warp does not visit contribute zero
     __syncwarp();
 
     // the last warp forms the right side of Eq. (9) (it depends on earlier iterations only)
@@ -234,12 +242,12 @@ __global__ void __launch_bounds__(LC_THREADS, 1) linear_cluster_kernel(const Par
     };
     float xc[RR][CPL], yc = 0.f;
     int b = wg;
-    if (b < n_batches) fetch(b, yc, xc);
-    while (b < n_batches) {
+    if (b < b_hi) fetch(b, yc, xc);
+    while (b < b_hi) {
       const int bn = b + nw_tot;
       float xn[RR][CPL], yn = 0.f;
       constexpr bool PREFETCH = RR * CPL <= 16;  // wider rows would not fit two batches in registers
-      if (PREFETCH && bn < n_batches) fetch(bn, yn, xn);
+      if (PREFETCH && bn < b_hi) fetch(bn, yn, xn);
       const int g = b / nb_g, rb = (b - g * nb_g) * RR;
       if (g != cur_g) {
         if (cur_g >= 0) {
@@ -293,7 +301,7 @@ __global__ void __launch_bounds__(LC_THREADS, 1) linear_cluster_kernel(const Par
           acc1[i] += e * xc[r][i];
         }
       }
-      if (!PREFETCH && bn < n_batches) fetch(bn, yn, xn);
+      if (!PREFETCH && bn < b_hi) fetch(bn, yn, xn);
       b = bn;
       yc = yn;
 #pragma unroll
@@ -313,7 +321,7 @@ __global__ void __launch_bounds__(LC_THREADS, 1) linear_cluster_kernel(const Par
 
     // ---- warps -> CTA partial (fixed order), published in this iteration's exchange buffer
     float* part = S.part + (size_t)(it & 1) * gp2;
-    for (int e = tid; e < gp2; e += LC_THREADS) {
+    for (int e = e_lo + tid; e < e_hi; e += LC_THREADS) {
       float s = 0.f;
 #pragma unroll
       for (int w = 0; w < LC_WARPS; ++w) s += S.accw[(size_t)w * gp2 + e];
@@ -325,13 +333,14 @@ __global__ void __launch_bounds__(LC_THREADS, 1) linear_cluster_kernel(const Par
     // thread; the 32 elements of a warp lie in one (group, point) row, so the warp also forms its share of
     // the squared innovation norm
     for (int e = tid; e < gp2; e += LC_THREADS) {
+      const int gq = e / pp, c = e - gq * pp, g = gq >> 1;
+      const int r_lo = (g * nb_g) / bpc, r_hi = ((g + 1) * nb_g - 1) / bpc;  // the CTAs that worked on group g
       float v[16];  // all remote loads in flight before the first add
 #pragma unroll
-      for (int r = 0; r < 16; ++r) v[r] = r < C ? cluster.map_shared_rank(part, r)[e] : 0.f;
+      for (int j = 0; j < 16; ++j) v[j] = r_lo + j <= r_hi ? cluster.map_shared_rank(part, r_lo + j)[e] : 0.f;
       float s = 0.f;
 #pragma unroll
-      for (int r = 0; r < 16; ++r) s += v[r];
-      const int gq = e / pp, c = e - gq * pp, g = gq >> 1;
+      for (int j = 0; j < 16; ++j) s += v[j];
       if (gq & 1) {
         S.innov[g * pp + c] = s;
         const double nrm = warp_sum((double)s * (double)s);
