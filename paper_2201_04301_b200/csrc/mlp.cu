@@ -9,11 +9,15 @@
 //
 // theta layout: for l = 1..L, W_l (n_l rows of n_{l-1}) then b_l (n_l).
 // Batch index z = q * G + g (q = point, g = group).
+#include <cooperative_groups.h>
+
 #include "mlp.h"
 
 #include "mlp_bf16.h"
 
 namespace gcada {
+
+namespace cg = cooperative_groups;
 
 namespace {
 
@@ -75,18 +79,27 @@ struct GemmArgs {
   long long bias_off;
   int relu;
   const float* mask;  // multiply by (mask(m, n) > 0); same indexing as C
+  int split;          // CTAs (one thread-block cluster along x) that share an output tile, each summing over
+  int kchunk;         // kchunk values of k (a multiple of TK); 1: no split
 };
 
 constexpr int TM = 64, TN = 64, TK = 16;
 
+// 64 x 64 output tile per CTA, 4 x 4 per thread; the next K step's operands are fetched into registers while
+// the current one is multiplied.  A product with few tiles and a long K (the first layer of a small network)
+// is split over the CTAs of one thread-block cluster: CTA r sums k in [r kchunk, (r+1) kchunk), the partial
+// tiles meet in CTA 0 through distributed shared memory in rank order (fixed, so results are reproducible).
 __global__ void __launch_bounds__(256) mlp_sgemm_kernel(const Params P, const GemmArgs a) {
   __shared__ float As[TK][TM + 4];
   __shared__ float Bs[TK][TN + 4];
+  __shared__ float4 red[4][256];  // this CTA's partial tile (split products only)
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   const int z = blockIdx.z, q = z / P.G, g = z - q * P.G;
   // rule PS (the selection is already known): selected groups at theta^k only
-  if (P.skip_unselected && (q != 0 || !P.mask_cur[g])) return;
-  const int m0 = blockIdx.y * TM, n0 = blockIdx.x * TN;
+  if (P.skip_unselected && (q != 0 || !P.mask_cur[g])) return;  // (the same for every CTA of a cluster)
+  const int rank = a.split > 1 ? (int)(blockIdx.x % a.split) : 0;
+  const int m0 = blockIdx.y * TM, n0 = (a.split > 1 ? (int)(blockIdx.x / a.split) : (int)blockIdx.x) * TN;
+  const int k_lo = rank * a.kchunk, k_hi = a.split > 1 ? (k_lo + a.kchunk < a.K ? k_lo + a.kchunk : a.K) : a.K;
   const long long k_it = P.st->k;
   const float* Ab = a.A.ring ? ring_ptr(P, g, q, k_it) + a.A.off : a.A.base + g * a.A.zg + q * a.A.zq;
   const float* Bb = a.Bm.ring ? ring_ptr(P, g, q, k_it) + a.Bm.off : a.Bm.base + g * a.Bm.zg + q * a.Bm.zq;
@@ -96,32 +109,45 @@ __global__ void __launch_bounds__(256) mlp_sgemm_kernel(const Params P, const Ge
 #pragma unroll
     for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
 
-  for (int k0 = 0; k0 < a.K; k0 += TK) {
+  // the four A and four B elements this thread moves per K step (the contiguous index runs fastest over threads)
+  int a_mm[4], a_kk[4], b_nn[4], b_kk[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int e = tid + 256 * i;
+    if (a.A.cs == 1) {
+      a_kk[i] = e & (TK - 1);
+      a_mm[i] = e >> 4;
+    } else {
+      a_mm[i] = e & (TM - 1);
+      a_kk[i] = e >> 6;
+    }
+    if (a.Bm.cs == 1) {
+      b_nn[i] = e & (TN - 1);
+      b_kk[i] = e >> 6;
+    } else {
+      b_kk[i] = e & (TK - 1);
+      b_nn[i] = e >> 4;
+    }
+  }
+  float ra[4], rb[4];
+  auto fetch = [&](int k0) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      const int e = tid + 256 * i;
-      int mm, kk;
-      if (a.A.cs == 1) {
-        kk = e & (TK - 1);
-        mm = e >> 4;
-      } else {
-        mm = e & (TM - 1);
-        kk = e >> 6;
-      }
-      const int m = m0 + mm, kx = k0 + kk;
-      As[kk][mm] = (m < a.M && kx < a.K) ? Ab[m * a.A.rs + kx * a.A.cs] : 0.f;
-      int nn, kb;
-      if (a.Bm.cs == 1) {
-        nn = e & (TN - 1);
-        kb = e >> 6;
-      } else {
-        kb = e & (TK - 1);
-        nn = e >> 4;
-      }
-      const int n = n0 + nn, ky = k0 + kb;
-      Bs[kb][nn] = (n < a.N && ky < a.K) ? Bb[ky * a.Bm.rs + n * a.Bm.cs] : 0.f;
+      const int m = m0 + a_mm[i], kx = k0 + a_kk[i];
+      ra[i] = (m < a.M && kx < k_hi) ? Ab[m * a.A.rs + kx * a.A.cs] : 0.f;
+      const int n = n0 + b_nn[i], ky = k0 + b_kk[i];
+      rb[i] = (n < a.N && ky < k_hi) ? Bb[ky * a.Bm.rs + n * a.Bm.cs] : 0.f;
+    }
+  };
+  if (k_lo < k_hi) fetch(k_lo);
+  for (int k0 = k_lo; k0 < k_hi; k0 += TK) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      As[a_kk[i]][a_mm[i]] = ra[i];
+      Bs[b_kk[i]][b_nn[i]] = rb[i];
     }
     __syncthreads();
+    if (k0 + TK < k_hi) fetch(k0 + TK);
 #pragma unroll
     for (int kk = 0; kk < TK; ++kk) {
       float av[4], bv[4];
@@ -135,6 +161,28 @@ __global__ void __launch_bounds__(256) mlp_sgemm_kernel(const Params P, const Ge
         for (int j = 0; j < 4; ++j) acc[i][j] += av[i] * bv[j];
     }
     __syncthreads();
+  }
+
+  if (a.split > 1) {
+    cg::cluster_group cluster = cg::this_cluster();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) red[i][tid] = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+    cluster.sync();
+    if (rank == 0) {
+      for (int r = 1; r < a.split; ++r) {
+        const float4* rr = cluster.map_shared_rank(&red[0][0], r);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float4 v = rr[i * 256 + tid];
+          acc[i][0] += v.x;
+          acc[i][1] += v.y;
+          acc[i][2] += v.z;
+          acc[i][3] += v.w;
+        }
+      }
+    }
+    cluster.sync();  // no CTA leaves while CTA 0 may still read its tile
+    if (rank != 0) return;
   }
 
   float* Cb;
@@ -158,6 +206,46 @@ __global__ void __launch_bounds__(256) mlp_sgemm_kernel(const Params P, const Ge
       if (Mb) v = Mb[m * a.c_rs + n] > 0.f ? v : 0.f;
       Cb[m * a.c_rs + n] = v;
     }
+  }
+}
+
+// Products with at most 16 output columns whose operands both run along k (the class scores of a small
+// network): a warp per output row, lanes stride over k, one shuffle reduction per column.
+constexpr int ROWDOT_MAX_N = 16;
+__global__ void __launch_bounds__(256) mlp_rowdot_kernel(const Params P, const GemmArgs a) {
+  const int w = (int)((blockIdx.x * 256 + threadIdx.x) >> 5), lane = threadIdx.x & 31;
+  if (w >= 2 * P.G * a.M) return;
+  const int z = w / a.M, m = w - z * a.M, q = z / P.G, g = z - q * P.G;
+  if (P.skip_unselected && (q != 0 || !P.mask_cur[g])) return;
+  const long long k_it = P.st->k;
+  const float* Ab = (a.A.ring ? ring_ptr(P, g, q, k_it) + a.A.off : a.A.base + g * a.A.zg + q * a.A.zq) + m * a.A.rs;
+  const float* Bb = a.Bm.ring ? ring_ptr(P, g, q, k_it) + a.Bm.off : a.Bm.base + g * a.Bm.zg + q * a.Bm.zq;
+  float part[ROWDOT_MAX_N];
+#pragma unroll
+  for (int n = 0; n < ROWDOT_MAX_N; ++n) part[n] = 0.f;
+  for (int k = lane; k < a.K; k += 32) {
+    const float av = Ab[k];
+#pragma unroll
+    for (int n = 0; n < ROWDOT_MAX_N; ++n)
+      if (n < a.N) part[n] += av * Bb[k + n * a.Bm.cs];
+  }
+  float mine = 0.f;
+#pragma unroll
+  for (int n = 0; n < ROWDOT_MAX_N; ++n) {
+    if (n < a.N) {  // (uniform)
+      float v = part[n];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+      if (lane == n) mine = v;
+    }
+  }
+  if (lane < a.N) {
+    float v = mine;
+    if (a.bias) v += (ring_ptr(P, g, q, k_it) + a.bias_off)[lane];
+    if (a.relu) v = fmaxf(v, 0.f);
+    const long long o = g * a.c_zg + q * a.c_zq + m * a.c_rs + lane;
+    if (a.mask) v = a.mask[o] > 0.f ? v : 0.f;
+    a.C[o] = v;
   }
 }
 
@@ -207,14 +295,55 @@ __global__ void __launch_bounds__(256) mlp_bias_grad_kernel(const Params P, cons
   if (P.skip_unselected && (q != 0 || !P.mask_cur[g])) return;
   const float* src = a.dz[l] + ((long long)z * P.B) * a.n[l] + n;
   float s = 0.f;
-  for (int r = 0; r < P.B; ++r) s += src[(long long)r * a.n[l]];
+  int r = 0;
+  for (; r + 8 <= P.B; r += 8) {  // eight loads in flight, added in row order
+    float v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) v[u] = src[(long long)(r + u) * a.n[l]];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) s += v[u];
+  }
+  for (; r < P.B; ++r) s += src[(long long)r * a.n[l]];
   ((q == 0 ? (P.skip_unselected ? last_row(P, g) : fresh_row(P, g)) : P.stale + (long long)g * P.p_pad) + a.b_off[l])[n] = s;
 }
 
-cudaError_t launch_gemm(const Params& P, const GemmArgs& a, cudaStream_t st) {
-  dim3 grid((a.N + TN - 1) / TN, (a.M + TM - 1) / TM, 2 * P.G);
-  mlp_sgemm_kernel<<<grid, 256, 0, st>>>(P, a);
-  return cudaGetLastError();
+cudaError_t launch_gemm(const Params& P, GemmArgs a, int sm_count, cudaStream_t st) {
+  if (a.N <= ROWDOT_MAX_N && a.A.cs == 1 && a.Bm.rs == 1 && !a.c_grad) {
+    const long long warps = 2LL * P.G * a.M;
+    mlp_rowdot_kernel<<<(unsigned)((warps * 32 + 255) / 256), 256, 0, st>>>(P, a);
+    return cudaGetLastError();
+  }
+  const int gx = (a.N + TN - 1) / TN, gy = (a.M + TM - 1) / TM;
+  const long long tiles = (long long)gx * gy * 2 * P.G;
+  // few tiles and a long K: split K over a cluster so that about two CTAs per SM are busy
+  a.split = 1;
+  a.kchunk = a.K;
+  if (a.K >= 16 * TK && tiles < sm_count) {
+    long long s = 2LL * sm_count / tiles;
+    if (s > 8) s = 8;
+    if (s > a.K / (4 * TK)) s = a.K / (4 * TK);
+    if (s > 1) {
+      a.kchunk = (int)(((a.K + s - 1) / s + TK - 1) / TK * TK);
+      a.split = (a.K + a.kchunk - 1) / a.kchunk;
+    }
+  }
+  if (a.split == 1) {
+    mlp_sgemm_kernel<<<dim3(gx, gy, 2 * P.G), 256, 0, st>>>(P, a);
+    return cudaGetLastError();
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(gx * a.split, gy, 2 * P.G);
+  cfg.blockDim = dim3(256);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = a.split;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, mlp_sgemm_kernel, P, a);
 }
 
 }  // namespace
@@ -304,7 +433,7 @@ cudaError_t launch_grad_mlp(const Params& P, const MlpPlan& pl, cudaStream_t st,
     a.bias = 1;
     a.bias_off = pl.b_off[l];
     a.relu = l < L;
-    if ((e = launch_gemm(P, a, st)) != cudaSuccess) return e;
+    if ((e = launch_gemm(P, a, pl.sm_count, st)) != cudaSuccess) return e;
     ++n;
   }
   mlp_softmax_grad_kernel<<<(unsigned)((2 * rows * 32 + 255) / 256), 256, 0, st>>>(P, pl.act[L], pl.yb, pl.dz[L],
@@ -326,7 +455,7 @@ cudaError_t launch_grad_mlp(const Params& P, const MlpPlan& pl, cudaStream_t st,
     w.c_grad = 1;
     w.c_off = pl.w_off[l];
     w.c_rs = ni;
-    if ((e = launch_gemm(P, w, st)) != cudaSuccess) return e;
+    if ((e = launch_gemm(P, w, pl.sm_count, st)) != cudaSuccess) return e;
     ++n;
     if (l > 1) {
       GemmArgs d{};  // dz_{l-1} = (dz_l W_l) masked by a_{l-1} > 0
@@ -340,7 +469,7 @@ cudaError_t launch_grad_mlp(const Params& P, const MlpPlan& pl, cudaStream_t st,
       d.c_zq = rows * ni;
       d.c_rs = ni;
       d.mask = pl.act[l - 1];
-      if ((e = launch_gemm(P, d, st)) != cudaSuccess) return e;
+      if ((e = launch_gemm(P, d, pl.sm_count, st)) != cudaSuccess) return e;
       ++n;
     }
   }
