@@ -83,7 +83,8 @@ struct GemmArgs {
   int kchunk;         // kchunk values of k (a multiple of TK); 1: no split
 };
 
-constexpr int TM = 64, TN = 64, TK = 16;
+constexpr int TM = 64, TN = 64, TK = 32;
+constexpr int EPT = TM * TK / 256;  // elements of each operand tile a thread moves per K step
 
 // 64 x 64 output tile per CTA, 4 x 4 per thread; the next K step's operands are fetched into registers while
 // the current one is multiplied.  A product with few tiles and a long K (the first layer of a small network)
@@ -110,13 +111,14 @@ __global__ void __launch_bounds__(256) mlp_sgemm_kernel(const Params P, const Ge
     for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
 
   // the four A and four B elements this thread moves per K step (the contiguous index runs fastest over threads)
-  int a_mm[4], a_kk[4], b_nn[4], b_kk[4];
+  static_assert(TM == 64 && TN == 64 && TK == 32, "index arithmetic below");
+  int a_mm[EPT], a_kk[EPT], b_nn[EPT], b_kk[EPT];
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
+  for (int i = 0; i < EPT; ++i) {
     const int e = tid + 256 * i;
     if (a.A.cs == 1) {
       a_kk[i] = e & (TK - 1);
-      a_mm[i] = e >> 4;
+      a_mm[i] = e >> 5;
     } else {
       a_mm[i] = e & (TM - 1);
       a_kk[i] = e >> 6;
@@ -126,13 +128,13 @@ __global__ void __launch_bounds__(256) mlp_sgemm_kernel(const Params P, const Ge
       b_kk[i] = e >> 6;
     } else {
       b_kk[i] = e & (TK - 1);
-      b_nn[i] = e >> 4;
+      b_nn[i] = e >> 5;
     }
   }
-  float ra[4], rb[4];
+  float ra[EPT], rb[EPT];
   auto fetch = [&](int k0) {
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < EPT; ++i) {
       const int m = m0 + a_mm[i], kx = k0 + a_kk[i];
       ra[i] = (m < a.M && kx < k_hi) ? Ab[m * a.A.rs + kx * a.A.cs] : 0.f;
       const int n = n0 + b_nn[i], ky = k0 + b_kk[i];
@@ -142,7 +144,7 @@ __global__ void __launch_bounds__(256) mlp_sgemm_kernel(const Params P, const Ge
   if (k_lo < k_hi) fetch(k_lo);
   for (int k0 = k_lo; k0 < k_hi; k0 += TK) {
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < EPT; ++i) {
       As[a_kk[i]][a_mm[i]] = ra[i];
       Bs[b_kk[i]][b_nn[i]] = rb[i];
     }
@@ -210,24 +212,45 @@ __global__ void __launch_bounds__(256) mlp_sgemm_kernel(const Params P, const Ge
 }
 
 // Products with at most 16 output columns whose operands both run along k (the class scores of a small
-// network): a warp per output row, lanes stride over k, one shuffle reduction per column.
+// network): the CTA stages the N x K weights of its (point, group) in shared memory, then a warp per output
+// row: lanes stride over k, one shuffle reduction per column.  Grid (ceil(M / 8), 2 G).
 constexpr int ROWDOT_MAX_N = 16;
 __global__ void __launch_bounds__(256) mlp_rowdot_kernel(const Params P, const GemmArgs a) {
-  const int w = (int)((blockIdx.x * 256 + threadIdx.x) >> 5), lane = threadIdx.x & 31;
-  if (w >= 2 * P.G * a.M) return;
-  const int z = w / a.M, m = w - z * a.M, q = z / P.G, g = z - q * P.G;
+  extern __shared__ float wsm[];  // [N][K]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int z = blockIdx.y, q = z / P.G, g = z - q * P.G;
   if (P.skip_unselected && (q != 0 || !P.mask_cur[g])) return;
   const long long k_it = P.st->k;
-  const float* Ab = (a.A.ring ? ring_ptr(P, g, q, k_it) + a.A.off : a.A.base + g * a.A.zg + q * a.A.zq) + m * a.A.rs;
   const float* Bb = a.Bm.ring ? ring_ptr(P, g, q, k_it) + a.Bm.off : a.Bm.base + g * a.Bm.zg + q * a.Bm.zq;
+  for (int e = threadIdx.x; e < a.N * a.K; e += 256) {
+    const int n = e / a.K, k = e - n * a.K;
+    wsm[e] = Bb[k + n * a.Bm.cs];
+  }
+  const int m = blockIdx.x * 8 + warp;
+  // the row's share of this lane, up to 8 values at a time, all loads in flight before the weights are needed
+  const float* Ab = (a.A.ring ? ring_ptr(P, g, q, k_it) + a.A.off : a.A.base + g * a.A.zg + q * a.A.zq) + (m < a.M ? m : 0) * a.A.rs;
   float part[ROWDOT_MAX_N];
 #pragma unroll
   for (int n = 0; n < ROWDOT_MAX_N; ++n) part[n] = 0.f;
-  for (int k = lane; k < a.K; k += 32) {
-    const float av = Ab[k];
+  float av[8];
 #pragma unroll
-    for (int n = 0; n < ROWDOT_MAX_N; ++n)
-      if (n < a.N) part[n] += av * Bb[k + n * a.Bm.cs];
+  for (int u = 0; u < 8; ++u) av[u] = lane + 32 * u < a.K ? Ab[lane + 32 * u] : 0.f;
+  __syncthreads();
+  for (int k0 = 0; k0 < a.K; k0 += 256) {
+    float nx[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) nx[u] = k0 + 256 + lane + 32 * u < a.K ? Ab[k0 + 256 + lane + 32 * u] : 0.f;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int k = k0 + lane + 32 * u;
+      if (k < a.K) {
+#pragma unroll
+        for (int n = 0; n < ROWDOT_MAX_N; ++n)
+          if (n < a.N) part[n] += av[u] * wsm[n * a.K + k];
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) av[u] = nx[u];
   }
   float mine = 0.f;
 #pragma unroll
@@ -239,7 +262,7 @@ __global__ void __launch_bounds__(256) mlp_rowdot_kernel(const Params P, const G
       if (lane == n) mine = v;
     }
   }
-  if (lane < a.N) {
+  if (m < a.M && lane < a.N) {
     float v = mine;
     if (a.bias) v += (ring_ptr(P, g, q, k_it) + a.bias_off)[lane];
     if (a.relu) v = fmaxf(v, 0.f);
@@ -308,9 +331,8 @@ __global__ void __launch_bounds__(256) mlp_bias_grad_kernel(const Params P, cons
 }
 
 cudaError_t launch_gemm(const Params& P, GemmArgs a, int sm_count, cudaStream_t st) {
-  if (a.N <= ROWDOT_MAX_N && a.A.cs == 1 && a.Bm.rs == 1 && !a.c_grad) {
-    const long long warps = 2LL * P.G * a.M;
-    mlp_rowdot_kernel<<<(unsigned)((warps * 32 + 255) / 256), 256, 0, st>>>(P, a);
+  if (a.N <= ROWDOT_MAX_N && a.A.cs == 1 && a.Bm.rs == 1 && !a.c_grad && (size_t)a.N * a.K * sizeof(float) <= 48 * 1024) {
+    mlp_rowdot_kernel<<<dim3((a.M + 7) / 8, 2 * P.G), 256, (size_t)a.N * a.K * sizeof(float), st>>>(P, a);
     return cudaGetLastError();
   }
   const int gx = (a.N + TN - 1) / TN, gy = (a.M + TM - 1) / TM;
@@ -318,10 +340,10 @@ cudaError_t launch_gemm(const Params& P, GemmArgs a, int sm_count, cudaStream_t 
   // few tiles and a long K: split K over a cluster so that about two CTAs per SM are busy
   a.split = 1;
   a.kchunk = a.K;
-  if (a.K >= 16 * TK && tiles < sm_count) {
+  if (a.K >= 8 * TK && tiles < sm_count) {
     long long s = 2LL * sm_count / tiles;
     if (s > 8) s = 8;
-    if (s > a.K / (4 * TK)) s = a.K / (4 * TK);
+    if (s > a.K / (2 * TK)) s = a.K / (2 * TK);
     if (s > 1) {
       a.kchunk = (int)(((a.K + s - 1) / s + TK - 1) / TK * TK);
       a.split = (a.K + a.kchunk - 1) / a.kchunk;
