@@ -86,14 +86,16 @@ struct GemmArgs {
 constexpr int TM = 64, TN = 64, TK = 32;
 constexpr int EPT = TM * TK / 256;  // elements of each operand tile a thread moves per K step
 
-// 64 x 64 output tile per CTA, 4 x 4 per thread; the next K step's operands are fetched into registers while
-// the current one is multiplied.  A product with few tiles and a long K (the first layer of a small network)
-// is split over the CTAs of one thread-block cluster: CTA r sums k in [r kchunk, (r+1) kchunk), the partial
-// tiles meet in CTA 0 through distributed shared memory in rank order (fixed, so results are reproducible).
+// 64 x 64 output tile per CTA, 4 x 4 per thread, K in steps of 32 through two shared-memory buffers: the next
+// step's operands are fetched into registers before the current step is multiplied and stored into the other
+// buffer after it, one block barrier per step.  A product with few tiles and a long K (the first layer of a
+// small network) is split over the CTAs of one thread-block cluster: CTA r sums k in [r kchunk, (r+1) kchunk),
+// the partial tiles meet in CTA 0 through distributed shared memory in rank order (fixed, so results are
+// reproducible).
 __global__ void __launch_bounds__(256) mlp_sgemm_kernel(const Params P, const GemmArgs a) {
-  __shared__ float As[TK][TM + 4];
-  __shared__ float Bs[TK][TN + 4];
-  __shared__ float4 red[4][256];  // this CTA's partial tile (split products only)
+  __shared__ __align__(16) float sm[2][2][TK][TM + 4];  // [buffer][A, B][k][m or n]
+  float4* red = reinterpret_cast<float4*>(&sm[0][0][0][0]);  // [4][256]: this CTA's partial tile (split products), after the loop
+  static_assert(sizeof(sm) >= 4 * 256 * sizeof(float4), "the partial tile reuses the operand buffers");
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   const int z = blockIdx.z, q = z / P.G, g = z - q * P.G;
   // rule PS (the selection is already known): selected groups at theta^k only
@@ -110,15 +112,18 @@ __global__ void __launch_bounds__(256) mlp_sgemm_kernel(const Params P, const Ge
 #pragma unroll
     for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
 
-  // the four A and four B elements this thread moves per K step (the contiguous index runs fastest over threads)
+  // The eight A and eight B elements this thread moves per K step.  An operand that runs along m (or n) is
+  // read and stored 32 consecutive m per warp.  One that runs along k is stored transposed: a warp takes
+  // 8 consecutive k of 4 rows, which are 32 different banks under the row pitch of 68 floats.
   static_assert(TM == 64 && TN == 64 && TK == 32, "index arithmetic below");
   int a_mm[EPT], a_kk[EPT], b_nn[EPT], b_kk[EPT];
 #pragma unroll
   for (int i = 0; i < EPT; ++i) {
     const int e = tid + 256 * i;
+    const int t_k = (e & 7) | (((e >> 5) & 3) << 3), t_m = ((e >> 3) & 3) | ((e >> 7) << 2);
     if (a.A.cs == 1) {
-      a_kk[i] = e & (TK - 1);
-      a_mm[i] = e >> 5;
+      a_kk[i] = t_k;
+      a_mm[i] = t_m;
     } else {
       a_mm[i] = e & (TM - 1);
       a_kk[i] = e >> 6;
@@ -127,8 +132,8 @@ __global__ void __launch_bounds__(256) mlp_sgemm_kernel(const Params P, const Ge
       b_nn[i] = e & (TN - 1);
       b_kk[i] = e >> 6;
     } else {
-      b_kk[i] = e & (TK - 1);
-      b_nn[i] = e >> 5;
+      b_kk[i] = t_k;
+      b_nn[i] = t_m;
     }
   }
   float ra[EPT], rb[EPT];
@@ -141,38 +146,44 @@ __global__ void __launch_bounds__(256) mlp_sgemm_kernel(const Params P, const Ge
       rb[i] = (n < a.N && ky < k_hi) ? Bb[ky * a.Bm.rs + n * a.Bm.cs] : 0.f;
     }
   };
-  if (k_lo < k_hi) fetch(k_lo);
-  for (int k0 = k_lo; k0 < k_hi; k0 += TK) {
+  auto stash = [&](int buf) {
 #pragma unroll
     for (int i = 0; i < EPT; ++i) {
-      As[a_kk[i]][a_mm[i]] = ra[i];
-      Bs[b_kk[i]][b_nn[i]] = rb[i];
+      sm[buf][0][a_kk[i]][a_mm[i]] = ra[i];
+      sm[buf][1][b_kk[i]][b_nn[i]] = rb[i];
     }
-    __syncthreads();
-    if (k0 + TK < k_hi) fetch(k0 + TK);
+  };
+  if (k_lo < k_hi) {
+    fetch(k_lo);
+    stash(0);
+  }
+  __syncthreads();
+  int buf = 0;
+  for (int k0 = k_lo; k0 < k_hi; k0 += TK, buf ^= 1) {
+    const bool more = k0 + TK < k_hi;
+    if (more) fetch(k0 + TK);
 #pragma unroll
     for (int kk = 0; kk < TK; ++kk) {
-      float av[4], bv[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) av[i] = As[kk][ty * 4 + i];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) bv[j] = Bs[kk][tx * 4 + j];
+      const float4 a4 = *reinterpret_cast<const float4*>(&sm[buf][0][kk][ty * 4]);
+      const float4 b4 = *reinterpret_cast<const float4*>(&sm[buf][1][kk][tx * 4]);
+      const float av[4] = {a4.x, a4.y, a4.z, a4.w}, bv[4] = {b4.x, b4.y, b4.z, b4.w};
 #pragma unroll
       for (int i = 0; i < 4; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] += av[i] * bv[j];
     }
+    if (more) stash(buf ^ 1);  // (last read before the barrier that ended the previous step)
     __syncthreads();
   }
 
   if (a.split > 1) {
     cg::cluster_group cluster = cg::this_cluster();
 #pragma unroll
-    for (int i = 0; i < 4; ++i) red[i][tid] = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+    for (int i = 0; i < 4; ++i) red[i * 256 + tid] = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
     cluster.sync();
     if (rank == 0) {
       for (int r = 1; r < a.split; ++r) {
-        const float4* rr = cluster.map_shared_rank(&red[0][0], r);
+        const float4* rr = cluster.map_shared_rank(red, r);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const float4 v = rr[i * 256 + tid];
