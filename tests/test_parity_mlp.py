@@ -22,6 +22,9 @@ def test_cfg4_teacher_forced():
     ((5, 3), 7, 2, 1, 2),                 # a single affine layer (softmax regression)
     ((33, 17, 9, 4), 10, 6, 2, 3),        # three layers, odd sizes
     ((70, 130, 65), 100, 3, 3, 4),        # sizes that straddle the 64-wide tiles, G = 1
+    ((300, 70, 5), 33, 6, 2, 2),          # first layer split over a cluster of 4 (K shares 96, 96, 96, 12)
+    ((600, 12), 20, 4, 2, 2),             # one layer of 12 outputs: warp-per-row product, K in three chunks
+    ((520, 64, 40, 16), 64, 2, 1, 3),     # split of 8, a 16-column output layer
 ])
 def test_odd_architectures(dims, batch, M, M_G, D):
     G = M // M_G
