@@ -119,6 +119,7 @@ void drop_graphs(gcada_ctx* ctx) {
 
 void free_all(gcada_ctx* ctx) {
   drop_graphs(ctx);
+  mlp_plan_release(&ctx->mlp);
   for (cudaEvent_t e : ctx->events)
     if (e) cudaEventDestroy(e);
   ctx->events.clear();

@@ -425,7 +425,30 @@ cudaError_t mlp_plan_create(const std::vector<int>& dims, int compute, int G, in
   }
   plan->launches_per_iter = 3 * L + 2;
   plan->skip_launches = 3 * L + 2;  // the same kernels; blocks of unselected groups and of the stale point exit at once
+  if (L >= 2) {
+    if ((e = cudaStreamCreateWithFlags(&plan->side, cudaStreamNonBlocking)) != cudaSuccess) return e;
+    for (int l = 1; l <= L; ++l)
+      if ((e = cudaEventCreateWithFlags(&plan->ev_dz[l], cudaEventDisableTiming)) != cudaSuccess) return e;
+    if ((e = cudaEventCreateWithFlags(&plan->ev_join, cudaEventDisableTiming)) != cudaSuccess) return e;
+  }
   return cudaSuccess;
+}
+
+void mlp_plan_release(MlpPlan* plan) {
+  if (plan->side) {
+    cudaStreamSynchronize(plan->side);
+    cudaStreamDestroy(plan->side);
+    plan->side = nullptr;
+  }
+  for (int l = 0; l <= MLP_MAX_LAYERS; ++l)
+    if (plan->ev_dz[l]) {
+      cudaEventDestroy(plan->ev_dz[l]);
+      plan->ev_dz[l] = nullptr;
+    }
+  if (plan->ev_join) {
+    cudaEventDestroy(plan->ev_join);
+    plan->ev_join = nullptr;
+  }
 }
 
 cudaError_t launch_grad_mlp_post(const Params& P, const MlpPlan& pl, cudaStream_t st, int* n_launches) {
@@ -474,7 +497,13 @@ cudaError_t launch_grad_mlp(const Params& P, const MlpPlan& pl, cudaStream_t st,
                                                                                   pl.dims[L]);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   ++n;
-  // backward
+  // backward.  Main stream: the back-propagation chain dz_L -> ... -> dz_1, then dW_1.  Second stream (when
+  // there is more than one layer): dW_l for l >= 2 as soon as dz_l is there, then all bias gradients.
+  cudaStream_t s2 = pl.side ? pl.side : st;
+  if (pl.side) {
+    if ((e = cudaEventRecord(pl.ev_dz[L], st)) != cudaSuccess) return e;
+    if ((e = cudaStreamWaitEvent(pl.side, pl.ev_dz[L], 0)) != cudaSuccess) return e;
+  }
   for (int l = L; l >= 1; --l) {
     const int ni = pl.dims[l - 1], no = pl.dims[l];
     GemmArgs w{};  // dW_l = dz_l^T a_{l-1}
@@ -489,7 +518,7 @@ cudaError_t launch_grad_mlp(const Params& P, const MlpPlan& pl, cudaStream_t st,
     w.c_grad = 1;
     w.c_off = pl.w_off[l];
     w.c_rs = ni;
-    if ((e = launch_gemm(P, w, pl.sm_count, st)) != cudaSuccess) return e;
+    if ((e = launch_gemm(P, w, pl.sm_count, l == 1 ? st : s2)) != cudaSuccess) return e;
     ++n;
     if (l > 1) {
       GemmArgs d{};  // dz_{l-1} = (dz_l W_l) masked by a_{l-1} > 0
@@ -505,6 +534,10 @@ cudaError_t launch_grad_mlp(const Params& P, const MlpPlan& pl, cudaStream_t st,
       d.mask = pl.act[l - 1];
       if ((e = launch_gemm(P, d, pl.sm_count, st)) != cudaSuccess) return e;
       ++n;
+      if (pl.side) {
+        if ((e = cudaEventRecord(pl.ev_dz[l - 1], st)) != cudaSuccess) return e;
+        if ((e = cudaStreamWaitEvent(pl.side, pl.ev_dz[l - 1], 0)) != cudaSuccess) return e;
+      }
     }
   }
   BiasArgs ba{};
@@ -515,9 +548,13 @@ cudaError_t launch_grad_mlp(const Params& P, const MlpPlan& pl, cudaStream_t st,
     ba.b_off[l] = pl.b_off[l];
     if (pl.dims[l] > maxn) maxn = pl.dims[l];
   }
-  mlp_bias_grad_kernel<<<dim3((maxn + 255) / 256, 2 * G, L), 256, 0, st>>>(P, ba);
+  mlp_bias_grad_kernel<<<dim3((maxn + 255) / 256, 2 * G, L), 256, 0, s2>>>(P, ba);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   ++n;
+  if (pl.side) {
+    if ((e = cudaEventRecord(pl.ev_join, pl.side)) != cudaSuccess) return e;
+    if ((e = cudaStreamWaitEvent(st, pl.ev_join, 0)) != cudaSuccess) return e;
+  }
   *n_launches = n;
   return cudaSuccess;
 }

@@ -28,6 +28,12 @@ struct MlpPlan {
   int* yb = nullptr;                          // [G*B] gathered class ids
   float* act[MLP_MAX_LAYERS + 1] = {nullptr}; // act[l], 1 <= l < L: [2][G*B][dims[l]] after ReLU; act[L]: class scores
   float* dz[MLP_MAX_LAYERS + 1] = {nullptr};  // dz[l], 1 <= l <= L: [2][G*B][dims[l]] gradient w.r.t. z_l
+  // fp32 path: the weight and bias gradients of the layers above the first do not feed the back-propagation
+  // chain, so they are enqueued on a second stream between a fork and a join event (branches of the graph
+  // when the iteration is captured)
+  cudaStream_t side = nullptr;
+  cudaEvent_t ev_dz[MLP_MAX_LAYERS + 1] = {nullptr};  // ev_dz[l]: dz_l is complete (on the main stream)
+  cudaEvent_t ev_join = nullptr;
   void* bf16_impl = nullptr;                  // opaque state of the bf16 tensor-core path
   std::vector<std::pair<void*, size_t>> state;  // device buffers that carry state across iterations (checkpoints)
   int norm_parts = 0;                         // > 0: the gradient kernels themselves deliver this many partial sums
@@ -40,6 +46,8 @@ const char* mlp_supported(const std::vector<int>& dims, int compute);
 cudaError_t mlp_plan_create(const std::vector<int>& dims, int compute, int G, int B, int D, long long p_pad,
                             int sm_count, cudaStream_t st, MlpPlan* plan, std::vector<void*>* owned,
                             const char** why);
+// Destroys the plan's stream and events (device buffers belong to the caller's `owned` list).
+void mlp_plan_release(MlpPlan* plan);
 // Enqueues the dual-point forward/backward of every group; writes each group's fresh-gradient row and P.stale.
 cudaError_t launch_grad_mlp(const Params& P, const MlpPlan& plan, cudaStream_t st, int* n_launches);
 // Work that must follow the selection kernel (none for the fp32 path; bf16: the selected groups' uploads
