@@ -420,6 +420,110 @@ __global__ void __launch_bounds__(256) update_kernel(const Params P) {
   }
 }
 
+// The same step for long parameter vectors (tens of thousands of 16-byte columns and more): one column per
+// thread, which folds every selected group itself in ascending order (loads of four groups in flight), so a
+// block is 256 columns wide and needs no exchange between its warps.
+__global__ void __launch_bounds__(256) update_wide_kernel(const Params P) {
+  extern __shared__ int sel_list[];  // selected groups, ascending; bit 30 set = the group's cur[] is 1
+  __shared__ int n_sel_sh;
+  __shared__ double scratch[40];
+  __shared__ bool is_last;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const long long cols4 = P.p_pad >> 2;
+  const long long k = P.st->k;
+  const int ring = P.D + 1;
+  const float alpha_k = step_size(P, k);
+  const long long i4 = (long long)blockIdx.x * 256 + tid;
+  const bool active = i4 < cols4;
+  const long long o = i4 * 4;
+  float4 ahi = make_float4(0.f, 0.f, 0.f, 0.f), alo = ahi, h = ahi, vh = ahi, th = ahi;
+  if (active) {  // independent of the selection: fetched first
+    ahi = ld4(P.agg_hi + o);
+    alo = ld4(P.agg_lo + o);
+    h = ld4(P.h + o);
+    vh = ld4(P.vhat + o);
+    th = ld4(P.theta_ring + (k % ring) * P.p_pad + o);
+  }
+  if (warp == 0) {
+    int cnt = 0;
+    for (int g0 = 0; g0 < P.G; g0 += 32) {
+      const int gg = g0 + lane;
+      const bool s = gg < P.G && P.mask_cur[gg] != 0;
+      const int cur = gg < P.G ? P.cur[gg] : 0;
+      const unsigned int b = __ballot_sync(0xffffffffu, s);
+      if (s) sel_list[cnt + __popc(b & ((1u << lane) - 1u))] = gg | (cur << 30);
+      cnt += __popc(b);
+    }
+    if (lane == 0) n_sel_sh = cnt;
+  }
+  __syncthreads();
+  const int n_sel = n_sel_sh;
+  double local = 0.0;
+  if (active) {
+    for (int j0 = 0; j0 < n_sel; j0 += 4) {
+      float4 f[4], l[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (j0 + u < n_sel) {
+          const int e = sel_list[j0 + u], g = e & 0x3fffffff, cur = e >> 30;
+          f[u] = ld4(P.gbuf + ((long long)cur * P.G + g) * P.p_pad + o);        // the fresh gradient (cur[g] already flipped)
+          l[u] = ld4(P.gbuf + ((long long)(1 - cur) * P.G + g) * P.p_pad + o);  // the gradient it replaces
+        }
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (j0 + u < n_sel) {
+          fold(ahi.x, alo.x, f[u].x, l[u].x);
+          fold(ahi.y, alo.y, f[u].y, l[u].y);
+          fold(ahi.z, alo.z, f[u].z, l[u].z);
+          fold(ahi.w, alo.w, f[u].w, l[u].w);
+        }
+    }
+    renorm(ahi.x, alo.x);
+    renorm(ahi.y, alo.y);
+    renorm(ahi.z, alo.z);
+    renorm(ahi.w, alo.w);
+    st4(P.agg_hi + o, ahi);
+    st4(P.agg_lo + o, alo);
+    float4 tn;
+#define GCADA_AMSGRAD(c)                                   \
+  {                                                        \
+    const float gr = ahi.c;                                \
+    h.c = P.beta1 * h.c + P.omb1 * gr;                     \
+    const float v = P.beta2 * vh.c + P.omb2 * (gr * gr);   \
+    vh.c = fmaxf(vh.c, v);                                 \
+    const float up = alpha_k * h.c / sqrtf(P.eps + vh.c);   \
+    tn.c = th.c - up;                                      \
+    local += (double)up * (double)up;                      \
+  }
+    GCADA_AMSGRAD(x)
+    GCADA_AMSGRAD(y)
+    GCADA_AMSGRAD(z)
+    GCADA_AMSGRAD(w)
+#undef GCADA_AMSGRAD
+    st4(P.h + o, h);
+    st4(P.vhat + o, vh);
+    st4(P.theta_ring + ((k + 1) % ring) * P.p_pad + o, tn);
+  }
+  const double tot = block_sum(local, scratch);
+  if (tid == 0) {
+    P.upd_part[blockIdx.x] = tot;
+    __threadfence();
+    is_last = atomicAdd(&P.st->ticket_update, 1u) == gridDim.x - 1u;
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  const volatile double* parts = P.upd_part;
+  double s = 0.0;
+  for (unsigned int b = tid; b < gridDim.x; b += 256) s += parts[b];
+  s = block_sum(s, scratch);
+  if (tid == 0) {
+    P.s_ring[k % P.D] = s;
+    P.st->k = k + 1;
+    P.st->ticket_update = 0u;
+  }
+}
+
 // Eq. (8a)-(8c) when the aggregate has already been formed in agg_hi (P.agg_direct): one float4 per thread.
 __global__ void __launch_bounds__(256) update_direct_kernel(const Params P) {
   __shared__ double scratch[40];
@@ -552,6 +656,10 @@ cudaError_t launch_select(const Params& P, const TailPlan& plan, cudaStream_t st
 cudaError_t launch_update(const Params& P, const TailPlan& plan, cudaStream_t st) {
   if (P.agg_direct) {
     update_direct_kernel<<<(plan.update_blocks + 7) / 8, 256, 0, st>>>(P);
+    return cudaGetLastError();
+  }
+  if (P.p_pad >= 4 * 256 * 128) {  // enough 16-byte columns to fill the machine with one per thread
+    update_wide_kernel<<<(plan.update_blocks + 7) / 8, 256, (size_t)P.G * sizeof(int), st>>>(P);
     return cudaGetLastError();
   }
   update_kernel<<<plan.update_blocks, 256, (size_t)P.G * sizeof(int), st>>>(P);
