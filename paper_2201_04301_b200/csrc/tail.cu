@@ -627,10 +627,9 @@ cudaError_t launch_ps_lhs(const Params& P, const TailPlan& plan, cudaStream_t st
 }
 
 void plan_tail(long long p_pad, int G, int sm_count, TailPlan* plan) {
-  (void)G;
-  (void)sm_count;
   const long long cols4 = p_pad / 4;
-  const int U = cols4 > 256 * 1024 ? 4 : 1;
+  // four columns per thread once one per thread would give more than four blocks per SM
+  const int U = (cols4 > 256 * 1024 || cols4 * G > 256LL * 4 * sm_count) ? 4 : 1;
   plan->select_cols4_per_block = 256 * U;
   plan->select_blocks_x = (int)((cols4 + 256 * U - 1) / (256 * U));
   plan->update_blocks = (int)((cols4 + 31) / 32);
