@@ -79,6 +79,14 @@ struct GemmB {
   int stages;
   int k_batched;     // 1: one output [M][N]; K runs over the batch entries of both operands (kpg K blocks each)
   int kpg, n_batch;
+  int agg_pass;      // k_batched products that maintain the aggregate of Eq. (3) from the last-upload store:
+                     // 0: sum over all n_batch entries, written (not added);
+                     // 1: before the selected groups' uploads are stored - minus the sum over the SELECTED
+                     //    groups' entries (their old uploads), added to the output;
+                     // 2: after they are stored - plus the sum over the selected groups' entries, added.
+                     // Passes 1 and 2 together replace the selected groups' terms.  When at least half of the
+                     // groups are selected, and every AGG_REFRESH-th iteration (so that rounding cannot pile
+                     // up), pass 1 does nothing and pass 2 is the full sum of pass 0.
   // epilogue operands
   __nv_bfloat16* out;    // row-major bf16 [z][M][ldo]
   __nv_bfloat16* outT;   // transposed bf16 [z][N][ldt]
@@ -197,6 +205,8 @@ __device__ __forceinline__ int ring_slot(const Params& P, int g, int q, long lon
 // the CTAs running together share operand tiles in L2); tensor memory holds
 // two 256-column accumulators, so the eight epilogue warps drain tile i while
 // the producer and the MMA warp work on tile i+1.
+constexpr int AGG_REFRESH = 16;  // the aggregate is recomputed in full at least every so many iterations (a replaced
+                                 // pair of uploads moves it by ~1e-7 of its norm from the recomputed value)
 constexpr int GN = 256;                                  // N tile of this kernel (the epilogue assumes 2 x 4 chunks of 32)
 constexpr int G_STAGE_BYTES = (BM + GN) * BK * 2;        // 48 KiB
 constexpr int G_STAGES = 4;
@@ -217,7 +227,24 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
   __shared__ uint32_t tmem_base_sm;
   unsigned char* tiles = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int nkb = a.k_batched ? a.kpg * a.n_batch : (a.K + BK - 1) / BK;
+  // aggregate passes: which batch entries, with which sign, written or added (the same in every thread of the grid)
+  int n_batch = a.n_batch;
+  bool listed = false, negate = false;
+  if (a.k_batched && a.agg_pass != 0) {
+    const int n_sel = P.sel_count[0];
+    const bool refresh = 2 * n_sel >= P.G || (P.st->k % AGG_REFRESH) == 0;
+    if (a.agg_pass == 1) {
+      if (refresh || n_sel == 0) return;
+      listed = negate = true;
+      n_batch = n_sel;
+    } else if (!refresh) {
+      if (n_sel == 0) return;  // no upload: the aggregate stands
+      listed = true;
+      n_batch = n_sel;
+    }
+  }
+  const bool accumulate = listed;
+  const int nkb = a.k_batched ? a.kpg * n_batch : (a.K + BK - 1) / BK;
   const int tiles_n = (a.N + GN - 1) / GN, tiles_m = (a.M + BM - 1) / BM;
   // batch entries: (point, group) for every group, or - when only the selected groups compute (rule PS:
   // Algorithm 1's own order, the selection is already known) - the selected groups at theta^k only
@@ -256,8 +283,10 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
         const int q = a.k_batched ? 0 : zi / n_grp;
         const int g = a.k_batched ? 0 : (P.skip_unselected ? P.sel_list[zi - q * n_grp] : zi - q * n_grp);
         const int z = q * P.G + g;
-        int zA = 0, zB = 0;
-        if (!a.k_batched) {
+        int zA = 0, zB = 0, ent = 0;
+        if (a.k_batched) {
+          zA = zB = listed ? P.sel_list[0] : 0;
+        } else {
           zA = a.a_shared ? g : z;
           zB = a.zb_mode == ZB_RING ? ring_slot(P, g, q, k_it) : (a.zb_mode == ZB_GROUP ? g : z);
         }
@@ -273,8 +302,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
           tma_load_3d(sa + BM * BK * 2, &tmB, kc, nt * GN, zB, &full_bar[s]);
           if (a.k_batched && ++kin == a.kpg) {
             kin = 0;
-            ++zA;
-            ++zB;
+            ++ent;
+            zA = zB = (listed && ent < n_batch) ? P.sel_list[ent] : ent;
           }
         }
       }
@@ -298,8 +327,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
           const uint64_t da = make_desc(sa), db = make_desc(sa + BM * BK * 2);
 #pragma unroll
           for (int kk = 0; kk < BK / 16; ++kk)  // 16 bf16 = 32 bytes = 2 descriptor units per MMA
-            tc_mma_bf16(tmem_base + (uint32_t)(slot * GN), da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), IDESC_G,
-                        (kb | kk) != 0 ? 1u : 0u);
+            tc_mma_bf16(tmem_base + (uint32_t)(slot * GN), da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2),
+                        negate ? (IDESC_G | (1u << 13)) : IDESC_G, (kb | kk) != 0 ? 1u : 0u);
           tc_commit(&empty_bar[s]);  // frees the stage once these MMAs have read it
         }
         if (ok) tc_commit(&tfull_bar[slot]);
@@ -372,11 +401,17 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
           if (row_ok) {
             if (full && ((a.c_off | a.ldc) & 3) == 0) {
 #pragma unroll
-              for (int j = 0; j < 32; j += 4)
-                *reinterpret_cast<float4*>(dst + j) = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
-                                                                  __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+              for (int j = 0; j < 32; j += 4) {
+                float4 o4 = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]),
+                                        __uint_as_float(v[j + 3]));
+                if (accumulate) {
+                  const float4 c4 = *reinterpret_cast<const float4*>(dst + j);
+                  o4 = make_float4(c4.x + o4.x, c4.y + o4.y, c4.z + o4.z, c4.w + o4.w);
+                }
+                *reinterpret_cast<float4*>(dst + j) = o4;
+              }
             } else {
-              for (int j = 0; j < 32 && nc + j < a.N; ++j) dst[j] = __uint_as_float(v[j]);
+              for (int j = 0; j < 32 && nc + j < a.N; ++j) dst[j] = (accumulate ? dst[j] : 0.f) + __uint_as_float(v[j]);
             }
           }
         } else if (a.epi == EPI_SCORES) {
@@ -1318,7 +1353,7 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
   e = cudaFuncSetAttribute(bf16_dw_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024);  // the kernel's static arrays take under 1 KiB
   if (e != cudaSuccess) return e;
   plan->launches_per_iter = 3 + L + 1 + L + (L - 1);
-  plan->post_launches = L + 2;
+  plan->post_launches = 2 * L + 2;
   plan->skip_launches = 2 + L + 1 + (L - 1) + 1;
   return cudaSuccess;
 }
@@ -1460,14 +1495,37 @@ BiasAggArgs bias_agg_args(const MlpPlan& pl, const Bf16Impl* im) {
 }  // namespace
 
 // After the selection, the server's side of Eq. (3): the selected groups' uploads replace their last
-// uploaded gradients (kept as factors), and the aggregate - the sum over ALL groups of the last uploaded
-// gradients - is formed anew as one product per layer whose K dimension runs over every group's rows.
-// Nothing is accumulated across iterations, so the aggregate carries no drift.
+// uploaded gradients (kept as factors) in the aggregate, the sum over ALL groups of the last uploaded
+// gradients.  Each layer's share is one product whose K dimension runs over groups' rows: over the selected
+// groups only - minus their old uploads before the store is updated, plus the new ones after it - when
+// fewer than half of the groups upload, over every group (the sum formed anew) otherwise and at least every
+// AGG_REFRESH iterations, which keeps the rounding of the running sum from piling up.
 cudaError_t mlp_bf16_launch_post(const Params& P, const MlpPlan& pl, cudaStream_t st, int* n_launches) {
   *n_launches = 0;
   const Bf16Impl* im = static_cast<const Bf16Impl*>(pl.bf16_impl);
   const int L = pl.n_layers, G = P.G, Bp = im->Bp;
   cudaError_t e;
+  auto aggregate = [&](int pass) -> cudaError_t {
+    for (int l = L; l >= 1; --l) {
+      GemmB a{};
+      a.M = pl.dims[l];
+      a.N = pl.dims[l - 1];
+      a.K = G * Bp;
+      a.k_batched = 1;
+      a.kpg = Bp / BK;
+      a.n_batch = G;
+      a.agg_pass = pass;
+      a.epi = EPI_AGG;
+      a.out_f32 = P.agg_hi;
+      a.c_off = pl.w_off[l];
+      a.ldc = pl.dims[l - 1];
+      cudaError_t e2 = launch_gemm(im->tm_agg_a[l], im->tm_agg_b[l], P, a, pl.sm_count, st);
+      if (e2 != cudaSuccess) return e2;
+      ++*n_launches;
+    }
+    return cudaSuccess;
+  };
+  if ((e = aggregate(1)) != cudaSuccess) return e;  // minus the uploads that are about to be replaced
   KeepArgs k{};
   for (int l = 1; l <= L; ++l) {
     k.src[k.n_seg] = im->dzT[l];
@@ -1483,21 +1541,7 @@ cudaError_t mlp_bf16_launch_post(const Params& P, const MlpPlan& pl, cudaStream_
   bf16_keep_kernel<<<dim3(64, G), 256, 0, st>>>(P, k);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   ++*n_launches;
-  for (int l = L; l >= 1; --l) {
-    GemmB a{};
-    a.M = pl.dims[l];
-    a.N = pl.dims[l - 1];
-    a.K = G * Bp;
-    a.k_batched = 1;
-    a.kpg = Bp / BK;
-    a.n_batch = G;
-    a.epi = EPI_AGG;
-    a.out_f32 = P.agg_hi;
-    a.c_off = pl.w_off[l];
-    a.ldc = pl.dims[l - 1];
-    if ((e = launch_gemm(im->tm_agg_a[l], im->tm_agg_b[l], P, a, pl.sm_count, st)) != cudaSuccess) return e;
-    ++*n_launches;
-  }
+  if ((e = aggregate(2)) != cudaSuccess) return e;  // plus the new ones (or the full sum, see GemmB::agg_pass)
   bf16_bias_agg_kernel<<<(im->nbias + 255) / 256, 256, 0, st>>>(P, bias_agg_args(pl, im), P.agg_hi);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   ++*n_launches;

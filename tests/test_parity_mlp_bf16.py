@@ -81,6 +81,33 @@ def test_aggregate_is_the_sum_of_last_uploads(dims, batch, G):
     assert 0 < m.sum() < m.size
 
 
+def test_running_aggregate_stays_the_sum_of_last_uploads():
+    """When fewer than half of the groups upload, the aggregate is not formed anew: the selected groups' old
+    uploads are taken out of it and their new ones put in (two products over the selected groups' rows), with
+    a full recomputation whenever half of the groups upload and at least every 16 iterations.  Under sparse
+    forced masks (none, one, a few, all) over several such periods it must stay equal to the sum of the
+    groups' last uploads, each rebuilt from its stored factors by a different kernel."""
+    G = 12
+    w = to_cuda(make_workload("cfg5", rows=G * 300, dims=(64, 128, 40), M=2 * G, M_G=2, D=100, batch=128, c=0.3))
+    g = binding.from_workload(w, stream=torch.cuda.Stream())
+    rng = np.random.default_rng(5)
+    worst = 0.0
+    for k in range(75):
+        mask = np.zeros((1, G), dtype=np.uint8)
+        if k == 0 or k == 40:
+            mask[:] = 1
+        elif k % 7 != 3:                                   # every seventh iteration uploads nothing
+            mask[0, rng.choice(G, size=int(rng.integers(1, 4)), replace=False)] = 1
+        g.step_forced(mask)
+        if k in (0, 1, 5, 15, 16, 17, 31, 39, 40, 41, 47, 63, 64, 74):
+            agg = g.get_debug(binding.DBG_AGG).astype(np.float64)
+            want = sum(g.get_group_gradient(binding.DBG_GLAST, gi).astype(np.float64) for gi in range(G))
+            err = np.linalg.norm(agg - want) / np.linalg.norm(want)
+            worst = max(worst, err)
+            assert err <= 5e-6, (k, err)
+    print("running aggregate: worst relative error", worst)
+
+
 def test_two_pass_norms_against_the_oracle():
     """The production path's left side of the test (difference accumulated in
     tensor memory) against the oracle, teacher-forced."""
