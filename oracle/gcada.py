@@ -158,8 +158,7 @@ class GCadaOracle:
         lhs = np.zeros(G)
         for g in range(G):
             _, Xb, yb = self.minibatch(g)
-            # the rule keeps tau_g <= D; a forced mask may let it grow, the stale iterate is then theta^{k-D}
-            theta_old = self.theta_at(k - min(int(self.tau[g]), self.D))
+            theta_old = self.theta_at(k - int(self.tau[g]))      # theta^{k - tau_g} (Eq. 3, Section IV)
             fresh[g] = self.model.grad(theta_k, Xb, yb, self.reduction)
             stale[g] = self.model.grad(theta_old, Xb, yb, self.reduction)
             if self.rule == "innov":

@@ -87,12 +87,21 @@ class MLP:
     before they are used; products, sums, the softmax and the loss are fp64.
     This is the reading of "bf16 inputs/weights with fp32 accumulation" for a
     multi-layer network: the input of layer l+1 is the bf16 output of layer l,
-    so both sides take each ReLU on/off decision from the same numbers."""
+    so both sides take each ReLU on/off decision from the same numbers.
+
+    With bf16="operands" only what the workload statement names is rounded:
+    the input features and the weight matrices W_l (the copy of the iterate
+    the products read); biases, hidden activations, back-propagated errors
+    and all arithmetic stay fp64.  This is the narrower reading of the same
+    phrase; the two differ by the rounding of the intermediate operands."""
     kind = "mlp"
 
     def __init__(self, dims, bf16=False):
         self.dims = tuple(int(n) for n in dims)
-        self.bf16 = bool(bf16)
+        if isinstance(bf16, str) and bf16 != "operands":
+            raise ValueError("bf16 must be False, True or 'operands'")
+        self.bf16_operands = isinstance(bf16, str)            # features and weight matrices only
+        self.bf16 = bool(bf16) and not self.bf16_operands     # every matrix-product operand rounded
         self.p = sum(self.dims[l] * self.dims[l - 1] + self.dims[l]
                      for l in range(1, len(self.dims)))
 
@@ -112,6 +121,9 @@ class MLP:
             theta = round_to_bf16(theta)
             Xb = round_to_bf16(Xb)
         layers = self.unpack(np.asarray(theta, dtype=np.float64))
+        if self.bf16_operands:
+            Xb = round_to_bf16(Xb)
+            layers = [(round_to_bf16(W), b) for W, b in layers]
         acts = [np.asarray(Xb, dtype=np.float64)]
         zs = []
         for l, (W, b) in enumerate(layers):

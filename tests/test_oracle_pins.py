@@ -563,3 +563,60 @@ def test_bf16_mode_rounds_every_matrix_operand():
     # and it stays close to the unrounded gradient
     exact = MLP((6, 5, 4, 3)).grad(theta, Xb, yb, "mean")
     assert 1e-5 < np.linalg.norm(got - exact) / np.linalg.norm(exact) < 3e-2
+
+
+def test_bf16_operands_mode_rounds_features_and_weight_matrices_only():
+    """The narrower reading of "bf16 inputs/weights": features and weight
+    matrices rounded, everything else exact.  Against torch autograd (library
+    routine) on explicitly cast leaves; the gradient is with respect to the
+    unrounded parameters, the rounding passing gradients through unchanged."""
+    rng = np.random.default_rng(11)
+    dims = (7, 6, 5, 3)
+    mlp = MLP(dims, bf16="operands")
+    theta = rng.normal(size=mlp.p)
+    Xb = rng.normal(size=(9, 7))
+    yb = rng.integers(0, 3, 9)
+    rb = lambda t: t.to(torch.float32).to(torch.bfloat16).to(torch.float64)
+    t = torch.tensor(theta, requires_grad=True)
+    o, a = 0, rb(torch.tensor(Xb))
+    for l in range(1, len(dims)):
+        W = t[o:o + dims[l] * dims[l - 1]].reshape(dims[l], dims[l - 1])
+        o += dims[l] * dims[l - 1]
+        b = t[o:o + dims[l]]
+        o += dims[l]
+        Wr = W + (rb(W.detach()) - W.detach())          # value rounded, gradient passed through
+        z = a @ Wr.T + b
+        a = torch.relu(z) if l < len(dims) - 1 else z
+    torch.nn.functional.cross_entropy(a, torch.tensor(yb), reduction="mean").backward()
+    got = mlp.grad(theta, Xb, yb, "mean")
+    assert np.allclose(got, t.grad.numpy(), rtol=1e-9, atol=1e-12)
+    # the three readings are distinct and ordered: exact -> operands -> every operand
+    exact = MLP(dims).grad(theta, Xb, yb, "mean")
+    every = MLP(dims, bf16=True).grad(theta, Xb, yb, "mean")
+    n = np.linalg.norm(exact)
+    assert 1e-5 < np.linalg.norm(got - exact) / n < 3e-2
+    assert 1e-5 < np.linalg.norm(every - got) / n < 3e-2
+    # rounding the inputs by hand and calling the unrounded model gives the same thing
+    th_r = theta.copy()
+    o = 0
+    for l in range(1, len(dims)):
+        n_w = dims[l] * dims[l - 1]
+        th_r[o:o + n_w] = round_to_bf16(theta[o:o + n_w])
+        o += n_w + dims[l]
+    assert np.array_equal(got, MLP(dims).grad(th_r, round_to_bf16(Xb), yb, "mean"))
+
+
+def test_stale_iterate_is_the_literal_one_under_forced_masks():
+    """Eq. (3) / Section IV: the stale iterate of a group is theta^{k - tau_g}, whatever tau_g is.  The
+    method's own rule keeps tau_g <= D; a forced mask can starve a group for longer, and the oracle then
+    still goes back tau_g iterates (to theta^0 at the earliest)."""
+    o = _toy_oracle(D=2)
+    masks = [[1, 1, 1], [1, 0, 1], [1, 0, 1], [1, 0, 1], [1, 0, 1]]
+    for k, m in enumerate(masks):
+        assert o.tau[1] == (2 if k == 0 else k)       # initial age D, then 1, 2, 3, 4: beyond D = 2 from k = 3
+        _, Xb, yb = o.minibatch(1)
+        want = o.model.grad(o.thetas[max(k - int(o.tau[1]), 0)], Xb, yb, "mean")
+        rec = o.step(forced_mask=m)
+        assert np.array_equal(rec["stale"][1], want)
+        if k >= 1:
+            assert np.array_equal(want, o.model.grad(o.thetas[0], Xb, yb, "mean"))   # last upload was at k = 0

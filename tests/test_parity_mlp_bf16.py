@@ -22,7 +22,7 @@ pytestmark = pytest.mark.gpu
 def test_small_architectures(dims, batch, M, M_G, D):
     G = M // M_G
     w = make_workload("cfg5", rows=G * 1000, dims=dims, M=M, M_G=M_G, D=D, batch=batch, c=0.3, alpha=1e-3)
-    flips, worst = forced_parity(w, 2 * D + 3, tol=TOL_BF16, stream=torch.cuda.Stream(), margin=None, rhs_tol=2e-2)
+    flips, worst = forced_parity(w, 2 * D + 3, tol=TOL_BF16, stream=torch.cuda.Stream(), rhs_tol=2e-2)
     print("bf16", dims, "worst", worst, "flips", flips)
 
 
