@@ -163,6 +163,142 @@ def mlp_flops_per_iteration(w):
     return rows * f
 
 
+MIN_REGION_MS = 50.0      # a timed region shorter than this is repeated (own event pair each) and the median kept
+SHORT_REPEATS = 7
+
+
+def time_steps(g, stream, steps, world, dev, sampler=None):
+    """Time gcada_step(steps) on the device: barrier + synchronize on both sides, one CUDA-event pair on the
+    launching stream, max over ranks.  When the region is short it is repeated SHORT_REPEATS times, each
+    repeat being exactly `steps` iterations under its own event pair.  Returns the per-repeat times (ms)."""
+    import torch
+    times = []
+    n_rep = 1
+    while len(times) < n_rep:
+        _barrier(world)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        g.step(steps)
+        e1.record(stream)
+        if sampler is not None:
+            sampler.sample_once()          # work is in flight
+        e1.synchronize()
+        _barrier(world)
+        times.append(_barrier_max(world, e0.elapsed_time(e1), dev))
+        if len(times) == 1 and times[0] < MIN_REGION_MS:
+            n_rep = SHORT_REPEATS
+    return times
+
+
+def _median(v):
+    s = sorted(v)
+    return s[len(s) // 2]
+
+
+def roofline_of(w, name, rule, peaks, ms_step, steps, launches_per_region, ms_grad, ms_grad_b2b, sel_frac, max_mhz):
+    """The roofline object of one workload: dominant kernel, algorithmic work per launch, achieved rate."""
+    if w["kind"] == "mlp" and w["compute"] == "fp32":
+        # plain fp32 FFMA tiles (a 1e-5 tolerance rules out single-pass tensor-core arithmetic):
+        # peak = SMs x 128 FMA lanes x 2 flop x max SM clock
+        import torch
+        flops = mlp_flops_per_iteration(w)
+        sms = torch.cuda.get_device_properties(0).multi_processor_count
+        peak = sms * 128 * 2 * (max_mhz or 1965) * 1e6 / 1e12
+        achieved = flops / (ms_grad * 1e-3) / 1e12 if ms_grad and ms_grad > 0 else None
+        return {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                "frac": achieved / peak if achieved else None, "traffic": None,
+                "kernel": "gradient (all launches of one iteration; latency-bound at this size)",
+                "peak_source": "derived: SMs x 128 lanes x 2 x max SM clock", "flops_per_iteration": flops,
+                "whole_step_tflops": flops / (ms_step * 1e-3) / 1e12}
+    if launches_per_region == 1:
+        # narrow model: the whole timed region was ONE launch of the cluster kernel (all iterations inside it)
+        bytes_launch = algorithmic_bytes_per_launch(w) * steps
+        achieved = bytes_launch / (ms_step * steps * 1e-3) / 1e9
+        return {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm"], "traffic": None,
+                "kernel": "linear_cluster_kernel (one launch = all %d iterations; latency-bound workload: "
+                          "%.0f KB per iteration)" % (steps, algorithmic_bytes_per_launch(w) / 1e3),
+                "peak_source": peaks["source"], "duration_ms": ms_step * steps,
+                "algorithmic_bytes_per_launch": bytes_launch}
+    if w["kind"] != "mlp":
+        bytes_launch = algorithmic_bytes_per_launch(w)
+        achieved = bytes_launch / (ms_grad_b2b * 1e-3) / 1e9 if ms_grad_b2b and ms_grad_b2b > 0 else None
+        traffic = None
+        rec = NCU_TRAFFIC.get(name)
+        if rec:
+            src = os.path.join(ROOT, "paper_2201_04301_b200", "csrc", rec[0])
+            if hashlib.sha256(open(src, "rb").read()).hexdigest() == rec[1]:
+                traffic = rec[2]
+        return {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm"] if achieved else None, "traffic": traffic,
+                "kernel": "gradient", "peak_source": peaks["source"],
+                "duration_ms": ms_grad_b2b, "duration_how": "200 back-to-back launches, one CUDA-event pair",
+                "achieved_from_bracketed_launches": bytes_launch / (ms_grad * 1e-3) / 1e9 if ms_grad and ms_grad > 0 else None,
+                "algorithmic_bytes_per_launch": bytes_launch,
+                "frac_of_nominal_8TBs": achieved / 8000.0 if achieved else None,
+                # the same bytes over the whole timed step (gradient + selection + update kernels)
+                "whole_step_gbs": bytes_launch / (ms_step * 1e-3) / 1e9,
+                "whole_step_frac": bytes_launch / (ms_step * 1e-3) / 1e9 / peaks["hbm"]}
+    # bf16 MLP: the dominant "kernel" is the chain of tensor-core products of one iteration; the flops are the
+    # dual-point forward/backward as specified (the aggregate products of the update phase are not counted),
+    # divided by the graph-replayed step the `value` comes from
+    flops = mlp_flops_per_iteration(w)
+    if rule == "ps":     # only the selected groups compute, at theta^k only
+        flops = flops / 2 * sel_frac
+    achieved = flops / (ms_step * 1e-3) / 1e12
+    grad = flops / (ms_grad * 1e-3) / 1e12 if ms_grad and ms_grad > 0 else None
+    return {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",
+            "frac": achieved / peaks["bf16_sustained"], "traffic": None,
+            "kernel": "whole iteration (all tensor-core launches; graph replay)",
+            "peak_source": peaks["source"] + " (sustained; the step runs for seconds under the power cap)",
+            "frac_of_burst_peak": achieved / peaks["bf16"], "burst_peak": peaks["bf16"],
+            "gradient_phase_tflops": grad,
+            "gradient_phase_frac": grad / peaks["bf16_sustained"] if grad else None,
+            "gradient_phase_how": "as-specified flops / event-bracketed gradient kernels (plain launches)",
+            "flops_per_iteration": flops}
+
+
+def measure(g, w, name, rule, stream, dev, world, local, steps, warmup, peaks, timing_iters=256):
+    """Warm up, time gcada_step(steps), then the per-kernel legs; returns the measured part of a bench line."""
+    import torch
+    from paper_2201_04301_b200 import binding
+    g.step(warmup)
+    if warmup < 16:
+        g.step(16)               # at least one replay of the 16-iteration graph before anything is timed
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    l0 = g.get_launch_count()
+    sampler.start()
+    times = time_steps(g, stream, steps, world, dev, sampler)
+    sampler.stop_flag = True
+    sampler.join()
+    launches = (g.get_launch_count() - l0) // len(times)
+    ms = _median(times)
+    n_hist = min(steps, 4096)
+    sel_frac = float(g.get_selection_mask(g.get_iteration() - n_hist, n_hist).mean())
+    # per-kernel times (plain launches bracketed by events)
+    g.set_option(binding.OPT_TIMING, 1)
+    g.step(min(steps, timing_iters))
+    (ms_grad, ms_sel, ms_upd), n_timed = g.get_kernel_times()
+    g.set_option(binding.OPT_TIMING, 0)
+    # the dominant kernel alone, back to back, one event pair (no per-launch bracket gaps); each repetition
+    # streams the same rows, more than four times the L2 on the wide workload, so nothing is served from cache
+    ms_grad_b2b = g.time_gradient(200 if w["kind"] != "mlp" else 5)
+    floor_us = g.time_empty_chain(max(16, min(steps, 2048)))
+    res = {
+        "value": aggregate_value(world, steps, ms), "unit": UNIT, "steps": steps, "warmup": warmup,
+        "ms_per_step": ms / steps, "ms_per_step_best": min(times) / steps, "timed_repeats": len(times),
+        "gpu_launches": int(launches), "selected_fraction": sel_frac, "clocks": sampler.result(),
+        "kernel_ms": {"gradient": ms_grad, "select": ms_sel, "update": ms_upd, "timed_iterations": n_timed},
+        "latency_floor_us": floor_us, "us_per_step": ms / steps * 1e3,
+        "latency_floor_how": "the iteration's launch structure replayed with empty kernels (same graph nodes, "
+                             "edges and launch shapes; for the one-cluster kernel: its cluster barrier per iteration)",
+    }
+    res["roofline"] = roofline_of(w, name, rule, peaks, ms / steps, steps, launches, ms_grad, ms_grad_b2b, sel_frac,
+                                  sampler.max_mhz)
+    return res
+
+
 def run_ours(args):
     import torch
     from paper_2201_04301_b200 import binding
@@ -175,6 +311,7 @@ def run_ours(args):
         _build.build()
     _barrier(world)
     binding.load()
+    peaks = _peaks()
     t0 = time.time()
     overrides = {}
     if args.workers:
@@ -182,7 +319,7 @@ def run_ours(args):
     w = make_workload(args.config, device=dev, data_seed=rank, rows=args.rows, **overrides)
     stream = torch.cuda.Stream(device=dev)
     torch.cuda.synchronize()
-    opts = {binding.OPT_GRAPH: 0.0 if args.no_graph else 1.0, binding.OPT_LINEAR_VARIANT: float(args.variant)}
+    opts = {binding.OPT_GRAPH: 0.0 if args.no_graph else 1.0}
     smooth = None
     if args.rule == "ps":      # Eq. (9) as printed, with one smoothness constant for every group
         opts[binding.OPT_RULE] = 1.0
@@ -192,35 +329,7 @@ def run_ours(args):
     G = g.G
 
     # --- device-resident timing ------------------------------------------------
-    g.step(args.warmup)
-    torch.cuda.synchronize()
-    sampler = ClockSampler(local)
-    l0 = g.get_launch_count()
-    _barrier(world)
-    sampler.start()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    g.step(args.steps)
-    e1.record(stream)
-    sampler.sample_once()          # work is in flight
-    e1.synchronize()
-    _barrier(world)
-    sampler.stop_flag = True
-    sampler.join()
-    ms = _barrier_max(world, e0.elapsed_time(e1), dev)
-    launches = g.get_launch_count() - l0
-    value = aggregate_value(world, args.steps, ms)
-    n_hist = min(args.steps, 4096)
-    sel_frac = float(g.get_selection_mask(g.get_iteration() - n_hist, n_hist).mean())
-
-    # --- per-kernel times (plain launches bracketed by events) -------------------
-    g.set_option(binding.OPT_TIMING, 1)
-    g.step(min(args.steps, 256))
-    (ms_grad, ms_sel, ms_upd), n_timed = g.get_kernel_times()
-    g.set_option(binding.OPT_TIMING, 0)
-    # the dominant kernel alone, back to back, one event pair (no per-launch bracket gaps); each repetition
-    # streams the same rows, more than four times the L2, so nothing is served from cache
-    ms_grad_b2b = g.time_gradient(200 if w["kind"] != "mlp" else 5)
+    m = measure(g, w, args.config, args.rule, stream, dev, world, local, args.steps, args.warmup, peaks)
 
     # --- end to end: minibatches fed from pinned host memory, theta read back ----
     e2e = None
@@ -256,10 +365,9 @@ def run_ours(args):
 
     if rank != 0:
         return
-    peaks = _peaks()
     out = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "metric": METRIC, "value": m["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": m["ms_per_step"], "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16" if w["compute"] == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": "%s: %s dims=%s N=%d M=%d M_G=%d batch=%d D=%d c=%g rule=%s" % (
             args.config, w["kind"], list(w["dims"]), w["X"].shape[0], w["M"], w["M_G"], w["batch"], w["D"], w["c"],
@@ -268,77 +376,26 @@ def run_ours(args):
             "l2": "inputs larger than L2: each step gathers its rows from the resident training set"
                   if w["X"].numel() * w["X"].element_size() > 126e6 else "training set smaller than L2 (latency-bound workload)",
             "setup_s": round(gen_s, 1)},
-        "clocks": sampler.result(),
-        "gpu_launches": int(launches),
-        "selected_fraction": sel_frac,
-        "kernel_ms": {"gradient": ms_grad, "select": ms_sel, "update": ms_upd, "timed_iterations": n_timed},
     }
+    for key in ("ms_per_step_best", "timed_repeats", "clocks", "gpu_launches", "selected_fraction", "kernel_ms",
+                "latency_floor_us", "latency_floor_how", "roofline"):
+        out[key] = m[key]
     if e2e:
         out["e2e"] = e2e
-    if w["kind"] == "mlp" and w["compute"] == "fp32":
-        # plain fp32 FFMA tiles (a 1e-5 tolerance rules out single-pass tensor-core arithmetic):
-        # peak = SMs x 128 FMA lanes x 2 flop x max SM clock
-        flops = mlp_flops_per_iteration(w)
-        import torch
-        sms = torch.cuda.get_device_properties(0).multi_processor_count
-        peak = sms * 128 * 2 * (sampler.max_mhz or 1965) * 1e6 / 1e12
-        achieved = flops / (ms_grad * 1e-3) / 1e12 if ms_grad > 0 else None
-        out["roofline"] = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                           "frac": achieved / peak if achieved else None, "traffic": None,
-                           "kernel": "gradient (all launches of one iteration; latency-bound at this size)",
-                           "peak_source": "derived: SMs x 128 lanes x 2 x max SM clock", "flops_per_iteration": flops}
-    elif launches == 1:
-        # narrow model: the whole timed region was ONE launch of the cluster kernel (all iterations inside it)
-        bytes_launch = algorithmic_bytes_per_launch(w) * args.steps
-        achieved = bytes_launch / (ms * 1e-3) / 1e9
-        out["roofline"] = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm"], "unit": "GB/s",
-                           "frac": achieved / peaks["hbm"], "traffic": None,
-                           "kernel": "linear_cluster_kernel (one launch = all %d iterations; latency-bound workload: "
-                                     "%.0f KB per iteration)" % (args.steps, algorithmic_bytes_per_launch(w) / 1e3),
-                           "peak_source": peaks["source"], "duration_ms": ms,
-                           "algorithmic_bytes_per_launch": bytes_launch}
-    elif w["kind"] != "mlp":
-        bytes_launch = algorithmic_bytes_per_launch(w)
-        achieved = bytes_launch / (ms_grad_b2b * 1e-3) / 1e9 if ms_grad_b2b > 0 else None
-        traffic = None
-        rec = NCU_TRAFFIC.get(args.config)
-        if rec:
-            src = os.path.join(ROOT, "paper_2201_04301_b200", "csrc", rec[0])
-            if hashlib.sha256(open(src, "rb").read()).hexdigest() == rec[1]:
-                traffic = rec[2]
-        out["roofline"] = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm"], "unit": "GB/s",
-                           "frac": achieved / peaks["hbm"] if achieved else None, "traffic": traffic,
-                           "kernel": "gradient", "peak_source": peaks["source"],
-                           "duration_ms": ms_grad_b2b, "duration_how": "200 back-to-back launches, one CUDA-event pair",
-                           "achieved_from_bracketed_launches": bytes_launch / (ms_grad * 1e-3) / 1e9 if ms_grad > 0 else None,
-                           "algorithmic_bytes_per_launch": bytes_launch,
-                           "frac_of_nominal_8TBs": achieved / 8000.0 if achieved else None,
-                           # the same bytes over the whole timed step (gradient + selection + update kernels)
-                           "whole_step_gbs": bytes_launch / (ms / args.steps * 1e-3) / 1e9,
-                           "whole_step_frac": bytes_launch / (ms / args.steps * 1e-3) / 1e9 / peaks["hbm"]}
-    else:
-        flops = mlp_flops_per_iteration(w)
-        if args.rule == "ps":     # only the selected groups compute, at theta^k only
-            flops = flops / 2 * sel_frac
-        achieved = flops / (ms_grad * 1e-3) / 1e12 if ms_grad > 0 else None
-        out["roofline"] = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_sustained"],
-                           "unit": "TFLOP/s", "frac": achieved / peaks["bf16_sustained"] if achieved else None,
-                           "traffic": None, "kernel": "gradient (all GEMM launches of one iteration)",
-                           "peak_source": peaks["source"] + " (sustained)", "flops_per_iteration": flops}
     if world == 1 and not (args.no_others or args.no_e2e or args.no_cpu):   # any --no-* switch: a short / profiling run
         # the remaining workloads of the statement, each for its own number of iterations (device-resident,
-        # same protocol: warm-up, one CUDA-event pair around gcada_step); parity cases elsewhere, here for context
+        # same protocol); parity cases elsewhere, here so that every workload's rate and roofline are on record
         g.close()
         del g, w
         torch.cuda.empty_cache()
-        out["other_workloads"] = other_workloads(args.config, dev, stream)
+        out["other_workloads"] = other_workloads(args.config, dev, stream, local, peaks)
     if world == 1 and not args.no_cpu:
-        out["cpu_baseline"] = cpu_baseline(args.config, budget_s=args.cpu_budget)
+        out["cpu_baseline"] = cpu_baseline_both(args.config, budget_s=args.cpu_budget)
     print(json.dumps(out), flush=True)
 
 
-def other_workloads(skip, dev, stream):
-    """Iterations per second of every other named workload, timed like the main one."""
+def other_workloads(skip, dev, stream, local, peaks):
+    """Every other named workload, timed like the main one, each with its own roofline, clocks and latency floor."""
     import torch
     from paper_2201_04301_b200 import binding
     from paper_2201_04301_b200.workloads import CONFIGS, make_workload
@@ -349,18 +406,10 @@ def other_workloads(skip, dev, stream):
         w = make_workload(name, device=dev)
         g = binding.from_workload(w, stream=stream, options={binding.OPT_GRAPH: 1.0})
         K = int(CONFIGS[name]["K"])
-        g.step(max(3, min(20, K // 10)))
-        torch.cuda.synchronize()
-        l0 = g.get_launch_count()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        g.step(K)
-        e1.record(stream)
-        e1.synchronize()
-        ms = e0.elapsed_time(e1)
-        res[name] = {"value": K / (ms * 1e-3), "unit": UNIT, "steps": K, "ms_per_step": ms / K,
-                     "gpu_launches": int(g.get_launch_count() - l0),
-                     "selected_fraction": float(g.get_selection_mask(g.get_iteration() - K, K).mean())}
+        m = measure(g, w, name, "innov", stream, dev, 1, local, K, max(3, min(20, K // 10)), peaks,
+                    timing_iters=64 if name == "cfg5" else 256)
+        m["dtype"] = "bf16" if w["compute"] == "bf16" else "f32"
+        res[name] = m
         g.close()
         del g, w
         torch.cuda.empty_cache()
@@ -430,6 +479,19 @@ def cpu_baseline(config, budget_s=15.0):
     return {"value": value, "unit": UNIT, "cores": _cores_used(), "kind": "oracle", "sample": sample}
 
 
+def cpu_baseline_both(config, budget_s=15.0):
+    """The oracle on the BLAS thread pool as it comes, and again held to one thread."""
+    res = cpu_baseline(config, budget_s)
+    try:
+        from threadpoolctl import threadpool_limits
+        with threadpool_limits(limits=1):
+            one = cpu_baseline(config, budget_s / 2)
+        res["one_thread"] = {"value": one["value"], "unit": UNIT, "cores": 1, "sample": one["sample"]}
+    except Exception as exc:       # no threadpoolctl: the pool figure stands alone
+        res["one_thread"] = {"unavailable": repr(exc)}
+    return res
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -483,7 +545,6 @@ def main():
     ap.add_argument("--rule", default="innov", choices=["innov", "ps"],
                     help="innov: measured gradient innovation (default); ps: left side of Eq. (9) as printed")
     ap.add_argument("--smoothness", type=float, default=0.25, help="L_g of every group for --rule ps")
-    ap.add_argument("--variant", type=int, default=0, help="GCADA_OPT_LINEAR_VARIANT (kernel shape knob)")
     ap.add_argument("--e2e-steps", type=int, default=60)
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     args = ap.parse_args()

@@ -27,10 +27,17 @@
  *     "host" pointers are ordinary host memory.  Borrowed buffers must outlive
  *     their use by the context; the library never frees caller memory.
  *     Output buffers are caller-allocated with the size passed.
- *   - gcada_step* only enqueue work on the context's stream; getters
- *     synchronise that stream.
- *   - Contexts are independent; there is no global state.  A context is bound
- *     to the device that was current in gcada_create.
+ *   - gcada_step only enqueues work on the context's stream (its first call
+ *     on a context also builds launch plans and captures its CUDA graphs,
+ *     which allocates); getters synchronise that stream.  The harness
+ *     variants gcada_step_forced and gcada_step_host_batch are not free of
+ *     host work: the first synchronises the stream, copies the mask with a
+ *     blocking copy and grows its device buffer when needed, the second
+ *     allocates a staging area on first use.
+ *   - Contexts are independent and share no state.  The only process-wide
+ *     state of the library is the fixed scratch array of
+ *     gcada_innovation_norms_noalloc (see there).  A context is bound to the
+ *     device that was current in gcada_create.
  *   - There is no CPU fallback: without a usable CUDA device gcada_create
  *     fails with GCADA_ECUDA.
  */
@@ -79,10 +86,7 @@ typedef struct {
 #define GCADA_OPT_TIMING 5     /* 1 = bracket each kernel phase with CUDA events (plain launches; see
                                   gcada_get_kernel_times); may be switched at any time (default 0) */
 
-#define GCADA_OPT_LINEAR_VARIANT 6 /* tuning knob of the d > 256 gradient kernel: 0 = default, 1 = one CTA per
-                                      SM with 4-row batches, 2 = two CTAs per SM with 2-row batches; results
-                                      differ only in summation order */
-
+/* (key 6 is not used) */
 #define GCADA_OPT_PERSISTENT 7     /* 1 (default) = logistic / quadratic models with d <= 256, at most 64 groups and
                                       1024 workers run free-running steps of the default rule as ONE launch of a
                                       single thread-block cluster per gcada_step call, whatever n_iters is (the
@@ -261,8 +265,11 @@ gcada_status gcada_get_kernel_times(gcada_ctx *ctx, double ms[3], int *n_timed);
  * use a context.  This call gives them the test quantity of the selection
  * rule on gradients they already hold:
  *     lhs_dev[g] = || fresh_dev[g*ld .. g*ld+p) - stale_dev[g*ld .. g*ld+p) ||^2
- * for g < G, the same arithmetic as the selection kernel (float difference,
- * double accumulation, fixed summation order).  All three pointers are device
+ * for g < G: each difference is taken in float, squared and accumulated in
+ * double in a fixed order (the order differs from a context's own reduction,
+ * and for logistic / quadratic models a context squares innovation partial
+ * sums that its gradient kernel formed directly, so the two agree to
+ * rounding, not bit for bit).  All three pointers are device
  * memory of the CURRENT device, owned by the caller; lhs_dev receives G
  * doubles.  The work is enqueued on cuda_stream (cudaStream_t as void*, NULL =
  * legacy default stream) and is asynchronous.
@@ -275,8 +282,11 @@ gcada_status gcada_get_kernel_times(gcada_ctx *ctx, double ms[3], int *n_timed);
  * between them) race and give wrong sums; order them.  The array keeps the
  * previous call's contents; the one word that must start at zero is cleared
  * on the stream by every call.  The first call on each device looks up the
- * array's device address (cudaGetSymbolAddress, with that device current):
- * make that first call outside any stream capture.  No call here uses
+ * array's device address (cudaGetSymbolAddress, with that device current)
+ * and keeps it for the life of the process: make that first call outside any
+ * stream capture, and do not use this entry point again on a device after
+ * cudaDeviceReset or from a second CUDA context on the same device (the kept
+ * address belongs to the context that first loaded the library).  No call here uses
  * cudaMalloc, cudaFree or any other allocating routine.
  * On failure a message is written to errbuf (if non-NULL, errbuf_len bytes).
  */
@@ -291,6 +301,15 @@ gcada_status gcada_innovation_norms_noalloc(const float *fresh_dev, const float 
  * a kernel that lasts tens of microseconds).  The repetitions recompute the same gradients and change no
  * state that an iteration reads.  Synchronises the stream before and after. */
 gcada_status gcada_time_gradient(gcada_ctx *ctx, int reps, double *ms_per_rep);
+
+/* Measurement aid: the latency floor of this context's iteration structure.  Enqueues what gcada_step(n_iters)
+ * would launch with all work removed - for the kernel chain a copy of the captured iteration graph (same
+ * nodes and dependencies, same grid, block, shared-memory and cluster shapes) whose kernels are empty, run in
+ * multiples of 16 iterations; for narrow linear models that run whole steps in one thread-block cluster, that
+ * cluster with nothing but its one cluster-wide barrier per iteration - and returns the device time per
+ * iteration in microseconds.  Touches no state of the run.  Needs a stream other than the default one
+ * (GCADA_ESTATE otherwise).  Synchronises the stream. */
+gcada_status gcada_time_empty_chain(gcada_ctx *ctx, int n_iters, double *us_per_iter);
 
 /* Reporting aid (not a step of Algorithm 1): the mean per-sample loss of the current iterate over rows
  * first_row .. first_row + n_rows - 1 of the resident training set, i.e. the objective of Eq. (1) restricted

@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(HERE, "libgcada.so")
 OK, EINVAL, ENOMEM, ECUDA, ESTATE, ETIMEOUT = range(6)
 MODEL_LOGISTIC, MODEL_MLP, MODEL_QUADRATIC = 0, 1, 2
 COMPUTE_FP32, COMPUTE_BF16 = 0, 1
-(OPT_RULE, OPT_REDUCTION, OPT_HISTORY, OPT_KEEP_STALE, OPT_GRAPH, OPT_TIMING, OPT_LINEAR_VARIANT,
+(OPT_RULE, OPT_REDUCTION, OPT_HISTORY, OPT_KEEP_STALE, OPT_GRAPH, OPT_TIMING, _OPT_UNUSED,
  OPT_PERSISTENT) = range(8)
 (DBG_FRESH, DBG_STALE, DBG_LHS, DBG_RHS, DBG_TAU, DBG_AGG, DBG_H, DBG_VHAT, DBG_TGROUP, DBG_GLAST,
  DBG_SRING) = range(11)
@@ -65,6 +65,7 @@ SIGNATURES = {
     "gcada_get_kernel_times": (C.c_int, [_VP, C.POINTER(C.c_double), C.POINTER(C.c_int)]),
     "gcada_innovation_norms_noalloc": (C.c_int, [_VP, _VP, C.c_int, _LL, _LL, _VP, _VP, C.c_char_p, C.c_size_t]),
     "gcada_time_gradient": (C.c_int, [_VP, C.c_int, C.POINTER(C.c_double)]),
+    "gcada_time_empty_chain": (C.c_int, [_VP, C.c_int, C.POINTER(C.c_double)]),
     "gcada_eval_loss": (C.c_int, [_VP, _LL, _LL, C.POINTER(C.c_double)]),
     "gcada_checkpoint_size": (C.c_int, [_VP, _ULLP]),
     "gcada_checkpoint_save": (C.c_int, [_VP, _VP, C.c_ulonglong]),
@@ -242,6 +243,12 @@ class GCada:
         ms = C.c_double()
         self._ck(self.lib.gcada_time_gradient(self.h, int(reps), C.byref(ms)))
         return ms.value
+
+    def time_empty_chain(self, n_iters):
+        """Device time per iteration (microseconds) of the iteration's launch structure with empty kernels."""
+        us = C.c_double()
+        self._ck(self.lib.gcada_time_empty_chain(self.h, int(n_iters), C.byref(us)))
+        return us.value
 
     def get_kernel_times(self):
         """(ms_gradient, ms_select, ms_update), n_timed: see GCADA_OPT_TIMING."""

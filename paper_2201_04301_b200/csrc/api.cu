@@ -36,7 +36,7 @@ struct gcada_ctx {
   double c = 0, alpha = 0, beta1 = 0, beta2 = 0, eps = 0;
   unsigned long long seed = 0;
   double shift = 1.0, rate = 1.0;
-  int rule = 0, reduction = 0, keep_stale = 0, use_graph = 1, linear_variant = 0, persistent = 1;
+  int rule = 0, reduction = 0, keep_stale = 0, use_graph = 1, persistent = 1;
   ClusterPlan cluster{};
   long long hist_cap = 65536;
   // data
@@ -270,8 +270,8 @@ gcada_status make_plans(gcada_ctx* ctx) {
     // the plan must also hold for the staging buffer of host-fed steps
     const void* xa = ctx->have_data ? ctx->X : nullptr;
     const long long ld = ctx->have_data ? ctx->ld : ((ctx->dims[0] + 3) / 4) * 4;
-    if (!plan_linear(ctx->dims[0], ld, xa, ctx->G, ctx->B, ctx->sm_count, ctx->smem_optin, ctx->linear_variant,
-                     &ctx->lin, &why))
+    if (!plan_linear(ctx->dims[0], ld, xa, ctx->G, ctx->B, ctx->sm_count, ctx->smem_optin, &ctx->lin,
+                     &why))
       return fail(ctx, GCADA_EINVAL, "%s", why);
     CK(prepare_grad_linear(ctx->lin, ctx->kind == GCADA_MODEL_QUADRATIC));
     // narrow models with few groups: whole iterations inside one thread-block cluster
@@ -384,7 +384,7 @@ gcada_status enqueue_iteration(gcada_ctx* ctx, const Params& P) {
   return GCADA_OK;
 }
 
-gcada_status capture(gcada_ctx* ctx, int iters, cudaGraphExec_t* out) {
+gcada_status capture_graph(gcada_ctx* ctx, int iters, cudaGraph_t* out) {
   cudaGraph_t graph = nullptr;
   const unsigned long long before = ctx->launches;
   CK(cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal));
@@ -399,11 +399,21 @@ gcada_status capture(gcada_ctx* ctx, int iters, cudaGraphExec_t* out) {
     return s;
   }
   CK(e);
-  e = cudaGraphInstantiate(out, graph, 0);
+  *out = graph;
+  return GCADA_OK;
+}
+
+gcada_status capture(gcada_ctx* ctx, int iters, cudaGraphExec_t* out) {
+  cudaGraph_t graph = nullptr;
+  TRY(capture_graph(ctx, iters, &graph));
+  cudaError_t e = cudaGraphInstantiate(out, graph, 0);
   cudaGraphDestroy(graph);
   CK(e);
   return GCADA_OK;
 }
+
+// A kernel that does nothing, for gcada_time_empty_chain.
+__global__ void empty_kernel() {}
 
 int kernels_per_iteration(const gcada_ctx* ctx) {
   if (is_linear(ctx)) return ctx->P.skip_unselected ? 5 : 3 + (ctx->rule == 1 ? 1 : 0);
@@ -669,10 +679,6 @@ gcada_status gcada_set_option(gcada_ctx* ctx, int key, double value) {
       if (!(value >= 1) || value > 1e9) return fail(ctx, GCADA_EINVAL, "history must be in [1, 1e9]");
       ctx->hist_cap = (long long)value;
       break;
-    case GCADA_OPT_LINEAR_VARIANT:
-      if (value != 0 && value != 1 && value != 2) return fail(ctx, GCADA_EINVAL, "variant must be 0, 1 or 2");
-      ctx->linear_variant = (int)value;
-      break;
     case GCADA_OPT_KEEP_STALE:
       ctx->keep_stale = value != 0;
       break;
@@ -746,8 +752,16 @@ static gcada_status run_iterations(gcada_ctx* ctx, int n_iters, const unsigned c
     ctx->cluster.usable = false;
   }
   if (ctx->use_graph && ctx->stream != nullptr && !ctx->timing) {
-    if (!ctx->graph1) TRY(capture(ctx, 1, &ctx->graph1));
-    if (!ctx->graphN && n_iters >= GRAPH_CHAIN) TRY(capture(ctx, GRAPH_CHAIN, &ctx->graphN));
+    // both graphs are captured, instantiated and uploaded by the first free-running step, whatever its
+    // length, so that no later call pays for a capture
+    if (!ctx->graph1) {
+      TRY(capture(ctx, 1, &ctx->graph1));
+      CK(cudaGraphUpload(ctx->graph1, ctx->stream));
+    }
+    if (!ctx->graphN) {
+      TRY(capture(ctx, GRAPH_CHAIN, &ctx->graphN));
+      CK(cudaGraphUpload(ctx->graphN, ctx->stream));
+    }
     const int kpi = kernels_per_iteration(ctx);
     while (left >= GRAPH_CHAIN && ctx->graphN) {
       CK(cudaGraphLaunch(ctx->graphN, ctx->stream));
@@ -1002,6 +1016,68 @@ gcada_status gcada_time_gradient(gcada_ctx* ctx, int reps, double* ms_per_rep) {
   cudaEventDestroy(e0);
   cudaEventDestroy(e1);
   *ms_per_rep = (double)ms / reps;
+  return GCADA_OK;
+}
+
+gcada_status gcada_time_empty_chain(gcada_ctx* ctx, int n_iters, double* us_per_iter) {
+  if (!ctx || !us_per_iter || n_iters < 1) return GCADA_EINVAL;
+  TRY(check_runnable(ctx, true));
+  DeviceGuard dg(ctx->device);
+  TRY(make_plans(ctx));
+  if (ctx->stream == nullptr) return fail(ctx, GCADA_ESTATE, "gcada_time_empty_chain needs a stream other than the default one");
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  CK(cudaEventCreate(&e0));
+  CK(cudaEventCreate(&e1));
+  float ms = 0.f;
+  int iters_run = 0;
+  if (is_linear(ctx) && ctx->cluster.usable) {
+    CK(launch_linear_cluster_empty(ctx->cluster, 16, ctx->stream));  // warm-up
+    CK(cudaStreamSynchronize(ctx->stream));
+    CK(cudaEventRecord(e0, ctx->stream));
+    CK(launch_linear_cluster_empty(ctx->cluster, n_iters, ctx->stream));
+    CK(cudaEventRecord(e1, ctx->stream));
+    iters_run = n_iters;
+  } else {
+    // the captured iterations with every kernel node's function replaced by an empty kernel: same nodes,
+    // same edges, same grids, blocks, shared-memory sizes and cluster shapes, no work
+    cudaGraph_t graph = nullptr;
+    TRY(capture_graph(ctx, GRAPH_CHAIN, &graph));
+    size_t n_nodes = 0;
+    CK(cudaGraphGetNodes(graph, nullptr, &n_nodes));
+    std::vector<cudaGraphNode_t> nodes(n_nodes);
+    CK(cudaGraphGetNodes(graph, nodes.data(), &n_nodes));
+    CK(cudaFuncSetAttribute(empty_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ctx->smem_optin));
+    CK(cudaFuncSetAttribute(empty_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+    for (cudaGraphNode_t nd : nodes) {
+      cudaGraphNodeType type;
+      CK(cudaGraphNodeGetType(nd, &type));
+      if (type != cudaGraphNodeTypeKernel) continue;
+      cudaKernelNodeParams kp{};
+      CK(cudaGraphKernelNodeGetParams(nd, &kp));
+      kp.func = reinterpret_cast<void*>(empty_kernel);
+      kp.kernelParams = nullptr;
+      kp.extra = nullptr;
+      CK(cudaGraphKernelNodeSetParams(nd, &kp));
+    }
+    cudaGraphExec_t exec = nullptr;
+    cudaError_t e = cudaGraphInstantiate(&exec, graph, 0);
+    cudaGraphDestroy(graph);
+    CK(e);
+    const int reps = (n_iters + GRAPH_CHAIN - 1) / GRAPH_CHAIN;
+    CK(cudaGraphLaunch(exec, ctx->stream));  // warm-up
+    CK(cudaStreamSynchronize(ctx->stream));
+    CK(cudaEventRecord(e0, ctx->stream));
+    for (int r = 0; r < reps; ++r) CK(cudaGraphLaunch(exec, ctx->stream));
+    CK(cudaEventRecord(e1, ctx->stream));
+    CK(cudaEventSynchronize(e1));
+    cudaGraphExecDestroy(exec);
+    iters_run = reps * GRAPH_CHAIN;
+  }
+  CK(cudaEventSynchronize(e1));
+  CK(cudaEventElapsedTime(&ms, e0, e1));
+  cudaEventDestroy(e0);
+  cudaEventDestroy(e1);
+  *us_per_iter = (double)ms * 1e3 / iters_run;
   return GCADA_OK;
 }
 

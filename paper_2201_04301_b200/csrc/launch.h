@@ -20,8 +20,7 @@ struct LinearPlan {
 };
 
 // Chooses the kernel and its shape; false (with *why) if the shape is not supported.
-// `variant`: 0 = default shape, 1 = one CTA per SM with 4-row batches, 2 = two CTAs per SM with 2-row batches.
-bool plan_linear(int d, long long ld, const void* X, int G, int B, int sm_count, size_t smem_optin, int variant,
+bool plan_linear(int d, long long ld, const void* X, int G, int B, int sm_count, size_t smem_optin,
                  LinearPlan* plan, const char** why);
 // One-time function attributes (dynamic shared memory size); call before the first launch.
 cudaError_t prepare_grad_linear(const LinearPlan& plan, bool quad);
@@ -49,6 +48,8 @@ struct ClusterPlan {
 };
 bool plan_linear_cluster(int d, int G, int M, int D, int B, long long p_pad, size_t smem_optin, ClusterPlan* plan);
 cudaError_t launch_linear_cluster(const Params& P, const ClusterPlan& plan, bool quad, int n_iters, cudaStream_t st);
+// Same launch shape, nothing but the per-iteration cluster barrier (measurement aid).
+cudaError_t launch_linear_cluster_empty(const ClusterPlan& plan, int n_iters, cudaStream_t st);
 
 // Mean loss of a logistic / quadratic model over rows [first, first + n) of the resident training set at
 // `theta` (device, d floats); result in scratch[0].  `scratch` holds eval_loss_scratch_doubles() doubles.

@@ -482,7 +482,37 @@ cudaError_t launch_cpl(const Params& P, const ClusterPlan& plan, bool quad, int 
   return cudaLaunchKernelEx(&cfg, kern, P, n_iters);
 }
 
+// The cluster kernel's launch shape with nothing in it but its one cluster-wide barrier per iteration:
+// the floor an iteration of this design cannot go below (measurement aid).
+__global__ void __launch_bounds__(LC_THREADS, 1) linear_cluster_empty_kernel(int n_iters) {
+  cg::cluster_group cluster = cg::this_cluster();
+  for (int i = 0; i < n_iters; ++i) cluster.sync();
+}
+
 }  // namespace
+
+cudaError_t launch_linear_cluster_empty(const ClusterPlan& plan, int n_iters, cudaStream_t st) {
+  cudaError_t e = cudaFuncSetAttribute(linear_cluster_empty_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)plan.smem_bytes);
+  if (e != cudaSuccess) return e;
+  if (plan.n_cta > 8) {
+    e = cudaFuncSetAttribute(linear_cluster_empty_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    if (e != cudaSuccess) return e;
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(plan.n_cta);
+  cfg.blockDim = dim3(LC_THREADS);
+  cfg.dynamicSmemBytes = plan.smem_bytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = plan.n_cta;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, linear_cluster_empty_kernel, n_iters);
+}
 
 bool plan_linear_cluster(int d, int G, int M, int D, int B, long long p_pad, size_t smem_optin, ClusterPlan* plan) {
   plan->usable = false;

@@ -1,5 +1,6 @@
 """Host logic of the multi-GPU benchmark path (replicas only: a barrier and a
 max over ranks, no data-path collective), run as two gloo ranks on CPU."""
+import json
 import os
 import subprocess
 import sys
@@ -34,7 +35,7 @@ def test_two_ranks_agree_on_the_slowest_time():
     for p in procs:
         out, err = p.communicate(timeout=180)
         assert p.returncode == 0, err[-2000:]
-        outs.append(eval(out.strip().splitlines()[-1].replace("true", "True")))
+        outs.append(json.loads(out.strip().splitlines()[-1]))
     assert {o["rank"] for o in outs} == {0, 1}
     for o in outs:
         assert o["ms"] == 15.0                      # max over ranks

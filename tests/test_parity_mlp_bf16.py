@@ -1,7 +1,11 @@
-"""CUDA tensor-core path (bf16 operands, fp32 accumulation) vs the CPU oracle
-with the same operand rounding, through the C ABI.  Tolerance 2e-2 relative
-L2: the CUDA path also rounds activations and back-propagated errors to bf16
-between layers, which the oracle (fp64 after operand rounding) does not."""
+"""CUDA tensor-core path (bf16 operands, fp32 accumulation) vs the CPU oracle,
+through the C ABI.  The oracle's bf16 mode rounds every matrix-product operand
+(features, weights, hidden activations, back-propagated errors) where the
+CUDA path does and computes in fp64, so these comparisons measure the
+kernels' arithmetic; tolerance 2e-2 relative L2.  How far the CUDA path is
+from the narrower reading (only features and weight matrices rounded) and
+from the unrounded gradient is measured and bounded in
+test_distance_from_the_other_readings."""
 import numpy as np
 import pytest
 import torch
@@ -9,7 +13,7 @@ import torch
 from paper_2201_04301_b200 import binding
 from paper_2201_04301_b200.workloads import make_workload
 
-from parity import TOL_BF16, forced_parity, to_cuda
+from parity import LHS_TOL_BF16, TOL_BF16, forced_parity, make_oracle, rel_l2, to_cuda
 
 pytestmark = pytest.mark.gpu
 
@@ -81,14 +85,15 @@ def test_aggregate_is_the_sum_of_last_uploads(dims, batch, G):
     assert 0 < m.sum() < m.size
 
 
-def test_running_aggregate_stays_the_sum_of_last_uploads():
+@pytest.mark.parametrize("dims,batch", [((64, 128, 40), 128), ((256, 300, 130), 256), ((512, 768, 520), 256)])
+def test_running_aggregate_stays_the_sum_of_last_uploads(dims, batch):
     """When fewer than half of the groups upload, the aggregate is not formed anew: the selected groups' old
     uploads are taken out of it and their new ones put in (two products over the selected groups' rows), with
     a full recomputation whenever half of the groups upload and at least every 16 iterations.  Under sparse
     forced masks (none, one, a few, all) over several such periods it must stay equal to the sum of the
     groups' last uploads, each rebuilt from its stored factors by a different kernel."""
     G = 12
-    w = to_cuda(make_workload("cfg5", rows=G * 300, dims=(64, 128, 40), M=2 * G, M_G=2, D=100, batch=128, c=0.3))
+    w = to_cuda(make_workload("cfg5", rows=G * 300, dims=dims, M=2 * G, M_G=2, D=100, batch=batch, c=0.3))
     g = binding.from_workload(w, stream=torch.cuda.Stream())
     rng = np.random.default_rng(5)
     worst = 0.0
@@ -104,8 +109,8 @@ def test_running_aggregate_stays_the_sum_of_last_uploads():
             want = sum(g.get_group_gradient(binding.DBG_GLAST, gi).astype(np.float64) for gi in range(G))
             err = np.linalg.norm(agg - want) / np.linalg.norm(want)
             worst = max(worst, err)
-            assert err <= 5e-6, (k, err)
-    print("running aggregate: worst relative error", worst)
+            assert err <= 2e-5, (k, err)        # up to 15 in-place updates of ~1e-6 each between two refreshes
+    print("running aggregate", dims, ": worst relative error", worst)
 
 
 def test_two_pass_norms_against_the_oracle():
@@ -171,3 +176,97 @@ def test_printed_rule_computes_only_the_selected_groups():
     before = h.get_group_gradient(binding.DBG_GLAST, 3)
     h.step_forced(np.zeros((1, G), dtype=np.uint8))
     assert np.array_equal(before, h.get_group_gradient(binding.DBG_GLAST, 3))
+
+
+def test_mid_size_every_cta_walks_several_tiles():
+    """64 groups x 128 rows on 512-1024-768-200: 128 row tiles per point, so the forward and backward-data
+    products have 512 / 384 / 128 output tiles for the 148 persistent CTAs (a CTA walks up to four tiles
+    and both accumulator slots change phase), K = 1024 wraps the four-stage operand ring four times, the
+    weight-gradient kernel runs units of up to four column tiles, and the last layer has a ragged tile.
+    The masks are chosen here (not by the rule) so that at every iteration from the third on the groups sit
+    at three different ages: the row tiles of one launch read three slots of the weight ring.  Two
+    contexts follow the oracle: one that materialises both gradients of every group (compared element by
+    element) and the production one (norm-only pass, uploads kept as factors, gradient rebuilt on demand)."""
+    G, D, K = 64, 3, 6
+    dims = (512, 1024, 768, 200)
+    w = make_workload("cfg5", rows=G * 400, dims=dims, M=2 * G, M_G=2, D=D, batch=128, c=0.3)
+    o = make_oracle(w)
+    wc = to_cuda(w)
+    a = binding.from_workload(wc, stream=torch.cuda.Stream(), options={binding.OPT_KEEP_STALE: 1.0})
+    b = binding.from_workload(wc, stream=torch.cuda.Stream())
+    gs = np.arange(G)
+    worst = dict(fresh=0.0, stale=0.0, lhs_a=0.0, lhs_b=0.0, upload=0.0, theta=0.0)
+    for k in range(K):
+        mask = np.ones(G, dtype=np.uint8) if k == 0 else ((k + gs) % 3 == 0).astype(np.uint8)
+        tau = o.tau.copy()
+        if k >= 3:
+            assert sorted(set(tau.tolist())) == [1, 2, 3]
+        rec = o.step(forced_mask=mask)
+        for ctx in (a, b):
+            ctx.step_forced(mask[None, :])
+        fresh, stale = a.get_debug(binding.DBG_FRESH), a.get_debug(binding.DBG_STALE)
+        for gi in range(G):
+            worst["fresh"] = max(worst["fresh"], rel_l2(fresh[gi], rec["fresh"][gi]))
+            worst["stale"] = max(worst["stale"], rel_l2(stale[gi], rec["stale"][gi]))
+        for name, ctx in (("lhs_a", a), ("lhs_b", b)):
+            lhs = ctx.get_debug(binding.DBG_LHS)
+            nz = rec["lhs"] > 0
+            # equal iterates: the two products cancel up to the fp32 rounding of their accumulation
+            f2 = np.sum(rec["fresh"].astype(np.float64) ** 2, axis=1)
+            assert np.all(lhs[~nz] <= 1e-10 * f2[~nz]), (k, name)
+            if nz.any():
+                worst[name] = max(worst[name], float(np.max(np.abs(lhs[nz] - rec["lhs"][nz]) / rec["lhs"][nz])))
+        for gi in np.nonzero(mask)[0][:6]:        # uploads of the production path, rebuilt from the kept factors
+            worst["upload"] = max(worst["upload"], rel_l2(b.get_group_gradient(binding.DBG_GLAST, gi), rec["fresh"][gi]))
+        for ctx in (a, b):
+            worst["theta"] = max(worst["theta"], rel_l2(ctx.get_theta(), rec["theta"]))
+        assert np.array_equal(a.get_theta(), b.get_theta())
+        assert worst["fresh"] <= TOL_BF16 and worst["stale"] <= TOL_BF16 and worst["upload"] <= TOL_BF16, (k, worst)
+        assert worst["lhs_a"] <= LHS_TOL_BF16 and worst["lhs_b"] <= LHS_TOL_BF16, (k, worst)
+        assert worst["theta"] <= TOL_BF16, (k, worst)
+    assert rel_l2(b.get_debug(binding.DBG_AGG), rec["agg"]) <= TOL_BF16
+    print("bf16 mid-size", dims, "worst", worst)
+
+
+def test_distance_from_the_other_readings():
+    """The CUDA path rounds hidden activations and back-propagated errors to bf16 between layers (they are
+    operands of the next product) and its bias copy too.  This test puts on record how far that is from
+    (i) the narrower reading - only the features and the weight matrices are bf16, everything else exact -
+    and (ii) the unrounded fp64 gradient of the fp32 master parameters, for fresh gradients and for the
+    left side of the selection test, on a network wide enough that the rounding flips ReLU units.  The
+    bounds asserted are about twice the values measured when the test was written."""
+    from oracle.models import MLP
+    from oracle import philox
+    G, D, K = 4, 3, 4
+    dims = (256, 768, 512, 100)
+    w = make_workload("cfg5", rows=G * 2000, dims=dims, M=G, M_G=1, D=D, batch=128, c=0.3, alpha=1e-3)
+    X = w["X"].float().numpy().astype(np.float64)
+    y = w["y"].numpy()
+    g = binding.from_workload(to_cuda(w), stream=torch.cuda.Stream(), options={binding.OPT_KEEP_STALE: 1.0})
+    models = {"operands": MLP(dims, bf16="operands"), "exact": MLP(dims), "all": MLP(dims, bf16=True)}
+    thetas = []
+    worst = {m: dict(fresh=0.0, lhs=0.0) for m in models}
+    tau = np.full(G, D)
+    n_g = X.shape[0] // G
+    for k in range(K):
+        thetas.append(g.get_theta().astype(np.float64))
+        mask = np.ones(G, dtype=np.uint8) if k == 0 else ((k + np.arange(G)) % 2 == 0).astype(np.uint8)
+        g.step_forced(mask[None, :])
+        fresh, lhs = g.get_debug(binding.DBG_FRESH), g.get_debug(binding.DBG_LHS)
+        for gi in range(G):
+            idx = philox.batch_indices(w["seed"], k, gi, w["batch"], n_g) + 0
+            Xb, yb = X[idx], y[idx]
+            for name, m in models.items():
+                f = m.grad(thetas[k], Xb, yb, "mean")
+                worst[name]["fresh"] = max(worst[name]["fresh"], rel_l2(fresh[gi], f))
+                if k > 0:
+                    s = m.grad(thetas[max(k - int(tau[gi]), 0)], Xb, yb, "mean")
+                    want = float(np.sum((f - s) ** 2))
+                    worst[name]["lhs"] = max(worst[name]["lhs"], abs(lhs[gi] - want) / want)
+        tau = np.where(mask, 1, tau + 1)
+    print("bf16 CUDA path vs readings (worst relative error; fresh = L2 of the gradient, lhs = squared norm):", worst)
+    assert worst["all"]["fresh"] <= TOL_BF16 and worst["all"]["lhs"] <= LHS_TOL_BF16
+    # measured on this case: gradient 2.7e-2 (features and weight matrices only) / 3.7e-2 (unrounded),
+    # left side of the test 5.7e-3 / 7.8e-3, against 2.0e-4 / 3.3e-5 for the reading the oracle shares
+    assert worst["operands"]["fresh"] <= 5e-2 and worst["exact"]["fresh"] <= 7e-2
+    assert worst["operands"]["lhs"] <= 2e-2 and worst["exact"]["lhs"] <= 2e-2
