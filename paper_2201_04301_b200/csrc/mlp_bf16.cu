@@ -6,8 +6,11 @@
 // weight gradients are never materialised on the production path: a first pass
 // forms only the squared innovation norms, and the server's aggregate (Eq. 3,
 // the sum over groups of each group's last uploaded gradient) is one product per
-// layer over the stored factors (dz_l^T, a_{l-1}^T) of every group's last
-// upload, with K running over all groups' rows.  Every product is an "NT" GEMM  C[M x N] = A[M x K] * B[N x K]^T
+// layer over the factors (dz_l^T, a_{l-1}^T) of every group's last
+// upload, with K running over all groups' rows.  The factors at theta^k are
+// written into one of two buffers per group; the other one holds the group's last
+// upload, and selecting the group flips the two (Params::cur), so an upload moves
+// no data.  Every product is an "NT" GEMM  C[M x N] = A[M x K] * B[N x K]^T
 // with both operands K-major, so one kernel serves all of them:
 //     forward   z_l   = a_{l-1} W_l^T        A = a_{l-1} [rows][n_{l-1}],  B = W_l   [n_l][n_{l-1}]
 //     backward  da    = dz_l W_l             A = dz_l    [rows][n_l],      B = W_l^T [n_{l-1}][n_l]
@@ -49,26 +52,25 @@ struct Bf16Impl {
   __nv_bfloat16* wb = nullptr;   // (D+1) slots
   float* bias = nullptr;         // (D+1) slots of rounded biases
   __nv_bfloat16* xb = nullptr;   // [G*Bp][ld0]
-  __nv_bfloat16* xbT = nullptr;  // [G][n_0][Bp]
   int* yb = nullptr;             // [G*Bp], -1 on padding rows
   __nv_bfloat16* act[MLP_MAX_LAYERS + 1] = {nullptr};   // [2][G*Bp][ld_l]
-  __nv_bfloat16* actT[MLP_MAX_LAYERS + 1] = {nullptr};  // [2][G][n_l][Bp]
   __nv_bfloat16* dz[MLP_MAX_LAYERS + 1] = {nullptr};
-  __nv_bfloat16* dzT[MLP_MAX_LAYERS + 1] = {nullptr};
   float* scores = nullptr;       // [2][G*Bp][n_L]
-  // factors of each group's last uploaded weight gradient, dW_l = lastA[l][g] * lastB[l][g]^T
-  __nv_bfloat16* lastA[MLP_MAX_LAYERS + 1] = {nullptr};  // [G][n_l][Bp]      dz_l^T at the upload
-  __nv_bfloat16* lastB[MLP_MAX_LAYERS + 1] = {nullptr};  // [G][n_{l-1}][Bp]  a_{l-1}^T at the upload
+  // Transposed copies = the factors of the weight gradients, dW_l(g) = dzT[l](g) * actT[l-1](g)^T.  Entries
+  // [0, 2G) are two upload buffers per group (entry b*G + g): buffer cur[g] holds the factors of the group's
+  // last upload, the other one receives the factors at theta^k; the selection flips cur[g] and thereby keeps
+  // the upload.  Entries [2G, 3G) hold the stale point's factors of this iteration (never kept).
+  __nv_bfloat16* xbT = nullptr;                         // [2][G][n_0][Bp] (the features serve both points)
+  __nv_bfloat16* actT[MLP_MAX_LAYERS + 1] = {nullptr};  // [3][G][n_l][Bp]
+  __nv_bfloat16* dzT[MLP_MAX_LAYERS + 1] = {nullptr};   // [3][G][n_l][Bp]
   int nbias = 0;                                         // bias entries of all layers
   int bias_loc[MLP_MAX_LAYERS + 2] = {0};                // first entry of layer l in the compact bias arrays
-  float* db_fresh = nullptr;     // [G][nbias] bias gradients at theta^k, this iteration
-  float* db_last = nullptr;      // [G][nbias] bias gradients of each group's last upload
+  float* db = nullptr;           // [2][G][nbias] bias gradients, the same two buffers per group
   int dw_part_base[MLP_MAX_LAYERS + 1] = {0}, bias_part_base[MLP_MAX_LAYERS + 1] = {0};
   int n_parts = 0;               // innovation-norm partial sums per group
   CUtensorMap tm_fwd_a[MLP_MAX_LAYERS + 1], tm_fwd_b[MLP_MAX_LAYERS + 1];
   CUtensorMap tm_da_a[MLP_MAX_LAYERS + 1], tm_da_b[MLP_MAX_LAYERS + 1];
-  CUtensorMap tm_dw_a[MLP_MAX_LAYERS + 1], tm_dw_b[MLP_MAX_LAYERS + 1];
-  CUtensorMap tm_agg_a[MLP_MAX_LAYERS + 1], tm_agg_b[MLP_MAX_LAYERS + 1];
+  CUtensorMap tm_dw_a[MLP_MAX_LAYERS + 1], tm_dw_b[MLP_MAX_LAYERS + 1];  // the factor arrays (also the aggregate's operands)
 };
 
 struct GemmB {
@@ -79,14 +81,13 @@ struct GemmB {
   int stages;
   int k_batched;     // 1: one output [M][N]; K runs over the batch entries of both operands (kpg K blocks each)
   int kpg, n_batch;
-  int agg_pass;      // k_batched products that maintain the aggregate of Eq. (3) from the last-upload store:
-                     // 0: sum over all n_batch entries, written (not added);
-                     // 1: before the selected groups' uploads are stored - minus the sum over the SELECTED
-                     //    groups' entries (their old uploads), added to the output;
-                     // 2: after they are stored - plus the sum over the selected groups' entries, added.
-                     // Passes 1 and 2 together replace the selected groups' terms.  When at least half of the
-                     // groups are selected, and every AGG_REFRESH-th iteration (so that rounding cannot pile
-                     // up), pass 1 does nothing and pass 2 is the full sum of pass 0.
+                     // k_batched products maintain the aggregate of Eq. (3) from the groups' upload buffers
+                     // (run after the selection has flipped cur[] of the selected groups).  When fewer than half
+                     // of the groups are selected, K runs over the SELECTED groups twice - their replaced
+                     // uploads (buffer 1 - cur[g]) with the A operand negated, then their new ones (buffer
+                     // cur[g]) - and the result is added to the output.  Otherwise, and every AGG_REFRESH-th
+                     // iteration (so that rounding cannot pile up), K runs over every group's buffer cur[g] and
+                     // the sum is written anew.
   // epilogue operands
   __nv_bfloat16* out;    // row-major bf16 [z][M][ldo]
   __nv_bfloat16* outT;   // transposed bf16 [z][N][ldt]
@@ -200,6 +201,15 @@ __device__ __forceinline__ int ring_slot(const Params& P, int g, int q, long lon
   return (int)(j % (P.D + 1));
 }
 
+// Upload buffer that receives group g's factors at theta^k.  Normally the gradients come before the
+// selection: the buffer that does not hold the last upload.  When the selection came first (printed rule,
+// only the selected groups compute) cur[g] has already been flipped and names the buffer to fill.
+__device__ __forceinline__ int fresh_buf(const Params& P, int g) { return P.skip_unselected ? P.cur[g] : 1 - P.cur[g]; }
+// Batch entry of (point q, group g) in the factor arrays.
+__device__ __forceinline__ int factor_entry(const Params& P, int g, int q) {
+  return q == 0 ? fresh_buf(P, g) * P.G + g : 2 * P.G + g;
+}
+
 // ----------------------------------------------------------------- GEMM (forward and backward-data products)
 // Persistent: one CTA per SM walks 128 x 256 output tiles (N fastest, so that
 // the CTAs running together share operand tiles in L2); tensor memory holds
@@ -229,18 +239,15 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // aggregate passes: which batch entries, with which sign, written or added (the same in every thread of the grid)
   int n_batch = a.n_batch;
-  bool listed = false, negate = false;
-  if (a.k_batched && a.agg_pass != 0) {
-    const int n_sel = P.sel_count[0];
+  int n_sel = 0;
+  bool listed = false;
+  if (a.k_batched) {
+    n_sel = P.sel_count[0];
     const bool refresh = 2 * n_sel >= P.G || (P.st->k % AGG_REFRESH) == 0;
-    if (a.agg_pass == 1) {
-      if (refresh || n_sel == 0) return;
-      listed = negate = true;
-      n_batch = n_sel;
-    } else if (!refresh) {
+    if (!refresh) {
       if (n_sel == 0) return;  // no upload: the aggregate stands
       listed = true;
-      n_batch = n_sel;
+      n_batch = 2 * n_sel;     // the replaced uploads (negated), then the new ones
     }
   }
   const bool accumulate = listed;
@@ -284,8 +291,15 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
         const int g = a.k_batched ? 0 : (P.skip_unselected ? P.sel_list[zi - q * n_grp] : zi - q * n_grp);
         const int z = q * P.G + g;
         int zA = 0, zB = 0, ent = 0;
+        // entry e of a k_batched product: every group's last upload, or (listed) the selected groups' replaced
+        // uploads followed by their new ones
+        auto agg_entry = [&](int e) {
+          if (!listed) return (int)P.cur[e] * P.G + e;
+          const int gs = P.sel_list[e < n_sel ? e : e - n_sel];
+          return (e < n_sel ? 1 - (int)P.cur[gs] : (int)P.cur[gs]) * P.G + gs;
+        };
         if (a.k_batched) {
-          zA = zB = listed ? P.sel_list[0] : 0;
+          zA = zB = agg_entry(0);
         } else {
           zA = a.a_shared ? g : z;
           zB = a.zb_mode == ZB_RING ? ring_slot(P, g, q, k_it) : (a.zb_mode == ZB_GROUP ? g : z);
@@ -303,7 +317,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
           if (a.k_batched && ++kin == a.kpg) {
             kin = 0;
             ++ent;
-            zA = zB = (listed && ent < n_batch) ? P.sel_list[ent] : ent;
+            if (ent < n_batch) zA = zB = agg_entry(ent);
           }
         }
       }
@@ -325,6 +339,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
           tc_fence_after();
           const uint32_t sa = smem_u32(tiles + (size_t)s * G_STAGE_BYTES);
           const uint64_t da = make_desc(sa), db = make_desc(sa + BM * BK * 2);
+          const bool negate = listed && kb < a.kpg * n_sel;  // the replaced uploads leave the sum (A negated, bit 13)
 #pragma unroll
           for (int kk = 0; kk < BK / 16; ++kk)  // 16 bf16 = 32 bytes = 2 descriptor units per MMA
             tc_mma_bf16(tmem_base + (uint32_t)(slot * GN), da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2),
@@ -349,6 +364,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
       const int q = a.k_batched ? 0 : zi / n_grp;
       const int g = a.k_batched ? 0 : (P.skip_unselected ? P.sel_list[zi - q * n_grp] : zi - q * n_grp);
       const int z = q * P.G + g;
+      const int zT = a.k_batched ? 0 : factor_entry(P, g, q);  // entry of the transposed copy (a factor array)
       const int m = mt * BM + quad * 32 + lane;
       const int n0 = nt * GN;
       // EPI_DA: the ReLU mask of this thread's row does not depend on the accumulator, so it is fetched (one
@@ -471,7 +487,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
               *reinterpret_cast<uint4*>(dst0 + (long long)r * a.ldo + qd * 8) = make_uint4(src[0], src[1], src[2], src[3]);
             }
             // transposed copy: lanes 4n..4n+3 write the 64 bytes (32 rows) of output row nc + n
-            __nv_bfloat16* dstT0 = a.outT + (long long)z * a.z_stride_outT + (long long)nc * a.ldt + (mt * BM + quad * 32);
+            __nv_bfloat16* dstT0 = a.outT + (long long)zT * a.z_stride_outT + (long long)nc * a.ldt + (mt * BM + quad * 32);
 #pragma unroll
             for (int it = 0; it < 4; ++it) {
               const int n = it * 8 + (lane >> 2), qd = lane & 3;
@@ -500,7 +516,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
               const uint32_t e1 = (lane & 1) ? (w1 >> 16) : (w1 & 0xFFFFu);
               o[r >> 1] = e0 | (e1 << 16);
             }
-            __nv_bfloat16* dstT = a.outT + (long long)z * a.z_stride_outT + (long long)(nc + lane) * a.ldt +
+            __nv_bfloat16* dstT = a.outT + (long long)zT * a.z_stride_outT + (long long)(nc + lane) * a.ldt +
                                   (mt * BM + quad * 32);
 #pragma unroll
             for (int j = 0; j < 16; j += 4)
@@ -558,7 +574,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
 // per-warp staging tile.
 struct DwArgs {
   int M, N, K;            // n_l, n_{l-1}, padded rows per group
-  int b_shared;           // 1: operand B has one entry per group (the gathered features)
+  int b_shared;           // 1: operand B is the same for both points (the gathered features)
   int nkb;                // K blocks per point
   int stages;
   int tiles_m, tiles_n, total_tiles;
@@ -630,13 +646,15 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
       int it = 0, ui = 0;
       for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
         const int mt = u % a.tiles_m, g = a.mode == DW_ONE ? a.g_only : u / a.tiles_m;
+        const int zone = (int)P.cur[g] * P.G + g;  // DW_ONE: the group's last upload
         // the unit's A blocks, once the MMAs of the previous unit have finished reading them
         ok = mbar_spin_bounded(&aempty_bar, (uint32_t)((ui & 1) ^ 1));
         if (!ok) break;
         mbar_expect_tx(&afull_bar, (uint32_t)(kb_per_tile * BLK));
         for (int j = 0; j < kb_per_tile; ++j) {
           const int q = j / a.nkb, kb = j - q * a.nkb;
-          tma_load_3d(a_res + (size_t)j * BLK, &tmA, kb * BK, mt * BM, q * P.G + g, &afull_bar);
+          tma_load_3d(a_res + (size_t)j * BLK, &tmA, kb * BK, mt * BM, a.mode == DW_ONE ? zone : factor_entry(P, g, q),
+                      &afull_bar);
         }
         ++ui;
         for (int nt = 0; nt < a.tiles_n && ok; ++nt) {
@@ -646,7 +664,8 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
             ok = mbar_spin_bounded(&empty_bar[s], (uint32_t)(((it / stages) & 1) ^ 1));
             if (!ok) break;
             mbar_expect_tx(&full_bar[s], BBLK);
-            tma_load_3d(tiles + (size_t)s * BBLK, &tmB, kb * BK, nt * DW_BN, a.b_shared ? g : q * P.G + g, &full_bar[s]);
+            tma_load_3d(tiles + (size_t)s * BBLK, &tmB, kb * BK, nt * DW_BN,
+                        a.mode == DW_ONE ? zone : factor_entry(P, g, a.b_shared ? 0 : q), &full_bar[s]);
           }
         }
       }
@@ -869,6 +888,7 @@ __global__ void __launch_bounds__(256) bf16_gather_kernel(const Params P, __nv_b
   const int g = blockIdx.y, rb = blockIdx.x * 32;
   const int tid = threadIdx.x;
   if (P.skip_unselected && !P.mask_cur[g]) return;
+  const int fb = fresh_buf(P, g);
   if (tid < 32) {
     const int j = rb + tid;
     long long row = -1;
@@ -908,7 +928,7 @@ __global__ void __launch_bounds__(256) bf16_gather_kernel(const Params P, __nv_b
     __syncthreads();
     for (int e = tid; e < GT_COLS * 32; e += 256) {
       const int c = e >> 5, r = e & 31;
-      if (c0 + c < d) xbT[((long long)g * d + c0 + c) * Bp + rb + r] = tile[r * GT_PITCH + c];
+      if (c0 + c < d) xbT[(((long long)fb * P.G + g) * d + c0 + c) * Bp + rb + r] = tile[r * GT_PITCH + c];
     }
     __syncthreads();
   }
@@ -961,7 +981,7 @@ __global__ void __launch_bounds__(256) bf16_softmax_grad_kernel(const Params P, 
     }
   }
   __syncthreads();
-  __nv_bfloat16* oT = dzT + ((long long)(q * P.G + g) * n_cls) * Bp + m0;
+  __nv_bfloat16* oT = dzT + ((long long)factor_entry(P, g, q) * n_cls) * Bp + m0;
   for (int c = warp; c < n_cls; c += 8) oT[(long long)c * Bp + lane] = sm_tile[lane * pitch + c];
 }
 
@@ -1023,7 +1043,7 @@ __global__ void __launch_bounds__(256) bf16_softmax_grad_pairs_kernel(const Para
     }
   }
   __syncthreads();
-  __nv_bfloat16* oT = dzT + ((long long)(q * P.G + g) * n_cls) * Bp + m0;
+  __nv_bfloat16* oT = dzT + ((long long)factor_entry(P, g, q) * n_cls) * Bp + m0;
   for (int c = warp; c < n_cls; c += 8) oT[(long long)c * Bp + lane] = sm_tile[lane * pitch + c];
 }
 
@@ -1036,7 +1056,7 @@ struct BiasArgsB {
   long long b_off[MLP_MAX_LAYERS + 1];
   int part_base[MLP_MAX_LAYERS + 1];
   int n_parts;
-  float* db_fresh;                    // [G][nbias]
+  float* db;                          // [2][G][nbias], buffer fresh_buf(g) receives this iteration's
   int bias_loc[MLP_MAX_LAYERS + 1];   // first entry of layer l in a db row
   int nbias;
 };
@@ -1080,7 +1100,7 @@ __global__ void __launch_bounds__(256) bf16_bias_grad_kernel(const Params P, con
         f += red[0][w][threadIdx.x];
         sv += red[1][w][threadIdx.x];
       }
-      a.db_fresh[(long long)g * a.nbias + a.bias_loc[l] + c] = f;
+      a.db[((long long)fresh_buf(P, g) * P.G + g) * a.nbias + a.bias_loc[l] + c] = f;
       if (P.gbuf) (fresh_row(P, g) + a.b_off[l])[c] = f;  // kept for inspection
       if (P.stale) (P.stale + (long long)g * P.p_pad + a.b_off[l])[c] = sv;
       d2 = (double)(f - sv) * (double)(f - sv);
@@ -1090,34 +1110,10 @@ __global__ void __launch_bounds__(256) bf16_bias_grad_kernel(const Params P, con
   if (threadIdx.x == 0) P.lhs_part[(long long)g * a.n_parts + a.part_base[l] + blockIdx.x] = d2;
 }
 
-// ----------------------------------------------------------------- upload: keep the selected groups' factors
-// A selected group's upload replaces its last uploaded gradient (Eq. 3).  The weight gradient is kept as its
-// two factors (dz_l^T and a_{l-1}^T at theta^k, bf16), the bias gradient as it is.  Grid (slices, G).
-struct KeepArgs {
-  const __nv_bfloat16* src[2 * MLP_MAX_LAYERS];
-  __nv_bfloat16* dst[2 * MLP_MAX_LAYERS];
-  long long elems[2 * MLP_MAX_LAYERS];  // per group; a multiple of 8
-  int n_seg;
-  const float* db_fresh;
-  float* db_last;
-  int nbias;
-};
-__global__ void __launch_bounds__(256) bf16_keep_kernel(const Params P, const KeepArgs a) {
-  const int g = blockIdx.y;
-  if (!P.mask_cur[g]) return;
-  for (int s = 0; s < a.n_seg; ++s) {
-    const uint4* src = reinterpret_cast<const uint4*>(a.src[s] + (long long)g * a.elems[s]);
-    uint4* dst = reinterpret_cast<uint4*>(a.dst[s] + (long long)g * a.elems[s]);
-    const long long n16 = a.elems[s] >> 3;
-    for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < n16; i += (long long)gridDim.x * 256) dst[i] = src[i];
-  }
-  for (int i = blockIdx.x * 256 + threadIdx.x; i < a.nbias; i += gridDim.x * 256)
-    a.db_last[(long long)g * a.nbias + i] = a.db_fresh[(long long)g * a.nbias + i];
-}
-
+// ----------------------------------------------------------------- bias part of the aggregate
 // Bias part of the aggregate: sum over groups (ascending) of the last uploaded bias gradients.
 struct BiasAggArgs {
-  const float* db_last;
+  const float* db;   // [2][G][nbias]; buffer cur[g] holds group g's last upload
   int nbias, n_layers;
   int bias_loc[MLP_MAX_LAYERS + 2];
   long long b_off[MLP_MAX_LAYERS + 1];
@@ -1126,19 +1122,19 @@ __global__ void __launch_bounds__(256) bf16_bias_agg_kernel(const Params P, cons
   const int i = blockIdx.x * 256 + threadIdx.x;
   if (i >= a.nbias) return;
   float s = 0.f;
-  for (int g = 0; g < P.G; ++g) s += a.db_last[(long long)g * a.nbias + i];
+  for (int g = 0; g < P.G; ++g) s += a.db[((long long)P.cur[g] * P.G + g) * a.nbias + i];
   int l = 1;
   while (l < a.n_layers && i >= a.bias_loc[l + 1]) ++l;
   agg[a.b_off[l] + (i - a.bias_loc[l])] = s;
 }
 
 // One group's bias gradient of its last upload into a p-vector (getters).
-__global__ void __launch_bounds__(256) bf16_bias_row_kernel(const BiasAggArgs a, int g, float* row) {
+__global__ void __launch_bounds__(256) bf16_bias_row_kernel(const Params P, const BiasAggArgs a, int g, float* row) {
   const int i = blockIdx.x * 256 + threadIdx.x;
   if (i >= a.nbias) return;
   int l = 1;
   while (l < a.n_layers && i >= a.bias_loc[l + 1]) ++l;
-  row[a.b_off[l] + (i - a.bias_loc[l])] = a.db_last[(long long)g * a.nbias + i];
+  row[a.b_off[l] + (i - a.bias_loc[l])] = a.db[((long long)P.cur[g] * P.G + g) * a.nbias + i];
 }
 
 // ----------------------------------------------------------------- host
@@ -1192,7 +1188,7 @@ cudaError_t launch_dw(const Params& P, const MlpPlan& pl, const Bf16Impl* im, in
   w.M = pl.dims[l];
   w.N = pl.dims[l - 1];
   w.K = im->Bp;
-  w.b_shared = (l == 1 || mode == DW_ONE) ? 1 : 0;  // the last-upload stores have one entry per group
+  w.b_shared = l == 1 ? 1 : 0;
   w.nkb = im->Bp / BK;
   // 32 KiB B blocks in whatever shared memory is left beside the resident A blocks (and the staging tile of
   // the modes that write gradients): the B stream is bound by bytes in flight, so every stage counts
@@ -1212,10 +1208,7 @@ cudaError_t launch_dw(const Params& P, const MlpPlan& pl, const Bf16Impl* im, in
   const int units = mode == DW_ONE ? w.tiles_m : w.tiles_m * P.G;
   const int ctas = units < pl.sm_count ? units : pl.sm_count;
   const size_t smem = (size_t)(2 * w.nkb + 2 * w.stages) * (BM * BK * 2) + 1024 + (size_t)stage_bytes;
-  if (mode == DW_ONE)
-    bf16_dw_kernel<<<ctas, DW_THREADS, smem, st>>>(im->tm_agg_a[l], im->tm_agg_b[l], P, w);
-  else
-    bf16_dw_kernel<<<ctas, DW_THREADS, smem, st>>>(im->tm_dw_a[l], im->tm_dw_b[l], P, w);
+  bf16_dw_kernel<<<ctas, DW_THREADS, smem, st>>>(im->tm_dw_a[l], im->tm_dw_b[l], P, w);
   return cudaGetLastError();
 }
 
@@ -1280,33 +1273,30 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
   A_(im->wb, (long long)(D + 1) * im->slot_elems, __nv_bfloat16);
   A_(im->bias, (long long)(D + 1) * im->bias_slot, float);
   A_(im->xb, rows * im->ld[0], __nv_bfloat16);
-  A_(im->xbT, (long long)G * plan->dims[0] * im->Bp, __nv_bfloat16);
+  A_(im->xbT, 2LL * G * plan->dims[0] * im->Bp, __nv_bfloat16);
   A_(im->yb, rows, int);
   for (int l = 1; l <= L; ++l) {
     if (l < L) {
       A_(im->act[l], 2 * rows * im->ld[l], __nv_bfloat16);
-      A_(im->actT[l], 2LL * G * plan->dims[l] * im->Bp, __nv_bfloat16);
+      A_(im->actT[l], 3LL * G * plan->dims[l] * im->Bp, __nv_bfloat16);
     }
     A_(im->dz[l], 2 * rows * im->ld[l], __nv_bfloat16);
-    A_(im->dzT[l], 2LL * G * plan->dims[l] * im->Bp, __nv_bfloat16);
+    A_(im->dzT[l], 3LL * G * plan->dims[l] * im->Bp, __nv_bfloat16);
   }
   A_(im->scores, 2 * rows * plan->dims[L], float);
-  for (int l = 1; l <= L; ++l) {
-    A_(im->lastA[l], (long long)G * plan->dims[l] * im->Bp, __nv_bfloat16);
-    A_(im->lastB[l], (long long)G * plan->dims[l - 1] * im->Bp, __nv_bfloat16);
-  }
-  A_(im->db_fresh, (long long)G * im->nbias, float);
-  A_(im->db_last, (long long)G * im->nbias, float);
+  A_(im->db, 2LL * G * im->nbias, float);
 #undef A_
   // what an iteration reads from earlier ones: the bf16 copies of the last D+1 iterates and every group's last upload
   plan->state.clear();
   plan->state.emplace_back(im->wb, sizeof(__nv_bfloat16) * (size_t)(D + 1) * im->slot_elems);
   plan->state.emplace_back(im->bias, sizeof(float) * (size_t)(D + 1) * im->bias_slot);
+  // (both upload buffers of every group: which of the two holds the last upload is in Params::cur)
+  plan->state.emplace_back(im->xbT, sizeof(__nv_bfloat16) * (size_t)2 * G * plan->dims[0] * im->Bp);
   for (int l = 1; l <= L; ++l) {
-    plan->state.emplace_back(im->lastA[l], sizeof(__nv_bfloat16) * (size_t)G * plan->dims[l] * im->Bp);
-    plan->state.emplace_back(im->lastB[l], sizeof(__nv_bfloat16) * (size_t)G * plan->dims[l - 1] * im->Bp);
+    plan->state.emplace_back(im->dzT[l], sizeof(__nv_bfloat16) * (size_t)2 * G * plan->dims[l] * im->Bp);
+    if (l < L) plan->state.emplace_back(im->actT[l], sizeof(__nv_bfloat16) * (size_t)2 * G * plan->dims[l] * im->Bp);
   }
-  plan->state.emplace_back(im->db_last, sizeof(float) * (size_t)G * im->nbias);
+  plan->state.emplace_back(im->db, sizeof(float) * (size_t)2 * G * im->nbias);
   if (!encode_fn()) {
     *why = "cuTensorMapEncodeTiled is not available from this driver";
     return cudaSuccess;
@@ -1325,14 +1315,13 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
     ok &= make_map(&im->tm_da_a[l], im->dz[l], no, Bp, 2LL * G, im->ld[l], Bp * im->ld[l], BM);
     ok &= make_map(&im->tm_da_b[l], im->wb + im->wt_pos[l], no, ni, D + 1, im->ld[l], im->slot_elems, GN);
     // weight gradient: A = dz_l^T, B = a_{l-1}^T
-    ok &= make_map(&im->tm_dw_a[l], im->dzT[l], Bp, no, 2LL * G, Bp, (long long)no * Bp, BM);
+    // (the aggregate reads the same two arrays: the groups' upload buffers are their first 2G entries)
+    static_assert(DW_BN == GN, "the weight-gradient and aggregate products share their B tensor map");
+    ok &= make_map(&im->tm_dw_a[l], im->dzT[l], Bp, no, 3LL * G, Bp, (long long)no * Bp, BM);
     if (l == 1)
-      ok &= make_map(&im->tm_dw_b[l], im->xbT, Bp, ni, G, Bp, (long long)ni * Bp, DW_BN);
+      ok &= make_map(&im->tm_dw_b[l], im->xbT, Bp, ni, 2LL * G, Bp, (long long)ni * Bp, DW_BN);
     else
-      ok &= make_map(&im->tm_dw_b[l], im->actT[l - 1], Bp, ni, 2LL * G, Bp, (long long)ni * Bp, DW_BN);
-    // aggregate: the same two operands, taken from the last-upload stores (one entry per group)
-    ok &= make_map(&im->tm_agg_a[l], im->lastA[l], Bp, no, G, Bp, (long long)no * Bp, BM);
-    ok &= make_map(&im->tm_agg_b[l], im->lastB[l], Bp, ni, G, Bp, (long long)ni * Bp, GN);
+      ok &= make_map(&im->tm_dw_b[l], im->actT[l - 1], Bp, ni, 3LL * G, Bp, (long long)ni * Bp, DW_BN);
   }
   if (!ok) {
     *why = "tensor map creation failed for this MLP shape";
@@ -1353,7 +1342,7 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
   e = cudaFuncSetAttribute(bf16_dw_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024);  // the kernel's static arrays take under 1 KiB
   if (e != cudaSuccess) return e;
   plan->launches_per_iter = 3 + L + 1 + L + (L - 1);
-  plan->post_launches = 2 * L + 2;
+  plan->post_launches = L + 1;
   plan->skip_launches = 2 + L + 1 + (L - 1) + 1;
   return cudaSuccess;
 }
@@ -1470,7 +1459,7 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
     if (pl.dims[l] > maxn) maxn = pl.dims[l];
   }
   ba.n_parts = im->n_parts;
-  ba.db_fresh = im->db_fresh;
+  ba.db = im->db;
   ba.nbias = im->nbias;
   bf16_bias_grad_kernel<<<dim3((maxn + 63) / 64, G, L), 256, 0, st>>>(P, ba, Bp);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
@@ -1485,7 +1474,7 @@ namespace gcada {
 namespace {
 BiasAggArgs bias_agg_args(const MlpPlan& pl, const Bf16Impl* im) {
   BiasAggArgs b{};
-  b.db_last = im->db_last;
+  b.db = im->db;
   b.nbias = im->nbias;
   b.n_layers = pl.n_layers;
   for (int l = 1; l <= pl.n_layers + 1; ++l) b.bias_loc[l] = im->bias_loc[l];
@@ -1494,54 +1483,32 @@ BiasAggArgs bias_agg_args(const MlpPlan& pl, const Bf16Impl* im) {
 }
 }  // namespace
 
-// After the selection, the server's side of Eq. (3): the selected groups' uploads replace their last
-// uploaded gradients (kept as factors) in the aggregate, the sum over ALL groups of the last uploaded
-// gradients.  Each layer's share is one product whose K dimension runs over groups' rows: over the selected
-// groups only - minus their old uploads before the store is updated, plus the new ones after it - when
-// fewer than half of the groups upload, over every group (the sum formed anew) otherwise and at least every
-// AGG_REFRESH iterations, which keeps the rounding of the running sum from piling up.
+// After the selection (which has flipped cur[] of the selected groups, so that their uploads are kept), the
+// server's side of Eq. (3): the aggregate is the sum over ALL groups of the last uploaded gradients.  Each
+// layer's share is one product whose K dimension runs over groups' rows: over the selected groups only - their
+// replaced uploads with a minus sign, then their new ones - when fewer than half of the groups upload, over
+// every group (the sum formed anew) otherwise and at least every AGG_REFRESH iterations, which keeps the
+// rounding of the running sum from piling up.
 cudaError_t mlp_bf16_launch_post(const Params& P, const MlpPlan& pl, cudaStream_t st, int* n_launches) {
   *n_launches = 0;
   const Bf16Impl* im = static_cast<const Bf16Impl*>(pl.bf16_impl);
   const int L = pl.n_layers, G = P.G, Bp = im->Bp;
   cudaError_t e;
-  auto aggregate = [&](int pass) -> cudaError_t {
-    for (int l = L; l >= 1; --l) {
-      GemmB a{};
-      a.M = pl.dims[l];
-      a.N = pl.dims[l - 1];
-      a.K = G * Bp;
-      a.k_batched = 1;
-      a.kpg = Bp / BK;
-      a.n_batch = G;
-      a.agg_pass = pass;
-      a.epi = EPI_AGG;
-      a.out_f32 = P.agg_hi;
-      a.c_off = pl.w_off[l];
-      a.ldc = pl.dims[l - 1];
-      cudaError_t e2 = launch_gemm(im->tm_agg_a[l], im->tm_agg_b[l], P, a, pl.sm_count, st);
-      if (e2 != cudaSuccess) return e2;
-      ++*n_launches;
-    }
-    return cudaSuccess;
-  };
-  if ((e = aggregate(1)) != cudaSuccess) return e;  // minus the uploads that are about to be replaced
-  KeepArgs k{};
-  for (int l = 1; l <= L; ++l) {
-    k.src[k.n_seg] = im->dzT[l];
-    k.dst[k.n_seg] = im->lastA[l];
-    k.elems[k.n_seg++] = (long long)pl.dims[l] * Bp;
-    k.src[k.n_seg] = l == 1 ? im->xbT : im->actT[l - 1];
-    k.dst[k.n_seg] = im->lastB[l];
-    k.elems[k.n_seg++] = (long long)pl.dims[l - 1] * Bp;
+  for (int l = L; l >= 1; --l) {
+    GemmB a{};
+    a.M = pl.dims[l];
+    a.N = pl.dims[l - 1];
+    a.K = G * Bp;
+    a.k_batched = 1;
+    a.kpg = Bp / BK;
+    a.n_batch = G;
+    a.epi = EPI_AGG;
+    a.out_f32 = P.agg_hi;
+    a.c_off = pl.w_off[l];
+    a.ldc = pl.dims[l - 1];
+    if ((e = launch_gemm(im->tm_dw_a[l], im->tm_dw_b[l], P, a, pl.sm_count, st)) != cudaSuccess) return e;
+    ++*n_launches;
   }
-  k.db_fresh = im->db_fresh;
-  k.db_last = im->db_last;
-  k.nbias = im->nbias;
-  bf16_keep_kernel<<<dim3(64, G), 256, 0, st>>>(P, k);
-  if ((e = cudaGetLastError()) != cudaSuccess) return e;
-  ++*n_launches;
-  if ((e = aggregate(2)) != cudaSuccess) return e;  // plus the new ones (or the full sum, see GemmB::agg_pass)
   bf16_bias_agg_kernel<<<(im->nbias + 255) / 256, 256, 0, st>>>(P, bias_agg_args(pl, im), P.agg_hi);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   ++*n_launches;
@@ -1555,7 +1522,7 @@ cudaError_t mlp_bf16_group_gradient(const Params& P, const MlpPlan& pl, int g, f
     cudaError_t e = launch_dw(P, pl, im, l, DW_ONE, st, g, row);
     if (e != cudaSuccess) return e;
   }
-  bf16_bias_row_kernel<<<(im->nbias + 255) / 256, 256, 0, st>>>(bias_agg_args(pl, im), g, row);
+  bf16_bias_row_kernel<<<(im->nbias + 255) / 256, 256, 0, st>>>(P, bias_agg_args(pl, im), g, row);
   return cudaGetLastError();
 }
 }  // namespace gcada
