@@ -66,6 +66,10 @@ struct Bf16Impl {
   int nbias = 0;                                         // bias entries of all layers
   int bias_loc[MLP_MAX_LAYERS + 2] = {0};                // first entry of layer l in the compact bias arrays
   float* db = nullptr;           // [2][G][nbias] bias gradients, the same two buffers per group
+  // column sums of dz_l over row blocks, written by the kernels that produce dz_l (the backward-data epilogue:
+  // blocks of 128 rows; the loss-gradient kernel: blocks of 32 rows): [2][G][blocks][n_l]
+  float* dbp[MLP_MAX_LAYERS + 1] = {nullptr};
+  int dbp_blocks[MLP_MAX_LAYERS + 1] = {0};
   int dw_part_base[MLP_MAX_LAYERS + 1] = {0}, bias_part_base[MLP_MAX_LAYERS + 1] = {0};
   int n_parts = 0;               // innovation-norm partial sums per group
   CUtensorMap tm_fwd_a[MLP_MAX_LAYERS + 1], tm_fwd_b[MLP_MAX_LAYERS + 1];
@@ -93,6 +97,7 @@ struct GemmB {
   __nv_bfloat16* outT;   // transposed bf16 [z][N][ldt]
   float* out_f32;        // EPI_SCORES: [z][M][N]
   const __nv_bfloat16* mask;  // EPI_DA: same indexing as out
+  float* colsum;              // EPI_DA: [z][tiles_m][N] column sums of the (bf16-rounded) output tile, or null
   const float* bias_ring;     // EPI_HIDDEN / EPI_SCORES: rounded biases, ring slots of bias_slot floats
   long long bias_slot, bias_pos;
   long long ldo, ldt;
@@ -223,6 +228,7 @@ constexpr int G_STAGES = 4;
 constexpr int G_EPI_WARPS = 8;
 constexpr int G_THREADS = 64 + 32 * G_EPI_WARPS;
 constexpr int G_TR_BYTES = G_EPI_WARPS * 32 * 17 * 4;  // per-warp transposition tiles of the epilogue
+constexpr int G_CS_BYTES = 2 * 4 * GN * 4;             // column sums of a tile per 32-row quadrant, two tiles in flight
 constexpr uint32_t IDESC_G = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(GN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
@@ -356,6 +362,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
     const int quad = warp & 3;
     const int half = ew >> 2;
     uint32_t* tr = reinterpret_cast<uint32_t*>(tiles + (size_t)G_STAGES * G_STAGE_BYTES) + ew * (32 * 17);
+    float* cs_all = reinterpret_cast<float*>(tiles + (size_t)G_STAGES * G_STAGE_BYTES + G_TR_BYTES);  // [2][4][GN]
     bool ok = true;
     int i = 0;
     for (int t = blockIdx.x; t < total_tiles; t += gridDim.x, ++i) {
@@ -400,7 +407,10 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
         ok = mbar_wait_bounded(&tfull_bar[slot], (uint32_t)((i >> 1) & 1));
         ok = __all_sync(0xffffffffu, ok);
       }
-      if (!ok) continue;
+      if (!ok) {  // (the barrier below is still taken: the other epilogue warps may be waiting at it)
+        if (a.colsum) asm volatile("bar.sync 1, %0;" ::"n"(32 * G_EPI_WARPS) : "memory");
+        continue;
+      }
       tc_fence_after();
       const float* bias = nullptr;
       if (a.epi == EPI_HIDDEN || a.epi == EPI_SCORES)
@@ -476,6 +486,17 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
 #pragma unroll
           for (int j = 0; j < 16; ++j) tr[lane * 17 + j] = h[j];
           __syncwarp();
+          if (a.colsum) {
+            // column `lane` of the warp's 32 x 32 block summed over its rows in row order (the rounded values:
+            // what the bias gradient is the column sum of); rows and columns outside the matrix hold zeros
+            float csum = 0.f;
+#pragma unroll
+            for (int r = 0; r < 32; ++r) {
+              const uint32_t wd = tr[r * 17 + (lane >> 1)];
+              csum += __uint_as_float((lane & 1) ? (wd & 0xFFFF0000u) : (wd << 16));
+            }
+            cs_all[((i & 1) * 4 + quad) * GN + c + lane] = csum;
+          }
           const int rows_here = a.M - (mt * BM + quad * 32);  // valid rows of this warp's block (>= 32 inside)
           if (full && rows_here >= 32) {
             // row-major copy: lanes 4r..4r+3 write the 64 bytes of row r, eight rows per instruction
@@ -545,6 +566,17 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&tempty_bar[slot]);
+      if (a.colsum) {
+        // the tile's column sums: the four 32-row quadrants added in order, one column per epilogue thread.
+        // The buffer alternates between tiles, so a warp that runs ahead writes the other half; it cannot
+        // reach this half again before every warp has passed the next tile's barrier.
+        asm volatile("bar.sync 1, %0;" ::"n"(32 * G_EPI_WARPS) : "memory");
+        const int col = ew * 32 + lane;  // 0..255
+        if (n0 + col < a.N) {
+          const float* cs = cs_all + (size_t)(i & 1) * 4 * GN + col;
+          a.colsum[((long long)z * tiles_m + mt) * a.N + n0 + col] = ((cs[0] + cs[GN]) + cs[2 * GN]) + cs[3 * GN];
+        }
+      }
     }
     if (!ok && lane == 0) atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
   }
@@ -940,7 +972,7 @@ __global__ void __launch_bounds__(256) bf16_gather_kernel(const Params P, __nv_b
 // results also go to a shared tile from which the transposed copy leaves in 64-byte runs.
 __global__ void __launch_bounds__(256) bf16_softmax_grad_kernel(const Params P, const float* scores, const int* yb,
                                                                 __nv_bfloat16* dz, __nv_bfloat16* dzT, int n_cls,
-                                                                int ldz, int Bp, int pitch) {
+                                                                int ldz, int Bp, int pitch, float* colsum) {
   extern __shared__ __nv_bfloat16 sm_tile[];  // [32][pitch]
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const long long rows = (long long)P.G * Bp;
@@ -983,6 +1015,14 @@ __global__ void __launch_bounds__(256) bf16_softmax_grad_kernel(const Params P, 
   __syncthreads();
   __nv_bfloat16* oT = dzT + ((long long)factor_entry(P, g, q) * n_cls) * Bp + m0;
   for (int c = warp; c < n_cls; c += 8) oT[(long long)c * Bp + lane] = sm_tile[lane * pitch + c];
+  // column sums of the block's 32 rows in row order: this block's share of the bias gradient of the last layer
+  float* cs = colsum + (((long long)(q * P.G + g)) * (Bp / 32) + m0 / 32) * n_cls;
+  for (int c = threadIdx.x; c < n_cls; c += 256) {
+    float v = 0.f;
+#pragma unroll 8
+    for (int r = 0; r < 32; ++r) v += __bfloat162float(sm_tile[r * pitch + c]);
+    cs[c] = v;
+  }
 }
 
 // The same for an even number of classes up to 64 * NP: a lane keeps its NP class pairs of a row in registers,
@@ -991,7 +1031,7 @@ __global__ void __launch_bounds__(256) bf16_softmax_grad_kernel(const Params P, 
 template <int NP>
 __global__ void __launch_bounds__(256) bf16_softmax_grad_pairs_kernel(const Params P, const float* scores, const int* yb,
                                                                       __nv_bfloat16* dz, __nv_bfloat16* dzT, int n_cls,
-                                                                      int ldz, int Bp, int pitch) {
+                                                                      int ldz, int Bp, int pitch, float* colsum) {
   extern __shared__ __nv_bfloat16 sm_tile[];  // [32][pitch]
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const long long rows = (long long)P.G * Bp;
@@ -1045,14 +1085,24 @@ __global__ void __launch_bounds__(256) bf16_softmax_grad_pairs_kernel(const Para
   __syncthreads();
   __nv_bfloat16* oT = dzT + ((long long)factor_entry(P, g, q) * n_cls) * Bp + m0;
   for (int c = warp; c < n_cls; c += 8) oT[(long long)c * Bp + lane] = sm_tile[lane * pitch + c];
+  // column sums of the block's 32 rows in row order: this block's share of the bias gradient of the last layer
+  float* cs = colsum + (((long long)(q * P.G + g)) * (Bp / 32) + m0 / 32) * n_cls;
+  for (int c = threadIdx.x; c < n_cls; c += 256) {
+    float v = 0.f;
+#pragma unroll 8
+    for (int r = 0; r < 32; ++r) v += __bfloat162float(sm_tile[r * pitch + c]);
+    cs[c] = v;
+  }
 }
 
 // ----------------------------------------------------------------- bias gradients
-// db_l at both points (column sums of dz_l over the group's rows), their
-// squared difference summed per block into the block's lhs_part slot.
+// db_l at both points = column sums of dz_l over the group's rows.  The kernels that produce dz_l leave the
+// sums of their row blocks (BiasArgsB::part); here the blocks are added in order, the fresh one is kept, and
+// the squared difference of the two points is summed per block of 64 columns into its lhs_part slot.
 struct BiasArgsB {
-  const __nv_bfloat16* dz[MLP_MAX_LAYERS + 1];
-  int n[MLP_MAX_LAYERS + 1], ld[MLP_MAX_LAYERS + 1];
+  const float* part[MLP_MAX_LAYERS + 1];  // [2][G][blocks[l]][n[l]]
+  int blocks[MLP_MAX_LAYERS + 1];
+  int n[MLP_MAX_LAYERS + 1];
   long long b_off[MLP_MAX_LAYERS + 1];
   int part_base[MLP_MAX_LAYERS + 1];
   int n_parts;
@@ -1060,51 +1110,27 @@ struct BiasArgsB {
   int bias_loc[MLP_MAX_LAYERS + 1];   // first entry of layer l in a db row
   int nbias;
 };
-// Block = 64 columns x 8 row slices: lane pairs of columns (bf16x2 loads), warp = row slice.
-__global__ void __launch_bounds__(256) bf16_bias_grad_kernel(const Params P, const BiasArgsB a, int Bp) {
-  __shared__ float red[2][8][64];
+__global__ void __launch_bounds__(64) bf16_bias_grad_kernel(const Params P, const BiasArgsB a) {
   __shared__ double scratch[40];
   const int l = blockIdx.z + 1;
   const int n_l = a.n[l];
   if ((int)blockIdx.x * 64 >= n_l) return;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = blockIdx.y;
-  if (P.skip_unselected && !P.mask_cur[g]) return;  // (its stale-point sums below are then unused)
-  const int n = blockIdx.x * 64 + 2 * lane;  // this lane's column pair (ld is even, so the pair is inside the row)
-  const long long rows = (long long)P.G * Bp;
-  float f0 = 0.f, f1 = 0.f, s0 = 0.f, s1 = 0.f;
-  if (n < n_l) {
-    const __nv_bfloat16* p0 = a.dz[l] + ((long long)g * Bp) * a.ld[l] + n;
-    const __nv_bfloat16* p1 = p0 + rows * a.ld[l];
-    for (int r = warp; r < Bp; r += 8) {
-      const __nv_bfloat162 u = *reinterpret_cast<const __nv_bfloat162*>(p0 + (long long)r * a.ld[l]);
-      const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(p1 + (long long)r * a.ld[l]);
-      f0 += __low2float(u);
-      f1 += __high2float(u);
-      s0 += __low2float(v);
-      s1 += __high2float(v);
-    }
-  }
-  red[0][warp][2 * lane] = f0;
-  red[0][warp][2 * lane + 1] = f1;
-  red[1][warp][2 * lane] = s0;
-  red[1][warp][2 * lane + 1] = s1;
-  __syncthreads();
+  if (P.skip_unselected && !P.mask_cur[g]) return;
+  const int c = blockIdx.x * 64 + threadIdx.x;
   double d2 = 0.0;
-  if (threadIdx.x < 64) {
-    const int c = blockIdx.x * 64 + threadIdx.x;
-    if (c < n_l) {
-      float f = 0.f, sv = 0.f;
-#pragma unroll
-      for (int w = 0; w < 8; ++w) {
-        f += red[0][w][threadIdx.x];
-        sv += red[1][w][threadIdx.x];
-      }
-      a.db[((long long)fresh_buf(P, g) * P.G + g) * a.nbias + a.bias_loc[l] + c] = f;
-      if (P.gbuf) (fresh_row(P, g) + a.b_off[l])[c] = f;  // kept for inspection
-      if (P.stale) (P.stale + (long long)g * P.p_pad + a.b_off[l])[c] = sv;
-      d2 = (double)(f - sv) * (double)(f - sv);
-    }
+  if (c < n_l) {
+    const int nb = a.blocks[l];
+    const float* p0 = a.part[l] + ((long long)g * nb) * n_l + c;
+    const float* p1 = p0 + (long long)P.G * nb * n_l;
+    float f = 0.f, sv = 0.f;
+    for (int b = 0; b < nb; ++b) f += p0[(long long)b * n_l];
+    if (!P.skip_unselected)                      // (no stale point when only the selected groups compute)
+      for (int b = 0; b < nb; ++b) sv += p1[(long long)b * n_l];
+    a.db[((long long)fresh_buf(P, g) * P.G + g) * a.nbias + a.bias_loc[l] + c] = f;
+    if (P.gbuf) (fresh_row(P, g) + a.b_off[l])[c] = f;  // kept for inspection
+    if (P.stale) (P.stale + (long long)g * P.p_pad + a.b_off[l])[c] = sv;
+    d2 = (double)(f - sv) * (double)(f - sv);
   }
   d2 = block_sum(d2, scratch);
   if (threadIdx.x == 0) P.lhs_part[(long long)g * a.n_parts + a.part_base[l] + blockIdx.x] = d2;
@@ -1176,7 +1202,7 @@ cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const Para
   a.stages = G_STAGES;
   const long long tiles = (long long)((a.N + GN - 1) / GN) * ((a.M + BM - 1) / BM) * (a.k_batched ? 1 : 2 * P.G);
   const int ctas = (int)(tiles < sm_count ? tiles : sm_count);
-  bf16_gemm_kernel<<<ctas, G_THREADS, (size_t)G_STAGES * G_STAGE_BYTES + 1024 + G_TR_BYTES, st>>>(ta, tb, P, a);
+  bf16_gemm_kernel<<<ctas, G_THREADS, (size_t)G_STAGES * G_STAGE_BYTES + 1024 + G_TR_BYTES + G_CS_BYTES, st>>>(ta, tb, P, a);
   return cudaGetLastError();
 }
 
@@ -1285,6 +1311,10 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
   }
   A_(im->scores, 2 * rows * plan->dims[L], float);
   A_(im->db, 2LL * G * im->nbias, float);
+  for (int l = 1; l <= L; ++l) {
+    im->dbp_blocks[l] = l < L ? im->Bp / BM : im->Bp / 32;
+    A_(im->dbp[l], 2LL * G * im->dbp_blocks[l] * plan->dims[l], float);
+  }
 #undef A_
   // what an iteration reads from earlier ones: the bf16 copies of the last D+1 iterates and every group's last upload
   plan->state.clear();
@@ -1328,7 +1358,7 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
     return cudaSuccess;
   }
   cudaError_t e = cudaFuncSetAttribute(bf16_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       G_STAGES * G_STAGE_BYTES + 1024 + G_TR_BYTES);
+                                       G_STAGES * G_STAGE_BYTES + 1024 + G_TR_BYTES + G_CS_BYTES);
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(bf16_softmax_grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            32 * (plan->dims[L] + 4) * 2);
@@ -1411,13 +1441,13 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
     const size_t sm = (size_t)32 * pitch * 2;
     if ((nc & 1) == 0 && nc <= 1024) {  // class pairs in registers
       if (nc <= 256)
-        bf16_softmax_grad_pairs_kernel<4><<<blocks, 256, sm, st>>>(P, im->scores, im->yb, im->dz[L], im->dzT[L], nc, im->ld[L], Bp, pitch);
+        bf16_softmax_grad_pairs_kernel<4><<<blocks, 256, sm, st>>>(P, im->scores, im->yb, im->dz[L], im->dzT[L], nc, im->ld[L], Bp, pitch, im->dbp[L]);
       else if (nc <= 512)
-        bf16_softmax_grad_pairs_kernel<8><<<blocks, 256, sm, st>>>(P, im->scores, im->yb, im->dz[L], im->dzT[L], nc, im->ld[L], Bp, pitch);
+        bf16_softmax_grad_pairs_kernel<8><<<blocks, 256, sm, st>>>(P, im->scores, im->yb, im->dz[L], im->dzT[L], nc, im->ld[L], Bp, pitch, im->dbp[L]);
       else
-        bf16_softmax_grad_pairs_kernel<16><<<blocks, 256, sm, st>>>(P, im->scores, im->yb, im->dz[L], im->dzT[L], nc, im->ld[L], Bp, pitch);
+        bf16_softmax_grad_pairs_kernel<16><<<blocks, 256, sm, st>>>(P, im->scores, im->yb, im->dz[L], im->dzT[L], nc, im->ld[L], Bp, pitch, im->dbp[L]);
     } else {
-      bf16_softmax_grad_kernel<<<blocks, 256, sm, st>>>(P, im->scores, im->yb, im->dz[L], im->dzT[L], nc, im->ld[L], Bp, pitch);
+      bf16_softmax_grad_kernel<<<blocks, 256, sm, st>>>(P, im->scores, im->yb, im->dz[L], im->dzT[L], nc, im->ld[L], Bp, pitch, im->dbp[L]);
     }
   }
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
@@ -1439,6 +1469,7 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
       d.out = im->dz[l - 1];
       d.outT = im->dzT[l - 1];
       d.mask = im->act[l - 1];
+      d.colsum = im->dbp[l - 1];
       d.ldo = im->ld[l - 1];
       d.ldt = Bp;
       d.z_stride_out = (long long)Bp * im->ld[l - 1];
@@ -1450,9 +1481,9 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
   BiasArgsB ba{};
   int maxn = 0;
   for (int l = 1; l <= L; ++l) {
-    ba.dz[l] = im->dz[l];
+    ba.part[l] = im->dbp[l];
+    ba.blocks[l] = im->dbp_blocks[l];
     ba.n[l] = pl.dims[l];
-    ba.ld[l] = im->ld[l];
     ba.b_off[l] = pl.b_off[l];
     ba.part_base[l] = im->bias_part_base[l];
     ba.bias_loc[l] = im->bias_loc[l];
@@ -1461,7 +1492,7 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
   ba.n_parts = im->n_parts;
   ba.db = im->db;
   ba.nbias = im->nbias;
-  bf16_bias_grad_kernel<<<dim3((maxn + 63) / 64, G, L), 256, 0, st>>>(P, ba, Bp);
+  bf16_bias_grad_kernel<<<dim3((maxn + 63) / 64, G, L), 64, 0, st>>>(P, ba);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   ++n;
   *n_launches = n;
