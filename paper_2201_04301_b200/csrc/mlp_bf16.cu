@@ -70,6 +70,11 @@ struct Bf16Impl {
   // blocks of 128 rows; the loss-gradient kernel: blocks of 32 rows): [2][G][blocks][n_l]
   float* dbp[MLP_MAX_LAYERS + 1] = {nullptr};
   int dbp_blocks[MLP_MAX_LAYERS + 1] = {0};
+  // differences between the two points, row-major [G*Bp][ld_l] (see bf16_gram_kernel)
+  __nv_bfloat16* dE[MLP_MAX_LAYERS + 1] = {nullptr};  // dz_l(theta^k) - dz_l(stale), l = 1..L
+  __nv_bfloat16* dF[MLP_MAX_LAYERS + 1] = {nullptr};  // a_l(theta^k) - a_l(stale),  l = 1..L-1
+  int gram_part_base[MLP_MAX_LAYERS + 1] = {0};
+  CUtensorMap tm_dE[MLP_MAX_LAYERS + 1], tm_dF[MLP_MAX_LAYERS + 1];
   int dw_part_base[MLP_MAX_LAYERS + 1] = {0}, bias_part_base[MLP_MAX_LAYERS + 1] = {0};
   int n_parts = 0;               // innovation-norm partial sums per group
   CUtensorMap tm_fwd_a[MLP_MAX_LAYERS + 1], tm_fwd_b[MLP_MAX_LAYERS + 1];
@@ -98,6 +103,9 @@ struct GemmB {
   float* out_f32;        // EPI_SCORES: [z][M][N]
   const __nv_bfloat16* mask;  // EPI_DA: same indexing as out
   float* colsum;              // EPI_DA: [z][tiles_m][N] column sums of the (bf16-rounded) output tile, or null
+  __nv_bfloat16* diff;        // EPI_HIDDEN / EPI_DA, or null: row-major [G][M][ldo]; the stale-point tile writes
+                              // (fresh output - its own output) here, rounded to bf16, instead of its transposed
+                              // copy: the small factors of the innovation's rank-one terms (see bf16_gram_kernel)
   const float* bias_ring;     // EPI_HIDDEN / EPI_SCORES: rounded biases, ring slots of bias_slot floats
   long long bias_slot, bias_pos;
   long long ldo, ldt;
@@ -231,6 +239,14 @@ constexpr int G_TR_BYTES = G_EPI_WARPS * 32 * 17 * 4;  // per-warp transposition
 constexpr int G_CS_BYTES = 2 * 4 * GN * 4;             // column sums of a tile per 32-row quadrant, two tiles in flight
 constexpr uint32_t IDESC_G = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(GN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
+// Difference of two packed bf16 pairs, each half exact in fp32 and rounded to nearest-even bf16.
+__device__ __forceinline__ uint32_t bf16x2_sub(uint32_t x, uint32_t y) {
+  const float lo = __uint_as_float(x << 16) - __uint_as_float(y << 16);
+  const float hi = __uint_as_float(x & 0xFFFF0000u) - __uint_as_float(y & 0xFFFF0000u);
+  const __nv_bfloat162 r = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&r);
+}
+
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
@@ -262,7 +278,12 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
   // batch entries: (point, group) for every group, or - when only the selected groups compute (rule PS:
   // Algorithm 1's own order, the selection is already known) - the selected groups at theta^k only
   const int n_grp = P.skip_unselected ? P.sel_count[0] : P.G;
-  const int total_tiles = a.k_batched ? tiles_n * tiles_m : tiles_n * tiles_m * (P.skip_unselected ? 1 : 2) * n_grp;
+  // A CTA walks units (column tile, row tile, group) and, inside a unit, the two points one after the other:
+  // the stale point's epilogue runs in the same threads, on the same rows and columns, as the fresh point's
+  // just before it, whose output it reads back to form the differences.
+  const int n_q = (a.k_batched || P.skip_unselected) ? 1 : 2;
+  const int total_units = tiles_n * tiles_m * (a.k_batched ? 1 : n_grp);
+  const int n_local = (int)blockIdx.x < total_units ? ((total_units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) * n_q : 0;
   const long long k_it = P.st->k;
 
   if (threadIdx.x == 0) {
@@ -291,10 +312,10 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
     if (lane == 0) {
       bool ok = true;
       int it = 0;
-      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-        const int nt = t % tiles_n, mt = (t / tiles_n) % tiles_m, zi = t / (tiles_n * tiles_m);
-        const int q = a.k_batched ? 0 : zi / n_grp;
-        const int g = a.k_batched ? 0 : (P.skip_unselected ? P.sel_list[zi - q * n_grp] : zi - q * n_grp);
+      for (int i = 0; i < n_local && ok; ++i) {
+        const int u = blockIdx.x + (i / n_q) * gridDim.x, q = i % n_q;
+        const int nt = u % tiles_n, mt = (u / tiles_n) % tiles_m, gi = u / (tiles_n * tiles_m);
+        const int g = a.k_batched ? 0 : (P.skip_unselected ? P.sel_list[gi] : gi);
         const int z = q * P.G + g;
         int zA = 0, zB = 0, ent = 0;
         // entry e of a k_batched product: every group's last upload, or (listed) the selected groups' replaced
@@ -332,8 +353,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
   } else if (warp == 1) {
     if (lane == 0) {
       bool ok = true;
-      int it = 0, i = 0;
-      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++i) {
+      int it = 0;
+      for (int i = 0; i < n_local && ok; ++i) {
         const int slot = i & 1;
         ok = mbar_spin_bounded(&tempty_bar[slot], (uint32_t)(((i >> 1) & 1) ^ 1));
         if (!ok) break;
@@ -364,13 +385,13 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
     uint32_t* tr = reinterpret_cast<uint32_t*>(tiles + (size_t)G_STAGES * G_STAGE_BYTES) + ew * (32 * 17);
     float* cs_all = reinterpret_cast<float*>(tiles + (size_t)G_STAGES * G_STAGE_BYTES + G_TR_BYTES);  // [2][4][GN]
     bool ok = true;
-    int i = 0;
-    for (int t = blockIdx.x; t < total_tiles; t += gridDim.x, ++i) {
+    for (int i = 0; i < n_local; ++i) {
       const int slot = i & 1;
-      const int nt = t % tiles_n, mt = (t / tiles_n) % tiles_m, zi = t / (tiles_n * tiles_m);
-      const int q = a.k_batched ? 0 : zi / n_grp;
-      const int g = a.k_batched ? 0 : (P.skip_unselected ? P.sel_list[zi - q * n_grp] : zi - q * n_grp);
+      const int u = blockIdx.x + (i / n_q) * gridDim.x, q = i % n_q;
+      const int nt = u % tiles_n, mt = (u / tiles_n) % tiles_m, gi = u / (tiles_n * tiles_m);
+      const int g = a.k_batched ? 0 : (P.skip_unselected ? P.sel_list[gi] : gi);
       const int z = q * P.G + g;
+      const bool write_diff = q == 1 && a.diff != nullptr;
       const int zT = a.k_batched ? 0 : factor_entry(P, g, q);  // entry of the transposed copy (a factor array)
       const int m = mt * BM + quad * 32 + lane;
       const int n0 = nt * GN;
@@ -500,13 +521,24 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
           const int rows_here = a.M - (mt * BM + quad * 32);  // valid rows of this warp's block (>= 32 inside)
           if (full && rows_here >= 32) {
             // row-major copy: lanes 4r..4r+3 write the 64 bytes of row r, eight rows per instruction
-            __nv_bfloat16* dst0 = a.out + (long long)z * a.z_stride_out + (long long)(mt * BM + quad * 32) * a.ldo + nc;
+            const long long off0 = (long long)(mt * BM + quad * 32) * a.ldo + nc;
+            __nv_bfloat16* dst0 = a.out + (long long)z * a.z_stride_out + off0;
 #pragma unroll
             for (int it = 0; it < 4; ++it) {
               const int r = it * 8 + (lane >> 2), qd = lane & 3;
               const uint32_t* src = tr + r * 17 + qd * 4;
-              *reinterpret_cast<uint4*>(dst0 + (long long)r * a.ldo + qd * 8) = make_uint4(src[0], src[1], src[2], src[3]);
+              const uint4 mine = make_uint4(src[0], src[1], src[2], src[3]);
+              *reinterpret_cast<uint4*>(dst0 + (long long)r * a.ldo + qd * 8) = mine;
+              if (write_diff) {
+                // the fresh point's 16 bytes at this place were stored by this very thread one tile ago
+                const uint4 fr = *reinterpret_cast<const uint4*>(a.out + (long long)g * a.z_stride_out + off0 +
+                                                                 (long long)r * a.ldo + qd * 8);
+                *reinterpret_cast<uint4*>(a.diff + (long long)g * a.z_stride_out + off0 + (long long)r * a.ldo + qd * 8) =
+                    make_uint4(bf16x2_sub(fr.x, mine.x), bf16x2_sub(fr.y, mine.y), bf16x2_sub(fr.z, mine.z),
+                               bf16x2_sub(fr.w, mine.w));
+              }
             }
+            if (write_diff) return;  // the stale point's transposed copy is not needed
             // transposed copy: lanes 4n..4n+3 write the 64 bytes (32 rows) of output row nc + n
             __nv_bfloat16* dstT0 = a.outT + (long long)zT * a.z_stride_outT + (long long)nc * a.ldt + (mt * BM + quad * 32);
 #pragma unroll
@@ -527,7 +559,14 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
           if (row_ok) {
             __nv_bfloat16* dst = a.out + (long long)z * a.z_stride_out + (long long)m * a.ldo + nc;
             for (int j = 0; j < 32 && nc + j < a.N; ++j) dst[j] = __float2bfloat16_rn(f[j]);
+            if (write_diff) {  // (this thread stored the fresh point's values of this row one tile ago)
+              const __nv_bfloat16* fr = a.out + (long long)g * a.z_stride_out + (long long)m * a.ldo + nc;
+              __nv_bfloat16* df = a.diff + (long long)g * a.z_stride_out + (long long)m * a.ldo + nc;
+              for (int j = 0; j < 32 && nc + j < a.N; ++j)
+                df[j] = __float2bfloat16_rn(__bfloat162float(fr[j]) - __bfloat162float(__float2bfloat16_rn(f[j])));
+            }
           }
+          if (write_diff) return;
           if (nc + lane < a.N) {
             uint32_t o[16];
 #pragma unroll
@@ -588,12 +627,190 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
   }
 }
 
+// ----------------------------------------------------------------- innovation norm of the weight gradients
+// ||dW_l(theta^k) - dW_l(stale)||_F^2 of one group without forming either gradient.  With r over the group's
+// minibatch rows, dz / a the back-propagated errors / input activations of layer l at theta^k and a tilde for
+// the stale point,
+//     dW - dW~ = sum_r dz_r (x) a_r - dz~_r (x) a~_r = sum_r (dz_r - dz~_r) (x) a_r + dz~_r (x) (a_r - a~_r),
+// a sum of 2B rank-one terms u_k (x) v_k in which one factor of every term is a small difference:
+//     U = [E; dz~],  V = [a; F],  E = dz - dz~,  F = a - a~   (E, F formed exactly from the bf16 values and
+//                                                              rounded to bf16 by the kernels that produce dz, a).
+// Then ||sum_k u_k (x) v_k||_F^2 = sum_{k,k'} (u_k . u_k') (v_k . v_k') = <U U^T, V V^T>: two Gram matrices of
+// 2B x 2B entries (K = n_l and n_{l-1}) and their elementwise product summed.  Every term is of the size of
+// the innovation itself, so nothing cancels (Grams of [dz; -dz~] and [a; a~] would sum terms of the size of
+// the gradients to a result of the size of the innovation).  Compared with forming dW - dW~ tile by tile the
+// tensor cores do 2 (2B)^2 (n_l + n_{l-1}) instead of 4 B n_l n_{l-1} flops and, decisive here, only 2 (2B)^2
+// accumulators per group and layer are read from tensor memory instead of n_l n_{l-1}: the direct pass was
+// bound by draining its accumulators.  Layer 1 has a = a~ (the features), so U = E, V = x.
+//
+// Unit = (group, 128-row block mi, column block nj of up to 256) of the two Grams: accumulator columns
+// [0, BN) receive U_mi U_nj^T, columns [BN, 2 BN) V_mi V_nj^T; the epilogue multiplies them elementwise and
+// adds up; one partial sum per unit goes to lhs_part.  Operand blocks of 128 rows come from up to two arrays
+// per matrix (part 0 / part 1) through their own tensor maps.
+struct GramArgs {
+  int parts;         // 1: U = E_l, V = a_{l-1} (layer 1); 2: U = [E_l; dz~_l], V = [a_{l-1}; F_{l-1}]
+  int nb;            // 128-row blocks per part (padded minibatch rows / 128)
+  int BN;            // column block of the Grams: min(parts * nb * 128, 256)
+  int Ku, Kv;        // n_l, n_{l-1}
+  int zu1_stale;     // 1: part 1 of U is entry G + g of its tensor map (the stale point's rows of dz_l)
+  int part_base, n_parts;
+};
+
+__global__ void __launch_bounds__(G_THREADS, 1) bf16_gram_kernel(const __grid_constant__ CUtensorMap tmU0,
+                                                                 const __grid_constant__ CUtensorMap tmU1,
+                                                                 const __grid_constant__ CUtensorMap tmV0,
+                                                                 const __grid_constant__ CUtensorMap tmV1,
+                                                                 const Params P, const GramArgs a) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  __shared__ uint64_t full_bar[G_STAGES], empty_bar[G_STAGES], tfull_bar, tempty_bar;
+  __shared__ uint32_t tmem_base_sm;
+  __shared__ double norm_sm[G_EPI_WARPS];
+  unsigned char* tiles = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int RB = a.parts * a.nb;             // 128-row blocks of U and V
+  const int bpn = a.BN / BM;                 // row blocks per column block
+  const int tiles_nj = RB / bpn;
+  const int units_per_group = RB * tiles_nj;
+  const int total_units = units_per_group * P.G;
+  const int nku = (a.Ku + BK - 1) / BK, nkv = (a.Kv + BK - 1) / BK;
+  const uint32_t stage_tx = (uint32_t)((BM + a.BN) * BK * 2);
+  const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(a.BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < G_STAGES; ++s) {
+      mbar_init(&full_bar[s], 1);
+      mbar_init(&empty_bar[s], 1);
+    }
+    mbar_init(&tfull_bar, 1);
+    mbar_init(&tempty_bar, G_EPI_WARPS);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_sm)),
+                 "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_sm;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      bool ok = true;
+      int it = 0;
+      for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
+        const int g = u / units_per_group, r = u - g * units_per_group;
+        const int mi = r / tiles_nj, nj = r - mi * tiles_nj;
+        for (int ph = 0; ph < 2 && ok; ++ph) {  // the U Gram, then the V Gram
+          const int nk = ph == 0 ? nku : nkv;
+          for (int kb = 0; kb < nk && ok; ++kb, ++it) {
+            const int s = it % G_STAGES;
+            ok = mbar_spin_bounded(&empty_bar[s], (uint32_t)(((it / G_STAGES) & 1) ^ 1));
+            if (!ok) break;
+            unsigned char* sa = tiles + (size_t)s * G_STAGE_BYTES;
+            mbar_expect_tx(&full_bar[s], stage_tx);
+            // block b of the matrix: part b / nb, rows (b % nb) * 128 of the group's entry in that part's array
+            auto load_block = [&](unsigned char* dst, int b) {
+              const int part = b / a.nb, row = (b - part * a.nb) * BM;
+              const CUtensorMap* tm = ph == 0 ? (part == 0 ? &tmU0 : &tmU1) : (part == 0 ? &tmV0 : &tmV1);
+              const int z = (ph == 0 && part == 1 && a.zu1_stale) ? P.G + g : g;
+              tma_load_3d(dst, tm, kb * BK, row, z, &full_bar[s]);
+            };
+            load_block(sa, mi);
+            for (int j = 0; j < bpn; ++j) load_block(sa + (size_t)(BM + j * BM) * BK * 2, nj * bpn + j);
+          }
+        }
+      }
+      if (!ok) atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      bool ok = true;
+      int it = 0, i = 0;
+      for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x, ++i) {
+        ok = mbar_spin_bounded(&tempty_bar, (uint32_t)((i & 1) ^ 1));  // the epilogue has drained the accumulators
+        if (!ok) break;
+        tc_fence_after();
+        for (int ph = 0; ph < 2 && ok; ++ph) {
+          const int nk = ph == 0 ? nku : nkv;
+          for (int kb = 0; kb < nk && ok; ++kb, ++it) {
+            const int s = it % G_STAGES;
+            ok = mbar_spin_bounded(&full_bar[s], (uint32_t)((it / G_STAGES) & 1));
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t sa = smem_u32(tiles + (size_t)s * G_STAGE_BYTES);
+            const uint64_t da = make_desc(sa), db = make_desc(sa + BM * BK * 2);
+#pragma unroll
+            for (int kk = 0; kk < BK / 16; ++kk)
+              tc_mma_bf16(tmem_base + (uint32_t)(ph * a.BN), da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc,
+                          (kb | kk) != 0 ? 1u : 0u);
+            tc_commit(&empty_bar[s]);
+          }
+        }
+        if (ok) tc_commit(&tfull_bar);
+      }
+      if (!ok) atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
+    }
+  } else {
+    const int ew = warp - 2, quad = warp & 3, half = ew >> 2;
+    bool ok = true;
+    int i = 0;
+    for (int u = blockIdx.x; u < total_units; u += gridDim.x, ++i) {
+      const int g = u / units_per_group, r = u - g * units_per_group;
+      double local = 0.0;
+      if (ok) {
+        ok = mbar_wait_bounded(&tfull_bar, (uint32_t)(i & 1));
+        ok = __all_sync(0xffffffffu, ok);
+      }
+      if (ok) {
+        tc_fence_after();
+        const uint32_t tbase = tmem_base + ((uint32_t)(quad * 32) << 16);
+        const int c0 = half * (a.BN / 2), c1 = c0 + a.BN / 2;  // this warp's columns of both accumulators
+        for (int c = c0; c < c1; c += 32) {
+          uint32_t gu[32], gv[32];
+          tc_ld32_issue(tbase + (uint32_t)c, gu);
+          tc_ld32_issue(tbase + (uint32_t)(a.BN + c), gv);
+          tc_ld_wait();
+          float part = 0.f;
+#pragma unroll
+          for (int j = 0; j < 32; ++j) part = fmaf(__uint_as_float(gu[j]), __uint_as_float(gv[j]), part);
+          local += (double)part;
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&tempty_bar);
+      }
+      // one partial sum per unit, the eight warps added in warp order (two barriers: the slots are reused)
+      local = warp_sum(local);
+      if (lane == 0) norm_sm[ew] = local;
+      asm volatile("bar.sync 1, %0;" ::"n"(32 * G_EPI_WARPS) : "memory");
+      if (ew == 0 && lane == 0) {
+        double tsum = 0.0;
+#pragma unroll
+        for (int w = 0; w < G_EPI_WARPS; ++w) tsum += norm_sm[w];
+        P.lhs_part[(long long)g * a.n_parts + a.part_base + r] = tsum;
+      }
+      asm volatile("bar.sync 1, %0;" ::"n"(32 * G_EPI_WARPS) : "memory");
+    }
+    if (!ok && lane == 0) atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
 // ----------------------------------------------------------------- weight gradients, both points in one CTA
 // dW_l of one group at theta^k (accumulator 0) and at the stale iterate
-// (accumulator 1), 128 x 256 tiles.  The epilogue forms the squared norm of
-// their difference - the tile's share of the left side of Eq. (9) - and stores
-// it in the tile's own slot of lhs_part; the gradients themselves are written
-// only when they are kept for inspection.
+// (accumulator 1), 128 x 256 tiles, written out: the inspection mode (every
+// group's two gradients are kept; the epilogue also forms the squared norm of
+// their difference, the tile's share of the left side of Eq. (9)) and the
+// getters' rebuild of one group's last upload from its kept factors.  The
+// production path never forms a group's weight gradient (bf16_gram_kernel).
 //
 // Persistent: one CTA per SM walks work units u = blockIdx.x, + gridDim.x,
 // ...; a unit is one (group, 128-row block of W_l) and its tiles are all the
@@ -612,15 +829,14 @@ struct DwArgs {
   int tiles_m, tiles_n, total_tiles;
   long long c_off, ldc;   // position of W_l inside the gradient vector, row stride
   int part_base, n_parts; // this layer's first slot in lhs_part and slots per group
-  int mode;               // DW_BOTH: both points in two accumulators, norm, gradients written for every group;
-                          // DW_NORM: one accumulator receives dW(theta^k) - dW(stale) (the second product enters
-                          //          negated), norm only, nothing written but lhs_part;
-                          // DW_ONE: one group's last uploaded gradient rebuilt from its stored factors (the
-                          //          operands are the last-upload stores) and written to out_row; used by getters
+  int mode;               // DW_BOTH: both points in two accumulators, norm, gradients written for every group
+                          //          (inspection mode; the production path takes the norm in bf16_gram_kernel);
+                          // DW_ONE: one group's last uploaded gradient rebuilt from its kept factors and
+                          //          written to out_row; used by getters
   int g_only;             // DW_ONE: the group
   float* out_row;         // DW_ONE: a p-vector
 };
-enum { DW_BOTH = 0, DW_NORM = 1, DW_ONE = 2 };
+enum { DW_BOTH = 0, DW_ONE = 2 };
 
 constexpr int DW_BN = 256;     // N tile: the MMA issue rate, not the tensor pipe, limits 128-wide instructions
 constexpr int DW_PITCH = 36;   // floats per staged row (16-byte aligned, conflict-free 16-byte stores)
@@ -724,13 +940,12 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
             tc_fence_after();
             const uint64_t da = make_desc(smem_u32(a_res + (size_t)j * BLK));
             const uint64_t db = make_desc(smem_u32(tiles + (size_t)s * BBLK));
-            // DW_NORM: the stale-point product is subtracted in the same accumulator (A negated, bit 13)
-            const uint32_t idesc = (a.mode == DW_NORM && q == 1) ? (IDESC_G | (1u << 13)) : IDESC_G;
+            const uint32_t idesc = IDESC_G;
             const uint32_t acc_col = (uint32_t)(slot * slot_cols + (a.mode == DW_BOTH ? q * DW_BN : 0));
 #pragma unroll
             for (int kk = 0; kk < BK / 16; ++kk)
               tc_mma_bf16(tmem_base + acc_col, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc,
-                          ((a.mode == DW_NORM ? j : kb) | kk) != 0 ? 1u : 0u);
+                          (kb | kk) != 0 ? 1u : 0u);
             tc_commit(&empty_bar[s]);
           }
           if (ok) tc_commit(&tfull_bar[slot]);
@@ -762,36 +977,11 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
       if (ok) {
         tc_fence_after();
         // kept for inspection: the fresh gradient goes to the row that is not the last uploaded one
-        float* fresh = a.mode == DW_NORM ? nullptr : (a.mode == DW_ONE ? a.out_row : fresh_row(P, g)) + a.c_off;
+        float* fresh = (a.mode == DW_ONE ? a.out_row : fresh_row(P, g)) + a.c_off;
         float* stale = (a.mode == DW_BOTH && P.stale) ? P.stale + (long long)g * P.p_pad + a.c_off : nullptr;
-        const int n_pass = a.mode == DW_NORM ? 0 : (stale ? 2 : 1);
+        const int n_pass = stale ? 2 : 1;
         const int mrow = mt * BM + quad * 32;
         const uint32_t tbase = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(slot * slot_cols);
-        if (a.mode == DW_NORM) {
-          // Norm only.  Rows and columns outside the matrix were zero-filled by the copies, so the whole
-          // 128 x 256 accumulator is summed without predicates; the four tensor-memory loads of this warp
-          // are pipelined (a load takes far longer than its issue).
-          const uint32_t cb = (uint32_t)(half * (DW_BN / 2));
-          uint32_t va[32], vb[32];
-          auto sq = [&](const uint32_t(&v)[32]) {
-            float part = 0.f;
-#pragma unroll
-            for (int j = 0; j < 32; ++j) part += __uint_as_float(v[j]) * __uint_as_float(v[j]);
-            local += (double)part;
-          };
-          tc_ld32_issue(tbase + cb, va);
-          tc_ld_wait();
-          tc_ld32_issue(tbase + cb + 32, vb);
-          sq(va);
-          tc_ld_wait();
-          tc_ld32_issue(tbase + cb + 64, va);
-          sq(vb);
-          tc_ld_wait();
-          tc_ld32_issue(tbase + cb + 96, vb);
-          sq(va);
-          tc_ld_wait();
-          sq(vb);
-        } else
 #pragma unroll 1
         for (int c = half * (DW_BN / 2); c < (half + 1) * (DW_BN / 2); c += 32) {
           const int nc = nt * DW_BN + c;
@@ -806,8 +996,7 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
             float part = 0.f;
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
-              // DW_NORM: the accumulator already holds the difference
-              const float d = a.mode == DW_BOTH ? __uint_as_float(v0[j]) - __uint_as_float(v1[j]) : __uint_as_float(v0[j]);
+              const float d = __uint_as_float(v0[j]) - __uint_as_float(v1[j]);
               if (interior || nc + j < a.N) part += d * d;
             }
             if (row_ok) local += (double)part;
@@ -968,60 +1157,74 @@ __global__ void __launch_bounds__(256) bf16_gather_kernel(const Params P, __nv_b
 
 // ----------------------------------------------------------------- loss gradient
 // dz = (softmax(scores) - onehot(y)) * scale in both orientations; padding rows (y < 0) get zeros.
-// Block = 32 consecutive rows of one (point, group); each of the 8 warps takes 4 rows; the bf16
-// results also go to a shared tile from which the transposed copy leaves in 64-byte runs.
+// Block = 32 consecutive rows of one group; each of the 8 warps takes 4 rows; the bf16 results also go to a
+// shared tile from which the transposed copy leaves in 64-byte runs and the column sums (the block's share
+// of the last layer's bias gradient) are taken.  With `both` the block handles the rows at theta^k and then
+// at the stale point, and writes the difference of the two (fresh - stale, rounded to bf16) to `diff` in
+// place of the stale point's transposed copy; otherwise grid.y selects the point.
 __global__ void __launch_bounds__(256) bf16_softmax_grad_kernel(const Params P, const float* scores, const int* yb,
                                                                 __nv_bfloat16* dz, __nv_bfloat16* dzT, int n_cls,
-                                                                int ldz, int Bp, int pitch, float* colsum) {
+                                                                int ldz, int Bp, int pitch, float* colsum,
+                                                                __nv_bfloat16* diff, int both) {
   extern __shared__ __nv_bfloat16 sm_tile[];  // [32][pitch]
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const long long rows = (long long)P.G * Bp;
-  const long long w0 = (long long)blockIdx.x * 32;  // first (point, row) of the block
-  const int q = (int)(w0 / rows);
-  const long long r0 = w0 - (long long)q * rows;
+  const long long r0 = (long long)blockIdx.x * 32;  // first row of the block inside a point
   const int g = (int)(r0 / Bp), m0 = (int)(r0 - (long long)g * Bp);
-  if (P.skip_unselected && (q != 0 || !P.mask_cur[g])) return;
-  for (int i = 0; i < 4; ++i) {
-    const int lr = warp * 4 + i;
-    const long long w = w0 + lr;
-    const float* s = scores + w * n_cls;
-    __nv_bfloat16* o = dz + w * ldz;
-    __nv_bfloat16* t = sm_tile + lr * pitch;
-    const int y = yb[r0 + lr];
-    if (y < 0) {
-      for (int c = lane; c < n_cls; c += 32) {
-        o[c] = __float2bfloat16_rn(0.f);
-        t[c] = __float2bfloat16_rn(0.f);
+  if (P.skip_unselected && (blockIdx.y != 0 || !P.mask_cur[g])) return;
+  const int q_first = both ? 0 : blockIdx.y, q_last = both ? 1 : blockIdx.y;
+  for (int q = q_first; q <= q_last; ++q) {
+    const long long w0 = (long long)q * rows + r0;
+    const bool write_diff = both && q == 1;
+    for (int i = 0; i < 4; ++i) {
+      const int lr = warp * 4 + i;
+      const long long w = w0 + lr;
+      const float* s = scores + w * n_cls;
+      __nv_bfloat16* o = dz + w * ldz;
+      const __nv_bfloat16* o0 = dz + (r0 + lr) * ldz;     // the same row at theta^k (written by this thread)
+      __nv_bfloat16* df = diff + (r0 + lr) * ldz;
+      __nv_bfloat16* t = sm_tile + lr * pitch;
+      const int y = yb[r0 + lr];
+      if (y < 0) {
+        for (int c = lane; c < n_cls; c += 32) {
+          o[c] = __float2bfloat16_rn(0.f);
+          t[c] = __float2bfloat16_rn(0.f);
+          if (write_diff) df[c] = __float2bfloat16_rn(0.f);
+        }
+        continue;
       }
-      continue;
-    }
-    float mx = -3.0e38f;
-    for (int c = lane; c < n_cls; c += 32) mx = fmaxf(mx, s[c]);
+      float mx = -3.0e38f;
+      for (int c = lane; c < n_cls; c += 32) mx = fmaxf(mx, s[c]);
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-    // p_y - 1 = -(sum of the other classes' exponentials) / sum, free of cancellation
-    float others = 0.f;
-    for (int c = lane; c < n_cls; c += 32)
-      if (c != y) others += expf(s[c] - mx);
-    others = warp_sum(others);
-    const float inv = 1.0f / (others + expf(s[y] - mx));
-    for (int c = lane; c < n_cls; c += 32) {
-      const float v = (c == y ? -others * inv : expf(s[c] - mx) * inv) * P.scale;
-      const __nv_bfloat16 b = __float2bfloat16_rn(v);
-      o[c] = b;
-      t[c] = b;
+      for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+      // p_y - 1 = -(sum of the other classes' exponentials) / sum, free of cancellation
+      float others = 0.f;
+      for (int c = lane; c < n_cls; c += 32)
+        if (c != y) others += expf(s[c] - mx);
+      others = warp_sum(others);
+      const float inv = 1.0f / (others + expf(s[y] - mx));
+      for (int c = lane; c < n_cls; c += 32) {
+        const float v = (c == y ? -others * inv : expf(s[c] - mx) * inv) * P.scale;
+        const __nv_bfloat16 b = __float2bfloat16_rn(v);
+        o[c] = b;
+        t[c] = b;
+        if (write_diff) df[c] = __float2bfloat16_rn(__bfloat162float(o0[c]) - __bfloat162float(b));
+      }
     }
-  }
-  __syncthreads();
-  __nv_bfloat16* oT = dzT + ((long long)factor_entry(P, g, q) * n_cls) * Bp + m0;
-  for (int c = warp; c < n_cls; c += 8) oT[(long long)c * Bp + lane] = sm_tile[lane * pitch + c];
-  // column sums of the block's 32 rows in row order: this block's share of the bias gradient of the last layer
-  float* cs = colsum + (((long long)(q * P.G + g)) * (Bp / 32) + m0 / 32) * n_cls;
-  for (int c = threadIdx.x; c < n_cls; c += 256) {
-    float v = 0.f;
+    __syncthreads();
+    if (!write_diff) {
+      __nv_bfloat16* oT = dzT + ((long long)factor_entry(P, g, q) * n_cls) * Bp + m0;
+      for (int c = warp; c < n_cls; c += 8) oT[(long long)c * Bp + lane] = sm_tile[lane * pitch + c];
+    }
+    // column sums of the block's 32 rows in row order: this block's share of the bias gradient of the last layer
+    float* cs = colsum + (((long long)(q * P.G + g)) * (Bp / 32) + m0 / 32) * n_cls;
+    for (int c = threadIdx.x; c < n_cls; c += 256) {
+      float v = 0.f;
 #pragma unroll 8
-    for (int r = 0; r < 32; ++r) v += __bfloat162float(sm_tile[r * pitch + c]);
-    cs[c] = v;
+      for (int r = 0; r < 32; ++r) v += __bfloat162float(sm_tile[r * pitch + c]);
+      cs[c] = v;
+    }
+    __syncthreads();  // the tile is reused for the second point
   }
 }
 
@@ -1031,67 +1234,79 @@ __global__ void __launch_bounds__(256) bf16_softmax_grad_kernel(const Params P, 
 template <int NP>
 __global__ void __launch_bounds__(256) bf16_softmax_grad_pairs_kernel(const Params P, const float* scores, const int* yb,
                                                                       __nv_bfloat16* dz, __nv_bfloat16* dzT, int n_cls,
-                                                                      int ldz, int Bp, int pitch, float* colsum) {
+                                                                      int ldz, int Bp, int pitch, float* colsum,
+                                                                      __nv_bfloat16* diff, int both) {
   extern __shared__ __nv_bfloat16 sm_tile[];  // [32][pitch]
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const long long rows = (long long)P.G * Bp;
-  const long long w0 = (long long)blockIdx.x * 32;  // first (point, row) of the block
-  const int q = (int)(w0 / rows);
-  const long long r0 = w0 - (long long)q * rows;
+  const long long r0 = (long long)blockIdx.x * 32;  // first row of the block inside a point
   const int g = (int)(r0 / Bp), m0 = (int)(r0 - (long long)g * Bp);
-  if (P.skip_unselected && (q != 0 || !P.mask_cur[g])) return;
-  for (int i = 0; i < 4; ++i) {
-    const int lr = warp * 4 + i;
-    const long long w = w0 + lr;
-    const float* s = scores + w * n_cls;
-    __nv_bfloat16* o = dz + w * ldz;
-    __nv_bfloat16* t = sm_tile + lr * pitch;
-    const int y = yb[r0 + lr];
-    float2 v[NP];
-    float mx = -3.0e38f;
+  if (P.skip_unselected && (blockIdx.y != 0 || !P.mask_cur[g])) return;
+  const int q_first = both ? 0 : blockIdx.y, q_last = both ? 1 : blockIdx.y;
+  for (int q = q_first; q <= q_last; ++q) {
+    const long long w0 = (long long)q * rows + r0;
+    const bool write_diff = both && q == 1;
+    for (int i = 0; i < 4; ++i) {
+      const int lr = warp * 4 + i;
+      const long long w = w0 + lr;
+      const float* s = scores + w * n_cls;
+      __nv_bfloat16* o = dz + w * ldz;
+      const __nv_bfloat16* o0 = dz + (r0 + lr) * ldz;     // the same row at theta^k (written by this thread)
+      __nv_bfloat16* df = diff + (r0 + lr) * ldz;
+      __nv_bfloat16* t = sm_tile + lr * pitch;
+      const int y = yb[r0 + lr];
+      float2 v[NP];
+      float mx = -3.0e38f;
 #pragma unroll
-    for (int j = 0; j < NP; ++j) {
-      const int c = 2 * lane + 64 * j;
-      v[j] = (y >= 0 && c < n_cls) ? *reinterpret_cast<const float2*>(s + c) : make_float2(-3.0e38f, -3.0e38f);
-      mx = fmaxf(mx, fmaxf(v[j].x, v[j].y));
-    }
+      for (int j = 0; j < NP; ++j) {
+        const int c = 2 * lane + 64 * j;
+        v[j] = (y >= 0 && c < n_cls) ? *reinterpret_cast<const float2*>(s + c) : make_float2(-3.0e38f, -3.0e38f);
+        mx = fmaxf(mx, fmaxf(v[j].x, v[j].y));
+      }
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-    // p_y - 1 = -(sum of the other classes' exponentials) / sum, free of cancellation
-    float others = 0.f, ey = 0.f;
+      for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+      // p_y - 1 = -(sum of the other classes' exponentials) / sum, free of cancellation
+      float others = 0.f, ey = 0.f;
 #pragma unroll
-    for (int j = 0; j < NP; ++j) {
-      const int c = 2 * lane + 64 * j;
-      v[j].x = expf(v[j].x - mx);  // classes beyond n_cls: exp of a huge negative number, zero
-      v[j].y = expf(v[j].y - mx);
-      if (c == y) ey = v[j].x; else others += v[j].x;
-      if (c + 1 == y) ey = v[j].y; else others += v[j].y;
-    }
-    others = warp_sum(others);
-    ey = warp_sum(ey);
-    const float inv = y >= 0 ? 1.0f / (others + ey) : 0.f;
+      for (int j = 0; j < NP; ++j) {
+        const int c = 2 * lane + 64 * j;
+        v[j].x = expf(v[j].x - mx);  // classes beyond n_cls: exp of a huge negative number, zero
+        v[j].y = expf(v[j].y - mx);
+        if (c == y) ey = v[j].x; else others += v[j].x;
+        if (c + 1 == y) ey = v[j].y; else others += v[j].y;
+      }
+      others = warp_sum(others);
+      ey = warp_sum(ey);
+      const float inv = y >= 0 ? 1.0f / (others + ey) : 0.f;
 #pragma unroll
-    for (int j = 0; j < NP; ++j) {
-      const int c = 2 * lane + 64 * j;
-      if (c < n_cls) {
-        const float a = y < 0 ? 0.f : (c == y ? -others * inv : v[j].x * inv) * P.scale;
-        const float b = y < 0 ? 0.f : (c + 1 == y ? -others * inv : v[j].y * inv) * P.scale;
-        const __nv_bfloat162 pr = __floats2bfloat162_rn(a, b);
-        *reinterpret_cast<__nv_bfloat162*>(o + c) = pr;
-        *reinterpret_cast<__nv_bfloat162*>(t + c) = pr;
+      for (int j = 0; j < NP; ++j) {
+        const int c = 2 * lane + 64 * j;
+        if (c < n_cls) {
+          const float a = y < 0 ? 0.f : (c == y ? -others * inv : v[j].x * inv) * P.scale;
+          const float b = y < 0 ? 0.f : (c + 1 == y ? -others * inv : v[j].y * inv) * P.scale;
+          const __nv_bfloat162 pr = __floats2bfloat162_rn(a, b);
+          *reinterpret_cast<__nv_bfloat162*>(o + c) = pr;
+          *reinterpret_cast<__nv_bfloat162*>(t + c) = pr;
+          if (write_diff) {
+            const uint32_t fr = *reinterpret_cast<const uint32_t*>(o0 + c);
+            *reinterpret_cast<uint32_t*>(df + c) = bf16x2_sub(fr, *reinterpret_cast<const uint32_t*>(&pr));
+          }
+        }
       }
     }
-  }
-  __syncthreads();
-  __nv_bfloat16* oT = dzT + ((long long)factor_entry(P, g, q) * n_cls) * Bp + m0;
-  for (int c = warp; c < n_cls; c += 8) oT[(long long)c * Bp + lane] = sm_tile[lane * pitch + c];
-  // column sums of the block's 32 rows in row order: this block's share of the bias gradient of the last layer
-  float* cs = colsum + (((long long)(q * P.G + g)) * (Bp / 32) + m0 / 32) * n_cls;
-  for (int c = threadIdx.x; c < n_cls; c += 256) {
-    float v = 0.f;
+    __syncthreads();
+    if (!write_diff) {
+      __nv_bfloat16* oT = dzT + ((long long)factor_entry(P, g, q) * n_cls) * Bp + m0;
+      for (int c = warp; c < n_cls; c += 8) oT[(long long)c * Bp + lane] = sm_tile[lane * pitch + c];
+    }
+    float* cs = colsum + (((long long)(q * P.G + g)) * (Bp / 32) + m0 / 32) * n_cls;
+    for (int c = threadIdx.x; c < n_cls; c += 256) {
+      float v2 = 0.f;
 #pragma unroll 8
-    for (int r = 0; r < 32; ++r) v += __bfloat162float(sm_tile[r * pitch + c]);
-    cs[c] = v;
+      for (int r = 0; r < 32; ++r) v2 += __bfloat162float(sm_tile[r * pitch + c]);
+      cs[c] = v2;
+    }
+    __syncthreads();  // the tile is reused for the second point
   }
 }
 
@@ -1200,8 +1415,8 @@ long long up(long long x, long long m) { return (x + m - 1) / m * m; }
 cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const Params& P, GemmB a, int sm_count,
                         cudaStream_t st) {
   a.stages = G_STAGES;
-  const long long tiles = (long long)((a.N + GN - 1) / GN) * ((a.M + BM - 1) / BM) * (a.k_batched ? 1 : 2 * P.G);
-  const int ctas = (int)(tiles < sm_count ? tiles : sm_count);
+  const long long units = (long long)((a.N + GN - 1) / GN) * ((a.M + BM - 1) / BM) * (a.k_batched ? 1 : P.G);
+  const int ctas = (int)(units < sm_count ? units : sm_count);
   bf16_gemm_kernel<<<ctas, G_THREADS, (size_t)G_STAGES * G_STAGE_BYTES + 1024 + G_TR_BYTES + G_CS_BYTES, st>>>(ta, tb, P, a);
   return cudaGetLastError();
 }
@@ -1218,7 +1433,7 @@ cudaError_t launch_dw(const Params& P, const MlpPlan& pl, const Bf16Impl* im, in
   w.nkb = im->Bp / BK;
   // 32 KiB B blocks in whatever shared memory is left beside the resident A blocks (and the staging tile of
   // the modes that write gradients): the B stream is bound by bytes in flight, so every stage counts
-  const long long stage_bytes = mode == DW_NORM ? 0 : (long long)DW_STAGE_FLOATS * 4;
+  const long long stage_bytes = (long long)DW_STAGE_FLOATS * 4;
   const long long room = 232448 - 1024 - 1024 - (long long)2 * w.nkb * (BM * BK * 2) - stage_bytes;
   w.stages = (int)(room / (DW_BN * BK * 2));
   if (w.stages > MAX_STAGES) w.stages = MAX_STAGES;
@@ -1281,6 +1496,11 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
     im->bias_part_base[l] = parts;
     parts += (plan->dims[l] + 63) / 64;
   }
+  for (int l = 1; l <= L; ++l) {  // units of the Gram products per group (slots that a mode does not use stay zero)
+    im->gram_part_base[l] = parts;
+    const int rb = (l == 1 ? 1 : 2) * (im->Bp / BM), bn = rb * BM < GN ? rb * BM : GN;
+    parts += rb * (rb * BM / bn);
+  }
   im->n_parts = parts;
   plan->norm_parts = parts;
   for (int l = 1; l <= L; ++l) im->bias_loc[l + 1] = im->bias_loc[l] + plan->dims[l];
@@ -1311,6 +1531,10 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
   }
   A_(im->scores, 2 * rows * plan->dims[L], float);
   A_(im->db, 2LL * G * im->nbias, float);
+  for (int l = 1; l <= L; ++l) {
+    A_(im->dE[l], rows * im->ld[l], __nv_bfloat16);
+    if (l < L) A_(im->dF[l], rows * im->ld[l], __nv_bfloat16);
+  }
   for (int l = 1; l <= L; ++l) {
     im->dbp_blocks[l] = l < L ? im->Bp / BM : im->Bp / 32;
     A_(im->dbp[l], 2LL * G * im->dbp_blocks[l] * plan->dims[l], float);
@@ -1345,6 +1569,9 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
     ok &= make_map(&im->tm_da_a[l], im->dz[l], no, Bp, 2LL * G, im->ld[l], Bp * im->ld[l], BM);
     ok &= make_map(&im->tm_da_b[l], im->wb + im->wt_pos[l], no, ni, D + 1, im->ld[l], im->slot_elems, GN);
     // weight gradient: A = dz_l^T, B = a_{l-1}^T
+    // differences of the two points (row-major, one entry per group): operands of the Gram products
+    ok &= make_map(&im->tm_dE[l], im->dE[l], no, Bp, G, im->ld[l], Bp * im->ld[l], BM);
+    if (l < L) ok &= make_map(&im->tm_dF[l], im->dF[l], no, Bp, G, im->ld[l], Bp * im->ld[l], BM);
     // (the aggregate reads the same two arrays: the groups' upload buffers are their first 2G entries)
     static_assert(DW_BN == GN, "the weight-gradient and aggregate products share their B tensor map");
     ok &= make_map(&im->tm_dw_a[l], im->dzT[l], Bp, no, 3LL * G, Bp, (long long)no * Bp, BM);
@@ -1370,6 +1597,8 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
   e = cudaFuncSetAttribute(bf16_softmax_grad_pairs_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 32 * (1024 + 4) * 2);
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(bf16_dw_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024);  // the kernel's static arrays take under 1 KiB
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(bf16_gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, G_STAGES * G_STAGE_BYTES + 1024);
   if (e != cudaSuccess) return e;
   plan->launches_per_iter = 3 + L + 1 + L + (L - 1);
   plan->post_launches = L + 1;
@@ -1409,6 +1638,9 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
   bf16_gather_kernel<<<dim3(Bp / 32, G), 256, 0, st>>>(P, im->xb, im->xbT, im->yb, pl.dims[0], im->ld[0], Bp);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   ++n;
+  // production: no group's weight gradient is formed; the stale point's epilogues write differences for the
+  // Gram form of the innovation norm.  Inspection mode keeps both gradients of every group instead.
+  const bool production = !P.stale && !P.skip_unselected;
   for (int l = 1; l <= L; ++l) {
     GemmB a{};
     a.M = Bp;
@@ -1427,6 +1659,7 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
       a.ldt = Bp;
       a.z_stride_out = (long long)Bp * im->ld[l];
       a.z_stride_outT = (long long)pl.dims[l] * Bp;
+      a.diff = production ? im->dF[l] : nullptr;
     } else {
       a.epi = EPI_SCORES;
       a.out_f32 = im->scores;
@@ -1437,25 +1670,44 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
   {
     const int pitch = pl.dims[L] + 2 + (pl.dims[L] & 1);  // even, and an odd number of 32-bit words when possible
     const int nc = pl.dims[L];
-    const unsigned blocks = (unsigned)(2 * rows / 32);
+    // production: a block takes both points of its rows and writes their difference; inspection mode (both
+    // gradients kept) and the printed rule (one point only): grid.y selects the point
+    const int both = (!P.stale && !P.skip_unselected) ? 1 : 0;
+    const dim3 blocks((unsigned)(rows / 32), both || P.skip_unselected ? 1 : 2);
     const size_t sm = (size_t)32 * pitch * 2;
     if ((nc & 1) == 0 && nc <= 1024) {  // class pairs in registers
       if (nc <= 256)
-        bf16_softmax_grad_pairs_kernel<4><<<blocks, 256, sm, st>>>(P, im->scores, im->yb, im->dz[L], im->dzT[L], nc, im->ld[L], Bp, pitch, im->dbp[L]);
+        bf16_softmax_grad_pairs_kernel<4><<<blocks, 256, sm, st>>>(P, im->scores, im->yb, im->dz[L], im->dzT[L], nc, im->ld[L], Bp, pitch, im->dbp[L], im->dE[L], both);
       else if (nc <= 512)
-        bf16_softmax_grad_pairs_kernel<8><<<blocks, 256, sm, st>>>(P, im->scores, im->yb, im->dz[L], im->dzT[L], nc, im->ld[L], Bp, pitch, im->dbp[L]);
+        bf16_softmax_grad_pairs_kernel<8><<<blocks, 256, sm, st>>>(P, im->scores, im->yb, im->dz[L], im->dzT[L], nc, im->ld[L], Bp, pitch, im->dbp[L], im->dE[L], both);
       else
-        bf16_softmax_grad_pairs_kernel<16><<<blocks, 256, sm, st>>>(P, im->scores, im->yb, im->dz[L], im->dzT[L], nc, im->ld[L], Bp, pitch, im->dbp[L]);
+        bf16_softmax_grad_pairs_kernel<16><<<blocks, 256, sm, st>>>(P, im->scores, im->yb, im->dz[L], im->dzT[L], nc, im->ld[L], Bp, pitch, im->dbp[L], im->dE[L], both);
     } else {
-      bf16_softmax_grad_kernel<<<blocks, 256, sm, st>>>(P, im->scores, im->yb, im->dz[L], im->dzT[L], nc, im->ld[L], Bp, pitch, im->dbp[L]);
+      bf16_softmax_grad_kernel<<<blocks, 256, sm, st>>>(P, im->scores, im->yb, im->dz[L], im->dzT[L], nc, im->ld[L], Bp, pitch, im->dbp[L], im->dE[L], both);
     }
   }
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   ++n;
-  const int dw_mode = P.stale ? DW_BOTH : DW_NORM;  // gradients of every group are materialised only on request
   for (int l = L; l >= 1; --l) {
-    if (!P.skip_unselected) {  // the innovation norms; not needed when the printed test has already decided
-      if ((e = launch_dw(P, pl, im, l, dw_mode, st)) != cudaSuccess) return e;
+    if (production) {  // the innovation norm of layer l's weight gradient from the two Gram products
+      GramArgs ga{};
+      ga.parts = l == 1 ? 1 : 2;
+      ga.nb = Bp / BM;
+      ga.BN = ga.parts * Bp < GN ? ga.parts * Bp : GN;
+      ga.Ku = pl.dims[l];
+      ga.Kv = pl.dims[l - 1];
+      ga.zu1_stale = 1;
+      ga.part_base = im->gram_part_base[l];
+      ga.n_parts = im->n_parts;
+      const int units = G * ga.parts * ga.nb * (ga.parts * Bp / ga.BN);
+      const int ctas = units < pl.sm_count ? units : pl.sm_count;
+      // U = [E_l; dz_l at the stale point], V = [a_{l-1} at theta^k; F_{l-1}]
+      bf16_gram_kernel<<<ctas, G_THREADS, (size_t)G_STAGES * G_STAGE_BYTES + 1024, st>>>(
+          im->tm_dE[l], im->tm_da_a[l], im->tm_fwd_a[l], l == 1 ? im->tm_fwd_a[l] : im->tm_dF[l - 1], P, ga);
+      if ((e = cudaGetLastError()) != cudaSuccess) return e;
+      ++n;
+    } else if (!P.skip_unselected) {  // inspection mode: both gradients of every group, norm from their difference
+      if ((e = launch_dw(P, pl, im, l, DW_BOTH, st)) != cudaSuccess) return e;
       ++n;
     }
     if (l > 1) {
@@ -1470,6 +1722,7 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
       d.outT = im->dzT[l - 1];
       d.mask = im->act[l - 1];
       d.colsum = im->dbp[l - 1];
+      d.diff = production ? im->dE[l - 1] : nullptr;
       d.ldo = im->ld[l - 1];
       d.ldt = Bp;
       d.z_stride_out = (long long)Bp * im->ld[l - 1];
