@@ -71,6 +71,7 @@ struct Bf16Impl {
   float* dbp[MLP_MAX_LAYERS + 1] = {nullptr};
   int dbp_blocks[MLP_MAX_LAYERS + 1] = {0};
   // differences between the two points, row-major [G*Bp][ld_l] (see bf16_gram_kernel)
+  uint32_t* relu_bits[MLP_MAX_LAYERS + 1] = {nullptr};  // [2G][(n_l + 31) / 32][Bp]: a_l > 0, l = 1..L-1
   __nv_bfloat16* dE[MLP_MAX_LAYERS + 1] = {nullptr};  // dz_l(theta^k) - dz_l(stale), l = 1..L
   __nv_bfloat16* dF[MLP_MAX_LAYERS + 1] = {nullptr};  // a_l(theta^k) - a_l(stale),  l = 1..L-1
   int gram_part_base[MLP_MAX_LAYERS + 1] = {0};
@@ -101,7 +102,10 @@ struct GemmB {
   __nv_bfloat16* out;    // row-major bf16 [z][M][ldo]
   __nv_bfloat16* outT;   // transposed bf16 [z][N][ldt]
   float* out_f32;        // EPI_SCORES: [z][M][N]
-  const __nv_bfloat16* mask;  // EPI_DA: same indexing as out
+  uint32_t* relu_bits;        // one bit per hidden unit: the (bf16-rounded) activation is positive.  Layout
+                              // [z][N / 32 rounded up][M] words (rows of a word position are contiguous).
+                              // EPI_HIDDEN writes them, EPI_DA of the same layer reads them as the ReLU derivative
+  int nw;                     // words per row: (N + 31) / 32
   float* colsum;              // EPI_DA: [z][tiles_m][N] column sums of the (bf16-rounded) output tile, or null
   __nv_bfloat16* diff;        // EPI_HIDDEN / EPI_DA, or null: row-major [G][M][ldo]; the stale-point tile writes
                               // (fresh output - its own output) here, rounded to bf16, instead of its transposed
@@ -395,33 +399,14 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
       const int zT = a.k_batched ? 0 : factor_entry(P, g, q);  // entry of the transposed copy (a factor array)
       const int m = mt * BM + quad * 32 + lane;
       const int n0 = nt * GN;
-      // EPI_DA: the ReLU mask of this thread's row does not depend on the accumulator, so it is fetched (one
-      // bit per column, four words for the four chunks) while the MMAs of the tile are still running
+      // EPI_DA: the ReLU derivative of this thread's row does not depend on the accumulator: its four words
+      // (one bit per column of the four chunks) are fetched while the MMAs of the tile are still running
       uint32_t mbits[4] = {0u, 0u, 0u, 0u};
-      const bool mask_in_regs = a.epi == EPI_DA && m < a.M;
-      if (mask_in_regs) {
-        const __nv_bfloat16* mk = a.mask + (long long)z * a.z_stride_out + (long long)m * a.ldo;
+      if (a.epi == EPI_DA && m < a.M) {
 #pragma unroll
         for (int ch = 0; ch < 4; ++ch) {
           const int nc = n0 + half * (GN / 2) + ch * 32;
-          if (nc + 32 <= a.N) {
-            uint4 pk[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) pk[j] = *reinterpret_cast<const uint4*>(mk + nc + 8 * j);
-            uint32_t bits = 0u;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const uint32_t wds[4] = {pk[j].x, pk[j].y, pk[j].z, pk[j].w};
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                // a bf16 is positive iff its bits are non-zero and its sign bit clear
-                const uint32_t lo = wds[e] & 0xFFFFu, hi = wds[e] >> 16;
-                bits |= (uint32_t)(lo != 0u && lo < 0x8000u) << (8 * j + 2 * e);
-                bits |= (uint32_t)(hi != 0u && hi < 0x8000u) << (8 * j + 2 * e + 1);
-              }
-            }
-            mbits[ch] = bits;
-          }
+          if (nc < a.N) mbits[ch] = a.relu_bits[((long long)z * a.nw + (nc >> 5)) * a.M + m];
         }
       }
       if (ok) {
@@ -479,19 +464,10 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
           if (a.epi == EPI_HIDDEN) {
 #pragma unroll
             for (int j = 0; j < 32; ++j) f[j] = fmaxf(__uint_as_float(v[j]) + (nc + j < a.N ? bias[nc + j] : 0.f), 0.f);
-          } else {  // EPI_DA: ReLU derivative of the layer below
-            const __nv_bfloat16* mk = a.mask + (long long)z * a.z_stride_out + (long long)m * a.ldo + nc;
-            if (full && row_ok) {
-              const uint32_t bits = mbits[(c - half * (GN / 2)) >> 5];
+          } else {  // EPI_DA: ReLU derivative of the layer below (bits of rows / columns outside the matrix are 0)
+            const uint32_t bits = mbits[(c - half * (GN / 2)) >> 5];
 #pragma unroll
-              for (int j = 0; j < 32; ++j) f[j] = ((bits >> j) & 1u) ? __uint_as_float(v[j]) : 0.f;
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                const bool on = row_ok && nc + j < a.N && __bfloat162float(mk[j]) > 0.f;
-                f[j] = on ? __uint_as_float(v[j]) : 0.f;
-              }
-            }
+            for (int j = 0; j < 32; ++j) f[j] = ((bits >> j) & 1u) ? __uint_as_float(v[j]) : 0.f;
           }
           // bf16 pairs of this thread's row
           uint32_t h[16];
@@ -499,6 +475,17 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
           for (int j = 0; j < 32; j += 2) {
             __nv_bfloat162 t2 = __floats2bfloat162_rn(f[j], f[j + 1]);
             h[j >> 1] = *reinterpret_cast<uint32_t*>(&t2);
+          }
+          if (a.epi == EPI_HIDDEN && row_ok) {
+            // a bf16 is positive iff its bits are non-zero and its sign bit clear
+            uint32_t bits = 0u;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const uint32_t lo = h[j] & 0xFFFFu, hi = h[j] >> 16;
+              bits |= (uint32_t)(lo != 0u && lo < 0x8000u) << (2 * j);
+              bits |= (uint32_t)(hi != 0u && hi < 0x8000u) << (2 * j + 1);
+            }
+            a.relu_bits[((long long)z * a.nw + (nc >> 5)) * a.M + m] = bits;
           }
           // The warp's 32 x 32 block goes through shared memory (rows of 17 words) for both copies, so that
           // every store instruction writes whole 32-byte sectors: a lane that stored 16 bytes of its own row
@@ -1534,6 +1521,7 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
   for (int l = 1; l <= L; ++l) {
     A_(im->dE[l], rows * im->ld[l], __nv_bfloat16);
     if (l < L) A_(im->dF[l], rows * im->ld[l], __nv_bfloat16);
+    if (l < L) A_(im->relu_bits[l], 2 * rows * ((plan->dims[l] + 31) / 32), uint32_t);
   }
   for (int l = 1; l <= L; ++l) {
     im->dbp_blocks[l] = l < L ? im->Bp / BM : im->Bp / 32;
@@ -1660,6 +1648,8 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
       a.z_stride_out = (long long)Bp * im->ld[l];
       a.z_stride_outT = (long long)pl.dims[l] * Bp;
       a.diff = production ? im->dF[l] : nullptr;
+      a.relu_bits = im->relu_bits[l];
+      a.nw = (pl.dims[l] + 31) / 32;
     } else {
       a.epi = EPI_SCORES;
       a.out_f32 = im->scores;
@@ -1720,7 +1710,8 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
       d.epi = EPI_DA;
       d.out = im->dz[l - 1];
       d.outT = im->dzT[l - 1];
-      d.mask = im->act[l - 1];
+      d.relu_bits = im->relu_bits[l - 1];
+      d.nw = (pl.dims[l - 1] + 31) / 32;
       d.colsum = im->dbp[l - 1];
       d.diff = production ? im->dE[l - 1] : nullptr;
       d.ldo = im->ld[l - 1];
