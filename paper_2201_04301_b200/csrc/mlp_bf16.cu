@@ -6,18 +6,18 @@
 // weight gradients are never materialised on the production path: a first pass
 // forms only the squared innovation norms, and the server's aggregate (Eq. 3,
 // the sum over groups of each group's last uploaded gradient) is one product per
-// layer over the factors (dz_l^T, a_{l-1}^T) of every group's last
+// layer over the factors (dz_l, a_{l-1}) of every group's last
 // upload, with K running over all groups' rows.  The factors at theta^k are
 // written into one of two buffers per group; the other one holds the group's last
 // upload, and selecting the group flips the two (Params::cur), so an upload moves
-// no data.  Every product is an "NT" GEMM  C[M x N] = A[M x K] * B[N x K]^T
-// with both operands K-major, so one kernel serves all of them:
-//     forward   z_l   = a_{l-1} W_l^T        A = a_{l-1} [rows][n_{l-1}],  B = W_l   [n_l][n_{l-1}]
-//     backward  da    = dz_l W_l             A = dz_l    [rows][n_l],      B = W_l^T [n_{l-1}][n_l]
-//     weights   dW_l  = dz_l^T a_{l-1}       A = dz_l^T  [n_l][rows],      B = a_{l-1}^T [n_{l-1}][rows]
-//     aggregate sum_g dW_l(last upload of g) the same with rows = all groups' rows of their last uploads
-// which is why activations, dz and the weights are kept in both orientations
-// (the epilogues write the second orientation for free).
+// no data.  One kernel serves every product  C[M x N] = sum_k A[m][k] B[n][k]:
+//     forward   z_l   = a_{l-1} W_l^T        A = a_{l-1} [rows][n_{l-1}],  B = W_l   [n_l][n_{l-1}]   (both K-major)
+//     backward  da    = dz_l W_l             A = dz_l    [rows][n_l],      B = W_l^T [n_{l-1}][n_l]   (both K-major)
+//     aggregate sum_g dz_l(g)^T a_{l-1}(g)   A = dz_l [rows][n_l], B = a_{l-1} [rows][n_{l-1}] of the groups' last
+//                                            uploads, K = rows: both operands are read as they lie (MN-major:
+//                                            the M / N index is the contiguous one), so no transposed copy of
+//                                            an activation or error matrix is ever written
+// (only the weights are kept in both orientations, by the conversion kernel).
 //
 // Kernels: persistent CTAs, one per SM; warp 0 = TMA producer
 // (cp.async.bulk.tensor, 128-byte swizzle, mbarrier ring), warp 1 = MMA issuer
@@ -51,18 +51,16 @@ struct Bf16Impl {
   int ld[MLP_MAX_LAYERS + 1] = {0};            // row stride (elements) of activation-like buffers of width n_l
   __nv_bfloat16* wb = nullptr;   // (D+1) slots
   float* bias = nullptr;         // (D+1) slots of rounded biases
-  __nv_bfloat16* xb = nullptr;   // [G*Bp][ld0]
   int* yb = nullptr;             // [G*Bp], -1 on padding rows
-  __nv_bfloat16* act[MLP_MAX_LAYERS + 1] = {nullptr};   // [2][G*Bp][ld_l]
-  __nv_bfloat16* dz[MLP_MAX_LAYERS + 1] = {nullptr};
   float* scores = nullptr;       // [2][G*Bp][n_L]
-  // Transposed copies = the factors of the weight gradients, dW_l(g) = dzT[l](g) * actT[l-1](g)^T.  Entries
-  // [0, 2G) are two upload buffers per group (entry b*G + g): buffer cur[g] holds the factors of the group's
-  // last upload, the other one receives the factors at theta^k; the selection flips cur[g] and thereby keeps
-  // the upload.  Entries [2G, 3G) hold the stale point's factors of this iteration (never kept).
-  __nv_bfloat16* xbT = nullptr;                         // [2][G][n_0][Bp] (the features serve both points)
-  __nv_bfloat16* actT[MLP_MAX_LAYERS + 1] = {nullptr};  // [3][G][n_l][Bp]
-  __nv_bfloat16* dzT[MLP_MAX_LAYERS + 1] = {nullptr};   // [3][G][n_l][Bp]
+  // Activations and back-propagated errors, row-major [entry][Bp][ld_l]: they are the operands of the next
+  // product AND the factors of the weight gradients, dW_l(g) = dz[l](g)^T act[l-1](g).  Entries [0, 2G) are
+  // two upload buffers per group (entry b*G + g): buffer cur[g] holds the factors of the group's last
+  // upload, the other one receives the factors at theta^k; the selection flips cur[g] and thereby keeps the
+  // upload.  Entries [2G, 3G) hold the stale point's matrices of this iteration (never kept).
+  __nv_bfloat16* xb = nullptr;                          // [2][G][Bp][ld_0] (the features serve both points)
+  __nv_bfloat16* act[MLP_MAX_LAYERS + 1] = {nullptr};   // [3][G][Bp][ld_l]
+  __nv_bfloat16* dz[MLP_MAX_LAYERS + 1] = {nullptr};    // [3][G][Bp][ld_l]
   int nbias = 0;                                         // bias entries of all layers
   int bias_loc[MLP_MAX_LAYERS + 2] = {0};                // first entry of layer l in the compact bias arrays
   float* db = nullptr;           // [2][G][nbias] bias gradients, the same two buffers per group
@@ -80,12 +78,12 @@ struct Bf16Impl {
   int n_parts = 0;               // innovation-norm partial sums per group
   CUtensorMap tm_fwd_a[MLP_MAX_LAYERS + 1], tm_fwd_b[MLP_MAX_LAYERS + 1];
   CUtensorMap tm_da_a[MLP_MAX_LAYERS + 1], tm_da_b[MLP_MAX_LAYERS + 1];
-  CUtensorMap tm_dw_a[MLP_MAX_LAYERS + 1], tm_dw_b[MLP_MAX_LAYERS + 1];  // the factor arrays (also the aggregate's operands)
+  CUtensorMap tm_dw_a[MLP_MAX_LAYERS + 1], tm_dw_b[MLP_MAX_LAYERS + 1];  // dz[l] / act[l-1] in boxes of 64 rows x 64 columns (MN-major operands)
 };
 
 struct GemmB {
   int M, N, K;
-  int a_shared;      // 1: operand A has one batch entry per group (the gathered features), else per (point, group)
+  int a_shared;      // 1: operand A is the same for both points (the gathered features)
   int zb_mode;       // ZB_*
   int epi;           // EPI_*
   int stages;
@@ -99,21 +97,20 @@ struct GemmB {
                      // iteration (so that rounding cannot pile up), K runs over every group's buffer cur[g] and
                      // the sum is written anew.
   // epilogue operands
-  __nv_bfloat16* out;    // row-major bf16 [z][M][ldo]
-  __nv_bfloat16* outT;   // transposed bf16 [z][N][ldt]
+  __nv_bfloat16* out;    // row-major bf16 [entry][M][ldo], entry = factor_entry(point, group)
   float* out_f32;        // EPI_SCORES: [z][M][N]
   uint32_t* relu_bits;        // one bit per hidden unit: the (bf16-rounded) activation is positive.  Layout
                               // [z][N / 32 rounded up][M] words (rows of a word position are contiguous).
                               // EPI_HIDDEN writes them, EPI_DA of the same layer reads them as the ReLU derivative
   int nw;                     // words per row: (N + 31) / 32
   float* colsum;              // EPI_DA: [z][tiles_m][N] column sums of the (bf16-rounded) output tile, or null
-  __nv_bfloat16* diff;        // EPI_HIDDEN / EPI_DA, or null: row-major [G][M][ldo]; the stale-point tile writes
-                              // (fresh output - its own output) here, rounded to bf16, instead of its transposed
-                              // copy: the small factors of the innovation's rank-one terms (see bf16_gram_kernel)
+  __nv_bfloat16* diff;        // EPI_HIDDEN / EPI_DA, or null: row-major [G][M][ldo]; the stale-point tile also
+                              // writes (fresh output - its own output) here, rounded to bf16: the small
+                              // factors of the innovation's rank-one terms (see bf16_gram_kernel)
   const float* bias_ring;     // EPI_HIDDEN / EPI_SCORES: rounded biases, ring slots of bias_slot floats
   long long bias_slot, bias_pos;
-  long long ldo, ldt;
-  long long z_stride_out, z_stride_outT;
+  long long ldo;
+  long long z_stride_out;
   long long c_off, ldc;       // EPI_AGG: offset inside out_f32 (a p-vector), row stride
 };
 
@@ -209,7 +206,17 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr) {
   return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
          (2ull << 61);
 }
-// Instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, N >> 3 at bit 17, M >> 4 at bit 24.
+// The same for an MN-major tile (the M / N index contiguous): 64 x 64 blocks as the copies deliver them, i.e.
+// 64 K-rows of 128 bytes (64 M / N values) under the 128-byte swizzle.  Atoms are 8 K-rows x 128 bytes; the
+// stride offset is the distance between K-groups of 8 rows (1024 bytes), the leading offset the distance
+// between blocks of 64 M / N values (one whole block: 8192 bytes).  One MMA (K = 16) spans two K-groups.
+__device__ __forceinline__ uint64_t make_desc_mn(uint32_t smem_addr) {
+  return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)(8192 >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+constexpr int MN_BLK = 64 * BK * 2;  // bytes of one 64 x 64 block
+// Instruction descriptor: fp32 accumulator, bf16 A and B, N >> 3 at bit 17, M >> 4 at bit 24; bits 15 / 16
+// set = A / B is MN-major (clear = K-major).
 
 __device__ __forceinline__ int ring_slot(const Params& P, int g, int q, long long k) {
   long long j = q == 0 ? k : k - P.tau[g];
@@ -242,6 +249,7 @@ constexpr int G_THREADS = 64 + 32 * G_EPI_WARPS;
 constexpr int G_TR_BYTES = G_EPI_WARPS * 32 * 17 * 4;  // per-warp transposition tiles of the epilogue
 constexpr int G_CS_BYTES = 2 * 4 * GN * 4;             // column sums of a tile per 32-row quadrant, two tiles in flight
 constexpr uint32_t IDESC_G = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(GN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+constexpr uint32_t IDESC_MN = IDESC_G | (1u << 15) | (1u << 16);
 
 // Difference of two packed bf16 pairs, each half exact in fp32 and rounded to nearest-even bf16.
 __device__ __forceinline__ uint32_t bf16x2_sub(uint32_t x, uint32_t y) {
@@ -332,7 +340,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
         if (a.k_batched) {
           zA = zB = agg_entry(0);
         } else {
-          zA = a.a_shared ? g : z;
+          zA = factor_entry(P, g, a.a_shared ? 0 : q);
           zB = a.zb_mode == ZB_RING ? ring_slot(P, g, q, k_it) : (a.zb_mode == ZB_GROUP ? g : z);
         }
         int kin = 0;  // K block inside the current batch entry (k_batched)
@@ -343,8 +351,16 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
           unsigned char* sa = tiles + (size_t)s * G_STAGE_BYTES;
           mbar_expect_tx(&full_bar[s], G_STAGE_BYTES);
           const int kc = (a.k_batched ? kin : kb) * BK;
-          tma_load_3d(sa, &tmA, kc, mt * BM, zA, &full_bar[s]);
-          tma_load_3d(sa + BM * BK * 2, &tmB, kc, nt * GN, zB, &full_bar[s]);
+          if (a.k_batched) {  // MN-major: 64-row x 64-column blocks of the row-major factors, two for A, four for B
+#pragma unroll
+            for (int j = 0; j < BM / 64; ++j) tma_load_3d(sa + j * MN_BLK, &tmA, mt * BM + j * 64, kc, zA, &full_bar[s]);
+#pragma unroll
+            for (int j = 0; j < GN / 64; ++j)
+              tma_load_3d(sa + BM * BK * 2 + j * MN_BLK, &tmB, nt * GN + j * 64, kc, zB, &full_bar[s]);
+          } else {
+            tma_load_3d(sa, &tmA, kc, mt * BM, zA, &full_bar[s]);
+            tma_load_3d(sa + BM * BK * 2, &tmB, kc, nt * GN, zB, &full_bar[s]);
+          }
           if (a.k_batched && ++kin == a.kpg) {
             kin = 0;
             ++ent;
@@ -369,12 +385,21 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
           if (!ok) break;
           tc_fence_after();
           const uint32_t sa = smem_u32(tiles + (size_t)s * G_STAGE_BYTES);
-          const uint64_t da = make_desc(sa), db = make_desc(sa + BM * BK * 2);
           const bool negate = listed && kb < a.kpg * n_sel;  // the replaced uploads leave the sum (A negated, bit 13)
+          if (a.k_batched) {
+            const uint64_t da = make_desc_mn(sa), db = make_desc_mn(sa + BM * BK * 2);
+            const uint32_t idesc = negate ? (IDESC_MN | (1u << 13)) : IDESC_MN;
 #pragma unroll
-          for (int kk = 0; kk < BK / 16; ++kk)  // 16 bf16 = 32 bytes = 2 descriptor units per MMA
-            tc_mma_bf16(tmem_base + (uint32_t)(slot * GN), da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2),
-                        negate ? (IDESC_G | (1u << 13)) : IDESC_G, (kb | kk) != 0 ? 1u : 0u);
+            for (int kk = 0; kk < BK / 16; ++kk)  // 16 K-rows = two K-groups of 1024 bytes = 128 descriptor units
+              tc_mma_bf16(tmem_base + (uint32_t)(slot * GN), da + (uint64_t)(kk * 128), db + (uint64_t)(kk * 128), idesc,
+                          (kb | kk) != 0 ? 1u : 0u);
+          } else {
+            const uint64_t da = make_desc(sa), db = make_desc(sa + BM * BK * 2);
+#pragma unroll
+            for (int kk = 0; kk < BK / 16; ++kk)  // 16 bf16 = 32 bytes = 2 descriptor units per MMA
+              tc_mma_bf16(tmem_base + (uint32_t)(slot * GN), da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), IDESC_G,
+                          (kb | kk) != 0 ? 1u : 0u);
+          }
           tc_commit(&empty_bar[s]);  // frees the stage once these MMAs have read it
         }
         if (ok) tc_commit(&tfull_bar[slot]);
@@ -396,7 +421,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
       const int g = a.k_batched ? 0 : (P.skip_unselected ? P.sel_list[gi] : gi);
       const int z = q * P.G + g;
       const bool write_diff = q == 1 && a.diff != nullptr;
-      const int zT = a.k_batched ? 0 : factor_entry(P, g, q);  // entry of the transposed copy (a factor array)
+      const int zT = a.k_batched ? 0 : factor_entry(P, g, q);  // entry of the output in its factor array
+      const int zF = a.k_batched ? 0 : factor_entry(P, g, 0);  // entry of the fresh point's output
       const int m = mt * BM + quad * 32 + lane;
       const int n0 = nt * GN;
       // EPI_DA: the ReLU derivative of this thread's row does not depend on the accumulator: its four words
@@ -487,9 +513,9 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
             }
             a.relu_bits[((long long)z * a.nw + (nc >> 5)) * a.M + m] = bits;
           }
-          // The warp's 32 x 32 block goes through shared memory (rows of 17 words) for both copies, so that
-          // every store instruction writes whole 32-byte sectors: a lane that stored 16 bytes of its own row
-          // touched half a sector, and the L2 counted twice the sectors the data needs.
+          // The warp's 32 x 32 block goes through shared memory (rows of 17 words), so that every store
+          // instruction writes whole 32-byte sectors: a lane that stored 16 bytes of its own row touched half
+          // a sector, and the L2 counted twice the sectors the data needs.
           __syncwarp();
 #pragma unroll
           for (int j = 0; j < 16; ++j) tr[lane * 17 + j] = h[j];
@@ -509,7 +535,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
           if (full && rows_here >= 32) {
             // row-major copy: lanes 4r..4r+3 write the 64 bytes of row r, eight rows per instruction
             const long long off0 = (long long)(mt * BM + quad * 32) * a.ldo + nc;
-            __nv_bfloat16* dst0 = a.out + (long long)z * a.z_stride_out + off0;
+            __nv_bfloat16* dst0 = a.out + (long long)zT * a.z_stride_out + off0;
 #pragma unroll
             for (int it = 0; it < 4; ++it) {
               const int r = it * 8 + (lane >> 2), qd = lane & 3;
@@ -518,56 +544,24 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
               *reinterpret_cast<uint4*>(dst0 + (long long)r * a.ldo + qd * 8) = mine;
               if (write_diff) {
                 // the fresh point's 16 bytes at this place were stored by this very thread one tile ago
-                const uint4 fr = *reinterpret_cast<const uint4*>(a.out + (long long)g * a.z_stride_out + off0 +
+                const uint4 fr = *reinterpret_cast<const uint4*>(a.out + (long long)zF * a.z_stride_out + off0 +
                                                                  (long long)r * a.ldo + qd * 8);
                 *reinterpret_cast<uint4*>(a.diff + (long long)g * a.z_stride_out + off0 + (long long)r * a.ldo + qd * 8) =
                     make_uint4(bf16x2_sub(fr.x, mine.x), bf16x2_sub(fr.y, mine.y), bf16x2_sub(fr.z, mine.z),
                                bf16x2_sub(fr.w, mine.w));
               }
             }
-            if (write_diff) return;  // the stale point's transposed copy is not needed
-            // transposed copy: lanes 4n..4n+3 write the 64 bytes (32 rows) of output row nc + n
-            __nv_bfloat16* dstT0 = a.outT + (long long)zT * a.z_stride_outT + (long long)nc * a.ldt + (mt * BM + quad * 32);
-#pragma unroll
-            for (int it = 0; it < 4; ++it) {
-              const int n = it * 8 + (lane >> 2), qd = lane & 3;
-              uint32_t o4[4];
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const uint32_t w0 = tr[(qd * 8 + 2 * e) * 17 + (n >> 1)], w1 = tr[(qd * 8 + 2 * e + 1) * 17 + (n >> 1)];
-                const uint32_t e0 = (n & 1) ? (w0 >> 16) : (w0 & 0xFFFFu);
-                const uint32_t e1 = (n & 1) ? (w1 >> 16) : (w1 & 0xFFFFu);
-                o4[e] = e0 | (e1 << 16);
-              }
-              *reinterpret_cast<uint4*>(dstT0 + (long long)n * a.ldt + qd * 8) = make_uint4(o4[0], o4[1], o4[2], o4[3]);
-            }
             return;
           }
           if (row_ok) {
-            __nv_bfloat16* dst = a.out + (long long)z * a.z_stride_out + (long long)m * a.ldo + nc;
+            __nv_bfloat16* dst = a.out + (long long)zT * a.z_stride_out + (long long)m * a.ldo + nc;
             for (int j = 0; j < 32 && nc + j < a.N; ++j) dst[j] = __float2bfloat16_rn(f[j]);
             if (write_diff) {  // (this thread stored the fresh point's values of this row one tile ago)
-              const __nv_bfloat16* fr = a.out + (long long)g * a.z_stride_out + (long long)m * a.ldo + nc;
+              const __nv_bfloat16* fr = a.out + (long long)zF * a.z_stride_out + (long long)m * a.ldo + nc;
               __nv_bfloat16* df = a.diff + (long long)g * a.z_stride_out + (long long)m * a.ldo + nc;
               for (int j = 0; j < 32 && nc + j < a.N; ++j)
                 df[j] = __float2bfloat16_rn(__bfloat162float(fr[j]) - __bfloat162float(__float2bfloat16_rn(f[j])));
             }
-          }
-          if (write_diff) return;
-          if (nc + lane < a.N) {
-            uint32_t o[16];
-#pragma unroll
-            for (int r = 0; r < 32; r += 2) {
-              const uint32_t w0 = tr[r * 17 + (lane >> 1)], w1 = tr[(r + 1) * 17 + (lane >> 1)];
-              const uint32_t e0 = (lane & 1) ? (w0 >> 16) : (w0 & 0xFFFFu);
-              const uint32_t e1 = (lane & 1) ? (w1 >> 16) : (w1 & 0xFFFFu);
-              o[r >> 1] = e0 | (e1 << 16);
-            }
-            __nv_bfloat16* dstT = a.outT + (long long)zT * a.z_stride_outT + (long long)(nc + lane) * a.ldt +
-                                  (mt * BM + quad * 32);
-#pragma unroll
-            for (int j = 0; j < 16; j += 4)
-              *reinterpret_cast<uint4*>(dstT + 2 * j) = make_uint4(o[j], o[j + 1], o[j + 2], o[j + 3]);
           }
         }
       };
@@ -639,7 +633,6 @@ struct GramArgs {
   int nb;            // 128-row blocks per part (padded minibatch rows / 128)
   int BN;            // column block of the Grams: min(parts * nb * 128, 256)
   int Ku, Kv;        // n_l, n_{l-1}
-  int zu1_stale;     // 1: part 1 of U is entry G + g of its tensor map (the stale point's rows of dz_l)
   int part_base, n_parts;
 };
 
@@ -702,7 +695,9 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gram_kernel(const __grid_co
             auto load_block = [&](unsigned char* dst, int b) {
               const int part = b / a.nb, row = (b - part * a.nb) * BM;
               const CUtensorMap* tm = ph == 0 ? (part == 0 ? &tmU0 : &tmU1) : (part == 0 ? &tmV0 : &tmV1);
-              const int z = (ph == 0 && part == 1 && a.zu1_stale) ? P.G + g : g;
+              // U: part 0 = E_l (entry g), part 1 = dz_l at the stale point; V: part 0 = a_{l-1} at theta^k (in
+              // the group's upload buffer being filled), part 1 = F_{l-1} (entry g)
+              const int z = ph == 0 ? (part == 1 ? factor_entry(P, g, 1) : g) : (part == 0 ? factor_entry(P, g, 0) : g);
               tma_load_3d(dst, tm, kb * BK, row, z, &full_bar[s]);
             };
             load_block(sa, mi);
@@ -801,8 +796,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gram_kernel(const __grid_co
 //
 // Persistent: one CTA per SM walks work units u = blockIdx.x, + gridDim.x,
 // ...; a unit is one (group, 128-row block of W_l) and its tiles are all the
-// column blocks.  The unit's A operand (dz_l^T at both points, 2 x K x 128
-// bf16) stays in shared memory for the whole unit and only B is streamed: with
+// column blocks.  The unit's A operand (128 columns of dz_l at both points, 2 x K x 128
+// bf16, read MN-major as it lies) stays in shared memory for the whole unit and only B is streamed: with
 // K = 128 the product is bound by operand traffic from L2, and this halves it.
 // Tensor memory holds two accumulator pairs (2 x 256 columns) so that the
 // eight epilogue warps drain tile i while the producer and the MMA warp work
@@ -888,8 +883,10 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
         mbar_expect_tx(&afull_bar, (uint32_t)(kb_per_tile * BLK));
         for (int j = 0; j < kb_per_tile; ++j) {
           const int q = j / a.nkb, kb = j - q * a.nkb;
-          tma_load_3d(a_res + (size_t)j * BLK, &tmA, kb * BK, mt * BM, a.mode == DW_ONE ? zone : factor_entry(P, g, q),
-                      &afull_bar);
+          const int zA = a.mode == DW_ONE ? zone : factor_entry(P, g, q);
+#pragma unroll
+          for (int h = 0; h < BM / 64; ++h)  // MN-major: 64 batch rows x 64 columns of dz_l per block
+            tma_load_3d(a_res + (size_t)j * BLK + h * MN_BLK, &tmA, mt * BM + h * 64, kb * BK, zA, &afull_bar);
         }
         ++ui;
         for (int nt = 0; nt < a.tiles_n && ok; ++nt) {
@@ -899,8 +896,10 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
             ok = mbar_spin_bounded(&empty_bar[s], (uint32_t)(((it / stages) & 1) ^ 1));
             if (!ok) break;
             mbar_expect_tx(&full_bar[s], BBLK);
-            tma_load_3d(tiles + (size_t)s * BBLK, &tmB, kb * BK, nt * DW_BN,
-                        a.mode == DW_ONE ? zone : factor_entry(P, g, a.b_shared ? 0 : q), &full_bar[s]);
+            const int zB = a.mode == DW_ONE ? zone : factor_entry(P, g, a.b_shared ? 0 : q);
+#pragma unroll
+            for (int h = 0; h < DW_BN / 64; ++h)
+              tma_load_3d(tiles + (size_t)s * BBLK + h * MN_BLK, &tmB, nt * DW_BN + h * 64, kb * BK, zB, &full_bar[s]);
           }
         }
       }
@@ -925,13 +924,13 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
             ok = mbar_spin_bounded(&full_bar[s], (uint32_t)((it / stages) & 1));
             if (!ok) break;
             tc_fence_after();
-            const uint64_t da = make_desc(smem_u32(a_res + (size_t)j * BLK));
-            const uint64_t db = make_desc(smem_u32(tiles + (size_t)s * BBLK));
-            const uint32_t idesc = IDESC_G;
+            const uint64_t da = make_desc_mn(smem_u32(a_res + (size_t)j * BLK));
+            const uint64_t db = make_desc_mn(smem_u32(tiles + (size_t)s * BBLK));
+            const uint32_t idesc = IDESC_MN;
             const uint32_t acc_col = (uint32_t)(slot * slot_cols + (a.mode == DW_BOTH ? q * DW_BN : 0));
 #pragma unroll
             for (int kk = 0; kk < BK / 16; ++kk)
-              tc_mma_bf16(tmem_base + acc_col, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc,
+              tc_mma_bf16(tmem_base + acc_col, da + (uint64_t)(kk * 128), db + (uint64_t)(kk * 128), idesc,
                           (kb | kk) != 0 ? 1u : 0u);
             tc_commit(&empty_bar[s]);
           }
@@ -1085,13 +1084,11 @@ __global__ void __launch_bounds__(256) bf16_convert_kernel(const Params P, const
   }
 }
 
-// ----------------------------------------------------------------- gather (rows and their transpose)
-// Block = 32 consecutive rows of one group; features move through a 32 x 256 tile: 16-byte loads and
-// row-major stores, 64-byte runs for the transposed copy.
-constexpr int GT_COLS = 256, GT_PITCH = GT_COLS + 2;  // pitch of 129 words: conflict-free column reads
-__global__ void __launch_bounds__(256) bf16_gather_kernel(const Params P, __nv_bfloat16* xb, __nv_bfloat16* xbT,
-                                                          int* yb, int d, int ld0, int Bp) {
-  __shared__ __nv_bfloat16 tile[32 * GT_PITCH];
+// ----------------------------------------------------------------- gather
+// Block = 32 consecutive minibatch rows of one group, copied with 16-byte loads and stores into the group's
+// upload buffer that receives this iteration's factors.
+__global__ void __launch_bounds__(256) bf16_gather_kernel(const Params P, __nv_bfloat16* xb, int* yb, int d, int ld0,
+                                                          int Bp) {
   __shared__ long long rows_sm[32];
   const int g = blockIdx.y, rb = blockIdx.x * 32;
   const int tid = threadIdx.x;
@@ -1106,53 +1103,36 @@ __global__ void __launch_bounds__(256) bf16_gather_kernel(const Params P, __nv_b
   }
   __syncthreads();
   const __nv_bfloat16* X = reinterpret_cast<const __nv_bfloat16*>(P.X);
+  __nv_bfloat16* out = xb + (((long long)fb * P.G + g) * Bp + rb) * ld0;
   const bool vec = (P.ld & 7) == 0 && (reinterpret_cast<uintptr_t>(X) & 15) == 0 && (d & 7) == 0;
-  for (int c0 = 0; c0 < d; c0 += GT_COLS) {
-    if (vec) {
-      for (int e = tid; e < 32 * (GT_COLS / 8); e += 256) {
-        const int r = e / (GT_COLS / 8), c = (e - r * (GT_COLS / 8)) * 8;
-        const long long row = rows_sm[r];
-        uint4 v = make_uint4(0u, 0u, 0u, 0u);
-        if (c0 + c < d) {
-          if (row >= 0) v = *reinterpret_cast<const uint4*>(X + row * P.ld + c0 + c);
-          *reinterpret_cast<uint4*>(xb + ((long long)g * Bp + rb + r) * ld0 + c0 + c) = v;
-        }
-        uint32_t* t = reinterpret_cast<uint32_t*>(tile + r * GT_PITCH + c);
-        t[0] = v.x;
-        t[1] = v.y;
-        t[2] = v.z;
-        t[3] = v.w;
-      }
-    } else {
-      for (int e = tid; e < 32 * GT_COLS; e += 256) {
-        const int r = e / GT_COLS, c = e - r * GT_COLS;
-        const long long row = rows_sm[r];
-        __nv_bfloat16 v = __float2bfloat16_rn(0.f);
-        if (row >= 0 && c0 + c < d) v = X[row * P.ld + c0 + c];
-        tile[r * GT_PITCH + c] = v;
-        if (c0 + c < d) xb[((long long)g * Bp + rb + r) * ld0 + c0 + c] = v;
-      }
+  if (vec) {
+    const int per_row = d / 8;
+    for (int e = tid; e < 32 * per_row; e += 256) {
+      const int r = e / per_row, c = (e - r * per_row) * 8;
+      const long long row = rows_sm[r];
+      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      if (row >= 0) v = *reinterpret_cast<const uint4*>(X + row * P.ld + c);
+      *reinterpret_cast<uint4*>(out + (long long)r * ld0 + c) = v;
     }
-    __syncthreads();
-    for (int e = tid; e < GT_COLS * 32; e += 256) {
-      const int c = e >> 5, r = e & 31;
-      if (c0 + c < d) xbT[(((long long)fb * P.G + g) * d + c0 + c) * Bp + rb + r] = tile[r * GT_PITCH + c];
+  } else {
+    for (int e = tid; e < 32 * d; e += 256) {
+      const int r = e / d, c = e - r * d;
+      const long long row = rows_sm[r];
+      out[(long long)r * ld0 + c] = row >= 0 ? X[row * P.ld + c] : __float2bfloat16_rn(0.f);
     }
-    __syncthreads();
   }
 }
 
 // ----------------------------------------------------------------- loss gradient
 // dz = (softmax(scores) - onehot(y)) * scale in both orientations; padding rows (y < 0) get zeros.
 // Block = 32 consecutive rows of one group; each of the 8 warps takes 4 rows; the bf16 results also go to a
-// shared tile from which the transposed copy leaves in 64-byte runs and the column sums (the block's share
-// of the last layer's bias gradient) are taken.  With `both` the block handles the rows at theta^k and then
-// at the stale point, and writes the difference of the two (fresh - stale, rounded to bf16) to `diff` in
-// place of the stale point's transposed copy; otherwise grid.y selects the point.
+// shared tile from which the column sums (the block's share of the last layer's bias gradient) are taken.
+// With `both` the block handles the rows at theta^k and then at the stale point, and also writes the
+// difference of the two (fresh - stale, rounded to bf16) to `diff`; otherwise grid.y selects the point.
 __global__ void __launch_bounds__(256) bf16_softmax_grad_kernel(const Params P, const float* scores, const int* yb,
-                                                                __nv_bfloat16* dz, __nv_bfloat16* dzT, int n_cls,
-                                                                int ldz, int Bp, int pitch, float* colsum,
-                                                                __nv_bfloat16* diff, int both) {
+                                                                __nv_bfloat16* dz, int n_cls, int ldz, int Bp,
+                                                                int pitch, float* colsum, __nv_bfloat16* diff,
+                                                                int both) {
   extern __shared__ __nv_bfloat16 sm_tile[];  // [32][pitch]
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const long long rows = (long long)P.G * Bp;
@@ -1167,8 +1147,8 @@ __global__ void __launch_bounds__(256) bf16_softmax_grad_kernel(const Params P, 
       const int lr = warp * 4 + i;
       const long long w = w0 + lr;
       const float* s = scores + w * n_cls;
-      __nv_bfloat16* o = dz + w * ldz;
-      const __nv_bfloat16* o0 = dz + (r0 + lr) * ldz;     // the same row at theta^k (written by this thread)
+      __nv_bfloat16* o = dz + (((long long)factor_entry(P, g, q) * Bp) + m0 + lr) * ldz;
+      const __nv_bfloat16* o0 = dz + (((long long)factor_entry(P, g, 0) * Bp) + m0 + lr) * ldz;  // the same row at theta^k (written by this thread)
       __nv_bfloat16* df = diff + (r0 + lr) * ldz;
       __nv_bfloat16* t = sm_tile + lr * pitch;
       const int y = yb[r0 + lr];
@@ -1199,10 +1179,6 @@ __global__ void __launch_bounds__(256) bf16_softmax_grad_kernel(const Params P, 
       }
     }
     __syncthreads();
-    if (!write_diff) {
-      __nv_bfloat16* oT = dzT + ((long long)factor_entry(P, g, q) * n_cls) * Bp + m0;
-      for (int c = warp; c < n_cls; c += 8) oT[(long long)c * Bp + lane] = sm_tile[lane * pitch + c];
-    }
     // column sums of the block's 32 rows in row order: this block's share of the bias gradient of the last layer
     float* cs = colsum + (((long long)(q * P.G + g)) * (Bp / 32) + m0 / 32) * n_cls;
     for (int c = threadIdx.x; c < n_cls; c += 256) {
@@ -1220,9 +1196,9 @@ __global__ void __launch_bounds__(256) bf16_softmax_grad_kernel(const Params P, 
 // pairs.
 template <int NP>
 __global__ void __launch_bounds__(256) bf16_softmax_grad_pairs_kernel(const Params P, const float* scores, const int* yb,
-                                                                      __nv_bfloat16* dz, __nv_bfloat16* dzT, int n_cls,
-                                                                      int ldz, int Bp, int pitch, float* colsum,
-                                                                      __nv_bfloat16* diff, int both) {
+                                                                      __nv_bfloat16* dz, int n_cls, int ldz, int Bp,
+                                                                      int pitch, float* colsum, __nv_bfloat16* diff,
+                                                                      int both) {
   extern __shared__ __nv_bfloat16 sm_tile[];  // [32][pitch]
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const long long rows = (long long)P.G * Bp;
@@ -1237,8 +1213,8 @@ __global__ void __launch_bounds__(256) bf16_softmax_grad_pairs_kernel(const Para
       const int lr = warp * 4 + i;
       const long long w = w0 + lr;
       const float* s = scores + w * n_cls;
-      __nv_bfloat16* o = dz + w * ldz;
-      const __nv_bfloat16* o0 = dz + (r0 + lr) * ldz;     // the same row at theta^k (written by this thread)
+      __nv_bfloat16* o = dz + (((long long)factor_entry(P, g, q) * Bp) + m0 + lr) * ldz;
+      const __nv_bfloat16* o0 = dz + (((long long)factor_entry(P, g, 0) * Bp) + m0 + lr) * ldz;  // the same row at theta^k (written by this thread)
       __nv_bfloat16* df = diff + (r0 + lr) * ldz;
       __nv_bfloat16* t = sm_tile + lr * pitch;
       const int y = yb[r0 + lr];
@@ -1282,10 +1258,6 @@ __global__ void __launch_bounds__(256) bf16_softmax_grad_pairs_kernel(const Para
       }
     }
     __syncthreads();
-    if (!write_diff) {
-      __nv_bfloat16* oT = dzT + ((long long)factor_entry(P, g, q) * n_cls) * Bp + m0;
-      for (int c = warp; c < n_cls; c += 8) oT[(long long)c * Bp + lane] = sm_tile[lane * pitch + c];
-    }
     float* cs = colsum + (((long long)(q * P.G + g)) * (Bp / 32) + m0 / 32) * n_cls;
     for (int c = threadIdx.x; c < n_cls; c += 256) {
       float v2 = 0.f;
@@ -1505,16 +1477,13 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
   } while (0)
   A_(im->wb, (long long)(D + 1) * im->slot_elems, __nv_bfloat16);
   A_(im->bias, (long long)(D + 1) * im->bias_slot, float);
-  A_(im->xb, rows * im->ld[0], __nv_bfloat16);
-  A_(im->xbT, 2LL * G * plan->dims[0] * im->Bp, __nv_bfloat16);
+  A_(im->xb, 2 * rows * im->ld[0], __nv_bfloat16);
   A_(im->yb, rows, int);
   for (int l = 1; l <= L; ++l) {
     if (l < L) {
-      A_(im->act[l], 2 * rows * im->ld[l], __nv_bfloat16);
-      A_(im->actT[l], 3LL * G * plan->dims[l] * im->Bp, __nv_bfloat16);
+      A_(im->act[l], 3 * rows * im->ld[l], __nv_bfloat16);
     }
-    A_(im->dz[l], 2 * rows * im->ld[l], __nv_bfloat16);
-    A_(im->dzT[l], 3LL * G * plan->dims[l] * im->Bp, __nv_bfloat16);
+    A_(im->dz[l], 3 * rows * im->ld[l], __nv_bfloat16);
   }
   A_(im->scores, 2 * rows * plan->dims[L], float);
   A_(im->db, 2LL * G * im->nbias, float);
@@ -1533,10 +1502,10 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
   plan->state.emplace_back(im->wb, sizeof(__nv_bfloat16) * (size_t)(D + 1) * im->slot_elems);
   plan->state.emplace_back(im->bias, sizeof(float) * (size_t)(D + 1) * im->bias_slot);
   // (both upload buffers of every group: which of the two holds the last upload is in Params::cur)
-  plan->state.emplace_back(im->xbT, sizeof(__nv_bfloat16) * (size_t)2 * G * plan->dims[0] * im->Bp);
+  plan->state.emplace_back(im->xb, sizeof(__nv_bfloat16) * (size_t)2 * rows * im->ld[0]);
   for (int l = 1; l <= L; ++l) {
-    plan->state.emplace_back(im->dzT[l], sizeof(__nv_bfloat16) * (size_t)2 * G * plan->dims[l] * im->Bp);
-    if (l < L) plan->state.emplace_back(im->actT[l], sizeof(__nv_bfloat16) * (size_t)2 * G * plan->dims[l] * im->Bp);
+    plan->state.emplace_back(im->dz[l], sizeof(__nv_bfloat16) * (size_t)2 * rows * im->ld[l]);
+    if (l < L) plan->state.emplace_back(im->act[l], sizeof(__nv_bfloat16) * (size_t)2 * rows * im->ld[l]);
   }
   plan->state.emplace_back(im->db, sizeof(float) * (size_t)2 * G * im->nbias);
   if (!encode_fn()) {
@@ -1549,24 +1518,24 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
     const int ni = plan->dims[l - 1], no = plan->dims[l];
     // forward: A = a_{l-1} rows, B = W_l (ring)
     if (l == 1)
-      ok &= make_map(&im->tm_fwd_a[l], im->xb, ni, Bp, G, im->ld[0], Bp * im->ld[0], BM);
+      ok &= make_map(&im->tm_fwd_a[l], im->xb, ni, Bp, 2LL * G, im->ld[0], Bp * im->ld[0], BM);
     else
-      ok &= make_map(&im->tm_fwd_a[l], im->act[l - 1], ni, Bp, 2LL * G, im->ld[l - 1], Bp * im->ld[l - 1], BM);
+      ok &= make_map(&im->tm_fwd_a[l], im->act[l - 1], ni, Bp, 3LL * G, im->ld[l - 1], Bp * im->ld[l - 1], BM);
     ok &= make_map(&im->tm_fwd_b[l], im->wb + im->w_pos[l], ni, no, D + 1, im->ld[l - 1], im->slot_elems, GN);
     // backward data: A = dz_l rows, B = W_l^T (ring)
-    ok &= make_map(&im->tm_da_a[l], im->dz[l], no, Bp, 2LL * G, im->ld[l], Bp * im->ld[l], BM);
+    ok &= make_map(&im->tm_da_a[l], im->dz[l], no, Bp, 3LL * G, im->ld[l], Bp * im->ld[l], BM);
     ok &= make_map(&im->tm_da_b[l], im->wb + im->wt_pos[l], no, ni, D + 1, im->ld[l], im->slot_elems, GN);
     // weight gradient: A = dz_l^T, B = a_{l-1}^T
     // differences of the two points (row-major, one entry per group): operands of the Gram products
     ok &= make_map(&im->tm_dE[l], im->dE[l], no, Bp, G, im->ld[l], Bp * im->ld[l], BM);
     if (l < L) ok &= make_map(&im->tm_dF[l], im->dF[l], no, Bp, G, im->ld[l], Bp * im->ld[l], BM);
-    // (the aggregate reads the same two arrays: the groups' upload buffers are their first 2G entries)
+    // weight gradient and aggregate: the same arrays read MN-major, in blocks of 64 batch rows x 64 columns
     static_assert(DW_BN == GN, "the weight-gradient and aggregate products share their B tensor map");
-    ok &= make_map(&im->tm_dw_a[l], im->dzT[l], Bp, no, 3LL * G, Bp, (long long)no * Bp, BM);
+    ok &= make_map(&im->tm_dw_a[l], im->dz[l], no, Bp, 3LL * G, im->ld[l], Bp * im->ld[l], 64);
     if (l == 1)
-      ok &= make_map(&im->tm_dw_b[l], im->xbT, Bp, ni, 2LL * G, Bp, (long long)ni * Bp, DW_BN);
+      ok &= make_map(&im->tm_dw_b[l], im->xb, ni, Bp, 2LL * G, im->ld[0], Bp * im->ld[0], 64);
     else
-      ok &= make_map(&im->tm_dw_b[l], im->actT[l - 1], Bp, ni, 3LL * G, Bp, (long long)ni * Bp, DW_BN);
+      ok &= make_map(&im->tm_dw_b[l], im->act[l - 1], ni, Bp, 3LL * G, im->ld[l - 1], Bp * im->ld[l - 1], 64);
   }
   if (!ok) {
     *why = "tensor map creation failed for this MLP shape";
@@ -1623,7 +1592,7 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     ++n;
   }
-  bf16_gather_kernel<<<dim3(Bp / 32, G), 256, 0, st>>>(P, im->xb, im->xbT, im->yb, pl.dims[0], im->ld[0], Bp);
+  bf16_gather_kernel<<<dim3(Bp / 32, G), 256, 0, st>>>(P, im->xb, im->yb, pl.dims[0], im->ld[0], Bp);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   ++n;
   // production: no group's weight gradient is formed; the stale point's epilogues write differences for the
@@ -1642,11 +1611,8 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
     if (l < L) {
       a.epi = EPI_HIDDEN;
       a.out = im->act[l];
-      a.outT = im->actT[l];
       a.ldo = im->ld[l];
-      a.ldt = Bp;
       a.z_stride_out = (long long)Bp * im->ld[l];
-      a.z_stride_outT = (long long)pl.dims[l] * Bp;
       a.diff = production ? im->dF[l] : nullptr;
       a.relu_bits = im->relu_bits[l];
       a.nw = (pl.dims[l] + 31) / 32;
@@ -1667,13 +1633,13 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
     const size_t sm = (size_t)32 * pitch * 2;
     if ((nc & 1) == 0 && nc <= 1024) {  // class pairs in registers
       if (nc <= 256)
-        bf16_softmax_grad_pairs_kernel<4><<<blocks, 256, sm, st>>>(P, im->scores, im->yb, im->dz[L], im->dzT[L], nc, im->ld[L], Bp, pitch, im->dbp[L], im->dE[L], both);
+        bf16_softmax_grad_pairs_kernel<4><<<blocks, 256, sm, st>>>(P, im->scores, im->yb, im->dz[L], nc, im->ld[L], Bp, pitch, im->dbp[L], im->dE[L], both);
       else if (nc <= 512)
-        bf16_softmax_grad_pairs_kernel<8><<<blocks, 256, sm, st>>>(P, im->scores, im->yb, im->dz[L], im->dzT[L], nc, im->ld[L], Bp, pitch, im->dbp[L], im->dE[L], both);
+        bf16_softmax_grad_pairs_kernel<8><<<blocks, 256, sm, st>>>(P, im->scores, im->yb, im->dz[L], nc, im->ld[L], Bp, pitch, im->dbp[L], im->dE[L], both);
       else
-        bf16_softmax_grad_pairs_kernel<16><<<blocks, 256, sm, st>>>(P, im->scores, im->yb, im->dz[L], im->dzT[L], nc, im->ld[L], Bp, pitch, im->dbp[L], im->dE[L], both);
+        bf16_softmax_grad_pairs_kernel<16><<<blocks, 256, sm, st>>>(P, im->scores, im->yb, im->dz[L], nc, im->ld[L], Bp, pitch, im->dbp[L], im->dE[L], both);
     } else {
-      bf16_softmax_grad_kernel<<<blocks, 256, sm, st>>>(P, im->scores, im->yb, im->dz[L], im->dzT[L], nc, im->ld[L], Bp, pitch, im->dbp[L], im->dE[L], both);
+      bf16_softmax_grad_kernel<<<blocks, 256, sm, st>>>(P, im->scores, im->yb, im->dz[L], nc, im->ld[L], Bp, pitch, im->dbp[L], im->dE[L], both);
     }
   }
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
@@ -1686,7 +1652,6 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
       ga.BN = ga.parts * Bp < GN ? ga.parts * Bp : GN;
       ga.Ku = pl.dims[l];
       ga.Kv = pl.dims[l - 1];
-      ga.zu1_stale = 1;
       ga.part_base = im->gram_part_base[l];
       ga.n_parts = im->n_parts;
       const int units = G * ga.parts * ga.nb * (ga.parts * Bp / ga.BN);
@@ -1709,15 +1674,12 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
       d.zb_mode = ZB_RING;
       d.epi = EPI_DA;
       d.out = im->dz[l - 1];
-      d.outT = im->dzT[l - 1];
       d.relu_bits = im->relu_bits[l - 1];
       d.nw = (pl.dims[l - 1] + 31) / 32;
       d.colsum = im->dbp[l - 1];
       d.diff = production ? im->dE[l - 1] : nullptr;
       d.ldo = im->ld[l - 1];
-      d.ldt = Bp;
       d.z_stride_out = (long long)Bp * im->ld[l - 1];
-      d.z_stride_outT = (long long)pl.dims[l - 1] * Bp;
       if ((e = launch_gemm(im->tm_da_a[l], im->tm_da_b[l], P, d, pl.sm_count, st)) != cudaSuccess) return e;
       ++n;
     }
