@@ -248,6 +248,8 @@ constexpr int G_EPI_WARPS = 8;
 constexpr int G_THREADS = 64 + 32 * G_EPI_WARPS;
 constexpr int G_TR_BYTES = G_EPI_WARPS * 32 * 17 * 4;  // per-warp transposition tiles of the epilogue
 constexpr int G_CS_BYTES = 2 * 4 * GN * 4;             // column sums of a tile per 32-row quadrant, two tiles in flight
+constexpr int G_BIAS_BYTES = G_EPI_WARPS * (GN / 2) * 4;  // each epilogue warp's 128 bias values of the current tile
+constexpr int G_SMEM_BYTES = G_STAGES * G_STAGE_BYTES + 1024 + G_TR_BYTES + G_CS_BYTES + G_BIAS_BYTES;
 constexpr uint32_t IDESC_G = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(GN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 constexpr uint32_t IDESC_MN = IDESC_G | (1u << 15) | (1u << 16);
 
@@ -413,6 +415,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
     const int half = ew >> 2;
     uint32_t* tr = reinterpret_cast<uint32_t*>(tiles + (size_t)G_STAGES * G_STAGE_BYTES) + ew * (32 * 17);
     float* cs_all = reinterpret_cast<float*>(tiles + (size_t)G_STAGES * G_STAGE_BYTES + G_TR_BYTES);  // [2][4][GN]
+    float* bias_w = reinterpret_cast<float*>(tiles + (size_t)G_STAGES * G_STAGE_BYTES + G_TR_BYTES + G_CS_BYTES) + ew * (GN / 2);
     bool ok = true;
     for (int i = 0; i < n_local; ++i) {
       const int slot = i & 1;
@@ -444,9 +447,23 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
         continue;
       }
       tc_fence_after();
-      const float* bias = nullptr;
-      if (a.epi == EPI_HIDDEN || a.epi == EPI_SCORES)
-        bias = a.bias_ring + (long long)ring_slot(P, g, q, k_it) * a.bias_slot + a.bias_pos;
+      if (a.epi == EPI_HIDDEN || a.epi == EPI_SCORES) {
+        // the 128 biases of this warp's columns, once per tile, into the warp's own shared-memory strip (read
+        // back as broadcasts); zeros beyond the matrix
+        const float* bias = a.bias_ring + (long long)ring_slot(P, g, q, k_it) * a.bias_slot + a.bias_pos;
+        const int col = n0 + half * (GN / 2) + lane * 4;
+        float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (col + 3 < a.N) {
+          b4 = *reinterpret_cast<const float4*>(bias + col);
+        } else {
+          if (col < a.N) b4.x = bias[col];
+          if (col + 1 < a.N) b4.y = bias[col + 1];
+          if (col + 2 < a.N) b4.z = bias[col + 2];
+        }
+        __syncwarp();
+        *reinterpret_cast<float4*>(bias_w + lane * 4) = b4;
+        __syncwarp();
+      }
       const uint32_t tbase = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(slot * GN);
       // one 32-column chunk of this thread's row
       auto chunk = [&](const uint32_t (&v)[32], int c) {
@@ -454,6 +471,19 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
         if (nc >= a.N) return;  // uniform across the warp
         const bool row_ok = m < a.M;
         const bool full = nc + 32 <= a.N;
+        const float* bw = bias_w + (c - half * (GN / 2));  // this chunk's biases (EPI_HIDDEN / EPI_SCORES)
+        // The stale point's tile also writes fresh - stale: the fresh point's values at the places this thread
+        // will store to (it stored them itself one tile ago) are fetched now, so that their latency is
+        // covered by the conversion work
+        const long long off0 = (long long)(mt * BM + quad * 32) * a.ldo + nc;
+        const bool fast = full && a.M - (mt * BM + quad * 32) >= 32;
+        uint4 frv[4] = {};
+        if (write_diff && fast) {
+#pragma unroll
+          for (int it = 0; it < 4; ++it)
+            frv[it] = *reinterpret_cast<const uint4*>(a.out + (long long)zF * a.z_stride_out + off0 +
+                                                      (long long)(it * 8 + (lane >> 2)) * a.ldo + (lane & 3) * 8);
+        }
         if (a.epi == EPI_AGG) {  // a block of the aggregated weight gradient, straight into the p-vector
           float* dst = a.out_f32 + a.c_off + (long long)m * a.ldc + nc;
           if (row_ok) {
@@ -479,17 +509,17 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
 #pragma unroll
               for (int j = 0; j < 32; j += 4)
                 *reinterpret_cast<float4*>(dst + j) =
-                    make_float4(__uint_as_float(v[j]) + bias[nc + j], __uint_as_float(v[j + 1]) + bias[nc + j + 1],
-                                __uint_as_float(v[j + 2]) + bias[nc + j + 2], __uint_as_float(v[j + 3]) + bias[nc + j + 3]);
+                    make_float4(__uint_as_float(v[j]) + bw[j], __uint_as_float(v[j + 1]) + bw[j + 1],
+                                __uint_as_float(v[j + 2]) + bw[j + 2], __uint_as_float(v[j + 3]) + bw[j + 3]);
             } else {
-              for (int j = 0; j < 32 && nc + j < a.N; ++j) dst[j] = __uint_as_float(v[j]) + bias[nc + j];
+              for (int j = 0; j < 32 && nc + j < a.N; ++j) dst[j] = __uint_as_float(v[j]) + bw[j];
             }
           }
         } else {
           float f[32];
           if (a.epi == EPI_HIDDEN) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) f[j] = fmaxf(__uint_as_float(v[j]) + (nc + j < a.N ? bias[nc + j] : 0.f), 0.f);
+            for (int j = 0; j < 32; ++j) f[j] = fmaxf(__uint_as_float(v[j]) + bw[j], 0.f);
           } else {  // EPI_DA: ReLU derivative of the layer below (bits of rows / columns outside the matrix are 0)
             const uint32_t bits = mbits[(c - half * (GN / 2)) >> 5];
 #pragma unroll
@@ -531,10 +561,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
             }
             cs_all[((i & 1) * 4 + quad) * GN + c + lane] = csum;
           }
-          const int rows_here = a.M - (mt * BM + quad * 32);  // valid rows of this warp's block (>= 32 inside)
-          if (full && rows_here >= 32) {
+          if (fast) {
             // row-major copy: lanes 4r..4r+3 write the 64 bytes of row r, eight rows per instruction
-            const long long off0 = (long long)(mt * BM + quad * 32) * a.ldo + nc;
             __nv_bfloat16* dst0 = a.out + (long long)zT * a.z_stride_out + off0;
 #pragma unroll
             for (int it = 0; it < 4; ++it) {
@@ -543,9 +571,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
               const uint4 mine = make_uint4(src[0], src[1], src[2], src[3]);
               *reinterpret_cast<uint4*>(dst0 + (long long)r * a.ldo + qd * 8) = mine;
               if (write_diff) {
-                // the fresh point's 16 bytes at this place were stored by this very thread one tile ago
-                const uint4 fr = *reinterpret_cast<const uint4*>(a.out + (long long)zF * a.z_stride_out + off0 +
-                                                                 (long long)r * a.ldo + qd * 8);
+                const uint4 fr = frv[it];
                 *reinterpret_cast<uint4*>(a.diff + (long long)g * a.z_stride_out + off0 + (long long)r * a.ldo + qd * 8) =
                     make_uint4(bf16x2_sub(fr.x, mine.x), bf16x2_sub(fr.y, mine.y), bf16x2_sub(fr.z, mine.z),
                                bf16x2_sub(fr.w, mine.w));
@@ -1376,7 +1402,7 @@ cudaError_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const Para
   a.stages = G_STAGES;
   const long long units = (long long)((a.N + GN - 1) / GN) * ((a.M + BM - 1) / BM) * (a.k_batched ? 1 : P.G);
   const int ctas = (int)(units < sm_count ? units : sm_count);
-  bf16_gemm_kernel<<<ctas, G_THREADS, (size_t)G_STAGES * G_STAGE_BYTES + 1024 + G_TR_BYTES + G_CS_BYTES, st>>>(ta, tb, P, a);
+  bf16_gemm_kernel<<<ctas, G_THREADS, (size_t)G_SMEM_BYTES, st>>>(ta, tb, P, a);
   return cudaGetLastError();
 }
 
@@ -1542,7 +1568,7 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
     return cudaSuccess;
   }
   cudaError_t e = cudaFuncSetAttribute(bf16_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       G_STAGES * G_STAGE_BYTES + 1024 + G_TR_BYTES + G_CS_BYTES);
+                                       G_SMEM_BYTES);
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(bf16_softmax_grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            32 * (plan->dims[L] + 4) * 2);
