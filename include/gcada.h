@@ -332,6 +332,20 @@ gcada_status gcada_checkpoint_size(gcada_ctx *ctx, unsigned long long *bytes);
 gcada_status gcada_checkpoint_save(gcada_ctx *ctx, void *host_buf, unsigned long long bytes);
 gcada_status gcada_checkpoint_load(gcada_ctx *ctx, const void *host_buf, unsigned long long bytes);
 
+/*
+ * The debug library.  libgcada_dbg.so is this same source compiled with -DGCADA_DEBUG: every store whose
+ * position a kernel computes at run time (partial-sum slots, innovation-norm partial sums, the mask history,
+ * the list of selected groups, gradient rows, the entries of the bf16 factor arrays) is checked against the
+ * size of its buffer first.  A failed check does not trap: the store is skipped, the run's device error word
+ * is raised, and from then on every getter returns GCADA_ECUDA with the buffer named in gcada_last_error
+ * (a bounded device-side wait that gave up is reported as GCADA_ETIMEOUT the same way, in both libraries).
+ * gcada_is_debug_build tells the two libraries apart (1 / 0).  gcada_debug_set_error writes the device error
+ * word from the host (dev_err: 0 none, 1 a wait gave up, 2 an index check failed) so that the reporting path
+ * can be exercised without any device-side failure; in the ordinary library it returns GCADA_ESTATE.
+ */
+int gcada_is_debug_build(void);
+gcada_status gcada_debug_set_error(gcada_ctx *ctx, int dev_err);
+
 /* Text of the last error of this context ("" if none); valid until the next
  * call on the context.  ctx == NULL returns the text of the last failed
  * gcada_create of the calling thread. */

@@ -11,6 +11,7 @@ import numpy as np
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libgcada.so")
+DEBUG_LIB_PATH = os.path.join(HERE, "libgcada_dbg.so")   # the same source with every computed store index checked
 
 OK, EINVAL, ENOMEM, ECUDA, ESTATE, ETIMEOUT = range(6)
 MODEL_LOGISTIC, MODEL_MLP, MODEL_QUADRATIC = 0, 1, 2
@@ -70,6 +71,8 @@ SIGNATURES = {
     "gcada_checkpoint_size": (C.c_int, [_VP, _ULLP]),
     "gcada_checkpoint_save": (C.c_int, [_VP, _VP, C.c_ulonglong]),
     "gcada_checkpoint_load": (C.c_int, [_VP, _VP, C.c_ulonglong]),
+    "gcada_is_debug_build": (C.c_int, []),
+    "gcada_debug_set_error": (C.c_int, [_VP, C.c_int]),
     "gcada_last_error": (C.c_char_p, [_VP]),
     "gcada_destroy": (None, [_VP]),
 }
@@ -274,6 +277,10 @@ class GCada:
     def checkpoint_load(self, buf):
         buf = np.ascontiguousarray(buf, dtype=np.uint8)
         self._ck(self.lib.gcada_checkpoint_load(self.h, _VP(buf.ctypes.data), buf.size))
+
+    def debug_set_error(self, dev_err):
+        """Debug library only: write the device error word (0 none, 1 a wait gave up, 2 an index check failed)."""
+        self._ck(self.lib.gcada_debug_set_error(self.h, int(dev_err)))
 
     def get_debug(self, what):
         G, p, D = self.G, self.p, self.D

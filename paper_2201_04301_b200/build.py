@@ -1,6 +1,6 @@
 """Compile the CUDA sources of this package into libgcada.so (in-tree).
 
-    python -m paper_2201_04301_b200.build [--force] [--verbose]
+    python -m paper_2201_04301_b200.build [--force] [--verbose] [--debug]
 
 nvcc cross-compiles for sm_100a; no GPU is needed to build.
 """
@@ -12,6 +12,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libgcada.so")
+DEBUG_LIB = os.path.join(HERE, "libgcada_dbg.so")
 SOURCES = ["api.cu", "grad_linear.cu", "tail.cu", "mlp.cu", "mlp_bf16.cu", "noalloc.cu", "eval.cu", "linear_cluster.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC,-Wall,-Wno-unused-function", "--expt-relaxed-constexpr"]
@@ -26,18 +27,23 @@ def _newest_header():
     return t
 
 
-def build(force=False, verbose=False):
+def build(force=False, verbose=False, debug=False):
+    """Compile libgcada.so, or with debug=True libgcada_dbg.so: the same sources with -DGCADA_DEBUG (every
+    store position a kernel computes is checked against its buffer; a failed check raises an error word)."""
     nvcc = os.environ.get("NVCC", "nvcc")
-    os.makedirs(OBJ, exist_ok=True)
+    obj_dir = OBJ + ("_dbg" if debug else "")
+    lib = DEBUG_LIB if debug else LIB
+    flags = NVCC_FLAGS + (["-DGCADA_DEBUG"] if debug else [])
+    os.makedirs(obj_dir, exist_ok=True)
     hdr_t = _newest_header()
     objs, rebuilt = [], False
     procs = []
     for src in SOURCES:
         s = os.path.join(CSRC, src)
-        o = os.path.join(OBJ, src.replace(".cu", ".o"))
+        o = os.path.join(obj_dir, src.replace(".cu", ".o"))
         objs.append(o)
         if force or not os.path.exists(o) or os.path.getmtime(o) < max(os.path.getmtime(s), hdr_t):
-            cmd = [nvcc, *NVCC_FLAGS, "-c", s, "-o", o]
+            cmd = [nvcc, *flags, "-c", s, "-o", o]
             if verbose:
                 cmd.insert(1, "-Xptxas=-v")
                 print(" ".join(cmd), flush=True)
@@ -49,13 +55,13 @@ def build(force=False, verbose=False):
             raise RuntimeError("nvcc failed on %s:\n%s" % (src, out))
         if verbose or out.strip():
             print(out)
-    if rebuilt or not os.path.exists(LIB):
-        cmd = [nvcc, "-shared", "-o", LIB, *objs, "-gencode", "arch=compute_100a,code=sm_100a"]
+    if rebuilt or not os.path.exists(lib):
+        cmd = [nvcc, "-shared", "-o", lib, *objs, "-gencode", "arch=compute_100a,code=sm_100a"]
         r = subprocess.run(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)
         if r.returncode != 0:
             raise RuntimeError("link failed:\n%s" % r.stdout)
-    return LIB
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, debug="--debug" in sys.argv))

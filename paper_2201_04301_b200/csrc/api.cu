@@ -210,6 +210,9 @@ gcada_status make_ready(gcada_ctx* ctx, const float* theta0, int on_device) {
   TRY(dev_alloc(ctx, &P.hist, (size_t)ctx->hist_cap * G));
   plan_tail(pp, G, ctx->sm_count, &ctx->tail);
   TRY(dev_alloc(ctx, &P.lhs_part, (size_t)G * ctx->tail.select_blocks_x));
+  P.lim.lhs_parts = (long long)G * ctx->tail.select_blocks_x;
+  P.lim.hist_bytes = ctx->hist_cap * G;
+  P.lim.grad_rows = P.gbuf ? 2LL * G : 0;
   TRY(dev_alloc(ctx, &P.upd_part, (size_t)ctx->tail.update_blocks));
   // everything an iteration inherits from earlier ones
   {
@@ -282,6 +285,7 @@ gcada_status make_plans(gcada_ctx* ctx) {
     P.pm.maxseg = ctx->lin.maxseg;
     P.pm.rows_per_group = ctx->B;
     TRY(dev_alloc(ctx, &P.partial, (size_t)ctx->lin.n_cta * ctx->lin.maxseg * 2 * ctx->p_pad));
+    P.lim.partial_slots = (long long)ctx->lin.n_cta * ctx->lin.maxseg;
   } else {
     P.pm.n_cta = 0;
     P.pm.maxseg = 0;
@@ -297,6 +301,7 @@ gcada_status make_plans(gcada_ctx* ctx) {
       P.pm.n_cta = -1;
       P.pm.maxseg = ctx->mlp.norm_parts;
       TRY(dev_alloc(ctx, &P.lhs_part, (size_t)ctx->G * ctx->mlp.norm_parts));
+      P.lim.lhs_parts = (long long)ctx->G * ctx->mlp.norm_parts;
     }
   }
   if (ctx->rule == 1) {
@@ -462,8 +467,13 @@ gcada_status group_row_dev(gcada_ctx* ctx, int what, int g, const std::vector<un
 gcada_status read_state(gcada_ctx* ctx, DevState* out) {
   CK(cudaStreamSynchronize(ctx->stream));
   CK(cudaMemcpy(out, ctx->st, sizeof(DevState), cudaMemcpyDeviceToHost));
-  if (out->err != DEV_OK)
-    return fail(ctx, GCADA_ETIMEOUT, "device-side error %d (a bounded wait on an asynchronous copy gave up)", out->err);
+  if (out->err == DEV_ERR_COPY_TIMEOUT)
+    return fail(ctx, GCADA_ETIMEOUT, "device-side error %d: a bounded wait on an asynchronous copy or a pipeline barrier gave up",
+                out->err);
+  if (out->err == DEV_ERR_BOUNDS)
+    return fail(ctx, GCADA_ECUDA, "device-side error %d: an index check of the debug library failed (buffer %d); the store was skipped",
+                out->err, out->err_info);
+  if (out->err != DEV_OK) return fail(ctx, GCADA_ECUDA, "device-side error %d", out->err);
   return GCADA_OK;
 }
 
@@ -1201,6 +1211,29 @@ gcada_status gcada_checkpoint_load(gcada_ctx* ctx, const void* host_buf, unsigne
   TRY(read_state(ctx, &s));
   ctx->k_host = s.k;
   return GCADA_OK;
+}
+
+int gcada_is_debug_build(void) {
+#ifdef GCADA_DEBUG
+  return 1;
+#else
+  return 0;
+#endif
+}
+
+gcada_status gcada_debug_set_error(gcada_ctx* ctx, int dev_err) {
+  if (!ctx) return GCADA_EINVAL;
+#ifdef GCADA_DEBUG
+  if (!ctx->have_theta) return fail(ctx, GCADA_ESTATE, "gcada_set_theta has not been called");
+  if (dev_err < 0 || dev_err > DEV_ERR_BOUNDS) return fail(ctx, GCADA_EINVAL, "unknown device error word %d", dev_err);
+  DeviceGuard dg(ctx->device);
+  CK(cudaStreamSynchronize(ctx->stream));
+  CK(cudaMemcpy(&ctx->st->err, &dev_err, sizeof(int), cudaMemcpyHostToDevice));
+  return GCADA_OK;
+#else
+  (void)dev_err;
+  return fail(ctx, GCADA_ESTATE, "gcada_debug_set_error exists in the debug library (libgcada_dbg.so) only");
+#endif
 }
 
 const char* gcada_last_error(const gcada_ctx* ctx) { return ctx ? ctx->err.c_str() : g_create_error.c_str(); }

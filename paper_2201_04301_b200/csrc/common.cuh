@@ -9,6 +9,8 @@ namespace gcada {
 
 // Device error words (DevState::err).
 enum { DEV_OK = 0, DEV_ERR_COPY_TIMEOUT = 1, DEV_ERR_BOUNDS = 2 };
+// What a failed index check was about to store to (DevState::err_info with DEV_ERR_BOUNDS).
+enum { CHK_PARTIAL = 1, CHK_LHS_PART = 2, CHK_HIST = 3, CHK_SEL_LIST = 4, CHK_GRAD_ROW = 5, CHK_FACTOR = 6 };
 
 // Mutable run state kept in device memory so that a captured graph can be
 // replayed without changing kernel arguments.
@@ -39,8 +41,18 @@ struct PartialMap {
   int rows_per_group;  // B
 };
 
+// Element counts of the buffers that kernels address with computed positions.  The library built with
+// -DGCADA_DEBUG checks every such position against them before it stores (see GCADA_INDEX_OK).
+struct Limits {
+  long long partial_slots;  // slots of 2 * p_pad floats in Params::partial
+  long long lhs_parts;      // doubles in Params::lhs_part
+  long long hist_bytes;     // bytes in Params::hist
+  long long grad_rows;      // rows of p_pad floats in Params::gbuf
+};
+
 struct Params {
   DevState* st;
+  Limits lim;
   // problem
   int G, M, M_G, D, B;
   long long n_g;        // shard rows per group
@@ -98,6 +110,20 @@ struct Params {
                                 // kernels work on the selected groups only (rule PS: Algorithm 1 as printed,
                                 // workers of unselected groups compute nothing)
 };
+
+// Index check of the debug library: true if 0 <= idx < limit; otherwise the run's error word is raised (first
+// failure wins; err_info says which buffer) and the caller skips the access - nothing traps, the context stays
+// usable and every getter then reports the failure.  Compiles to `true` in the ordinary library.
+#ifdef GCADA_DEBUG
+__device__ __forceinline__ bool index_ok(DevState* st, long long idx, long long limit, int what) {
+  if (idx >= 0 && idx < limit) return true;
+  if (atomicCAS(&st->err, (int)DEV_OK, (int)DEV_ERR_BOUNDS) == (int)DEV_OK) st->err_info = what;
+  return false;
+}
+#define GCADA_INDEX_OK(st, idx, limit, what) gcada::index_ok((st), (long long)(idx), (long long)(limit), (what))
+#else
+#define GCADA_INDEX_OK(st, idx, limit, what) true
+#endif
 
 // ---------------------------------------------------------------------------
 // Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11).

@@ -124,8 +124,12 @@ __global__ void __launch_bounds__(THREADS, MINB) grad_linear_large_kernel(const 
   const int n_groups = build_group_list(P, sel_sm, &n_groups_sm);
   const bool skip = P.skip_unselected != 0;
   const long long Rtot = (long long)n_groups * B;
-  const long long r0 = (long long)blockIdx.x * Rtot / gridDim.x;
-  const long long r1 = (long long)(blockIdx.x + 1) * Rtot / gridDim.x;
+  // (when only the selected groups compute there may be fewer rows than CTAs: the first Rtot CTAs take one each,
+  // so that no CTA with an empty range sits between two that hold a group's partial sums)
+  const long long n_eff = Rtot < (long long)gridDim.x ? Rtot : (long long)gridDim.x;
+  if ((long long)blockIdx.x >= n_eff) return;
+  const long long r0 = (long long)blockIdx.x * Rtot / n_eff;
+  const long long r1 = (long long)(blockIdx.x + 1) * Rtot / n_eff;
   if (r0 >= r1) return;
   const int rows_cta = (int)(r1 - r0);
   const int g_first = (int)(r0 / B);
@@ -169,7 +173,11 @@ __global__ void __launch_bounds__(THREADS, MINB) grad_linear_large_kernel(const 
   int failed = 0;
 
   auto flush = [&](int g) {
-    float* dst = P.partial + ((long long)(blockIdx.x * P.pm.maxseg + (g - g_first)) * 2) * P.p_pad;
+    const long long slot = (long long)blockIdx.x * P.pm.maxseg + (g - g_first);
+    if (!GCADA_INDEX_OK(P.st, g - g_first, P.pm.maxseg, CHK_PARTIAL) ||
+        !GCADA_INDEX_OK(P.st, slot, P.lim.partial_slots, CHK_PARTIAL))
+      return;
+    float* dst = P.partial + (slot * 2) * P.p_pad;
 #pragma unroll
     for (int i = 0; i < CPT; ++i) {
       if (!own[i]) continue;
@@ -389,8 +397,10 @@ __global__ void __launch_bounds__(256) grad_linear_small_kernel(const Params P) 
   const int n_groups = build_group_list(P, sel_sm, &n_groups_sm);  // positions in this list are called g below
   const bool skip = P.skip_unselected != 0;
   const long long Rtot = (long long)n_groups * P.B;
-  const long long r0 = (long long)blockIdx.x * Rtot / gridDim.x;
-  const long long r1 = (long long)(blockIdx.x + 1) * Rtot / gridDim.x;
+  const long long n_eff = Rtot < (long long)gridDim.x ? Rtot : (long long)gridDim.x;  // see the wide kernel
+  if ((long long)blockIdx.x >= n_eff) return;
+  const long long r0 = (long long)blockIdx.x * Rtot / n_eff;
+  const long long r1 = (long long)(blockIdx.x + 1) * Rtot / n_eff;
   if (r0 >= r1) return;
   const int g_first = (int)(r0 / P.B);
 
@@ -468,8 +478,11 @@ __global__ void __launch_bounds__(256) grad_linear_small_kernel(const Params P) 
       accw[warp][1][lane + 32 * i] = acc1[i];
     }
     __syncthreads();
-    float* dst = P.partial + ((long long)(blockIdx.x * P.pm.maxseg + (g - g_first)) * 2) * P.p_pad;
-    for (int e = tid; e < 2 * 32 * CPL; e += 256) {
+    const long long slot = (long long)blockIdx.x * P.pm.maxseg + (g - g_first);
+    const bool slot_ok = GCADA_INDEX_OK(P.st, g - g_first, P.pm.maxseg, CHK_PARTIAL) &&
+                         GCADA_INDEX_OK(P.st, slot, P.lim.partial_slots, CHK_PARTIAL);
+    float* dst = P.partial + (slot * 2) * P.p_pad;
+    for (int e = tid; slot_ok && e < 2 * 32 * CPL; e += 256) {
       const int pt = e / (32 * CPL), c = e - pt * 32 * CPL;
       if (c < d) {
         float s = 0.f;

@@ -364,7 +364,8 @@ __global__ void __launch_bounds__(LC_THREADS, 1) linear_cluster_kernel(const Par
       S.tg[g] = t;
       S.mask[g] = sel ? 1 : 0;
       S.tau[g] = sel ? 1 : tau + 1;
-      if (cta == 0) P.hist[(long long)hslot * G + g] = sel ? 1 : 0;
+      if (cta == 0 && GCADA_INDEX_OK(P.st, (long long)hslot * G + g, P.lim.hist_bytes, CHK_HIST))
+        P.hist[(long long)hslot * G + g] = sel ? 1 : 0;
     }
     __syncthreads();
     int nsel = 0;

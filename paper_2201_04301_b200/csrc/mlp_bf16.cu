@@ -103,6 +103,7 @@ struct GemmB {
                               // [z][N / 32 rounded up][M] words (rows of a word position are contiguous).
                               // EPI_HIDDEN writes them, EPI_DA of the same layer reads them as the ReLU derivative
   int nw;                     // words per row: (N + 31) / 32
+  int n_entries;              // entries of `out` (checked by the debug library)
   float* colsum;              // EPI_DA: [z][tiles_m][N] column sums of the (bf16-rounded) output tile, or null
   __nv_bfloat16* diff;        // EPI_HIDDEN / EPI_DA, or null: row-major [G][M][ldo]; the stale-point tile also
                               // writes (fresh output - its own output) here, rounded to bf16: the small
@@ -426,6 +427,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
       const bool write_diff = q == 1 && a.diff != nullptr;
       const int zT = a.k_batched ? 0 : factor_entry(P, g, q);  // entry of the output in its factor array
       const int zF = a.k_batched ? 0 : factor_entry(P, g, 0);  // entry of the fresh point's output
+      // (debug library) the entry of the factor array this tile stores to
+      const bool entry_ok = a.k_batched || a.epi == EPI_SCORES || GCADA_INDEX_OK(P.st, zT, a.n_entries, CHK_FACTOR);
       const int m = mt * BM + quad * 32 + lane;
       const int n0 = nt * GN;
       // EPI_DA: the ReLU derivative of this thread's row does not depend on the accumulator: its four words
@@ -468,7 +471,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
       // one 32-column chunk of this thread's row
       auto chunk = [&](const uint32_t (&v)[32], int c) {
         const int nc = n0 + c;
-        if (nc >= a.N) return;  // uniform across the warp
+        if (nc >= a.N || !entry_ok) return;  // uniform across the warp
         const bool row_ok = m < a.M;
         const bool full = nc + 32 <= a.N;
         const float* bw = bias_w + (c - half * (GN / 2));  // this chunk's biases (EPI_HIDDEN / EPI_SCORES)
@@ -798,7 +801,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gram_kernel(const __grid_co
         double tsum = 0.0;
 #pragma unroll
         for (int w = 0; w < G_EPI_WARPS; ++w) tsum += norm_sm[w];
-        P.lhs_part[(long long)g * a.n_parts + a.part_base + r] = tsum;
+        if (GCADA_INDEX_OK(P.st, (long long)g * a.n_parts + a.part_base + r, P.lim.lhs_parts, CHK_LHS_PART))
+          P.lhs_part[(long long)g * a.n_parts + a.part_base + r] = tsum;
       }
       asm volatile("bar.sync 1, %0;" ::"n"(32 * G_EPI_WARPS) : "memory");
     }
@@ -1054,7 +1058,8 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
         double tsum = 0.0;
 #pragma unroll
         for (int w = 0; w < DW_EPI_WARPS; ++w) tsum += norm_sm[ui & 1][w];
-        P.lhs_part[(long long)g * a.n_parts + a.part_base + mt] = tsum;
+        if (GCADA_INDEX_OK(P.st, (long long)g * a.n_parts + a.part_base + mt, P.lim.lhs_parts, CHK_LHS_PART))
+          P.lhs_part[(long long)g * a.n_parts + a.part_base + mt] = tsum;
       }
     }
     if (!ok && lane == 0) atomicExch(&P.st->err, DEV_ERR_COPY_TIMEOUT);
@@ -1333,7 +1338,9 @@ __global__ void __launch_bounds__(64) bf16_bias_grad_kernel(const Params P, cons
     d2 = (double)(f - sv) * (double)(f - sv);
   }
   d2 = block_sum(d2, scratch);
-  if (threadIdx.x == 0) P.lhs_part[(long long)g * a.n_parts + a.part_base[l] + blockIdx.x] = d2;
+  if (threadIdx.x == 0 &&
+      GCADA_INDEX_OK(P.st, (long long)g * a.n_parts + a.part_base[l] + blockIdx.x, P.lim.lhs_parts, CHK_LHS_PART))
+    P.lhs_part[(long long)g * a.n_parts + a.part_base[l] + blockIdx.x] = d2;
 }
 
 // ----------------------------------------------------------------- bias part of the aggregate
@@ -1640,6 +1647,7 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
       a.ldo = im->ld[l];
       a.z_stride_out = (long long)Bp * im->ld[l];
       a.diff = production ? im->dF[l] : nullptr;
+      a.n_entries = 3 * G;
       a.relu_bits = im->relu_bits[l];
       a.nw = (pl.dims[l] + 31) / 32;
     } else {
@@ -1704,6 +1712,7 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
       d.nw = (pl.dims[l - 1] + 31) / 32;
       d.colsum = im->dbp[l - 1];
       d.diff = production ? im->dE[l - 1] : nullptr;
+      d.n_entries = 3 * G;
       d.ldo = im->ld[l - 1];
       d.z_stride_out = (long long)Bp * im->ld[l - 1];
       if ((e = launch_gemm(im->tm_da_a[l], im->tm_da_b[l], P, d, pl.sm_count, st)) != cudaSuccess) return e;

@@ -58,11 +58,15 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
       gi = (int)(block_sum((double)before, scratch) + 0.5);
       n_groups = (int)(block_sum((double)total, scratch) + 0.5);
     }
+    if (!GCADA_INDEX_OK(P.st, P.cur[g], 2, CHK_GRAD_ROW) ||
+        !GCADA_INDEX_OK(P.st, (long long)P.G + g, P.lim.grad_rows, CHK_GRAD_ROW))
+      return;  // (debug library: the group's two gradient rows are rows g and G + g of gbuf)
     float* fresh_g = what == SEL_REDUCE ? last_row(P, g) : fresh_row(P, g);
     int c_lo = 0, c_hi = -1;
     const long long Rtot = (long long)n_groups * P.pm.rows_per_group;
-    const int n = P.pm.n_cta;
-    // CTA c of the gradient kernel owns rows [c*Rtot/n, (c+1)*Rtot/n); 32-bit arithmetic where the products fit
+    // CTA c of the gradient kernel owns rows [c*Rtot/n, (c+1)*Rtot/n), n = the CTAs that got rows (all of them
+    // unless only a few selected groups compute); 32-bit arithmetic where the products fit
+    const int n = (P.pm.n_cta > 0 && Rtot < (long long)P.pm.n_cta) ? (int)Rtot : P.pm.n_cta;
     const bool small = (Rtot + 1) * (long long)(n + 1) < 0x7fffffffLL;
     if (n > 0) {
       const long long x0 = (long long)gi * P.pm.rows_per_group;
@@ -120,7 +124,8 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
     if (what == SEL_REDUCE) return;
     const double tot = block_sum(local, scratch);
     if (tid == 0) {
-      P.lhs_part[(long long)g * blocks_x + blockIdx.x] = tot;
+      if (GCADA_INDEX_OK(P.st, (long long)g * blocks_x + blockIdx.x, P.lim.lhs_parts, CHK_LHS_PART))
+        P.lhs_part[(long long)g * blocks_x + blockIdx.x] = tot;
       __threadfence();
       const unsigned int total = (unsigned int)blocks_x * (unsigned int)P.G;
       is_last = atomicAdd(&P.st->ticket_select, 1u) == total - 1u;
@@ -215,7 +220,8 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
       P.lhs[gg] = lhs;
       P.t_g[gg] = t;
       P.mask_cur[gg] = sel ? 1 : 0;
-      P.hist[(k % P.hist_cap) * P.G + gg] = sel ? 1 : 0;
+      if (GCADA_INDEX_OK(P.st, (k % P.hist_cap) * P.G + gg, P.lim.hist_bytes, CHK_HIST))
+        P.hist[(k % P.hist_cap) * P.G + gg] = sel ? 1 : 0;
       P.tau[gg] = sel ? 1 : tau + 1;
       if (sel) P.cur[gg] ^= 1;  // the fresh gradient's row becomes the last uploaded one
       if (sel) {
@@ -234,7 +240,8 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
         if (w < warp) base += sh_cnt[w];
         all += sh_cnt[w];
       }
-      if (sel) P.sel_list[base + __popc(b & ((1u << lane) - 1u))] = gg;
+      if (sel && GCADA_INDEX_OK(P.st, base + __popc(b & ((1u << lane) - 1u)), P.G, CHK_SEL_LIST))
+        P.sel_list[base + __popc(b & ((1u << lane) - 1u))] = gg;
       listed += all;
     }
   }

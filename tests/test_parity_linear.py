@@ -230,3 +230,13 @@ def test_rule_ps_wide_model_skips_work():
     L = [0.5 + 0.1 * g for g in range(16)]
     flips, worst = forced_parity(w, 14, stream=_stream(), L=L)
     print("rule PS wide worst", worst, "flips", flips)
+
+
+def test_rule_ps_wide_model_with_fewer_selected_rows_than_ctas():
+    """Printed rule on the row-ring kernel when the selected groups' rows are fewer than the kernel's CTAs
+    (small minibatches): only the first rows-many CTAs work, one row each, and the selection kernel must add
+    up exactly those (a CTA without rows between two that hold a group's partial sums would contribute
+    whatever its slot held before)."""
+    w = make_workload("cfg3", rows=6 * 300, M=12, M_G=2, D=3, batch=40)
+    flips, worst = forced_parity(w, 8, stream=_stream(), L=[3.0, 0.2, 1.4, 0.05, 2.0, 0.5])
+    print("rule PS, few rows, worst", worst, "flips", flips)
