@@ -341,6 +341,96 @@ __global__ void __launch_bounds__(256) mlp_bias_grad_kernel(const Params P, cons
   ((q == 0 ? (P.skip_unselected ? last_row(P, g) : fresh_row(P, g)) : P.stale + (long long)g * P.p_pad) + a.b_off[l])[n] = s;
 }
 
+// ------------------------------------------------------------------ small output layer, fused
+// Networks whose last layer is small (at most 16 classes on at most 256 hidden units: the 784-200-10 workload)
+// spend their time in launch and dependency latency, not in arithmetic.  Everything on the back-propagation
+// chain above the last hidden layer is local to a minibatch row, so one launch does it, a warp per row:
+// class scores z_L = a_{L-1} W_L^T + b_L, the loss gradient dz_L, and the back-propagated error
+// dz_{L-1} = (dz_L W_L) masked by a_{L-1} > 0.  It replaces three dependent launches (scores, loss gradient,
+// backward-data).  Grid (ceil(B / 8), 2 G); the CTA stages W_L of its (point, group) in shared memory.
+constexpr int HEAD_MAX_N = 16;   // classes
+constexpr int HEAD_CH = 8;       // hidden units per lane: up to 256 hidden units
+struct HeadArgs {
+  int n1, nL;                    // hidden units n_{L-1}, classes n_L
+  long long w_off, b_off;        // W_L and b_L inside theta
+  const float* a1;               // [2][G*B][n1]  activations of the last hidden layer
+  const int* yb;                 // [G*B]
+  float* dzL;                    // [2][G*B][nL]
+  float* dz1;                    // [2][G*B][n1]
+};
+
+__global__ void __launch_bounds__(256) mlp_head_kernel(const Params P, const HeadArgs a) {
+  extern __shared__ float hsm[];  // W_L [nL][n1]
+  const int n1 = a.n1, nL = a.nL;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int z = blockIdx.y, q = z / P.G, g = z - q * P.G;
+  if (P.skip_unselected && (q != 0 || !P.mask_cur[g])) return;
+  const long long k_it = P.st->k;
+  const float* theta = ring_ptr(P, g, q, k_it);
+  const int r = blockIdx.x * 8 + warp;
+  const long long row = (long long)q * P.G * P.B + (long long)g * P.B + (r < P.B ? r : 0);
+  // the row's activations and label are on their way while the weights are staged
+  const float* ar = a.a1 + row * n1;
+  float av[HEAD_CH];
+#pragma unroll
+  for (int u = 0; u < HEAD_CH; ++u) av[u] = lane + 32 * u < n1 ? ar[lane + 32 * u] : 0.f;
+  const int y = a.yb[(long long)g * P.B + (r < P.B ? r : 0)];
+  const float bl = lane < nL ? theta[a.b_off + lane] : 0.f;
+  for (int e = threadIdx.x; e < nL * n1; e += 256) hsm[e] = theta[a.w_off + e];
+  __syncthreads();
+  if (r >= P.B) return;
+  // class scores: lane c ends up with z_L[c]
+  float mine = 0.f;
+#pragma unroll
+  for (int c = 0; c < HEAD_MAX_N; ++c) {
+    if (c < nL) {  // (uniform)
+      float v = 0.f;
+#pragma unroll
+      for (int u = 0; u < HEAD_CH; ++u)
+        if (lane + 32 * u < n1) v += av[u] * hsm[c * n1 + lane + 32 * u];
+      v = warp_sum(v);
+      if (lane == c) mine = v + bl;
+    }
+  }
+  // loss gradient across the lanes; p_y - 1 = -(sum of the other classes' exponentials) / sum, free of cancellation
+  float mx = lane < nL ? mine : -3.0e38f;
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+  const float ex = lane < nL ? expf(mine - mx) : 0.f;
+  const float others = warp_sum(lane == y ? 0.f : ex);
+  const float ey = __shfl_sync(0xffffffffu, ex, y & 31);
+  const float inv = 1.0f / (others + ey);
+  const float dzc = lane < nL ? (lane == y ? -others * inv : ex * inv) * P.scale : 0.f;
+  if (lane < nL) a.dzL[row * nL + lane] = dzc;
+  // back-propagated error of the last hidden layer
+  float acc[HEAD_CH];
+#pragma unroll
+  for (int u = 0; u < HEAD_CH; ++u) acc[u] = 0.f;
+#pragma unroll
+  for (int c = 0; c < HEAD_MAX_N; ++c) {
+    if (c < nL) {
+      const float d = __shfl_sync(0xffffffffu, dzc, c);
+#pragma unroll
+      for (int u = 0; u < HEAD_CH; ++u)
+        if (lane + 32 * u < n1) acc[u] += d * hsm[c * n1 + lane + 32 * u];
+    }
+  }
+  float* d1 = a.dz1 + row * n1;
+#pragma unroll
+  for (int u = 0; u < HEAD_CH; ++u)
+    if (lane + 32 * u < n1) d1[lane + 32 * u] = av[u] > 0.f ? acc[u] : 0.f;
+}
+
+size_t head_smem_bytes(const MlpPlan& pl) {
+  const int L = pl.n_layers;
+  return (size_t)pl.dims[L] * pl.dims[L - 1] * sizeof(float);
+}
+bool head_fits(const MlpPlan& pl) {
+  const int L = pl.n_layers;
+  return pl.compute == 0 && L >= 2 && pl.dims[L] <= HEAD_MAX_N && pl.dims[L - 1] <= 32 * HEAD_CH &&
+         head_smem_bytes(pl) <= 96 * 1024;
+}
+
 cudaError_t launch_gemm(const Params& P, GemmArgs a, int sm_count, cudaStream_t st) {
   if (a.N <= ROWDOT_MAX_N && a.A.cs == 1 && a.Bm.rs == 1 && !a.c_grad && (size_t)a.N * a.K * sizeof(float) <= 48 * 1024) {
     mlp_rowdot_kernel<<<dim3((a.M + 7) / 8, 2 * P.G), 256, (size_t)a.N * a.K * sizeof(float), st>>>(P, a);
@@ -424,7 +514,12 @@ cudaError_t mlp_plan_create(const std::vector<int>& dims, int compute, int G, in
     if ((e = alloc(reinterpret_cast<void**>(&plan->dz[l]), sizeof(float) * 2 * rows * dims[l])) != cudaSuccess) return e;
   }
   plan->launches_per_iter = 3 * L + 2;
-  plan->skip_launches = 3 * L + 2;  // the same kernels; blocks of unselected groups and of the stale point exit at once
+  if (head_fits(*plan)) {  // scores, loss gradient and the first backward-data product in one launch
+    plan->launches_per_iter = 3 * L;
+    if ((e = cudaFuncSetAttribute(mlp_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)head_smem_bytes(*plan))) != cudaSuccess)
+      return e;
+  }
+  plan->skip_launches = plan->launches_per_iter;  // the same kernels; blocks of unselected groups and of the stale point exit at once
   if (L >= 2) {
     if ((e = cudaStreamCreateWithFlags(&plan->side, cudaStreamNonBlocking)) != cudaSuccess) return e;
     for (int l = 1; l <= L; ++l)
@@ -471,8 +566,12 @@ cudaError_t launch_grad_mlp(const Params& P, const MlpPlan& pl, cudaStream_t st,
   mlp_gather_kernel<<<(unsigned)((rows * 32 + 255) / 256), 256, 0, st>>>(P, pl.xb, pl.yb, pl.dims[0]);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   ++n;
+  // a small output layer: everything above the last hidden layer in one launch (see mlp_head_kernel)
+  const size_t head_smem = head_smem_bytes(pl);
+  const bool head = head_fits(pl);
+  const int L_top = head ? L - 1 : L;   // layers handled by the tile kernels
   // forward
-  for (int l = 1; l <= L; ++l) {
+  for (int l = 1; l <= L_top; ++l) {
     const int ni = pl.dims[l - 1], no = pl.dims[l];
     GemmArgs a{};
     a.M = B;
@@ -493,14 +592,29 @@ cudaError_t launch_grad_mlp(const Params& P, const MlpPlan& pl, cudaStream_t st,
     if ((e = launch_gemm(P, a, pl.sm_count, st)) != cudaSuccess) return e;
     ++n;
   }
-  mlp_softmax_grad_kernel<<<(unsigned)((2 * rows * 32 + 255) / 256), 256, 0, st>>>(P, pl.act[L], pl.yb, pl.dz[L],
-                                                                                  pl.dims[L]);
+  if (head) {
+    HeadArgs h{};
+    h.n1 = pl.dims[L - 1];
+    h.nL = pl.dims[L];
+    h.w_off = pl.w_off[L];
+    h.b_off = pl.b_off[L];
+    h.a1 = pl.act[L - 1];
+    h.yb = pl.yb;
+    h.dzL = pl.dz[L];
+    h.dz1 = pl.dz[L - 1];
+    mlp_head_kernel<<<dim3((B + 7) / 8, 2 * G), 256, head_smem, st>>>(P, h);
+  } else {
+    mlp_softmax_grad_kernel<<<(unsigned)((2 * rows * 32 + 255) / 256), 256, 0, st>>>(P, pl.act[L], pl.yb, pl.dz[L],
+                                                                                    pl.dims[L]);
+  }
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   ++n;
   // backward.  Main stream: the back-propagation chain dz_L -> ... -> dz_1, then dW_1.  Second stream (when
   // there is more than one layer): dW_l for l >= 2 as soon as dz_l is there, then all bias gradients.
-  cudaStream_t s2 = pl.side ? pl.side : st;
-  if (pl.side) {
+  // (with the fused output layer dz_L and dz_{L-1} are both there already)
+  const bool side = pl.side != nullptr;
+  cudaStream_t s2 = side ? pl.side : st;
+  if (side) {
     if ((e = cudaEventRecord(pl.ev_dz[L], st)) != cudaSuccess) return e;
     if ((e = cudaStreamWaitEvent(pl.side, pl.ev_dz[L], 0)) != cudaSuccess) return e;
   }
@@ -520,7 +634,7 @@ cudaError_t launch_grad_mlp(const Params& P, const MlpPlan& pl, cudaStream_t st,
     w.c_rs = ni;
     if ((e = launch_gemm(P, w, pl.sm_count, l == 1 ? st : s2)) != cudaSuccess) return e;
     ++n;
-    if (l > 1) {
+    if (l > 1 && !(head && l == L)) {
       GemmArgs d{};  // dz_{l-1} = (dz_l W_l) masked by a_{l-1} > 0
       d.M = B;
       d.N = ni;
@@ -534,24 +648,27 @@ cudaError_t launch_grad_mlp(const Params& P, const MlpPlan& pl, cudaStream_t st,
       d.mask = pl.act[l - 1];
       if ((e = launch_gemm(P, d, pl.sm_count, st)) != cudaSuccess) return e;
       ++n;
-      if (pl.side) {
+      if (side) {
         if ((e = cudaEventRecord(pl.ev_dz[l - 1], st)) != cudaSuccess) return e;
         if ((e = cudaStreamWaitEvent(pl.side, pl.ev_dz[l - 1], 0)) != cudaSuccess) return e;
       }
     }
   }
-  BiasArgs ba{};
-  int maxn = 0;
-  for (int l = 1; l <= L; ++l) {
-    ba.dz[l] = pl.dz[l];
-    ba.n[l] = pl.dims[l];
-    ba.b_off[l] = pl.b_off[l];
-    if (pl.dims[l] > maxn) maxn = pl.dims[l];
+  const int L_bias = L;
+  {
+    BiasArgs ba{};
+    int maxn = 0;
+    for (int l = 1; l <= L_bias; ++l) {
+      ba.dz[l] = pl.dz[l];
+      ba.n[l] = pl.dims[l];
+      ba.b_off[l] = pl.b_off[l];
+      if (pl.dims[l] > maxn) maxn = pl.dims[l];
+    }
+    mlp_bias_grad_kernel<<<dim3((maxn + 255) / 256, 2 * G, L_bias), 256, 0, s2>>>(P, ba);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    ++n;
   }
-  mlp_bias_grad_kernel<<<dim3((maxn + 255) / 256, 2 * G, L), 256, 0, s2>>>(P, ba);
-  if ((e = cudaGetLastError()) != cudaSuccess) return e;
-  ++n;
-  if (pl.side) {
+  if (side) {
     if ((e = cudaEventRecord(pl.ev_join, pl.side)) != cudaSuccess) return e;
     if ((e = cudaStreamWaitEvent(st, pl.ev_join, 0)) != cudaSuccess) return e;
   }
