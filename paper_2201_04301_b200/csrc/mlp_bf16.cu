@@ -671,7 +671,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gram_kernel(const __grid_co
                                                                  const __grid_constant__ CUtensorMap tmV1,
                                                                  const Params P, const GramArgs a) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
-  __shared__ uint64_t full_bar[G_STAGES], empty_bar[G_STAGES], tfull_bar, tempty_bar;
+  __shared__ uint64_t full_bar[MAX_STAGES], empty_bar[MAX_STAGES], tfull_bar, tempty_bar;
   __shared__ uint32_t tmem_base_sm;
   __shared__ double norm_sm[G_EPI_WARPS];
   unsigned char* tiles = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -682,11 +682,17 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gram_kernel(const __grid_co
   const int units_per_group = RB * tiles_nj;
   const int total_units = units_per_group * P.G;
   const int nku = (a.Ku + BK - 1) / BK, nkv = (a.Kv + BK - 1) / BK;
-  const uint32_t stage_tx = (uint32_t)((BM + a.BN) * BK * 2);
+  // The 128 rows of the A operand are rows of the same matrix as the B operand's: when they lie inside the B
+  // tile (always, if one column block covers the whole Gram) they are not fetched a second time and the
+  // stages shrink to the B tile, which makes the ring deeper.
+  const bool always_inside = tiles_nj == 1;
+  const int stage_bytes = (always_inside ? a.BN : BM + a.BN) * BK * 2;
+  const int stages = (G_STAGES * G_STAGE_BYTES) / stage_bytes < MAX_STAGES ? (G_STAGES * G_STAGE_BYTES) / stage_bytes : MAX_STAGES;
+  const int b_off = always_inside ? 0 : BM * BK * 2;  // where the B tile starts inside a stage
   const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(a.BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < G_STAGES; ++s) {
+    for (int s = 0; s < stages; ++s) {
       mbar_init(&full_bar[s], 1);
       mbar_init(&empty_bar[s], 1);
     }
@@ -712,14 +718,15 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gram_kernel(const __grid_co
       for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
         const int g = u / units_per_group, r = u - g * units_per_group;
         const int mi = r / tiles_nj, nj = r - mi * tiles_nj;
+        const bool inside = mi / bpn == nj;  // the A rows are among the B rows of this unit
         for (int ph = 0; ph < 2 && ok; ++ph) {  // the U Gram, then the V Gram
           const int nk = ph == 0 ? nku : nkv;
           for (int kb = 0; kb < nk && ok; ++kb, ++it) {
-            const int s = it % G_STAGES;
-            ok = mbar_spin_bounded(&empty_bar[s], (uint32_t)(((it / G_STAGES) & 1) ^ 1));
+            const int s = it % stages;
+            ok = mbar_spin_bounded(&empty_bar[s], (uint32_t)(((it / stages) & 1) ^ 1));
             if (!ok) break;
-            unsigned char* sa = tiles + (size_t)s * G_STAGE_BYTES;
-            mbar_expect_tx(&full_bar[s], stage_tx);
+            unsigned char* sa = tiles + (size_t)s * stage_bytes;
+            mbar_expect_tx(&full_bar[s], (uint32_t)((inside ? a.BN : BM + a.BN) * BK * 2));
             // block b of the matrix: part b / nb, rows (b % nb) * 128 of the group's entry in that part's array
             auto load_block = [&](unsigned char* dst, int b) {
               const int part = b / a.nb, row = (b - part * a.nb) * BM;
@@ -729,8 +736,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gram_kernel(const __grid_co
               const int z = ph == 0 ? (part == 1 ? factor_entry(P, g, 1) : g) : (part == 0 ? factor_entry(P, g, 0) : g);
               tma_load_3d(dst, tm, kb * BK, row, z, &full_bar[s]);
             };
-            load_block(sa, mi);
-            for (int j = 0; j < bpn; ++j) load_block(sa + (size_t)(BM + j * BM) * BK * 2, nj * bpn + j);
+            if (!inside) load_block(sa, mi);
+            for (int j = 0; j < bpn; ++j) load_block(sa + b_off + (size_t)(j * BM) * BK * 2, nj * bpn + j);
           }
         }
       }
@@ -741,18 +748,21 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gram_kernel(const __grid_co
       bool ok = true;
       int it = 0, i = 0;
       for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x, ++i) {
+        const int r = u % units_per_group, mi = r / tiles_nj, nj = r - mi * tiles_nj;
+        const bool inside = mi / bpn == nj;
         ok = mbar_spin_bounded(&tempty_bar, (uint32_t)((i & 1) ^ 1));  // the epilogue has drained the accumulators
         if (!ok) break;
         tc_fence_after();
         for (int ph = 0; ph < 2 && ok; ++ph) {
           const int nk = ph == 0 ? nku : nkv;
           for (int kb = 0; kb < nk && ok; ++kb, ++it) {
-            const int s = it % G_STAGES;
-            ok = mbar_spin_bounded(&full_bar[s], (uint32_t)((it / G_STAGES) & 1));
+            const int s = it % stages;
+            ok = mbar_spin_bounded(&full_bar[s], (uint32_t)((it / stages) & 1));
             if (!ok) break;
             tc_fence_after();
-            const uint32_t sa = smem_u32(tiles + (size_t)s * G_STAGE_BYTES);
-            const uint64_t da = make_desc(sa), db = make_desc(sa + BM * BK * 2);
+            const uint32_t sa = smem_u32(tiles + (size_t)s * stage_bytes);
+            const uint64_t db = make_desc(sa + b_off);
+            const uint64_t da = make_desc(inside ? sa + b_off + (uint32_t)((mi % bpn) * BM * BK * 2) : sa);
 #pragma unroll
             for (int kk = 0; kk < BK / 16; ++kk)
               tc_mma_bf16(tmem_base + (uint32_t)(ph * a.BN), da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc,
