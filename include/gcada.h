@@ -313,8 +313,10 @@ gcada_status gcada_time_empty_chain(gcada_ctx *ctx, int n_iters, double *us_per_
 
 /* Reporting aid (not a step of Algorithm 1): the mean per-sample loss of the current iterate over rows
  * first_row .. first_row + n_rows - 1 of the resident training set, i.e. the objective of Eq. (1) restricted
- * to those rows, in double precision, to *mean_loss (host).  Logistic and quadratic models only
- * (GCADA_EINVAL for an MLP).  Synchronises the stream. */
+ * to those rows, to *mean_loss (host).  Logistic / quadratic models: double precision.  MLPs: the softmax
+ * cross-entropy of the fp32 master parameters in fp32 arithmetic (whatever the model's compute type; the
+ * per-row terms and their sum in double), rows pushed through the tile kernels in slabs; scratch buffers are
+ * allocated on the first call.  Synchronises the stream. */
 gcada_status gcada_eval_loss(gcada_ctx *ctx, long long first_row, long long n_rows, double *mean_loss);
 
 /*

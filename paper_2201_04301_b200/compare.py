@@ -60,8 +60,6 @@ def main():
     ap.add_argument("--c-cada", type=float, default=2.0, help="threshold constant of the CADA run (the paper's 2)")
     args = ap.parse_args()
     w = make_workload(args.config, device="cuda")
-    if w["kind"] == "mlp":
-        raise SystemExit("loss curves need a logistic or quadratic model")
     stream = torch.cuda.Stream()
     for name, kw in schemes(w, args.c_cada).items():
         for rec in run_scheme(w, kw["M_G"], kw["c"], args.iters, args.every, min(args.eval_rows, w["X"].shape[0]),

@@ -66,6 +66,7 @@ struct gcada_ctx {
   long long stage_ld = 0;
   std::vector<std::pair<void*, size_t>> state;  // device buffers a checkpoint holds (besides the plan's)
   double* eval_scratch = nullptr;
+  MlpEvalScratch mlp_eval{};
   float* row_scratch = nullptr;  // one p-vector for getters that rebuild a group's gradient on demand
   // graphs (free-running resident-data mode only)
   cudaGraphExec_t graph1 = nullptr, graphN = nullptr;
@@ -134,6 +135,7 @@ void free_all(gcada_ctx* ctx) {
   ctx->stage_x = ctx->stage_y = nullptr;
   ctx->row_scratch = nullptr;  // was in `owned`
   ctx->eval_scratch = nullptr;
+  ctx->mlp_eval = MlpEvalScratch{};
   ctx->state.clear();
   ctx->st = nullptr;
   ctx->ready = false;
@@ -1094,7 +1096,6 @@ gcada_status gcada_time_empty_chain(gcada_ctx* ctx, int n_iters, double* us_per_
 gcada_status gcada_eval_loss(gcada_ctx* ctx, long long first_row, long long n_rows, double* mean_loss) {
   if (!ctx) return GCADA_EINVAL;
   if (!mean_loss) return fail(ctx, GCADA_EINVAL, "mean_loss is NULL");
-  if (!is_linear(ctx)) return fail(ctx, GCADA_EINVAL, "gcada_eval_loss supports logistic and quadratic models only");
   TRY(check_runnable(ctx, true));
   if (first_row < 0 || n_rows < 1 || first_row + n_rows > ctx->N)
     return fail(ctx, GCADA_EINVAL, "rows [%lld, %lld) are outside the training set of %lld rows", first_row,
@@ -1104,6 +1105,21 @@ gcada_status gcada_eval_loss(gcada_ctx* ctx, long long first_row, long long n_ro
   if (!ctx->eval_scratch) TRY(dev_alloc(ctx, &ctx->eval_scratch, (size_t)eval_loss_scratch_doubles()));
   DevState s;
   TRY(read_state(ctx, &s));
+  if (!is_linear(ctx)) {
+    if (!ctx->mlp_eval.part) {  // slab buffers, on first use
+      int widest = 0;
+      for (int v : ctx->dims) widest = v > widest ? v : widest;
+      TRY(dev_alloc(ctx, &ctx->mlp_eval.buf[0], (size_t)MLP_EVAL_SLAB * widest));
+      TRY(dev_alloc(ctx, &ctx->mlp_eval.buf[1], (size_t)MLP_EVAL_SLAB * widest));
+      TRY(dev_alloc(ctx, &ctx->mlp_eval.ones, (size_t)MLP_EVAL_SLAB / 64));
+      CK(cudaMemsetAsync(ctx->mlp_eval.ones, 1, (size_t)MLP_EVAL_SLAB / 64, ctx->stream));
+      TRY(dev_alloc(ctx, &ctx->mlp_eval.part, (size_t)1024));
+    }
+    CK(mlp_eval_loss(ctx->P, ctx->mlp, first_row, n_rows, ctx->mlp_eval, ctx->eval_scratch, ctx->stream));
+    CK(cudaStreamSynchronize(ctx->stream));
+    CK(cudaMemcpy(mean_loss, ctx->eval_scratch, sizeof(double), cudaMemcpyDeviceToHost));
+    return GCADA_OK;
+  }
   const float* theta = ctx->P.theta_ring + (s.k % (ctx->D + 1)) * ctx->p_pad;
   CK(launch_eval_loss_linear(ctx->P, theta, ctx->kind == GCADA_MODEL_QUADRATIC, first_row, n_rows, ctx->eval_scratch,
                              ctx->stream));

@@ -10,6 +10,7 @@
 // theta layout: for l = 1..L, W_l (n_l rows of n_{l-1}) then b_l (n_l).
 // Batch index z = q * G + g (q = point, g = group).
 #include <cooperative_groups.h>
+#include <cuda_bf16.h>
 
 #include "mlp.h"
 
@@ -555,6 +556,112 @@ cudaError_t launch_grad_mlp_post(const Params& P, const MlpPlan& pl, cudaStream_
 cudaError_t mlp_group_gradient(const Params& P, const MlpPlan& pl, int g, float* row, cudaStream_t st) {
   if (pl.compute != 1) return cudaErrorNotSupported;
   return mlp_bf16_group_gradient(P, pl, g, row, st);
+}
+
+// ------------------------------------------------------------------ loss of the current iterate (reporting)
+namespace {
+constexpr int EVAL_CHUNK = 64;  // rows per "group" of the tile kernels
+__global__ void __launch_bounds__(256) mlp_eval_convert_kernel(const __nv_bfloat16* X, long long ld, int d, long long rows,
+                                                               float* out) {
+  const long long n = rows * d;
+  for (long long e = (long long)blockIdx.x * 256 + threadIdx.x; e < n; e += (long long)gridDim.x * 256) {
+    const long long r = e / d;
+    out[e] = __bfloat162float(X[r * ld + (e - r * d)]);
+  }
+}
+// Warp per row: -ln softmax(scores)[y] in double; one partial sum per block.
+__global__ void __launch_bounds__(256) mlp_eval_rows_kernel(const float* scores, const int* y, long long rows, int n_cls,
+                                                            double* part) {
+  __shared__ double scratch[40];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  double local = 0.0;
+  for (long long r = (long long)blockIdx.x * 8 + warp; r < rows; r += (long long)gridDim.x * 8) {
+    const float* s = scores + r * n_cls;
+    float mx = -3.0e38f;
+    for (int c = lane; c < n_cls; c += 32) mx = fmaxf(mx, s[c]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    double sum = 0.0;
+    for (int c = lane; c < n_cls; c += 32) sum += exp((double)s[c] - (double)mx);
+    sum = warp_sum(sum);
+    if (lane == 0) local += log(sum) + (double)mx - (double)s[y[r]];
+  }
+  const double tot = block_sum(local, scratch);
+  if (threadIdx.x == 0) part[blockIdx.x] = tot;
+}
+// out[0] = (add ? out[0] : 0) + sum(part), divided by `div` when div > 0 (the last slab).
+__global__ void __launch_bounds__(256) mlp_eval_add_kernel(const double* part, int n_part, int add, double div, double* out) {
+  __shared__ double scratch[40];
+  double s = 0.0;
+  for (int i = threadIdx.x; i < n_part; i += 256) s += part[i];
+  s = block_sum(s, scratch);
+  if (threadIdx.x == 0) {
+    double v = (add ? out[0] : 0.0) + s;
+    if (div > 0.0) v /= div;
+    out[0] = v;
+  }
+}
+}  // namespace
+
+cudaError_t mlp_eval_loss(const Params& P, const MlpPlan& pl, long long first, long long n, const MlpEvalScratch& sc,
+                          double* out, cudaStream_t st) {
+  const int L = pl.n_layers;
+  cudaError_t e;
+  for (long long s0 = 0; s0 < n; s0 += MLP_EVAL_SLAB) {
+    const long long m = n - s0 < MLP_EVAL_SLAB ? n - s0 : MLP_EVAL_SLAB;
+    const float* in = nullptr;
+    long long in_ld = 0;
+    int cur = 0;
+    if (pl.compute == 1) {  // bf16 features: a dense fp32 copy of the slab
+      mlp_eval_convert_kernel<<<592, 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(P.X) + (first + s0) * P.ld, P.ld,
+                                                   pl.dims[0], m, sc.buf[0]);
+      if ((e = cudaGetLastError()) != cudaSuccess) return e;
+      in = sc.buf[0];
+      in_ld = pl.dims[0];
+      cur = 1;
+    } else {
+      in = reinterpret_cast<const float*>(P.X) + (first + s0) * P.ld;
+      in_ld = P.ld;
+    }
+    for (int l = 1; l <= L; ++l) {
+      const int ni = pl.dims[l - 1], no = pl.dims[l];
+      float* outp = sc.buf[cur];
+      // whole chunks of 64 rows as "groups" of the tile kernels at the current iterate, then the remaining rows
+      for (int part = 0; part < 2; ++part) {
+        const long long chunks = m / EVAL_CHUNK, done = chunks * EVAL_CHUNK;
+        const long long rows_here = part == 0 ? EVAL_CHUNK : m - done;
+        const long long groups = part == 0 ? chunks : 1;
+        if (groups == 0 || rows_here == 0) continue;
+        Params Q = P;
+        Q.G = (int)groups;
+        Q.B = (int)rows_here;
+        Q.skip_unselected = 1;   // point 0 only ...
+        Q.mask_cur = sc.ones;    // ... of every "group"
+        GemmArgs a{};
+        a.M = (int)rows_here;
+        a.N = no;
+        a.K = ni;
+        a.A = Operand{in + (part == 0 ? 0 : done * in_ld), 0, (long long)EVAL_CHUNK * in_ld, 0, in_ld, 1, 0};
+        a.Bm = Operand{nullptr, pl.w_off[l], 0, 0, 1, ni, 1};
+        a.C = outp + (part == 0 ? 0 : done * no);
+        a.c_zg = (long long)EVAL_CHUNK * no;
+        a.c_zq = 0;
+        a.c_rs = no;
+        a.bias = 1;
+        a.bias_off = pl.b_off[l];
+        a.relu = l < L;
+        if ((e = launch_gemm(Q, a, pl.sm_count, st)) != cudaSuccess) return e;
+      }
+      in = outp;
+      in_ld = no;
+      cur ^= 1;
+    }
+    mlp_eval_rows_kernel<<<512, 256, 0, st>>>(in, reinterpret_cast<const int*>(P.y) + first + s0, m, pl.dims[L], sc.part);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    mlp_eval_add_kernel<<<1, 256, 0, st>>>(sc.part, 512, s0 > 0 ? 1 : 0, s0 + m >= n ? (double)n : 0.0, out);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  }
+  return cudaSuccess;
 }
 
 cudaError_t launch_grad_mlp(const Params& P, const MlpPlan& pl, cudaStream_t st, int* n_launches) {

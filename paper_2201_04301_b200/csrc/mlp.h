@@ -56,4 +56,18 @@ cudaError_t launch_grad_mlp_post(const Params& P, const MlpPlan& plan, cudaStrea
 // bf16 path without kept per-group gradients: group g's last uploaded gradient rebuilt into `row` (device).
 cudaError_t mlp_group_gradient(const Params& P, const MlpPlan& plan, int g, float* row, cudaStream_t st);
 
+// Reporting aid (not a step of Algorithm 1): the mean softmax cross-entropy of the CURRENT iterate (the fp32
+// master parameters, fp32 arithmetic, whatever the model's compute type) over rows [first, first + n) of the
+// resident training set, into out[0] (device).  The rows are pushed through the fp32 tile kernels in slabs of
+// MLP_EVAL_SLAB rows; `buf` are two device buffers of MLP_EVAL_SLAB * (widest layer, input included) floats,
+// `ones` MLP_EVAL_SLAB / 64 bytes of value 1, `part` 1024 doubles.
+constexpr int MLP_EVAL_SLAB = 4096;
+struct MlpEvalScratch {
+  float* buf[2] = {nullptr, nullptr};
+  unsigned char* ones = nullptr;
+  double* part = nullptr;
+};
+cudaError_t mlp_eval_loss(const Params& P, const MlpPlan& plan, long long first, long long n, const MlpEvalScratch& sc,
+                          double* out, cudaStream_t st);
+
 }  // namespace gcada
