@@ -134,22 +134,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait for the single-thread producer / MMA loops: non-blocking polls, so that the thread
-// reacts within a few cycles of the phase flipping (try_wait may park the thread for a while).
+// Bounded wait of the single-thread producer / MMA loops: the hardware parks the thread for at most about a
+// microsecond per try (suspend-time hint) and wakes it when the phase flips, so a waiting thread issues next
+// to nothing (busy polling with test_wait reacted no faster in practice and cost the step ~0.5 % under the
+// power cap).  2^20 tries: about a second before the wait is given up.
 __device__ __forceinline__ bool mbar_spin_bounded(uint64_t* bar, uint32_t parity) {
-  for (uint32_t it = 0; it < (1u << 26); ++it)
-    if (mbar_test_wait(bar, parity)) return true;
+  for (uint32_t it = 0; it < (1u << 20); ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(1000u)
+        : "memory");
+    if (ok) return true;
+  }
   return false;
 }
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
