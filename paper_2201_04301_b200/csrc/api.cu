@@ -208,6 +208,7 @@ gcada_status make_ready(gcada_ctx* ctx, const float* theta0, int on_device) {
   TRY(dev_alloc(ctx, &P.s_ring, (size_t)D));
   TRY(dev_alloc(ctx, &P.mask_cur, (size_t)G));
   TRY(dev_alloc(ctx, &P.sel_list, (size_t)G));
+  TRY(dev_alloc(ctx, &P.age_order, (size_t)G));
   TRY(dev_alloc(ctx, &P.sel_count, (size_t)1));
   TRY(dev_alloc(ctx, &P.hist, (size_t)ctx->hist_cap * G));
   plan_tail(pp, G, ctx->sm_count, &ctx->tail);

@@ -104,6 +104,9 @@ struct Params {
   const double* ps_L2;          // [G] squared smoothness constants, or null (rule INNOV)
   double* ps_lhs;               // [G] the printed left side, written by ps_lhs_kernel
   double* ps_part;              // [D][blocks] partial sums of ||theta^k - theta^{k-d}||^2
+  int* age_order;               // [G] the groups sorted by age of information (stable), rewritten at the start of
+                                // every iteration of the bf16 MLP path: tiles of groups of equal age read the
+                                // same slot of the weight ring, so they are scheduled next to each other
   int* sel_list;                // [G] groups selected this iteration, ascending (written with the mask)
   int* sel_count;               // [1] how many
   int skip_unselected;          // 1: the selection of this iteration is already in mask_cur and the gradient

@@ -330,7 +330,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
       for (int i = 0; i < n_local && ok; ++i) {
         const int u = blockIdx.x + (i / n_q) * gridDim.x, q = i % n_q;
         const int nt = u % tiles_n, mt = (u / tiles_n) % tiles_m, gi = u / (tiles_n * tiles_m);
-        const int g = a.k_batched ? 0 : (P.skip_unselected ? P.sel_list[gi] : gi);
+        const int g = a.k_batched ? 0 : (P.skip_unselected ? P.sel_list[gi] : P.age_order[gi]);
         const int z = q * P.G + g;
         int zA = 0, zB = 0, ent = 0;
         // entry e of a k_batched product: every group's last upload, or (listed) the selected groups' replaced
@@ -422,7 +422,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
       const int slot = i & 1;
       const int u = blockIdx.x + (i / n_q) * gridDim.x, q = i % n_q;
       const int nt = u % tiles_n, mt = (u / tiles_n) % tiles_m, gi = u / (tiles_n * tiles_m);
-      const int g = a.k_batched ? 0 : (P.skip_unselected ? P.sel_list[gi] : gi);
+      const int g = a.k_batched ? 0 : (P.skip_unselected ? P.sel_list[gi] : P.age_order[gi]);
       const int z = q * P.G + g;
       const bool write_diff = q == 1 && a.diff != nullptr;
       const int zT = a.k_batched ? 0 : factor_entry(P, g, q);  // entry of the output in its factor array
@@ -1122,6 +1122,29 @@ __global__ void __launch_bounds__(256) bf16_convert_kernel(const Params P, const
   if (blockIdx.x == 0 && blockIdx.y == 0) {
     float* bo = bias + (long long)slot * a.bias_slot + a.bias_pos[l];
     for (int n = threadIdx.x; n < no; n += 256) bo[n] = __bfloat162float(__float2bfloat16_rn(th[a.b_off[l] + n]));
+  }
+  // One warp of one block also lists the groups by age (stable; ages beyond D, which only forced masks
+  // produce, count as D + 1): groups of equal age read the same slot of the weight ring at the stale point,
+  // and the products schedule their tiles in this order so that the CTAs running together touch few slots.
+  // The order has no influence on any result.
+  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x < 32) {
+    const int lane = threadIdx.x, G = P.G, chunks = (G + 31) / 32;
+    if ((long long)(P.D + 1) * chunks <= 8192) {
+      int base = 0;
+      for (int age = 1; age <= P.D + 1; ++age) {
+        for (int c = 0; c < chunks; ++c) {
+          const int g = c * 32 + lane;
+          int t = g < G ? P.tau[g] : 0;
+          if (t > P.D + 1) t = P.D + 1;
+          if (t < 1 && g < G) t = 1;
+          const unsigned int m = __ballot_sync(0xffffffffu, t == age);
+          if (t == age) P.age_order[base + __popc(m & ((1u << lane) - 1u))] = g;
+          base += __popc(m);
+        }
+      }
+    } else {
+      for (int g = lane; g < G; g += 32) P.age_order[g] = g;
+    }
   }
 }
 
