@@ -104,6 +104,11 @@ struct GemmB {
                               // EPI_HIDDEN writes them, EPI_DA of the same layer reads them as the ReLU derivative
   int nw;                     // words per row: (N + 31) / 32
   int n_entries;              // entries of `out` (checked by the debug library)
+  int point;                  // forward / backward-data products: the point this launch computes (0: theta^k,
+                              // 1: the stale iterates).  One launch per point: all tiles of the first share one
+                              // slot of the weight ring, which then stays in L2; the second walks the groups by
+                              // age, one stale slot after the other; interleaving the two kept two slots (64 MB
+                              // at 4096 x 4096) live at a time and every wave of CTAs fetched both from HBM again
   float* colsum;              // EPI_DA: [z][tiles_m][N] column sums of the (bf16-rounded) output tile, or null
   __nv_bfloat16* diff;        // EPI_HIDDEN / EPI_DA, or null: row-major [G][M][ldo]; the stale-point tile also
                               // writes (fresh output - its own output) here, rounded to bf16: the small
@@ -239,7 +244,9 @@ __device__ __forceinline__ int factor_entry(const Params& P, int g, int q) {
 // Persistent: one CTA per SM walks 128 x 256 output tiles (N fastest, so that
 // the CTAs running together share operand tiles in L2); tensor memory holds
 // two 256-column accumulators, so the eight epilogue warps drain tile i while
-// the producer and the MMA warp work on tile i+1.
+// the producer and the MMA warp work on tile i+1.  A forward / backward-data
+// product is two launches, theta^k for all groups and then the stale iterates
+// with the groups taken in order of age (GemmB::point).
 constexpr int AGG_REFRESH = 16;  // the aggregate is recomputed in full at least every so many iterations (a replaced
                                  // pair of uploads moves it by ~1e-7 of its norm from the recomputed value)
 constexpr int GN = 256;                                  // N tile of this kernel (the epilogue assumes 2 x 4 chunks of 32)
@@ -293,10 +300,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
   // batch entries: (point, group) for every group, or - when only the selected groups compute (rule PS:
   // Algorithm 1's own order, the selection is already known) - the selected groups at theta^k only
   const int n_grp = P.skip_unselected ? P.sel_count[0] : P.G;
-  // A CTA walks units (column tile, row tile, group) and, inside a unit, the two points one after the other:
-  // the stale point's epilogue runs in the same threads, on the same rows and columns, as the fresh point's
-  // just before it, whose output it reads back to form the differences.
-  const int n_q = (a.k_batched || P.skip_unselected) ? 1 : 2;
+  // A CTA walks units (column tile, row tile, group) of the launch's point.
+  constexpr int n_q = 1;
   const int total_units = tiles_n * tiles_m * (a.k_batched ? 1 : n_grp);
   const int n_local = (int)blockIdx.x < total_units ? ((total_units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) * n_q : 0;
   const long long k_it = P.st->k;
@@ -328,7 +333,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
       bool ok = true;
       int it = 0;
       for (int i = 0; i < n_local && ok; ++i) {
-        const int u = blockIdx.x + (i / n_q) * gridDim.x, q = i % n_q;
+        const int u = blockIdx.x + (i / n_q) * gridDim.x, q = a.k_batched ? 0 : a.point;
         const int nt = u % tiles_n, mt = (u / tiles_n) % tiles_m, gi = u / (tiles_n * tiles_m);
         const int g = a.k_batched ? 0 : (P.skip_unselected ? P.sel_list[gi] : P.age_order[gi]);
         const int z = q * P.G + g;
@@ -420,7 +425,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
     bool ok = true;
     for (int i = 0; i < n_local; ++i) {
       const int slot = i & 1;
-      const int u = blockIdx.x + (i / n_q) * gridDim.x, q = i % n_q;
+      const int u = blockIdx.x + (i / n_q) * gridDim.x, q = a.k_batched ? 0 : a.point;
       const int nt = u % tiles_n, mt = (u / tiles_n) % tiles_m, gi = u / (tiles_n * tiles_m);
       const int g = a.k_batched ? 0 : (P.skip_unselected ? P.sel_list[gi] : P.age_order[gi]);
       const int z = q * P.G + g;
@@ -475,9 +480,9 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
         const bool row_ok = m < a.M;
         const bool full = nc + 32 <= a.N;
         const float* bw = bias_w + (c - half * (GN / 2));  // this chunk's biases (EPI_HIDDEN / EPI_SCORES)
-        // The stale point's tile also writes fresh - stale: the fresh point's values at the places this thread
-        // will store to (it stored them itself one tile ago) are fetched now, so that their latency is
-        // covered by the conversion work
+        // The stale point's tile also writes fresh - stale: the fresh point's values (written by the launch
+        // before this one) at the places this thread will store to are fetched now, so that their latency
+        // is covered by the conversion work
         const long long off0 = (long long)(mt * BM + quad * 32) * a.ldo + nc;
         const bool fast = full && a.M - (mt * BM + quad * 32) >= 32;
         uint4 frv[4] = {};
@@ -585,7 +590,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
           if (row_ok) {
             __nv_bfloat16* dst = a.out + (long long)zT * a.z_stride_out + (long long)m * a.ldo + nc;
             for (int j = 0; j < 32 && nc + j < a.N; ++j) dst[j] = __float2bfloat16_rn(f[j]);
-            if (write_diff) {  // (this thread stored the fresh point's values of this row one tile ago)
+            if (write_diff) {
               const __nv_bfloat16* fr = a.out + (long long)zF * a.z_stride_out + (long long)m * a.ldo + nc;
               __nv_bfloat16* df = a.diff + (long long)g * a.z_stride_out + (long long)m * a.ldo + nc;
               for (int j = 0; j < 32 && nc + j < a.N; ++j)
@@ -1623,7 +1628,7 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(bf16_gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, G_STAGES * G_STAGE_BYTES + 1024);
   if (e != cudaSuccess) return e;
-  plan->launches_per_iter = 3 + L + 1 + L + (L - 1);
+  plan->launches_per_iter = 3 + 2 * L + 1 + L + 2 * (L - 1);
   plan->post_launches = L + 1;
   plan->skip_launches = 2 + L + 1 + (L - 1) + 1;
   return cudaSuccess;
@@ -1687,8 +1692,11 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
       a.epi = EPI_SCORES;
       a.out_f32 = im->scores;
     }
-    if ((e = launch_gemm(im->tm_fwd_a[l], im->tm_fwd_b[l], P, a, pl.sm_count, st)) != cudaSuccess) return e;
-    ++n;
+    for (int q = 0; q < (P.skip_unselected ? 1 : 2); ++q) {  // theta^k, then the stale iterates
+      a.point = q;
+      if ((e = launch_gemm(im->tm_fwd_a[l], im->tm_fwd_b[l], P, a, pl.sm_count, st)) != cudaSuccess) return e;
+      ++n;
+    }
   }
   {
     const int pitch = pl.dims[L] + 2 + (pl.dims[L] & 1);  // even, and an odd number of 32-bit words when possible
@@ -1748,8 +1756,11 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
       d.n_entries = 3 * G;
       d.ldo = im->ld[l - 1];
       d.z_stride_out = (long long)Bp * im->ld[l - 1];
-      if ((e = launch_gemm(im->tm_da_a[l], im->tm_da_b[l], P, d, pl.sm_count, st)) != cudaSuccess) return e;
-      ++n;
+      for (int q = 0; q < (P.skip_unselected ? 1 : 2); ++q) {
+        d.point = q;
+        if ((e = launch_gemm(im->tm_da_a[l], im->tm_da_b[l], P, d, pl.sm_count, st)) != cudaSuccess) return e;
+        ++n;
+      }
     }
   }
   BiasArgsB ba{};
