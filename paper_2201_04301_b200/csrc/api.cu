@@ -295,6 +295,7 @@ gcada_status make_plans(gcada_ctx* ctx) {
     P.pm.rows_per_group = ctx->B;
     const char* why = "";
     std::vector<void*> bufs;
+    ctx->mlp.inspect = ctx->keep_stale;
     cudaError_t e = mlp_plan_create(ctx->dims, ctx->compute, ctx->G, ctx->B, ctx->D, ctx->p_pad, ctx->sm_count,
                                     ctx->stream, &ctx->mlp, &bufs, &why);
     for (void* q : bufs) ctx->owned.push_back(q);

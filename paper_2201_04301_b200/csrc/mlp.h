@@ -17,6 +17,8 @@ struct MlpPlan {
   int skip_launches = 0;      // kernels before the update when only the selected groups compute (rule PS)
   int post_launches = 0;      // kernels that follow the selection kernel (bf16 path: upload + aggregate)
   int compute = 0;            // 0 fp32, 1 bf16 operands
+  int inspect = 0;            // set by the caller before the plan is created: both gradients of every group
+                              // are kept (GCADA_OPT_KEEP_STALE); decides which partial sums of the norm exist
   int G = 0, B = 0, D = 0;
   long long p_pad = 0;
   int dims[MLP_MAX_LAYERS + 1] = {0};

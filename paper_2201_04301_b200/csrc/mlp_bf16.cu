@@ -1341,7 +1341,9 @@ __global__ void __launch_bounds__(256) bf16_softmax_grad_pairs_kernel(const Para
 // ----------------------------------------------------------------- bias gradients
 // db_l at both points = column sums of dz_l over the group's rows.  The kernels that produce dz_l leave the
 // sums of their row blocks (BiasArgsB::part); here the blocks are added in order, the fresh one is kept, and
-// the squared difference of the two points is summed per block of 64 columns into its lhs_part slot.
+// the squared difference of the two points is summed into the layer's lhs_part slot of the group.  One block
+// per (group, layer): the selection kernel's single scheduling block adds up every group's partial sums, so
+// there should be few of them.
 struct BiasArgsB {
   const float* part[MLP_MAX_LAYERS + 1];  // [2][G][blocks[l]][n[l]]
   int blocks[MLP_MAX_LAYERS + 1];
@@ -1353,16 +1355,14 @@ struct BiasArgsB {
   int bias_loc[MLP_MAX_LAYERS + 1];   // first entry of layer l in a db row
   int nbias;
 };
-__global__ void __launch_bounds__(64) bf16_bias_grad_kernel(const Params P, const BiasArgsB a) {
+__global__ void __launch_bounds__(256) bf16_bias_grad_kernel(const Params P, const BiasArgsB a) {
   __shared__ double scratch[40];
-  const int l = blockIdx.z + 1;
+  const int l = blockIdx.y + 1;
   const int n_l = a.n[l];
-  if ((int)blockIdx.x * 64 >= n_l) return;
-  const int g = blockIdx.y;
+  const int g = blockIdx.x;
   if (P.skip_unselected && !P.mask_cur[g]) return;
-  const int c = blockIdx.x * 64 + threadIdx.x;
   double d2 = 0.0;
-  if (c < n_l) {
+  for (int c = threadIdx.x; c < n_l; c += 256) {
     const int nb = a.blocks[l];
     const float* p0 = a.part[l] + ((long long)g * nb) * n_l + c;
     const float* p1 = p0 + (long long)P.G * nb * n_l;
@@ -1373,12 +1373,11 @@ __global__ void __launch_bounds__(64) bf16_bias_grad_kernel(const Params P, cons
     a.db[((long long)fresh_buf(P, g) * P.G + g) * a.nbias + a.bias_loc[l] + c] = f;
     if (P.gbuf) (fresh_row(P, g) + a.b_off[l])[c] = f;  // kept for inspection
     if (P.stale) (P.stale + (long long)g * P.p_pad + a.b_off[l])[c] = sv;
-    d2 = (double)(f - sv) * (double)(f - sv);
+    d2 += (double)(f - sv) * (double)(f - sv);
   }
   d2 = block_sum(d2, scratch);
-  if (threadIdx.x == 0 &&
-      GCADA_INDEX_OK(P.st, (long long)g * a.n_parts + a.part_base[l] + blockIdx.x, P.lim.lhs_parts, CHK_LHS_PART))
-    P.lhs_part[(long long)g * a.n_parts + a.part_base[l] + blockIdx.x] = d2;
+  if (threadIdx.x == 0 && GCADA_INDEX_OK(P.st, (long long)g * a.n_parts + a.part_base[l], P.lim.lhs_parts, CHK_LHS_PART))
+    P.lhs_part[(long long)g * a.n_parts + a.part_base[l]] = d2;
 }
 
 // ----------------------------------------------------------------- bias part of the aggregate
@@ -1517,19 +1516,14 @@ cudaError_t mlp_bf16_plan_create(MlpPlan* plan, cudaStream_t st, std::vector<voi
   }
   im->slot_elems = pos;
   im->bias_slot = bpos;
+  // partial sums of the innovation norm per group: one per layer for the biases, and for the weights either one
+  // per unit of the Gram products or (inspection mode) one per 128-row block of W_l
   int parts = 0;
+  for (int l = 1; l <= L; ++l) im->bias_part_base[l] = parts++;
   for (int l = 1; l <= L; ++l) {
-    im->dw_part_base[l] = parts;
-    parts += (plan->dims[l] + BM - 1) / BM;  // one per (group, 128-row block of W_l)
-  }
-  for (int l = 1; l <= L; ++l) {
-    im->bias_part_base[l] = parts;
-    parts += (plan->dims[l] + 63) / 64;
-  }
-  for (int l = 1; l <= L; ++l) {  // units of the Gram products per group (slots that a mode does not use stay zero)
-    im->gram_part_base[l] = parts;
+    im->dw_part_base[l] = im->gram_part_base[l] = parts;
     const int rb = (l == 1 ? 1 : 2) * (im->Bp / BM), bn = rb * BM < GN ? rb * BM : GN;
-    parts += rb * (rb * BM / bn);
+    parts += plan->inspect ? (plan->dims[l] + BM - 1) / BM : rb * (rb * BM / bn);
   }
   im->n_parts = parts;
   plan->norm_parts = parts;
@@ -1777,7 +1771,7 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
   ba.n_parts = im->n_parts;
   ba.db = im->db;
   ba.nbias = im->nbias;
-  bf16_bias_grad_kernel<<<dim3((maxn + 63) / 64, G, L), 64, 0, st>>>(P, ba);
+  bf16_bias_grad_kernel<<<dim3(G, L), 256, 0, st>>>(P, ba);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   ++n;
   *n_launches = n;
