@@ -322,6 +322,9 @@ gcada_status make_plans(gcada_ctx* ctx) {
     P.ps_L2 = nullptr;
     P.skip_unselected = 0;
   }
+  P.k_off = 0;  // outside a captured chain every iteration is a chain of its own
+  P.chain_last = 1;
+  P.pdl = 0;
   CK(cudaStreamSynchronize(ctx->stream));
   ctx->ready = true;
   return GCADA_OK;
@@ -363,8 +366,17 @@ gcada_status enqueue_iteration(gcada_ctx* ctx, const Params& P) {
     }
     return GCADA_OK;
   }
+  // Inside a captured chain the linear models' gradient and selection kernels are launched programmatically
+  // dependent.  The selection kernel's blocks become resident while the gradient kernel drains; the update
+  // kernel, launched in the ordinary way, lets the next iteration's gradient kernel start at once, which
+  // computes its draw and starts copying its first rows while the update runs.  Measured on the d = 4096
+  // workload (us per iteration, same GPU): plain launches 107.2, this arrangement 102.7; with the update
+  // kernel programmatically dependent too, so that the copies also run under the selection kernel, 104.7
+  // (the selection's chain of dependent loads queues behind them); every kernel releasing its dependents at
+  // its start 109.8.
+  const bool pdl = P.pdl != 0;
   if (is_linear(ctx)) {
-    CK(launch_grad_linear(P, ctx->lin, ctx->kind == GCADA_MODEL_QUADRATIC, ctx->stream));
+    CK(launch_grad_linear(P, ctx->lin, ctx->kind == GCADA_MODEL_QUADRATIC, ctx->stream, pdl && P.k_off > 0));
     ctx->launches += 1;
   } else {
     int n = 0;
@@ -373,10 +385,10 @@ gcada_status enqueue_iteration(gcada_ctx* ctx, const Params& P) {
   }
   if (ev) CK(cudaEventRecord(ev[1], ctx->stream));
   if (P.ps_L2) {
-    CK(launch_ps_lhs(P, ctx->tail, ctx->stream));
+    CK(launch_ps_lhs(P, ctx->tail, ctx->stream, pdl));
     ctx->launches += 1;
   }
-  CK(launch_select(P, ctx->tail, ctx->stream));
+  CK(launch_select(P, ctx->tail, ctx->stream, 0, pdl));
   if (ev) CK(cudaEventRecord(ev[2], ctx->stream));
   if (!is_linear(ctx)) {  // bf16 MLP: the uploads are kept and the aggregate is formed (counted with the update phase)
     int n = 0;
@@ -384,7 +396,7 @@ gcada_status enqueue_iteration(gcada_ctx* ctx, const Params& P) {
     ctx->launches += (unsigned long long)n;
   }
   if (ev) CK(cudaEventRecord(ev[3], ctx->stream));
-  CK(launch_update(P, ctx->tail, ctx->stream));
+  CK(launch_update(P, ctx->tail, ctx->stream, false));
   if (ev) {
     CK(cudaEventRecord(ev[4], ctx->stream));
     ctx->timed += 1;
@@ -399,7 +411,13 @@ gcada_status capture_graph(gcada_ctx* ctx, int iters, cudaGraph_t* out) {
   CK(cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal));
   gcada_status s = GCADA_OK;
   ctx->capturing = true;
-  for (int i = 0; i < iters && s == GCADA_OK; ++i) s = enqueue_iteration(ctx, ctx->P);
+  for (int i = 0; i < iters && s == GCADA_OK; ++i) {
+    Params Q = ctx->P;
+    Q.k_off = i;
+    Q.chain_last = i == iters - 1;
+    Q.pdl = (is_linear(ctx) && !Q.skip_unselected) ? 1 : 0;
+    s = enqueue_iteration(ctx, Q);
+  }
   ctx->capturing = false;
   cudaError_t e = cudaStreamEndCapture(ctx->stream, &graph);
   ctx->launches = before;
@@ -477,6 +495,9 @@ gcada_status read_state(gcada_ctx* ctx, DevState* out) {
   if (out->err == DEV_ERR_BOUNDS)
     return fail(ctx, GCADA_ECUDA, "device-side error %d: an index check of the debug library failed (buffer %d); the store was skipped",
                 out->err, out->err_info);
+  if (out->err == DEV_ERR_CHAIN)
+    return fail(ctx, GCADA_ECUDA, "device-side error %d: a gradient kernel started inside a chain of iterations found the iteration counter elsewhere than the chain's bookkeeping",
+                out->err);
   if (out->err != DEV_OK) return fail(ctx, GCADA_ECUDA, "device-side error %d", out->err);
   return GCADA_OK;
 }

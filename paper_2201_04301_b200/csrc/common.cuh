@@ -8,7 +8,7 @@
 namespace gcada {
 
 // Device error words (DevState::err).
-enum { DEV_OK = 0, DEV_ERR_COPY_TIMEOUT = 1, DEV_ERR_BOUNDS = 2 };
+enum { DEV_OK = 0, DEV_ERR_COPY_TIMEOUT = 1, DEV_ERR_BOUNDS = 2, DEV_ERR_CHAIN = 3 };
 // What a failed index check was about to store to (DevState::err_info with DEV_ERR_BOUNDS).
 enum { CHK_PARTIAL = 1, CHK_LHS_PART = 2, CHK_HIST = 3, CHK_SEL_LIST = 4, CHK_GRAD_ROW = 5, CHK_FACTOR = 6 };
 
@@ -27,7 +27,8 @@ struct DevState {
   unsigned int ticket_select;     // "last block done" counters
   unsigned int ticket_update;
   unsigned int ticket_aux;
-  unsigned int pad_;
+  unsigned int k_chain;           // low 32 bits of k as it was when the running chain of iterations began (a chain
+                                  // = the iterations captured in one graph; see Params::k_off)
 };
 
 // How a per-group gradient is spread over partial-sum slots by the linear
@@ -109,10 +110,41 @@ struct Params {
                                 // same slot of the weight ring, so they are scheduled next to each other
   int* sel_list;                // [G] groups selected this iteration, ascending (written with the mask)
   int* sel_count;               // [1] how many
+  // Iterations captured back to back in one graph form a chain; iteration number k_off of the chain runs
+  // iteration st->k_chain + k_off (st->k_chain is rewritten by the update kernel of the chain's last iteration
+  // only, so it can be read while the previous iteration is still running).  pdl = 1: the linear models'
+  // gradient and selection kernels of the chain carry the programmatic-dependent-launch attribute, and the
+  // wide models' gradient kernel starts the copies of its first rows (they depend on the draw, not on the
+  // iterate) before it waits for the previous iteration's update to finish.
+  int k_off, chain_last, pdl;
   int skip_unselected;          // 1: the selection of this iteration is already in mask_cur and the gradient
                                 // kernels work on the selected groups only (rule PS: Algorithm 1 as printed,
                                 // workers of unselected groups compute nothing)
 };
+
+// Programmatic dependent launch.  Every kernel of an iteration calls pdl_wait() before it reads or writes
+// anything that another kernel writes: when launched with the attribute it returns once the previous kernel
+// of the stream has finished and its writes are visible, otherwise at once.  pdl_launch_dependents() lets the
+// next kernel's blocks become resident (and sit in their own pdl_wait) as soon as every block of this one has
+// started.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KA, typename... A>
+inline cudaError_t launch_k(void (*kern)(KA...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool pdl,
+                            A&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KA>(args)...);
+}
 
 // Index check of the debug library: true if 0 <= idx < limit; otherwise the run's error word is raised (first
 // failure wins; err_info says which buffer) and the caller skips the access - nothing traps, the context stays

@@ -110,19 +110,23 @@ __global__ void __launch_bounds__(THREADS, MINB) grad_linear_large_kernel(const 
   unsigned char* slots = reinterpret_cast<unsigned char*>(res + 32);
   slots = reinterpret_cast<unsigned char*>(((uintptr_t)slots + 127) & ~(uintptr_t)127);
 
-  const long long k = P.st->k;
-  const uint32_t k32 = (uint32_t)k;
-  const int ring = P.D + 1;
-  const float* theta_k = P.theta_ring + (k % ring) * P.p_pad;
   const float* Xf = reinterpret_cast<const float*>(P.X);
   const float* yf = reinterpret_cast<const float*>(P.y);
   const int B = P.B;
+  const bool skip = P.skip_unselected != 0;
+  // Inside a chain of captured iterations the kernel may start while the previous iteration's selection and
+  // update kernels are still running.  Which rows it reads follows from the draw alone (Section II-A: the
+  // minibatch does not depend on the iterate), so the first copies are started before the wait below; the
+  // iteration number for the draw then comes from the chain's start, which no running kernel writes.
+  const bool early = P.pdl != 0 && !skip;
+  pdl_launch_dependents();
+  if (!early) pdl_wait();
+  const uint32_t k32 = early ? P.st->k_chain + (uint32_t)P.k_off : (uint32_t)P.st->k;
 
   // group numbers below are positions in the list of groups worked on (all groups, or the selected ones)
   __shared__ int sel_sm[SKIP_MAX_GROUPS];
   __shared__ int n_groups_sm;
   const int n_groups = build_group_list(P, sel_sm, &n_groups_sm);
-  const bool skip = P.skip_unselected != 0;
   const long long Rtot = (long long)n_groups * B;
   // (when only the selected groups compute there may be fewer rows than CTAs: the first Rtot CTAs take one each,
   // so that no CTA with an empty range sits between two that hold a group's partial sums)
@@ -139,6 +143,47 @@ __global__ void __launch_bounds__(THREADS, MINB) grad_linear_large_kernel(const 
     for (int s = 0; s < nslot; ++s) mbar_init(&bars[s], 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+
+  // Index and label of the rows of a chunk, then the first copies (as many as the ring has slots).
+  // Returns how many copies were issued (meaningful in the issuing thread).
+  int cslot = 0;          // ring slot of the next row to consume
+  auto stage_chunk = [&](int cs, int nrows) -> int {
+    __syncthreads();  // previous chunk fully consumed; barriers initialised (first pass)
+    for (int i = tid; i < nrows; i += THREADS) {
+      const int pos = in_g0 + cs + i;
+      const int gi = pos / B;
+      const long long row = batch_row(P, k32, skip ? sel_sm[g_first + gi] : g_first + gi, pos - gi * B);
+      row_sm[i] = row * P.ld;
+      y_sm[i] = yf[row];
+    }
+    __syncthreads();
+    int issued = 0;
+    if (tid == ISSUER) {
+      const int n0 = nrows < nslot ? nrows : nslot;
+      for (; issued < n0; ++issued) {
+        int s = cslot + issued;
+        if (s >= nslot) s -= nslot;
+        mbar_expect_tx(&bars[s], rowbytes);
+        bulk_load(slots + (size_t)s * rowbytes, Xf + row_sm[issued], rowbytes, &bars[s]);
+      }
+    }
+    return issued;
+  };
+  int issued_early = 0;
+  if (early) {
+    issued_early = stage_chunk(0, rows_cta < LG_CHUNK_ROWS ? rows_cta : LG_CHUNK_ROWS);
+    pdl_wait();
+  }
+  const long long k = P.st->k;
+  int failed = 0;
+  if ((uint32_t)k != k32) {  // the chain's bookkeeping and the iteration counter disagree: nothing is computed
+    if (tid == 0) atomicCAS(&P.st->err, (int)DEV_OK, (int)DEV_ERR_CHAIN);
+    if (tid == ISSUER)  // the copies already started get a bounded chance to land before the CTA leaves
+      for (int j = 0; j < issued_early; ++j) mbar_wait_bounded(&bars[j], 0u);
+    return;
+  }
+  const int ring = P.D + 1;
+  const float* theta_k = P.theta_ring + (k % ring) * P.p_pad;
 
   // column ownership
   bool own[CPT];
@@ -168,9 +213,7 @@ __global__ void __launch_bounds__(THREADS, MINB) grad_linear_large_kernel(const 
 
   int cur_g = -1;
   int g_end = 0;          // CTA-local row at which the current group ends
-  int cslot = 0;          // ring slot of the next row to consume
   uint32_t cphase = 0;    // barrier parity of that slot's current fill
-  int failed = 0;
 
   auto flush = [&](int g) {
     const long long slot = (long long)blockIdx.x * P.pm.maxseg + (g - g_first);
@@ -198,25 +241,7 @@ __global__ void __launch_bounds__(THREADS, MINB) grad_linear_large_kernel(const 
 
   for (int cs = 0; cs < rows_cta && !failed; cs += LG_CHUNK_ROWS) {
     const int nrows = rows_cta - cs < LG_CHUNK_ROWS ? rows_cta - cs : LG_CHUNK_ROWS;
-    __syncthreads();  // previous chunk fully consumed; barriers initialised (first pass)
-    for (int i = tid; i < nrows; i += THREADS) {
-      const int pos = in_g0 + cs + i;
-      const int gi = pos / B;
-      const long long row = batch_row(P, k32, skip ? sel_sm[g_first + gi] : g_first + gi, pos - gi * B);
-      row_sm[i] = row * P.ld;
-      y_sm[i] = yf[row];
-    }
-    __syncthreads();
-    int issued = 0;
-    if (tid == ISSUER) {
-      const int n0 = nrows < nslot ? nrows : nslot;
-      for (; issued < n0; ++issued) {
-        int s = cslot + issued;
-        if (s >= nslot) s -= nslot;
-        mbar_expect_tx(&bars[s], rowbytes);
-        bulk_load(slots + (size_t)s * rowbytes, Xf + row_sm[issued], rowbytes, &bars[s]);
-      }
-    }
+    int issued = (early && cs == 0) ? issued_early : stage_chunk(cs, nrows);
     int consumed = 0;
     while (consumed < nrows) {
       const int lr = cs + consumed;
@@ -386,6 +411,8 @@ __global__ void __launch_bounds__(256) grad_linear_small_kernel(const Params P) 
   __shared__ float accw[NW][2][32 * CPL];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int d = P.d;
+  pdl_launch_dependents();
+  pdl_wait();
   const long long k = P.st->k;
   const uint32_t k32 = (uint32_t)k;
   const int ring = P.D + 1;
@@ -502,7 +529,7 @@ static size_t large_smem_fixed(int threads, int R) {
 
 template <int CPT, int R, int MINB>
 static cudaError_t launch_large(const Params& P, const LinearPlan& plan, bool quad, cudaStream_t st,
-                                bool attr_only) {
+                                bool attr_only, bool pdl) {
   void (*kern)(const Params, int);
   if (plan.full)
     kern = quad ? grad_linear_large_kernel<256, CPT, R, MINB, true, true>
@@ -512,17 +539,13 @@ static cudaError_t launch_large(const Params& P, const LinearPlan& plan, bool qu
                 : grad_linear_large_kernel<256, CPT, R, MINB, false, false>;
   if (attr_only)
     return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
-  kern<<<plan.n_cta, 256, plan.smem_bytes, st>>>(P, plan.nslot);
-  return cudaGetLastError();
+  return launch_k(kern, dim3(plan.n_cta), dim3(256), plan.smem_bytes, st, pdl, P, plan.nslot);
 }
 
 template <int CPL>
-static cudaError_t launch_small(const Params& P, const LinearPlan& plan, bool quad, cudaStream_t st) {
-  if (quad)
-    grad_linear_small_kernel<CPL, true><<<plan.n_cta, 256, 0, st>>>(P);
-  else
-    grad_linear_small_kernel<CPL, false><<<plan.n_cta, 256, 0, st>>>(P);
-  return cudaGetLastError();
+static cudaError_t launch_small(const Params& P, const LinearPlan& plan, bool quad, cudaStream_t st, bool pdl) {
+  if (quad) return launch_k(grad_linear_small_kernel<CPL, true>, dim3(plan.n_cta), dim3(256), 0, st, pdl, P);
+  return launch_k(grad_linear_small_kernel<CPL, false>, dim3(plan.n_cta), dim3(256), 0, st, pdl, P);
 }
 
 bool plan_linear(int d, long long ld, const void* X, int G, int B, int sm_count, size_t smem_optin,
@@ -574,29 +597,29 @@ bool plan_linear(int d, long long ld, const void* X, int G, int B, int sm_count,
 }
 
 static cudaError_t dispatch_large(const Params& P, const LinearPlan& plan, bool quad, cudaStream_t st,
-                                  bool attr_only) {
+                                  bool attr_only, bool pdl) {
   switch (plan.cpt) {
-    case 1: return launch_large<1, 2, 2>(P, plan, quad, st, attr_only);
-    case 2: return launch_large<2, 2, 2>(P, plan, quad, st, attr_only);
-    default: return launch_large<4, 2, 2>(P, plan, quad, st, attr_only);
+    case 1: return launch_large<1, 2, 2>(P, plan, quad, st, attr_only, pdl);
+    case 2: return launch_large<2, 2, 2>(P, plan, quad, st, attr_only, pdl);
+    default: return launch_large<4, 2, 2>(P, plan, quad, st, attr_only, pdl);
   }
 }
 
 cudaError_t prepare_grad_linear(const LinearPlan& plan, bool quad) {
   if (plan.small) return cudaSuccess;
-  return dispatch_large(Params{}, plan, quad, nullptr, true);
+  return dispatch_large(Params{}, plan, quad, nullptr, true, false);
 }
 
-cudaError_t launch_grad_linear(const Params& P, const LinearPlan& plan, bool quad, cudaStream_t st) {
+cudaError_t launch_grad_linear(const Params& P, const LinearPlan& plan, bool quad, cudaStream_t st, bool pdl) {
   if (plan.small) {
     switch (plan.cpl) {
-      case 1: return launch_small<1>(P, plan, quad, st);
-      case 2: return launch_small<2>(P, plan, quad, st);
-      case 4: return launch_small<4>(P, plan, quad, st);
-      default: return launch_small<8>(P, plan, quad, st);
+      case 1: return launch_small<1>(P, plan, quad, st, pdl);
+      case 2: return launch_small<2>(P, plan, quad, st, pdl);
+      case 4: return launch_small<4>(P, plan, quad, st, pdl);
+      default: return launch_small<8>(P, plan, quad, st, pdl);
     }
   }
-  return dispatch_large(P, plan, quad, st, false);
+  return dispatch_large(P, plan, quad, st, false, pdl);
 }
 
 }  // namespace gcada

@@ -24,7 +24,8 @@ bool plan_linear(int d, long long ld, const void* X, int G, int B, int sm_count,
                  LinearPlan* plan, const char** why);
 // One-time function attributes (dynamic shared memory size); call before the first launch.
 cudaError_t prepare_grad_linear(const LinearPlan& plan, bool quad);
-cudaError_t launch_grad_linear(const Params& P, const LinearPlan& plan, bool quad, cudaStream_t st);
+// pdl (here and below): the launch carries the programmatic-dependent-launch attribute (see pdl_wait)
+cudaError_t launch_grad_linear(const Params& P, const LinearPlan& plan, bool quad, cudaStream_t st, bool pdl = false);
 
 struct TailPlan {
   int select_cols4_per_block;  // float4 columns per block of the selection kernel
@@ -34,10 +35,10 @@ struct TailPlan {
 };
 void plan_tail(long long p_pad, int G, int sm_count, TailPlan* plan);
 // Rule PS only: the printed left side of Eq. (9) for every group (run before the selection kernel).
-cudaError_t launch_ps_lhs(const Params& P, const TailPlan& plan, cudaStream_t st);
+cudaError_t launch_ps_lhs(const Params& P, const TailPlan& plan, cudaStream_t st, bool pdl = false);
 // what: 0 = reduce the gradient partial sums and schedule, 1 = schedule only, 2 = reduce only (skip mode).
-cudaError_t launch_select(const Params& P, const TailPlan& plan, cudaStream_t st, int what = 0);
-cudaError_t launch_update(const Params& P, const TailPlan& plan, cudaStream_t st);
+cudaError_t launch_select(const Params& P, const TailPlan& plan, cudaStream_t st, int what = 0, bool pdl = false);
+cudaError_t launch_update(const Params& P, const TailPlan& plan, cudaStream_t st, bool pdl = false);
 
 // Narrow linear models, free-running default rule: any number of iterations in one launch of a single
 // thread-block cluster (see linear_cluster.cu).

@@ -39,6 +39,7 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = blockIdx.y;
   const long long cols4 = P.p_pad >> 2;
+  pdl_wait();  // (no pdl_launch_dependents here: see enqueue_iteration)
   const long long k = P.st->k;
 
   // ---- phase 1: partial sums -> fresh_g (and stale_g), innovation norm
@@ -306,6 +307,8 @@ __global__ void __launch_bounds__(256) update_kernel(const Params P) {
   __shared__ bool is_last;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const long long cols4 = P.p_pad >> 2;
+  pdl_launch_dependents();
+  pdl_wait();
   const long long k = P.st->k;
   const int ring = P.D + 1;
   const float alpha_k = step_size(P, k);
@@ -423,6 +426,7 @@ __global__ void __launch_bounds__(256) update_kernel(const Params P) {
   if (tid == 0) {
     P.s_ring[k % P.D] = s;
     P.st->k = k + 1;
+    if (P.chain_last) P.st->k_chain = (unsigned int)(k + 1);
     P.st->ticket_update = 0u;
   }
 }
@@ -437,6 +441,8 @@ __global__ void __launch_bounds__(256) update_wide_kernel(const Params P) {
   __shared__ bool is_last;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const long long cols4 = P.p_pad >> 2;
+  pdl_launch_dependents();
+  pdl_wait();
   const long long k = P.st->k;
   const int ring = P.D + 1;
   const float alpha_k = step_size(P, k);
@@ -527,6 +533,7 @@ __global__ void __launch_bounds__(256) update_wide_kernel(const Params P) {
   if (tid == 0) {
     P.s_ring[k % P.D] = s;
     P.st->k = k + 1;
+    if (P.chain_last) P.st->k_chain = (unsigned int)(k + 1);
     P.st->ticket_update = 0u;
   }
 }
@@ -537,6 +544,8 @@ __global__ void __launch_bounds__(256) update_direct_kernel(const Params P) {
   __shared__ bool is_last;
   const int tid = threadIdx.x;
   const long long cols4 = P.p_pad >> 2;
+  pdl_launch_dependents();
+  pdl_wait();
   const long long k = P.st->k;
   const int ring = P.D + 1;
   const float alpha_k = step_size(P, k);
@@ -583,6 +592,7 @@ __global__ void __launch_bounds__(256) update_direct_kernel(const Params P) {
   if (tid == 0) {
     P.s_ring[k % P.D] = s;
     P.st->k = k + 1;
+    if (P.chain_last) P.st->k_chain = (unsigned int)(k + 1);
     P.st->ticket_update = 0u;
   }
 }
@@ -596,6 +606,7 @@ __global__ void __launch_bounds__(256) ps_lhs_kernel(const Params P) {
   const int tid = threadIdx.x;
   const int d = blockIdx.y + 1;
   const long long cols4 = P.p_pad >> 2;
+  pdl_wait();
   const long long k = P.st->k;
   const int ring = P.D + 1;
   long long j = k - d;
@@ -628,9 +639,8 @@ __global__ void __launch_bounds__(256) ps_lhs_kernel(const Params P) {
   if (tid == 0) P.st->ticket_aux = 0u;
 }
 
-cudaError_t launch_ps_lhs(const Params& P, const TailPlan& plan, cudaStream_t st) {
-  ps_lhs_kernel<<<dim3(plan.ps_blocks, P.D), 256, 0, st>>>(P);
-  return cudaGetLastError();
+cudaError_t launch_ps_lhs(const Params& P, const TailPlan& plan, cudaStream_t st, bool pdl) {
+  return launch_k(ps_lhs_kernel, dim3(plan.ps_blocks, P.D), dim3(256), 0, st, pdl, P);
 }
 
 void plan_tail(long long p_pad, int G, int sm_count, TailPlan* plan) {
@@ -644,32 +654,26 @@ void plan_tail(long long p_pad, int G, int sm_count, TailPlan* plan) {
   plan->ps_blocks = (int)(pb < 1 ? 1 : (pb > 1024 ? 1024 : pb));
 }
 
-cudaError_t launch_select(const Params& P, const TailPlan& plan, cudaStream_t st, int what) {
+cudaError_t launch_select(const Params& P, const TailPlan& plan, cudaStream_t st, int what, bool pdl) {
   if (what == SEL_SCHEDULE || P.pm.n_cta < 0) {
     // nothing to reduce: with n_cta < 0 the norm partial sums are already in lhs_part (maxseg per group);
     // in skip mode (rule PS) the left sides come from ps_lhs and lhs_part is not read (0 slots)
-    select_kernel<1><<<dim3(1, 1), 256, 0, st>>>(P, P.pm.n_cta < 0 ? P.pm.maxseg : 0, SEL_SCHEDULE);
-    return cudaGetLastError();
+    return launch_k(select_kernel<1>, dim3(1, 1), dim3(256), 0, st, pdl, P, P.pm.n_cta < 0 ? P.pm.maxseg : 0,
+                    (int)SEL_SCHEDULE);
   }
   dim3 grid(plan.select_blocks_x, P.G);
   if (plan.select_cols4_per_block == 256)
-    select_kernel<1><<<grid, 256, 0, st>>>(P, plan.select_blocks_x, what);
-  else
-    select_kernel<4><<<grid, 256, 0, st>>>(P, plan.select_blocks_x, what);
-  return cudaGetLastError();
+    return launch_k(select_kernel<1>, grid, dim3(256), 0, st, pdl, P, plan.select_blocks_x, what);
+  return launch_k(select_kernel<4>, grid, dim3(256), 0, st, pdl, P, plan.select_blocks_x, what);
 }
 
-cudaError_t launch_update(const Params& P, const TailPlan& plan, cudaStream_t st) {
-  if (P.agg_direct) {
-    update_direct_kernel<<<(plan.update_blocks + 7) / 8, 256, 0, st>>>(P);
-    return cudaGetLastError();
-  }
-  if (P.p_pad >= 4 * 256 * 128) {  // enough 16-byte columns to fill the machine with one per thread
-    update_wide_kernel<<<(plan.update_blocks + 7) / 8, 256, (size_t)P.G * sizeof(int), st>>>(P);
-    return cudaGetLastError();
-  }
-  update_kernel<<<plan.update_blocks, 256, (size_t)P.G * sizeof(int), st>>>(P);
-  return cudaGetLastError();
+cudaError_t launch_update(const Params& P, const TailPlan& plan, cudaStream_t st, bool pdl) {
+  if (P.agg_direct)
+    return launch_k(update_direct_kernel, dim3((plan.update_blocks + 7) / 8), dim3(256), 0, st, pdl, P);
+  if (P.p_pad >= 4 * 256 * 128)  // enough 16-byte columns to fill the machine with one per thread
+    return launch_k(update_wide_kernel, dim3((plan.update_blocks + 7) / 8), dim3(256), (size_t)P.G * sizeof(int), st,
+                    pdl, P);
+  return launch_k(update_kernel, dim3(plan.update_blocks), dim3(256), (size_t)P.G * sizeof(int), st, pdl, P);
 }
 
 }  // namespace gcada

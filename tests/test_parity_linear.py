@@ -86,18 +86,30 @@ def test_free_running_masks_match_until_a_near_tie():
     assert got[0].all()                 # first iteration selects every group
 
 
-def test_graph_replay_equals_plain_launches_bitwise():
-    w = to_cuda(make_workload("cfg2", rows=50000))
+@pytest.mark.parametrize("name,rows,over", [("cfg2", 50000, {}), ("cfg3", 20000, {}),
+                                            ("cfg3", 9000, dict(dims=(1004,), M=40, M_G=4, batch=77, D=3))])
+def test_graph_replay_equals_plain_launches_bitwise(name, rows, over):
+    """Replayed graphs hold chains of 16 iterations whose kernels are launched programmatically dependent; in
+    a chain the wide models' gradient kernel starts copying rows before the previous iteration has finished
+    and takes the iteration number for its draw from the chain's start.  Nothing of that may change a bit,
+    however the run is cut into calls, and also when plain (forced) iterations sit between two chains."""
+    w = to_cuda(make_workload(name, rows=rows, **over))
+    G = w["M"] // w["M_G"]
+    forced = np.ones((3, G), np.uint8)
+    forced[1, ::2] = 0
     runs = []
-    for graph, chunks in ((1.0, [37]), (0.0, [37]), (1.0, [16, 5, 16])):
+    for graph, chunks in ((1.0, [40]), (0.0, [40]), (1.0, [16, 5, 19]), (1.0, [33, -3, 4]), (0.0, [33, -3, 4])):
         g = binding.from_workload(w, stream=_stream(), options={binding.OPT_GRAPH: graph, binding.OPT_PERSISTENT: 0.0})
         for n in chunks:
-            g.step(n)
-        runs.append((g.get_theta(), g.get_selection_mask(0, 37), g.get_wallclock(), g.get_comm_count()))
+            if n < 0:
+                g.step_forced(forced)
+            else:
+                g.step(n)
+        runs.append((g.get_theta(), g.get_selection_mask(0, 40), g.get_wallclock(), g.get_comm_count()))
         g.close()
-    for r in runs[1:]:
-        assert np.array_equal(r[0], runs[0][0]) and np.array_equal(r[1], runs[0][1])
-        assert r[2] == runs[0][2] and r[3] == runs[0][3]
+    for a, b in ((0, 1), (0, 2), (3, 4)):
+        assert np.array_equal(runs[a][0], runs[b][0]) and np.array_equal(runs[a][1], runs[b][1])
+        assert runs[a][2] == runs[b][2] and runs[a][3] == runs[b][3]
 
 
 @pytest.mark.parametrize("name,rows,over", [("cfg1", None, {}), ("cfg2", 60000, {}),
