@@ -374,7 +374,7 @@ gcada_status enqueue_iteration(gcada_ctx* ctx, const Params& P) {
   // kernel programmatically dependent too, so that the copies also run under the selection kernel, 104.7
   // (the selection's chain of dependent loads queues behind them); every kernel releasing its dependents at
   // its start 109.8.
-  const bool pdl = P.pdl != 0;
+  const bool pdl = P.pdl != 0 && is_linear(ctx);
   if (is_linear(ctx)) {
     CK(launch_grad_linear(P, ctx->lin, ctx->kind == GCADA_MODEL_QUADRATIC, ctx->stream, pdl && P.k_off > 0));
     ctx->launches += 1;
@@ -415,7 +415,7 @@ gcada_status capture_graph(gcada_ctx* ctx, int iters, cudaGraph_t* out) {
     Params Q = ctx->P;
     Q.k_off = i;
     Q.chain_last = i == iters - 1;
-    Q.pdl = (is_linear(ctx) && !Q.skip_unselected) ? 1 : 0;
+    Q.pdl = Q.skip_unselected ? 0 : 1;
     s = enqueue_iteration(ctx, Q);
   }
   ctx->capturing = false;

@@ -1156,17 +1156,25 @@ __global__ void __launch_bounds__(256) bf16_convert_kernel(const Params P, const
 // ----------------------------------------------------------------- gather
 // Block = 32 consecutive minibatch rows of one group, copied with 16-byte loads and stores into the group's
 // upload buffer that receives this iteration's factors.
+// Inside a chain of captured iterations (P.pdl) the kernel runs beside the previous iteration's update kernel:
+// the draw does not depend on the iterate (Section II-A), the iteration number comes from the chain's start,
+// and neither cur[] nor the buffer written here is touched by the update.  It waits for the update at its end,
+// so that its completion implies the update's.
 __global__ void __launch_bounds__(256) bf16_gather_kernel(const Params P, __nv_bfloat16* xb, int* yb, int d, int ld0,
                                                           int Bp) {
   __shared__ long long rows_sm[32];
   const int g = blockIdx.y, rb = blockIdx.x * 32;
   const int tid = threadIdx.x;
+  const bool early = P.pdl != 0 && !P.skip_unselected;
+  pdl_launch_dependents();
+  if (!early) pdl_wait();
+  const uint32_t k32 = early ? P.st->k_chain + (uint32_t)P.k_off : (uint32_t)P.st->k;
   if (P.skip_unselected && !P.mask_cur[g]) return;
   const int fb = fresh_buf(P, g);
   if (tid < 32) {
     const int j = rb + tid;
     long long row = -1;
-    if (j < P.B) row = batch_row(P, (uint32_t)P.st->k, g, j);
+    if (j < P.B) row = batch_row(P, k32, g, j);
     rows_sm[tid] = row;
     yb[(long long)g * Bp + j] = row >= 0 ? reinterpret_cast<const int*>(P.y)[row] : -1;
   }
@@ -1189,6 +1197,11 @@ __global__ void __launch_bounds__(256) bf16_gather_kernel(const Params P, __nv_b
       const long long row = rows_sm[r];
       out[(long long)r * ld0 + c] = row >= 0 ? X[row * P.ld + c] : __float2bfloat16_rn(0.f);
     }
+  }
+  if (early) {
+    pdl_wait();
+    if (blockIdx.x == 0 && g == 0 && tid == 0 && (uint32_t)P.st->k != k32)
+      atomicCAS(&P.st->err, (int)DEV_OK, (int)DEV_ERR_CHAIN);
   }
 }
 
@@ -1634,6 +1647,12 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
   const long long rows = (long long)G * Bp;
   int n = 0;
   cudaError_t e;
+  // the minibatch rows first: inside a captured chain this launch is programmatically dependent on the previous
+  // iteration's update kernel and runs beside it
+  if ((e = launch_k(bf16_gather_kernel, dim3(Bp / 32, G), dim3(256), 0, st, P.pdl != 0 && P.k_off > 0, P, im->xb,
+                    im->yb, pl.dims[0], im->ld[0], Bp)) != cudaSuccess)
+    return e;
+  ++n;
   // weights of theta^k -> bf16 ring slot k (both orientations) and rounded biases
   {
     ConvArgs c{};
@@ -1657,9 +1676,6 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     ++n;
   }
-  bf16_gather_kernel<<<dim3(Bp / 32, G), 256, 0, st>>>(P, im->xb, im->yb, pl.dims[0], im->ld[0], Bp);
-  if ((e = cudaGetLastError()) != cudaSuccess) return e;
-  ++n;
   // production: no group's weight gradient is formed; the stale point's epilogues write differences for the
   // Gram form of the innovation norm.  Inspection mode keeps both gradients of every group instead.
   const bool production = !P.stale && !P.skip_unselected;

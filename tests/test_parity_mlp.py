@@ -79,3 +79,29 @@ def test_printed_rule_computes_only_the_selected_groups():
     masks = g.get_selection_mask(0, K)
     assert masks[0].all() and 0 < masks.sum() < masks.size
     assert g.get_comm_count() == (o.uploads, o.comm, o.comp)
+
+
+@pytest.mark.parametrize("name,over", [("cfg4", dict(rows=5 * 400)),
+                                       ("cfg5", dict(rows=6000, dims=(64, 128, 96, 40), M=12, M_G=2, D=5, batch=128, c=1.0))])
+def test_graph_replay_equals_plain_launches_bitwise(name, over):
+    """Inside a replayed chain of iterations the kernel that gathers the minibatch rows is launched programmatically
+    dependent on the previous iteration's update kernel and runs beside it, with the iteration number of its
+    draw taken from the chain's start.  The run must not depend on that in any bit, however it is cut into
+    calls and with plain (forced) iterations between two chains."""
+    w = to_cuda(make_workload(name, **over))
+    G = w["M"] // w["M_G"]
+    forced = np.ones((3, G), np.uint8)
+    forced[1, ::2] = 0
+    runs = []
+    for graph, chunks in ((1.0, [40]), (0.0, [40]), (1.0, [16, 5, 19]), (1.0, [33, -3, 4]), (0.0, [33, -3, 4])):
+        g = binding.from_workload(w, stream=torch.cuda.Stream(), options={binding.OPT_GRAPH: graph})
+        for n in chunks:
+            if n < 0:
+                g.step_forced(forced)
+            else:
+                g.step(n)
+        runs.append((g.get_theta(), g.get_selection_mask(0, 40), g.get_wallclock(), g.get_comm_count()))
+        g.close()
+    for a, b in ((0, 1), (0, 2), (3, 4)):
+        assert np.array_equal(runs[a][0], runs[b][0]) and np.array_equal(runs[a][1], runs[b][1])
+        assert runs[a][2] == runs[b][2] and runs[a][3] == runs[b][3]
