@@ -1291,50 +1291,65 @@ __global__ void __launch_bounds__(256) bf16_softmax_grad_pairs_kernel(const Para
   for (int q = q_first; q <= q_last; ++q) {
     const long long w0 = (long long)q * rows + r0;
     const bool write_diff = both && q == 1;
-    for (int i = 0; i < 4; ++i) {
-      const int lr = warp * 4 + i;
-      const long long w = w0 + lr;
-      const float* s = scores + w * n_cls;
-      __nv_bfloat16* o = dz + (((long long)factor_entry(P, g, q) * Bp) + m0 + lr) * ldz;
-      const __nv_bfloat16* o0 = dz + (((long long)factor_entry(P, g, 0) * Bp) + m0 + lr) * ldz;  // the same row at theta^k (written by this thread)
-      __nv_bfloat16* df = diff + (r0 + lr) * ldz;
-      __nv_bfloat16* t = sm_tile + lr * pitch;
-      const int y = yb[r0 + lr];
-      float2 v[NP];
-      float mx = -3.0e38f;
+    const long long zq = (long long)factor_entry(P, g, q) * Bp + m0;
+    for (int i = 0; i < 4; i += 2) {  // two rows at a time: the loads of both are in flight together
+      float2 v[2][NP];
+      int y[2];
+      float mx[2];
 #pragma unroll
-      for (int j = 0; j < NP; ++j) {
-        const int c = 2 * lane + 64 * j;
-        v[j] = (y >= 0 && c < n_cls) ? *reinterpret_cast<const float2*>(s + c) : make_float2(-3.0e38f, -3.0e38f);
-        mx = fmaxf(mx, fmaxf(v[j].x, v[j].y));
+      for (int u = 0; u < 2; ++u) {
+        const int lr = warp * 4 + i + u;
+        const float* s = scores + (w0 + lr) * n_cls;
+        y[u] = yb[r0 + lr];
+        mx[u] = -3.0e38f;
+#pragma unroll
+        for (int j = 0; j < NP; ++j) {
+          const int c = 2 * lane + 64 * j;
+          v[u][j] = (y[u] >= 0 && c < n_cls) ? *reinterpret_cast<const float2*>(s + c) : make_float2(-3.0e38f, -3.0e38f);
+        }
       }
 #pragma unroll
-      for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-      // p_y - 1 = -(sum of the other classes' exponentials) / sum, free of cancellation
-      float others = 0.f, ey = 0.f;
+      for (int u = 0; u < 2; ++u) {
 #pragma unroll
-      for (int j = 0; j < NP; ++j) {
-        const int c = 2 * lane + 64 * j;
-        v[j].x = expf(v[j].x - mx);  // classes beyond n_cls: exp of a huge negative number, zero
-        v[j].y = expf(v[j].y - mx);
-        if (c == y) ey = v[j].x; else others += v[j].x;
-        if (c + 1 == y) ey = v[j].y; else others += v[j].y;
+        for (int j = 0; j < NP; ++j) mx[u] = fmaxf(mx[u], fmaxf(v[u][j].x, v[u][j].y));
       }
-      others = warp_sum(others);
-      ey = warp_sum(ey);
-      const float inv = y >= 0 ? 1.0f / (others + ey) : 0.f;
 #pragma unroll
-      for (int j = 0; j < NP; ++j) {
-        const int c = 2 * lane + 64 * j;
-        if (c < n_cls) {
-          const float a = y < 0 ? 0.f : (c == y ? -others * inv : v[j].x * inv) * P.scale;
-          const float b = y < 0 ? 0.f : (c + 1 == y ? -others * inv : v[j].y * inv) * P.scale;
-          const __nv_bfloat162 pr = __floats2bfloat162_rn(a, b);
-          *reinterpret_cast<__nv_bfloat162*>(o + c) = pr;
-          *reinterpret_cast<__nv_bfloat162*>(t + c) = pr;
-          if (write_diff) {
-            const uint32_t fr = *reinterpret_cast<const uint32_t*>(o0 + c);
-            *reinterpret_cast<uint32_t*>(df + c) = bf16x2_sub(fr, *reinterpret_cast<const uint32_t*>(&pr));
+      for (int off = 16; off > 0; off >>= 1) {
+        mx[0] = fmaxf(mx[0], __shfl_xor_sync(0xffffffffu, mx[0], off));
+        mx[1] = fmaxf(mx[1], __shfl_xor_sync(0xffffffffu, mx[1], off));
+      }
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        const int lr = warp * 4 + i + u;
+        __nv_bfloat16* o = dz + (zq + lr) * ldz;
+        __nv_bfloat16* df = diff + (r0 + lr) * ldz;
+        __nv_bfloat16* t = sm_tile + lr * pitch;
+        // p_y - 1 = -(sum of the other classes' exponentials) / sum, free of cancellation
+        float others = 0.f, ey = 0.f;
+#pragma unroll
+        for (int j = 0; j < NP; ++j) {
+          const int c = 2 * lane + 64 * j;
+          v[u][j].x = expf(v[u][j].x - mx[u]);  // classes beyond n_cls: exp of a huge negative number, zero
+          v[u][j].y = expf(v[u][j].y - mx[u]);
+          if (c == y[u]) ey = v[u][j].x; else others += v[u][j].x;
+          if (c + 1 == y[u]) ey = v[u][j].y; else others += v[u][j].y;
+        }
+        others = warp_sum(others);
+        ey = warp_sum(ey);
+        const float inv = y[u] >= 0 ? 1.0f / (others + ey) : 0.f;
+#pragma unroll
+        for (int j = 0; j < NP; ++j) {
+          const int c = 2 * lane + 64 * j;
+          if (c < n_cls) {
+            const float a = y[u] < 0 ? 0.f : (c == y[u] ? -others * inv : v[u][j].x * inv) * P.scale;
+            const float b = y[u] < 0 ? 0.f : (c + 1 == y[u] ? -others * inv : v[u][j].y * inv) * P.scale;
+            const __nv_bfloat162 pr = __floats2bfloat162_rn(a, b);
+            *reinterpret_cast<__nv_bfloat162*>(o + c) = pr;
+            if (write_diff) {  // the tile still holds this row at theta^k (this thread put it there)
+              const uint32_t fr = *reinterpret_cast<const uint32_t*>(t + c);
+              *reinterpret_cast<uint32_t*>(df + c) = bf16x2_sub(fr, *reinterpret_cast<const uint32_t*>(&pr));
+            }
+            *reinterpret_cast<__nv_bfloat162*>(t + c) = pr;
           }
         }
       }
