@@ -1088,7 +1088,8 @@ __global__ void __launch_bounds__(DW_THREADS, 1) bf16_dw_kernel(const __grid_con
 }
 
 // ----------------------------------------------------------------- weights -> bf16 (both orientations)
-// grid (col tiles, row tiles, layer-1); 32 x 32 tiles through shared memory.
+// grid (col tiles, row tiles, layer-1); 64 x 64 tiles through shared memory, two elements per thread so that a warp
+// reads 256 bytes of a row and writes 128 bytes of a row in either orientation.
 struct ConvArgs {
   int n_out[MLP_MAX_LAYERS + 1], n_in[MLP_MAX_LAYERS + 1];
   long long w_off[MLP_MAX_LAYERS + 1], b_off[MLP_MAX_LAYERS + 1];
@@ -1099,10 +1100,10 @@ struct ConvArgs {
 
 __global__ void __launch_bounds__(256) bf16_convert_kernel(const Params P, const ConvArgs a, __nv_bfloat16* wb,
                                                            float* bias) {
-  __shared__ float tile[32][33];
+  __shared__ float tile[64][65];
   const int l = blockIdx.z + 1;
   const int no = a.n_out[l], ni = a.n_in[l];
-  const int r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
+  const int r0 = blockIdx.y * 64, c0 = blockIdx.x * 64;
   if (r0 >= no || c0 >= ni) return;
   const long long k = P.st->k;
   const int slot = (int)(k % (P.D + 1));
@@ -1110,19 +1111,39 @@ __global__ void __launch_bounds__(256) bf16_convert_kernel(const Params P, const
   __nv_bfloat16* W = wb + (long long)slot * a.slot_elems + a.w_pos[l];
   __nv_bfloat16* WT = wb + (long long)slot * a.slot_elems + a.wt_pos[l];
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-  for (int i = ty; i < 32; i += 8) {
-    const int r = r0 + i, c = c0 + tx;
-    float v = 0.f;
-    if (r < no && c < ni) {
-      v = th[a.w_off[l] + (long long)r * ni + c];
-      W[(long long)r * a.ldk[l] + c] = __float2bfloat16_rn(v);
+  const bool pair_ok = ((a.w_off[l] | (long long)ni) & 1) == 0;  // 8-byte loads of the fp32 master weights
+  for (int i = ty; i < 64; i += 8) {
+    const int r = r0 + i, c = c0 + 2 * tx;
+    float v0 = 0.f, v1 = 0.f;
+    if (r < no) {
+      const float* src = th + a.w_off[l] + (long long)r * ni + c;
+      if (pair_ok && c + 1 < ni) {
+        const float2 t = *reinterpret_cast<const float2*>(src);
+        v0 = t.x;
+        v1 = t.y;
+      } else {
+        if (c < ni) v0 = src[0];
+        if (c + 1 < ni) v1 = src[1];
+      }
+      __nv_bfloat16* dst = W + (long long)r * a.ldk[l] + c;  // (even leading dimension, even c: 4-byte aligned)
+      if (c + 1 < ni)
+        *reinterpret_cast<__nv_bfloat162*>(dst) = __floats2bfloat162_rn(v0, v1);
+      else if (c < ni)
+        dst[0] = __float2bfloat16_rn(v0);
     }
-    tile[i][tx] = v;
+    tile[i][2 * tx] = v0;
+    tile[i][2 * tx + 1] = v1;
   }
   __syncthreads();
-  for (int i = ty; i < 32; i += 8) {
-    const int c = c0 + i, r = r0 + tx;
-    if (r < no && c < ni) WT[(long long)c * a.ldn[l] + r] = __float2bfloat16_rn(tile[tx][i]);
+  for (int i = ty; i < 64; i += 8) {
+    const int c = c0 + i, r = r0 + 2 * tx;
+    if (c < ni) {
+      __nv_bfloat16* dst = WT + (long long)c * a.ldn[l] + r;
+      if (r + 1 < no)
+        *reinterpret_cast<__nv_bfloat162*>(dst) = __floats2bfloat162_rn(tile[2 * tx][i], tile[2 * tx + 1][i]);
+      else if (r < no)
+        dst[0] = __float2bfloat16_rn(tile[2 * tx][i]);
+    }
   }
   if (blockIdx.x == 0 && blockIdx.y == 0) {
     float* bo = bias + (long long)slot * a.bias_slot + a.bias_pos[l];
@@ -1687,7 +1708,7 @@ cudaError_t mlp_bf16_launch(const Params& P, const MlpPlan& pl, cudaStream_t st,
     }
     c.slot_elems = im->slot_elems;
     c.bias_slot = im->bias_slot;
-    bf16_convert_kernel<<<dim3((max_ni + 31) / 32, (max_no + 31) / 32, L), 256, 0, st>>>(P, c, im->wb, im->bias);
+    bf16_convert_kernel<<<dim3((max_ni + 63) / 64, (max_no + 63) / 64, L), 256, 0, st>>>(P, c, im->wb, im->bias);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     ++n;
   }
