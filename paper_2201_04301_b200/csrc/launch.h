@@ -31,6 +31,7 @@ struct TailPlan {
   int select_cols4_per_block;  // float4 columns per block of the selection kernel
   int select_blocks_x;         // blocks per group
   int update_blocks;
+  int direct_blocks;  // blocks of update_direct_kernel (a few per SM; each walks the columns with the grid's stride)
   int ps_blocks;               // column blocks of ps_lhs_kernel
 };
 void plan_tail(long long p_pad, int G, int sm_count, TailPlan* plan);

@@ -549,32 +549,48 @@ __global__ void __launch_bounds__(256) update_direct_kernel(const Params P) {
   const long long k = P.st->k;
   const int ring = P.D + 1;
   const float alpha_k = step_size(P, k);
-  const long long i4 = (long long)blockIdx.x * 256 + tid;
+  // a block walks the columns with the grid's stride, two columns of a thread in flight together (a few
+  // blocks per SM: one partial sum and one ticket per block, not per 256 columns)
+  const long long stride = (long long)gridDim.x * 256;
+  const float* th_k = P.theta_ring + (k % ring) * P.p_pad;
+  float* th_n = P.theta_ring + ((k + 1) % ring) * P.p_pad;
   double local = 0.0;
-  if (i4 < cols4) {
-    const long long o = i4 * 4;
-    const float4 ahi = ld4(P.agg_hi + o);
-    float4 h = ld4(P.h + o), vh = ld4(P.vhat + o);
-    const float4 th = ld4(P.theta_ring + (k % ring) * P.p_pad + o);
-    float4 tn;
-#define GCADA_AMSGRAD(c)                                   \
-  {                                                        \
-    const float gr = ahi.c;                                \
-    h.c = P.beta1 * h.c + P.omb1 * gr;                     \
-    const float v = P.beta2 * vh.c + P.omb2 * (gr * gr);   \
-    vh.c = fmaxf(vh.c, v);                                 \
-    const float up = alpha_k * h.c / sqrtf(P.eps + vh.c);   \
-    tn.c = th.c - up;                                      \
-    local += (double)up * (double)up;                      \
+  for (long long i4 = (long long)blockIdx.x * 256 + tid; i4 < cols4; i4 += 2 * stride) {
+    const long long o[2] = {i4 * 4, (i4 + stride) * 4};
+    const bool have[2] = {true, i4 + stride < cols4};
+    float4 ahi[2], h[2], vh[2], th[2];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      if (have[u]) {
+        ahi[u] = ld4(P.agg_hi + o[u]);
+        h[u] = ld4(P.h + o[u]);
+        vh[u] = ld4(P.vhat + o[u]);
+        th[u] = ld4(th_k + o[u]);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      if (!have[u]) continue;
+      float4 tn;
+#define GCADA_AMSGRAD(c)                                        \
+  {                                                             \
+    const float gr = ahi[u].c;                                  \
+    h[u].c = P.beta1 * h[u].c + P.omb1 * gr;                    \
+    const float v = P.beta2 * vh[u].c + P.omb2 * (gr * gr);     \
+    vh[u].c = fmaxf(vh[u].c, v);                                \
+    const float up = alpha_k * h[u].c / sqrtf(P.eps + vh[u].c); \
+    tn.c = th[u].c - up;                                        \
+    local += (double)up * (double)up;                           \
   }
-    GCADA_AMSGRAD(x)
-    GCADA_AMSGRAD(y)
-    GCADA_AMSGRAD(z)
-    GCADA_AMSGRAD(w)
+      GCADA_AMSGRAD(x)
+      GCADA_AMSGRAD(y)
+      GCADA_AMSGRAD(z)
+      GCADA_AMSGRAD(w)
 #undef GCADA_AMSGRAD
-    st4(P.h + o, h);
-    st4(P.vhat + o, vh);
-    st4(P.theta_ring + ((k + 1) % ring) * P.p_pad + o, tn);
+      st4(P.h + o[u], h[u]);
+      st4(P.vhat + o[u], vh[u]);
+      st4(th_n + o[u], tn);
+    }
   }
   const double tot = block_sum(local, scratch);
   if (tid == 0) {
@@ -650,6 +666,8 @@ void plan_tail(long long p_pad, int G, int sm_count, TailPlan* plan) {
   plan->select_cols4_per_block = 256 * U;
   plan->select_blocks_x = (int)((cols4 + 256 * U - 1) / (256 * U));
   plan->update_blocks = (int)((cols4 + 31) / 32);
+  const long long db = (cols4 + 255) / 256;
+  plan->direct_blocks = (int)(db < 8LL * sm_count ? db : 8LL * sm_count);
   long long pb = (cols4 + 256 * 8 - 1) / (256 * 8);  // about eight float4 per thread
   plan->ps_blocks = (int)(pb < 1 ? 1 : (pb > 1024 ? 1024 : pb));
 }
@@ -669,7 +687,7 @@ cudaError_t launch_select(const Params& P, const TailPlan& plan, cudaStream_t st
 
 cudaError_t launch_update(const Params& P, const TailPlan& plan, cudaStream_t st, bool pdl) {
   if (P.agg_direct)
-    return launch_k(update_direct_kernel, dim3((plan.update_blocks + 7) / 8), dim3(256), 0, st, pdl, P);
+    return launch_k(update_direct_kernel, dim3(plan.direct_blocks), dim3(256), 0, st, pdl, P);
   if (P.p_pad >= 4 * 256 * 128)  // enough 16-byte columns to fill the machine with one per thread
     return launch_k(update_wide_kernel, dim3((plan.update_blocks + 7) / 8), dim3(256), (size_t)P.G * sizeof(int), st,
                     pdl, P);
