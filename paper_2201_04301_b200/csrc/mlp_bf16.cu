@@ -254,19 +254,31 @@ constexpr int G_STAGE_BYTES = (BM + GN) * BK * 2;        // 48 KiB
 constexpr int G_STAGES = 4;
 constexpr int G_EPI_WARPS = 8;
 constexpr int G_THREADS = 64 + 32 * G_EPI_WARPS;
-constexpr int G_TR_BYTES = G_EPI_WARPS * 32 * 17 * 4;  // per-warp transposition tiles of the epilogue
+constexpr int TRP = 20;  // words per row of a transposition tile: rows 16-byte aligned, and the eight lanes of a
+                        // 128-bit access phase (row stride 20 words) fall on 32 different banks
+constexpr int G_TR_BYTES = G_EPI_WARPS * 32 * TRP * 4;  // per-warp transposition tiles of the epilogue
 constexpr int G_CS_BYTES = 2 * 4 * GN * 4;             // column sums of a tile per 32-row quadrant, two tiles in flight
 constexpr int G_BIAS_BYTES = G_EPI_WARPS * (GN / 2) * 4;  // each epilogue warp's 128 bias values of the current tile
 constexpr int G_SMEM_BYTES = G_STAGES * G_STAGE_BYTES + 1024 + G_TR_BYTES + G_CS_BYTES + G_BIAS_BYTES;
 constexpr uint32_t IDESC_G = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(GN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 constexpr uint32_t IDESC_MN = IDESC_G | (1u << 15) | (1u << 16);
 
-// Difference of two packed bf16 pairs, each half exact in fp32 and rounded to nearest-even bf16.
+// Difference of two packed bf16 pairs: each half is the exact difference rounded once to nearest-even bf16.
 __device__ __forceinline__ uint32_t bf16x2_sub(uint32_t x, uint32_t y) {
-  const float lo = __uint_as_float(x << 16) - __uint_as_float(y << 16);
-  const float hi = __uint_as_float(x & 0xFFFF0000u) - __uint_as_float(y & 0xFFFF0000u);
-  const __nv_bfloat162 r = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<const uint32_t*>(&r);
+  uint32_t r;
+  asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(x), "r"(y));
+  return r;
+}
+// (lo, hi) -> packed bf16 pair, round to nearest even; the second form also replaces negative values by zero.
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+__device__ __forceinline__ uint32_t pack_relu_bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
 }
 
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
@@ -419,7 +431,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
     const int ew = warp - 2;
     const int quad = warp & 3;
     const int half = ew >> 2;
-    uint32_t* tr = reinterpret_cast<uint32_t*>(tiles + (size_t)G_STAGES * G_STAGE_BYTES) + ew * (32 * 17);
+    uint32_t* tr = reinterpret_cast<uint32_t*>(tiles + (size_t)G_STAGES * G_STAGE_BYTES) + ew * (32 * TRP);
     float* cs_all = reinterpret_cast<float*>(tiles + (size_t)G_STAGES * G_STAGE_BYTES + G_TR_BYTES);  // [2][4][GN]
     float* bias_w = reinterpret_cast<float*>(tiles + (size_t)G_STAGES * G_STAGE_BYTES + G_TR_BYTES + G_CS_BYTES) + ew * (GN / 2);
     bool ok = true;
@@ -524,30 +536,34 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
             }
           }
         } else {
+          // bf16 pairs of this thread's row
           float f[32];
-          if (a.epi == EPI_HIDDEN) {
+          uint32_t h[16];
+          if (a.epi == EPI_HIDDEN) {  // bias, ReLU and rounding (the conversion clamps at zero)
 #pragma unroll
-            for (int j = 0; j < 32; ++j) f[j] = fmaxf(__uint_as_float(v[j]) + bw[j], 0.f);
+            for (int j = 0; j < 32; j += 4) {
+              const float4 b4 = *reinterpret_cast<const float4*>(bw + j);
+              f[j] = __uint_as_float(v[j]) + b4.x;
+              f[j + 1] = __uint_as_float(v[j + 1]) + b4.y;
+              f[j + 2] = __uint_as_float(v[j + 2]) + b4.z;
+              f[j + 3] = __uint_as_float(v[j + 3]) + b4.w;
+              h[j >> 1] = pack_relu_bf16x2(f[j], f[j + 1]);
+              h[(j >> 1) + 1] = pack_relu_bf16x2(f[j + 2], f[j + 3]);
+            }
           } else {  // EPI_DA: ReLU derivative of the layer below (bits of rows / columns outside the matrix are 0)
             const uint32_t bits = mbits[(c - half * (GN / 2)) >> 5];
 #pragma unroll
             for (int j = 0; j < 32; ++j) f[j] = ((bits >> j) & 1u) ? __uint_as_float(v[j]) : 0.f;
-          }
-          // bf16 pairs of this thread's row
-          uint32_t h[16];
 #pragma unroll
-          for (int j = 0; j < 32; j += 2) {
-            __nv_bfloat162 t2 = __floats2bfloat162_rn(f[j], f[j + 1]);
-            h[j >> 1] = *reinterpret_cast<uint32_t*>(&t2);
+            for (int j = 0; j < 32; j += 2) h[j >> 1] = pack_bf16x2(f[j], f[j + 1]);
           }
           if (a.epi == EPI_HIDDEN && row_ok) {
-            // a bf16 is positive iff its bits are non-zero and its sign bit clear
+            // after the clamp a value is positive iff its bits are non-zero (a NaN counts as positive, as before)
             uint32_t bits = 0u;
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
-              const uint32_t lo = h[j] & 0xFFFFu, hi = h[j] >> 16;
-              bits |= (uint32_t)(lo != 0u && lo < 0x8000u) << (2 * j);
-              bits |= (uint32_t)(hi != 0u && hi < 0x8000u) << (2 * j + 1);
+              bits |= (uint32_t)((h[j] & 0xFFFFu) != 0u) << (2 * j);
+              bits |= (uint32_t)((h[j] >> 16) != 0u) << (2 * j + 1);
             }
             a.relu_bits[((long long)z * a.nw + (nc >> 5)) * a.M + m] = bits;
           }
@@ -556,7 +572,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
           // a sector, and the L2 counted twice the sectors the data needs.
           __syncwarp();
 #pragma unroll
-          for (int j = 0; j < 16; ++j) tr[lane * 17 + j] = h[j];
+          for (int j = 0; j < 16; j += 4)
+            *reinterpret_cast<uint4*>(tr + lane * TRP + j) = make_uint4(h[j], h[j + 1], h[j + 2], h[j + 3]);
           __syncwarp();
           if (a.colsum) {
             // column `lane` of the warp's 32 x 32 block summed over its rows in row order (the rounded values:
@@ -564,7 +581,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
             float csum = 0.f;
 #pragma unroll
             for (int r = 0; r < 32; ++r) {
-              const uint32_t wd = tr[r * 17 + (lane >> 1)];
+              const uint32_t wd = tr[r * TRP + (lane >> 1)];
               csum += __uint_as_float((lane & 1) ? (wd & 0xFFFF0000u) : (wd << 16));
             }
             cs_all[((i & 1) * 4 + quad) * GN + c + lane] = csum;
@@ -575,8 +592,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
 #pragma unroll
             for (int it = 0; it < 4; ++it) {
               const int r = it * 8 + (lane >> 2), qd = lane & 3;
-              const uint32_t* src = tr + r * 17 + qd * 4;
-              const uint4 mine = make_uint4(src[0], src[1], src[2], src[3]);
+              const uint4 mine = *reinterpret_cast<const uint4*>(tr + r * TRP + qd * 4);
               *reinterpret_cast<uint4*>(dst0 + (long long)r * a.ldo + qd * 8) = mine;
               if (write_diff) {
                 const uint4 fr = frv[it];
@@ -589,12 +605,16 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
           }
           if (row_ok) {
             __nv_bfloat16* dst = a.out + (long long)zT * a.z_stride_out + (long long)m * a.ldo + nc;
-            for (int j = 0; j < 32 && nc + j < a.N; ++j) dst[j] = __float2bfloat16_rn(f[j]);
+            const unsigned short* hv = reinterpret_cast<const unsigned short*>(h);  // the row's 32 rounded values
+            unsigned short* dst16 = reinterpret_cast<unsigned short*>(dst);
+            for (int j = 0; j < 32 && nc + j < a.N; ++j) dst16[j] = hv[j];
             if (write_diff) {
-              const __nv_bfloat16* fr = a.out + (long long)zF * a.z_stride_out + (long long)m * a.ldo + nc;
-              __nv_bfloat16* df = a.diff + (long long)g * a.z_stride_out + (long long)m * a.ldo + nc;
+              const unsigned short* fr =
+                  reinterpret_cast<const unsigned short*>(a.out + (long long)zF * a.z_stride_out + (long long)m * a.ldo + nc);
+              unsigned short* df =
+                  reinterpret_cast<unsigned short*>(a.diff + (long long)g * a.z_stride_out + (long long)m * a.ldo + nc);
               for (int j = 0; j < 32 && nc + j < a.N; ++j)
-                df[j] = __float2bfloat16_rn(__bfloat162float(fr[j]) - __bfloat162float(__float2bfloat16_rn(f[j])));
+                df[j] = (unsigned short)(bf16x2_sub((uint32_t)fr[j], (uint32_t)hv[j]) & 0xFFFFu);
             }
           }
         }
