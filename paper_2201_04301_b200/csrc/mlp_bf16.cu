@@ -558,12 +558,17 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
             for (int j = 0; j < 32; j += 2) h[j >> 1] = pack_bf16x2(f[j], f[j + 1]);
           }
           if (a.epi == EPI_HIDDEN && row_ok) {
-            // after the clamp a value is positive iff its bits are non-zero (a NaN counts as positive, as before)
+            // After the clamp a value is positive iff its 16 bits are non-zero (a NaN counts as positive, as
+            // before), i.e. iff adding 0x7FFF sets bit 15 (no half exceeds 0x7FFF, so nothing carries over).  The
+            // four flag bytes of two words are gathered into one word and a multiplication moves their top bits
+            // next to each other: (a 2^7 + b 2^15 + c 2^23 + d 2^31) * (2^21 + 2^14 + 2^7 + 1) has a, b, c, d at
+            // bits 28..31 and every other product below bit 24 or beyond bit 31.
             uint32_t bits = 0u;
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              bits |= (uint32_t)((h[j] & 0xFFFFu) != 0u) << (2 * j);
-              bits |= (uint32_t)((h[j] >> 16) != 0u) << (2 * j + 1);
+            for (int k = 0; k < 8; ++k) {
+              const uint32_t s0 = h[2 * k] + 0x7FFF7FFFu, s1 = h[2 * k + 1] + 0x7FFF7FFFu;
+              const uint32_t x = __byte_perm(s0, s1, 0x7531) & 0x80808080u;
+              bits |= ((x * 0x00204081u) >> 28) << (4 * k);
             }
             a.relu_bits[((long long)z * a.nw + (nc >> 5)) * a.M + m] = bits;
           }
