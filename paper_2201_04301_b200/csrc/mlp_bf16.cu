@@ -313,9 +313,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
   // Algorithm 1's own order, the selection is already known) - the selected groups at theta^k only
   const int n_grp = P.skip_unselected ? P.sel_count[0] : P.G;
   // A CTA walks units (column tile, row tile, group) of the launch's point.
-  constexpr int n_q = 1;
   const int total_units = tiles_n * tiles_m * (a.k_batched ? 1 : n_grp);
-  const int n_local = (int)blockIdx.x < total_units ? ((total_units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) * n_q : 0;
+  const int n_local = (int)blockIdx.x < total_units ? (total_units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
   const long long k_it = P.st->k;
 
   if (threadIdx.x == 0) {
@@ -345,7 +344,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
       bool ok = true;
       int it = 0;
       for (int i = 0; i < n_local && ok; ++i) {
-        const int u = blockIdx.x + (i / n_q) * gridDim.x, q = a.k_batched ? 0 : a.point;
+        const int u = blockIdx.x + i * gridDim.x, q = a.k_batched ? 0 : a.point;
         const int nt = u % tiles_n, mt = (u / tiles_n) % tiles_m, gi = u / (tiles_n * tiles_m);
         const int g = a.k_batched ? 0 : (P.skip_unselected ? P.sel_list[gi] : P.age_order[gi]);
         const int z = q * P.G + g;
@@ -437,7 +436,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) bf16_gemm_kernel(const __grid_co
     bool ok = true;
     for (int i = 0; i < n_local; ++i) {
       const int slot = i & 1;
-      const int u = blockIdx.x + (i / n_q) * gridDim.x, q = a.k_batched ? 0 : a.point;
+      const int u = blockIdx.x + i * gridDim.x, q = a.k_batched ? 0 : a.point;
       const int nt = u % tiles_n, mt = (u / tiles_n) % tiles_m, gi = u / (tiles_n * tiles_m);
       const int g = a.k_batched ? 0 : (P.skip_unselected ? P.sel_list[gi] : P.age_order[gi]);
       const int z = q * P.G + g;
