@@ -342,7 +342,9 @@ gcada_status gcada_checkpoint_load(gcada_ctx *ctx, const void *host_buf, unsigne
  * is raised, and from then on every getter returns GCADA_ECUDA with the buffer named in gcada_last_error
  * (a bounded device-side wait that gave up is reported as GCADA_ETIMEOUT the same way, in both libraries).
  * gcada_is_debug_build tells the two libraries apart (1 / 0).  gcada_debug_set_error writes the device error
- * word from the host (dev_err: 0 none, 1 a wait gave up, 2 an index check failed) so that the reporting path
+ * word from the host (dev_err: 0 none, 1 a wait gave up, 2 an index check failed, 3 a kernel that started early
+ * inside a replayed chain of iterations found the iteration counter elsewhere than the chain's bookkeeping:
+ * reported as GCADA_ECUDA) so that the reporting path
  * can be exercised without any device-side failure; in the ordinary library it returns GCADA_ESTATE.
  */
 int gcada_is_debug_build(void);

@@ -1264,7 +1264,7 @@ gcada_status gcada_debug_set_error(gcada_ctx* ctx, int dev_err) {
   if (!ctx) return GCADA_EINVAL;
 #ifdef GCADA_DEBUG
   if (!ctx->have_theta) return fail(ctx, GCADA_ESTATE, "gcada_set_theta has not been called");
-  if (dev_err < 0 || dev_err > DEV_ERR_BOUNDS) return fail(ctx, GCADA_EINVAL, "unknown device error word %d", dev_err);
+  if (dev_err < 0 || dev_err > DEV_ERR_CHAIN) return fail(ctx, GCADA_EINVAL, "unknown device error word %d", dev_err);
   DeviceGuard dg(ctx->device);
   CK(cudaStreamSynchronize(ctx->stream));
   CK(cudaMemcpy(&ctx->st->err, &dev_err, sizeof(int), cudaMemcpyHostToDevice));

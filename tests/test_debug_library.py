@@ -78,7 +78,8 @@ def test_a_raised_error_word_reaches_every_getter(debug_lib):
     g = binding.from_workload(to_cuda(make_workload("cfg1", rows=3000)), stream=torch.cuda.Stream())
     g.step(3)
     g.get_theta()
-    for word, status, text in ((1, binding.ETIMEOUT, "wait"), (2, binding.ECUDA, "index check")):
+    for word, status, text in ((1, binding.ETIMEOUT, "wait"), (2, binding.ECUDA, "index check"),
+                               (3, binding.ECUDA, "chain of iterations")):
         g.debug_set_error(word)
         for call in (g.get_theta, g.get_iteration, g.get_comm_count, g.get_wallclock,
                      lambda: g.get_selection_mask(0, 1), lambda: g.get_debug(binding.DBG_LHS), g.checkpoint_save):
