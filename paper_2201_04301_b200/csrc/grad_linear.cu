@@ -303,8 +303,11 @@ __global__ void __launch_bounds__(THREADS, MINB) grad_linear_large_kernel(const 
                 if (c0 + 3 >= d) x[r][i].w = 0.f;
               }
             }
-            pz[r] += x[r][i].x * th[i].x + x[r][i].y * th[i].y + x[r][i].z * th[i].z + x[r][i].w * th[i].w;
-            pz[R + r] += x[r][i].x * ths[i].x + x[r][i].y * ths[i].y + x[r][i].z * ths[i].z + x[r][i].w * ths[i].w;
+            // (one fused multiply-add per term: written as a sum of products the compiler must keep the
+            // grouping and spends a multiplication and an addition more per four columns)
+            pz[r] = fmaf(x[r][i].w, th[i].w, fmaf(x[r][i].z, th[i].z, fmaf(x[r][i].y, th[i].y, fmaf(x[r][i].x, th[i].x, pz[r]))));
+            pz[R + r] = fmaf(x[r][i].w, ths[i].w,
+                             fmaf(x[r][i].z, ths[i].z, fmaf(x[r][i].y, ths[i].y, fmaf(x[r][i].x, ths[i].x, pz[R + r]))));
           }
         } else {
 #pragma unroll
