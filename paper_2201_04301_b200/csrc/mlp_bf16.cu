@@ -3,8 +3,9 @@
 //
 // Operands are bf16 (features as stored; weights rounded from the fp32 master
 // iterate once per iteration), accumulation is fp32 in tensor memory.  Per-group
-// weight gradients are never materialised on the production path: a first pass
-// forms only the squared innovation norms, and the server's aggregate (Eq. 3,
+// weight gradients are never materialised on the production path: the squared
+// innovation norms come from two Gram products per group and layer over the
+// differences of the two points (bf16_gram_kernel), and the server's aggregate (Eq. 3,
 // the sum over groups of each group's last uploaded gradient) is one product per
 // layer over the factors (dz_l, a_{l-1}) of every group's last
 // upload, with K running over all groups' rows.  The factors at theta^k are
@@ -68,8 +69,8 @@ struct Bf16Impl {
   // blocks of 128 rows; the loss-gradient kernel: blocks of 32 rows): [2][G][blocks][n_l]
   float* dbp[MLP_MAX_LAYERS + 1] = {nullptr};
   int dbp_blocks[MLP_MAX_LAYERS + 1] = {0};
-  // differences between the two points, row-major [G*Bp][ld_l] (see bf16_gram_kernel)
   uint32_t* relu_bits[MLP_MAX_LAYERS + 1] = {nullptr};  // [2G][(n_l + 31) / 32][Bp]: a_l > 0, l = 1..L-1
+  // differences between the two points, row-major [G*Bp][ld_l] (see bf16_gram_kernel)
   __nv_bfloat16* dE[MLP_MAX_LAYERS + 1] = {nullptr};  // dz_l(theta^k) - dz_l(stale), l = 1..L
   __nv_bfloat16* dF[MLP_MAX_LAYERS + 1] = {nullptr};  // a_l(theta^k) - a_l(stale),  l = 1..L-1
   int gram_part_base[MLP_MAX_LAYERS + 1] = {0};
