@@ -27,8 +27,9 @@ struct DevState {
   unsigned int ticket_select;     // "last block done" counters
   unsigned int ticket_update;
   unsigned int ticket_aux;
-  unsigned int k_chain;           // low 32 bits of k as it was when the running chain of iterations began (a chain
-                                  // = the iterations captured in one graph; see Params::k_off)
+  unsigned int pad_;
+  long long k_chain;              // k as it was when the running chain of iterations began (a chain = the
+                                  // iterations captured in one graph; see Params::k_off)
 };
 
 // How a per-group gradient is spread over partial-sum slots by the linear

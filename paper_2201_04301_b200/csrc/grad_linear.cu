@@ -121,7 +121,9 @@ __global__ void __launch_bounds__(THREADS, MINB) grad_linear_large_kernel(const 
   const bool early = P.pdl != 0 && !skip;
   pdl_launch_dependents();
   if (!early) pdl_wait();
-  const uint32_t k32 = early ? P.st->k_chain + (uint32_t)P.k_off : (uint32_t)P.st->k;
+  const long long k_pre = early ? P.st->k_chain + P.k_off : P.st->k;  // the iteration (confirmed after the wait)
+  const uint32_t k32 = (uint32_t)k_pre;
+  const int ring = P.D + 1;
 
   // group numbers below are positions in the list of groups worked on (all groups, or the selected ones)
   __shared__ int sel_sm[SKIP_MAX_GROUPS];
@@ -169,27 +171,35 @@ __global__ void __launch_bounds__(THREADS, MINB) grad_linear_large_kernel(const 
     }
     return issued;
   };
-  int issued_early = 0;
-  if (early) {
-    issued_early = stage_chunk(0, rows_cta < LG_CHUNK_ROWS ? rows_cta : LG_CHUNK_ROWS);
-    pdl_wait();
-  }
-  const long long k = P.st->k;
-  int failed = 0;
-  if ((uint32_t)k != k32) {  // the chain's bookkeeping and the iteration counter disagree: nothing is computed
-    if (tid == 0) atomicCAS(&P.st->err, (int)DEV_OK, (int)DEV_ERR_CHAIN);
-    if (tid == ISSUER)  // the copies already started get a bounded chance to land before the CTA leaves
-      for (int j = 0; j < issued_early; ++j) mbar_wait_bounded(&bars[j], 0u);
-    return;
-  }
-  const int ring = P.D + 1;
-  const float* theta_k = P.theta_ring + (k % ring) * P.p_pad;
-
   // column ownership
   bool own[CPT];
   float4 th[CPT], ths[CPT], acc0[CPT], acc1[CPT];
   const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
   const bool ragged = !FULL && (d & 3) != 0;
+#pragma unroll
+  for (int i = 0; i < CPT; ++i) ths[i] = zero4;
+  int issued_early = 0;
+  // The stale iterate of the CTA's first group can be fetched early as well: the ages were written by the
+  // previous selection kernel, which had finished before the update kernel started, and theta^{k - tau} with
+  // tau >= 1 sits in a slot of the ring that the running update does not write.
+  bool ths_raw = false;  // ths[] holds the first group's stale iterate itself, not yet theta^k minus it
+  if (early) {
+    issued_early = stage_chunk(0, rows_cta < LG_CHUNK_ROWS ? rows_cta : LG_CHUNK_ROWS);
+    if (FULL) {
+      long long js = k_pre - P.tau[g_first];
+      if (js < k_pre - P.D) js = k_pre - P.D;
+      if (js < 0) js = 0;
+      const float* theta_s = P.theta_ring + (js % ring) * P.p_pad;
+#pragma unroll
+      for (int i = 0; i < CPT; ++i) ths[i] = *reinterpret_cast<const float4*>(theta_s + (tid + THREADS * i) * 4);
+      ths_raw = true;
+    }
+    pdl_wait();
+  }
+  // theta^k: its slot follows from the iteration number already at hand, so these loads and the one that
+  // confirms the number leave together
+  const long long k = early ? *reinterpret_cast<volatile const long long*>(&P.st->k) : k_pre;
+  const float* theta_k = P.theta_ring + (k_pre % ring) * P.p_pad;
 #pragma unroll
   for (int i = 0; i < CPT; ++i) {
     const int q = tid + THREADS * i;
@@ -206,9 +216,15 @@ __global__ void __launch_bounds__(THREADS, MINB) grad_linear_large_kernel(const 
         th[i].w = c0 + 3 < d ? theta_k[c0 + 3] : 0.f;
       }
     }
-    ths[i] = zero4;
     acc0[i] = zero4;
     acc1[i] = zero4;
+  }
+  int failed = 0;
+  if (k != k_pre) {  // the chain's bookkeeping and the iteration counter disagree: nothing is computed
+    if (tid == 0) atomicCAS(&P.st->err, (int)DEV_OK, (int)DEV_ERR_CHAIN);
+    if (tid == ISSUER)  // the copies already started get a bounded chance to land before the CTA leaves
+      for (int j = 0; j < issued_early; ++j) mbar_wait_bounded(&bars[j], 0u);
+    return;
   }
 
   int cur_g = -1;
@@ -249,7 +265,7 @@ __global__ void __launch_bounds__(THREADS, MINB) grad_linear_large_kernel(const 
         if (cur_g >= 0) flush(cur_g);
         cur_g = cur_g < 0 ? g_first : cur_g + 1;
         g_end = (cur_g + 1 - g_first) * B - in_g0;
-        long long js = k - P.tau[skip ? sel_sm[cur_g] : cur_g];
+        long long js = k - (ths_raw ? 0 : P.tau[skip ? sel_sm[cur_g] : cur_g]);
         if (js < k - P.D) js = k - P.D;  // ages beyond D only arise under forced masks: oldest kept iterate
         if (js < 0) js = 0;
         const float* theta_s = P.theta_ring + (js % ring) * P.p_pad;
@@ -260,7 +276,7 @@ __global__ void __launch_bounds__(THREADS, MINB) grad_linear_large_kernel(const 
           if (own[i]) {
             const int c0 = (tid + THREADS * i) * 4;
             if (FULL) {
-              const float4 t = *reinterpret_cast<const float4*>(theta_s + c0);
+              const float4 t = ths_raw ? ths[i] : *reinterpret_cast<const float4*>(theta_s + c0);
               ths[i] = make_float4(th[i].x - t.x, th[i].y - t.y, th[i].z - t.z, th[i].w - t.w);
             } else {
               ths[i].x = th[i].x - theta_s[c0];
@@ -270,6 +286,7 @@ __global__ void __launch_bounds__(THREADS, MINB) grad_linear_large_kernel(const 
             }
           }
         }
+        ths_raw = false;
       }
       int lim = (g_end < cs + nrows ? g_end : cs + nrows) - lr;
       const int nb = lim < R ? lim : R;

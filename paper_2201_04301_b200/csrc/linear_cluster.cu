@@ -453,7 +453,7 @@ __global__ void __launch_bounds__(LC_THREADS, 1) linear_cluster_kernel(const Par
     }
     if (tid == 0) {
       st.err = P.st->err;
-      st.k_chain = (unsigned int)st.k;
+      st.k_chain = st.k;
       *P.st = st;
     }
   }

@@ -1214,7 +1214,7 @@ __global__ void __launch_bounds__(256) bf16_gather_kernel(const Params P, __nv_b
   const bool early = P.pdl != 0 && !P.skip_unselected;
   pdl_launch_dependents();
   if (!early) pdl_wait();
-  const uint32_t k32 = early ? P.st->k_chain + (uint32_t)P.k_off : (uint32_t)P.st->k;
+  const uint32_t k32 = (uint32_t)(early ? P.st->k_chain + P.k_off : P.st->k);
   if (P.skip_unselected && !P.mask_cur[g]) return;
   const int fb = fresh_buf(P, g);
   if (tid < 32) {

@@ -426,7 +426,7 @@ __global__ void __launch_bounds__(256) update_kernel(const Params P) {
   if (tid == 0) {
     P.s_ring[k % P.D] = s;
     P.st->k = k + 1;
-    if (P.chain_last) P.st->k_chain = (unsigned int)(k + 1);
+    if (P.chain_last) P.st->k_chain = k + 1;
     P.st->ticket_update = 0u;
   }
 }
@@ -533,7 +533,7 @@ __global__ void __launch_bounds__(256) update_wide_kernel(const Params P) {
   if (tid == 0) {
     P.s_ring[k % P.D] = s;
     P.st->k = k + 1;
-    if (P.chain_last) P.st->k_chain = (unsigned int)(k + 1);
+    if (P.chain_last) P.st->k_chain = k + 1;
     P.st->ticket_update = 0u;
   }
 }
@@ -608,7 +608,7 @@ __global__ void __launch_bounds__(256) update_direct_kernel(const Params P) {
   if (tid == 0) {
     P.s_ring[k % P.D] = s;
     P.st->k = k + 1;
-    if (P.chain_last) P.st->k_chain = (unsigned int)(k + 1);
+    if (P.chain_last) P.st->k_chain = k + 1;
     P.st->ticket_update = 0u;
   }
 }
