@@ -44,7 +44,17 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
 
   // ---- phase 1: partial sums -> fresh_g (and stale_g), innovation norm
   // (skipped when the gradient kernels have already delivered the norm partial sums)
+  const bool tg_early = P.pm.n_cta >= 0 && what == SEL_ALL;  // the groups' computing times are taken in phase 1
   if (P.pm.n_cta >= 0 && what != SEL_SCHEDULE) {
+    // The group's computing time (fastest of its workers, Section II-B) needs nothing from the gradients: the
+    // first warp of the group's first block takes it here, off the single block's chain of phase 2.
+    if (tg_early && blockIdx.x == 0 && warp == 0) {
+      double t = 1.0e300;
+      for (int j = lane; j < P.M_G; j += 32) t = fmin(t, worker_time(P, (uint32_t)k, g * P.M_G + j));
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) t = fmin(t, __shfl_xor_sync(0xffffffffu, t, o));
+      if (lane == 0) P.t_g[g] = t;  // (thread 0: published by the fence before this block's ticket)
+    }
     // skip mode: the group's rank among the selected ones locates its partial sums, and its fresh gradient
     // goes to the row that the flip of cur[g] has already made the last uploaded one
     int gi = g, n_groups = P.G;
@@ -151,6 +161,15 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
   double rhs = 0.0;
   const uint32_t k32 = (uint32_t)k;
   const volatile double* parts = P.lhs_part;
+  // (the counters that thread 0 advances at the end are fetched now, with everything else)
+  unsigned long long up0 = 0ull, comm0 = 0ull, comp0 = 0ull;
+  double wall0 = 0.0;
+  if (tid == 0) {
+    up0 = P.st->uploads;
+    comm0 = P.st->comm;
+    comp0 = P.st->comp;
+    wall0 = P.st->wall;
+  }
   int nsel = 0;
   int listed = 0;  // selected groups of earlier chunks (the same in every thread)
   double tmax = 0.0;
@@ -184,7 +203,8 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
     // computing times: one thread per worker into shared memory (tiles of 1024
     // workers), then each group's thread takes the minimum over its workers
     double t = 1.0e300;
-    const long long w_lo = (long long)gc * P.M_G, w_hi = (long long)(gc + ng) * P.M_G;
+    if (tg_early && have) t = reinterpret_cast<const volatile double*>(P.t_g)[gg];
+    const long long w_lo = (long long)gc * P.M_G, w_hi = tg_early ? w_lo : (long long)(gc + ng) * P.M_G;
     for (long long m0 = w_lo; m0 < w_hi; m0 += 1024) {
       const int cnt = (int)(w_hi - m0 < 1024 ? w_hi - m0 : 1024);
       __syncthreads();
@@ -266,10 +286,10 @@ __global__ void __launch_bounds__(256) select_kernel(const Params P, int blocks_
       tm = fmax(tm, sh_tmax[w]);
     }
     DevState* st = P.st;
-    st->uploads += (unsigned long long)ns;
-    st->comm += (unsigned long long)ns * (unsigned long long)(P.M_G + 1);
-    st->comp += (unsigned long long)ns * (unsigned long long)P.M_G;
-    st->wall += tm;
+    st->uploads = up0 + (unsigned long long)ns;
+    st->comm = comm0 + (unsigned long long)ns * (unsigned long long)(P.M_G + 1);
+    st->comp = comp0 + (unsigned long long)ns * (unsigned long long)P.M_G;
+    st->wall = wall0 + tm;
     st->last_dt = tm;
     st->rhs = rhs;
     st->ticket_select = 0u;
